@@ -1,0 +1,284 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, independent of the oracle's own code.
+
+Each test is chosen so that a plausible mistake in the oracle (a dropped scale, a wrong
+sign, a transposed operand, an off-by-one in the window, a wrong GQA map) fails it.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+
+import wmtp_inputs as wi
+from oracle import reference as R
+from oracle import twin
+
+BF = wi.f32_to_bf16_bits
+F64 = wi.bf16_bits_to_f64
+
+
+def _rand(seed, tid, shape, scale=1.0):
+    return wi.normal_bf16(seed, tid, shape, scale=scale, threads=1)
+
+
+# ---------------------------------------------------------------- golden fixtures (hand-worked)
+def _read_golden(path):
+    rows = []
+    for line in open(path):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        rows.append(line)
+    return rows
+
+
+def test_keep_set_matches_hand_worked_examples(golden_dir):
+    for line in _read_golden(os.path.join(golden_dir, "keep_sets.txt")):
+        lhs, rhs = line.split(":")
+        S, n_sink, W = (int(t) for t in lhs.split())
+        want = [int(t) for t in rhs.split()]
+        assert R.keep_set(S, n_sink, W) == want, line
+        st = R.WindowStore(n_sink, W)
+        for p in range(S):
+            st.append(p, p)
+        assert st.positions() == want, line
+
+
+def test_kv_bytes_per_token_match_paper(golden_dir):
+    for line in _read_golden(os.path.join(golden_dir, "kv_bytes.txt")):
+        Hkv, D, nbytes = (int(t) for t in line.split())
+        cfg = wi.scaled(wi.CONFIGS[2], Hkv=Hkv, D=D)
+        assert cfg.kv_bytes_per_token == nbytes
+    # the million-token configuration reads ~2 GB per full-context step, ~8 MB windowed
+    c3 = wi.CONFIGS[2]
+    assert c3.S0 * c3.kv_bytes_per_token == 2 << 30
+    assert (c3.W + c3.n_sink) * c3.kv_bytes_per_token == 4100 * 2048
+
+
+# ---------------------------------------------------------------- key set / stores, brute force
+@pytest.mark.parametrize("n_sink,W", [(0, 1), (1, 1), (2, 3), (4, 8), (0, 5), (3, 1)])
+def test_window_store_brute_force(n_sink, W):
+    st = R.WindowStore(n_sink, W)
+    for S in range(1, n_sink + W + 71):
+        st.append(("k", S - 1), ("v", S - 1))
+        brute = [p for p in range(S) if p < n_sink or p >= S - W]          # written independently
+        assert st.positions() == brute
+        assert R.keep_set(S, n_sink, W) == brute
+        assert twin.window_positions(S, n_sink, W) == brute
+        assert len(brute) == min(S, n_sink + W)                            # reads min(seq, W + n_sink) tokens
+        assert all(e[1] == ("k", e[0]) and e[2] == ("v", e[0]) for e in st.entries())
+
+
+@pytest.mark.parametrize("n_sink,W,slack", [(0, 1, 0), (1, 1, 0), (2, 3, 0), (4, 8, 0), (4, 8, 3), (2, 5, 7)])
+def test_ring_sim_holds_sink_and_last_W(n_sink, W, slack):
+    cap = W + slack
+    Hkv, D = 2, 4
+    ring = R.RingSim(n_sink, cap, Hkv, D)
+    rows = {}
+    for p in range(3 * (n_sink + cap) + 6):
+        k = np.full((Hkv, D), p * 2 + 1, dtype=np.uint16)
+        v = np.full((Hkv, D), p * 2 + 2, dtype=np.uint16)
+        rows[p] = (k, v)
+        slot = ring.append(k, v)
+        S = p + 1
+        # footprint independent of S; closed-form slot (sink fixed, window region circular)
+        assert slot == (p if p < n_sink else n_sink + (p - n_sink) % cap)
+        assert ring.length == S
+        held = {int(x) for x in ring.slot_pos if x >= 0}
+        want = {q for q in range(S) if q < n_sink or q >= S - cap}
+        assert held == want                                   # ring = sink U last `cap` tokens
+        assert set(R.keep_set(S, n_sink, W)) <= held          # everything the draft reads is present
+        for s, q in enumerate(ring.slot_pos):
+            if q >= 0:
+                assert (ring.K[:, s] == rows[int(q)][0]).all() and (ring.V[:, s] == rows[int(q)][1]).all()
+            else:
+                assert not ring.written[s]
+
+
+# ---------------------------------------------------------------- softmax attention, closed forms
+def test_uniform_keys_give_mean_of_values():
+    Hq, Hkv, D, n = 8, 2, 16, 37
+    q = _rand(1, 1, (Hq, D))
+    krow = _rand(1, 2, (Hkv, 1, D))
+    K = np.repeat(krow, n, axis=1)
+    V = _rand(1, 3, (Hkv, n, D))
+    out, lse = R.attention(q, K, V)
+    G = Hq // Hkv
+    for h in range(Hq):
+        g = h // G
+        np.testing.assert_allclose(out[h], F64(V[g]).mean(axis=0), rtol=0, atol=1e-13)
+        z = (F64(q[h]) * F64(krow[g, 0])).sum() / math.sqrt(D)
+        assert abs(lse[h] - (z + math.log(n))) < 1e-12
+
+
+def test_zero_query_gives_mean_and_log_count():
+    Hq, Hkv, D, n = 4, 4, 8, 11
+    q = np.zeros((Hq, D), dtype=np.uint16)
+    K, V = _rand(2, 2, (Hkv, n, D)), _rand(2, 3, (Hkv, n, D))
+    out, lse = R.attention(q, K, V)
+    for h in range(Hq):
+        np.testing.assert_allclose(out[h], F64(V[h]).mean(axis=0), atol=1e-14)
+        assert abs(lse[h] - math.log(n)) < 1e-14
+
+
+def test_single_key_returns_its_value_exactly():
+    Hq, Hkv, D = 6, 3, 8
+    q, K, V = _rand(3, 1, (Hq, D)), _rand(3, 2, (Hkv, 1, D)), _rand(3, 3, (Hkv, 1, D))
+    out, lse = R.attention(q, K, V)
+    for h in range(Hq):
+        g = h // 2
+        assert (out[h] == F64(V[g, 0])).all()
+        assert abs(lse[h] - (F64(q[h]) * F64(K[g, 0])).sum() / math.sqrt(D)) < 1e-14
+
+
+def test_two_keys_logistic_closed_form_and_scale():
+    # q = 4*e_0 ; k_a = 3*e_0, k_b = -1*e_0 ; logits = scale*12, scale*(-4).
+    D = 4
+    q = BF(np.array([[4, 0, 0, 0]], dtype=np.float32))
+    K = BF(np.array([[[3, 9, 9, 9], [-1, 5, 5, 5]]], dtype=np.float32))
+    V = BF(np.array([[[1, 0, 2, 8], [0, 1, -2, 4]]], dtype=np.float32))
+    for scale in (None, 0.125, 1.0):
+        s = 1 / math.sqrt(D) if scale is None else scale
+        out, lse = R.attention(q, K, V, sm_scale=scale)
+        wa = 1.0 / (1.0 + math.exp(-(12 * s - (-4 * s))))       # logistic of the logit gap
+        want = wa * np.array([1, 0, 2, 8.0]) + (1 - wa) * np.array([0, 1, -2, 4.0])
+        np.testing.assert_allclose(out[0], want, rtol=1e-14, atol=1e-15)
+        assert abs(lse[0] - (12 * s + math.log1p(math.exp(-16 * s)))) < 1e-13
+
+
+def test_dominant_key_wins():
+    Hq, Hkv, D, n = 4, 1, 16, 50
+    q = BF(np.ones((Hq, D), dtype=np.float32) * 2)
+    Kf = np.zeros((Hkv, n, D), dtype=np.float32)
+    Kf[0, 17] = 8.0                                   # logit 2*8*16/4 = 64 above the rest (0)
+    K, V = BF(Kf), _rand(4, 3, (Hkv, n, D))
+    out, lse = R.attention(q, K, V)
+    np.testing.assert_allclose(out, np.broadcast_to(F64(V[0, 17]), (Hq, D)), atol=1e-20 + 50 * math.exp(-64) * 5)
+    np.testing.assert_allclose(lse, 64.0, atol=1e-12)
+
+
+def test_gqa_head_map_is_consecutive_groups():
+    Hq, Hkv, D, n = 8, 4, 4, 5
+    q = _rand(5, 1, (Hq, D))
+    K = _rand(5, 2, (Hkv, n, D))
+    Vf = np.zeros((Hkv, n, D), dtype=np.float32)
+    for g in range(Hkv):
+        Vf[g] = g + 1
+    out, _ = R.attention(q, K, BF(Vf))
+    np.testing.assert_allclose(out[:, 0], [1, 1, 2, 2, 3, 3, 4, 4], atol=1e-14)
+
+
+def test_shift_and_permutation_invariance():
+    Hq, Hkv, D, n = 4, 2, 8, 23
+    rs = np.random.RandomState(0)
+    q = BF(rs.randint(-3, 4, (Hq, D)).astype(np.float32))
+    Kf = rs.randint(-4, 5, (Hkv, n, D)).astype(np.float32)
+    c = rs.randint(-2, 3, (Hkv, 1, D)).astype(np.float32)
+    V = _rand(6, 3, (Hkv, n, D))
+    o0, l0 = R.attention(q, BF(Kf), V)
+    o1, l1 = R.attention(q, BF(Kf + c), V)                       # K + c exact in bf16 (small integers)
+    np.testing.assert_allclose(o1, o0, atol=1e-13)
+    for h in range(Hq):
+        shift = (F64(q[h]) * c[h // 2, 0]).sum() / math.sqrt(D)
+        assert abs((l1[h] - l0[h]) - shift) < 1e-12
+    perm = rs.permutation(n)
+    o2, l2 = R.attention(q, BF(Kf), V, keys=perm)
+    np.testing.assert_allclose(o2, o0, atol=1e-14)
+    np.testing.assert_allclose(l2, l0, atol=1e-14)
+    # a strict subset lowers lse and equals attention over the gathered rows
+    sub = np.sort(perm[: n // 2])
+    o3, l3 = R.attention(q, BF(Kf), V, keys=sub)
+    o4, l4 = R.attention(q, np.ascontiguousarray(BF(Kf)[:, sub]), np.ascontiguousarray(V[:, sub]))
+    assert (o3 == o4).all() and (l3 == l4).all() and (l3 < l0).all()
+
+
+def test_empty_key_set():
+    q = _rand(7, 1, (2, 4))
+    K = np.zeros((1, 0, 4), dtype=np.uint16)
+    out, lse = R.attention(q, K, K)
+    assert (out == 0).all() and np.isneginf(lse).all()
+
+
+# ---------------------------------------------------------------- brute force and library cross-check
+@pytest.mark.parametrize("n", [1, 2, 7, 33, 64])
+def test_against_pure_python_twin(n):
+    Hq, Hkv, D = 4, 2, 8
+    q, K, V = _rand(8, (1, n), (Hq, D)), _rand(8, (2, n), (Hkv, n, D), scale=2.0), _rand(8, (3, n), (Hkv, n, D))
+    out, lse = R.attention(q, K, V, sm_scale=0.3)
+    o_py, l_py = twin.attention_py(q.tolist(), K.tolist(), V.tolist(), Hq // Hkv, 0.3)
+    np.testing.assert_allclose(out, np.array(o_py), rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(lse, np.array(l_py), rtol=1e-13, atol=1e-13)
+
+
+def test_against_torch_sdpa_fp64():
+    import torch
+    Hq, Hkv, D, n = 16, 2, 128, 777
+    q, K, V = _rand(9, 1, (Hq, D)), _rand(9, 2, (Hkv, n, D)), _rand(9, 3, (Hkv, n, D))
+    out, lse = R.attention(q, K, V)
+    tq = torch.from_numpy(F64(q)).view(1, Hq, 1, D)
+    tk = torch.from_numpy(F64(K)).repeat_interleave(Hq // Hkv, dim=0).unsqueeze(0)
+    tv = torch.from_numpy(F64(V)).repeat_interleave(Hq // Hkv, dim=0).unsqueeze(0)
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv)[0, :, 0, :].numpy()
+    np.testing.assert_allclose(out, ref, rtol=1e-11, atol=1e-13)
+    z = (tq @ tk.transpose(-1, -2))[0, :, 0, :] / math.sqrt(D)
+    np.testing.assert_allclose(lse, torch.logsumexp(z, dim=-1).numpy(), rtol=1e-13)
+
+
+# ---------------------------------------------------------------- windowed vs full relations
+def _small_cfg(**kw):
+    base = dict(name="t", batch=1, S0=40, Hq=4, Hkv=2, D=16, W=8, n_sink=2, gamma=3, seed=77)
+    base.update(kw)
+    return wi.DraftConfig(**base)
+
+
+@pytest.mark.parametrize("S0", [0, 1, 2, 5, 7])
+def test_windowed_equals_full_when_window_covers_context(S0):
+    cfg = _small_cfg(S0=S0)          # S0 + gamma <= n_sink + W = 10
+    wl = wi.make_workload(cfg, threads=1)
+    o = R.DraftOracle(wl.K[0], wl.V[0], cfg.Hq, cfg.n_sink, cfg.W)
+    for i in range(cfg.gamma):
+        r = o.step(wl.q[i, 0], wl.k_new[i, 0], wl.v_new[i, 0])
+        assert (r["win"][0] == r["full"][0]).all() and (r["win"][1] == r["full"][1]).all()
+
+
+def test_windowed_store_equals_keep_set_applied_to_full_kv():
+    cfg = _small_cfg(S0=61)
+    wl = wi.make_workload(cfg, threads=1)
+    o = R.DraftOracle(wl.K[0], wl.V[0], cfg.Hq, cfg.n_sink, cfg.W)
+    for i in range(cfg.gamma):
+        r = o.step(wl.q[i, 0], wl.k_new[i, 0], wl.v_new[i, 0])
+        keep = R.keep_set(o.S, cfg.n_sink, cfg.W)
+        ow, lw = R.attention(wl.q[i, 0], o.Kfull[:, : o.S], o.Vfull[:, : o.S], keys=keep)
+        np.testing.assert_allclose(r["win"][0], ow, atol=1e-15)
+        np.testing.assert_allclose(r["win"][1], lw, atol=1e-15)
+        # the ring simulation holds exactly the rows the store holds
+        held = {int(p): s for s, p in enumerate(o.ring.slot_pos) if p >= 0}
+        assert sorted(held) == keep
+        for p in keep:
+            assert (o.ring.K[:, held[p]] == o.Kfull[:, p]).all() and (o.ring.V[:, held[p]] == o.Vfull[:, p]).all()
+
+
+def test_mass_identity_and_needle():
+    cfg = _small_cfg(S0=300, W=32, n_sink=4, D=32)
+    wl = wi.make_workload(cfg, threads=1)
+    K0, V0 = wl.K[0].copy(), wl.V[0].copy()
+    # plant a far key aligned with query head 0 of step 0 (outside sink and window)
+    qf = wi.bf16_bits_to_f32(wl.q[0, 0, 0])
+    K0[0, 100] = BF(qf * 3.0)
+    o = R.DraftOracle(K0, V0, cfg.Hq, cfg.n_sink, cfg.W)
+    r = o.step(wl.q[0, 0], wl.k_new[0, 0], wl.v_new[0, 0])
+    (ow, lw), (of, lf) = r["win"], r["full"]
+    S = o.S
+    keep = set(R.keep_set(S, cfg.n_sink, cfg.W))
+    far = [p for p in range(S) if p not in keep]
+    ofar, lfar = R.attention(wl.q[0, 0], o.Kfull[:, :S], o.Vfull[:, :S], keys=far)
+    mu = R.in_window_mass(lw, lf)
+    assert ((mu > 0) & (mu <= 1)).all() and (lw <= lf).all()
+    np.testing.assert_allclose(mu + np.exp(lfar - lf), 1.0, atol=1e-13)            # Z_win/Z + Z_far/Z = 1
+    np.testing.assert_allclose(of, mu[:, None] * ow + (1 - mu)[:, None] * ofar, atol=1e-13)
+    # head 0 of the full read-out is pulled to the needle's value row; the windowed one is not
+    needle_v = F64(V0[0, 100])
+    assert mu[0] < 1e-3
+    assert np.abs(of[0] - needle_v).max() < 1e-2
+    assert np.abs(ow[0] - needle_v).max() > 0.5
+    assert R.win_perturb(of, ow)[0] > 0.5
