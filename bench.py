@@ -1,0 +1,352 @@
+#!/usr/bin/env python
+"""Benchmark of the draft-attention hot path (windowed ring + full-context), one JSON line on stdout.
+
+A *step* is one pass of the whole path over one batch of synthetic input: a gamma-step windowed draft
+loop (ring append -> windowed attention) followed by a gamma-step full-context draft loop (KV append ->
+full attention) on the same q / k_new / v_new. `value` is the mean time per draft-attention step of that
+pass in microseconds (2*gamma draft-attention steps per pass); the `variants` object splits it into the
+windowed and the full-context figure with their achieved bytes/s.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload million]
+
+N > 1 (under torchrun) runs N independent replicas: the path has no cross-GPU exchange.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "us_per_draft_attention_step"
+UNIT = "us"
+WORKLOADS = {"tiny": 0, "s128k": 1, "million": 2, "batched": 3, "sweep": 4}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (full-context partial
+# kernel), from the ncu capture summarised under profiles/; keyed by workload. None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, STREAM-style copy)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.proc, self.gpu_id = None, gpu_id
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def pick_config(name: str, steps_total: int):
+    import wmtp_inputs as wi
+    cfg = wi.CONFIGS[WORKLOADS[name]]
+    return cfg
+
+
+def oracle_sample(wl, n_threads_hint=None):
+    """Times the CPU oracle, as it stands, on one windowed and one full-context draft step (sequence 0)."""
+    from oracle import reference as R
+    cfg = wl.cfg
+    S = int(wl.seq_lens[0])
+    K0, V0 = wl.K[0], wl.V[0]
+    q = wl.q[0, 0]
+    keep = R.keep_set(S, cfg.n_sink, cfg.W)
+    t0 = time.perf_counter()
+    R.attention(q, K0, V0, keys=keep)
+    t_win = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    R.attention(q, K0, V0)
+    t_full = time.perf_counter() - t0
+    return t_win, t_full, R.threads()
+
+
+def run_reference(args, rank):
+    """The reference arm: the CPU oracle timed on the host cores, same metric and workload."""
+    if rank != 0:
+        return
+    import wmtp_inputs as wi
+    from oracle import reference as R
+    R.build()
+    cfg = pick_config(args.workload, 0)
+    wl = wi.make_workload(cfg, poison_unused=False)
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_sample(wl)
+    tw, tf = [], []
+    for _ in range(args.steps):
+        a, b, thr = oracle_sample(wl)
+        tw.append(a); tf.append(b)
+    per_step_us = (statistics.mean(tw) + statistics.mean(tf)) / 2 * 1e6
+    sample = (f"per bench step: 1 windowed + 1 full-context draft-attention step of sequence 0, all {cfg.Hq} query heads "
+              f"(of the {2 * cfg.gamma * cfg.batch} per pass)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": per_step_us, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": (statistics.mean(tw) + statistics.mean(tf)) * 1e3,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": config_dict(cfg, args),
+        "variants": {"windowed": {"us_per_step": statistics.mean(tw) * 1e6}, "full": {"us_per_step": statistics.mean(tf) * 1e6}},
+        "cpu_baseline": {"value": per_step_us, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": sample},
+        "e2e": {"value": per_step_us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def config_dict(cfg, args):
+    return {
+        "workload": f"{cfg.name}: batch {cfg.batch}, S={'log-uniform ' + str(cfg.S0_range) if cfg.S0_range else cfg.S0}, "
+                    f"Hq={cfg.Hq}, Hkv={cfg.Hkv}, head_dim={cfg.D}, W={cfg.W}, sink={cfg.n_sink}, gamma={cfg.gamma}, "
+                    f"{'paged(64)' if cfg.paged else 'contiguous'} bf16 KV",
+        "step": "gamma windowed draft steps (ring append + attention) + gamma full-context draft steps (KV append + attention)",
+        "draft_steps_per_pass": 2 * cfg.gamma,
+        "l2": "inputs larger than L2: every full-context draft step streams the whole KV "
+              f"({cfg.kv_bytes_per_token * (cfg.S0 or 0) / 2**20:.0f} MiB at batch 1) between windowed loops",
+        "parallelism": f"replicas x{args.gpus} (no cross-GPU exchange)" if args.gpus > 1 else "single GPU",
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="million", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2607_21535_b200 as wm
+    import wmtp_inputs as wi
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    wm.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = pick_config(args.workload, 0)
+    gam, B = cfg.gamma, cfg.batch
+    total_passes = args.warmup + 3 * args.steps + 8          # timed + breakdown + e2e passes, plus slack
+    t0 = time.perf_counter()
+    wl = wi.make_workload(cfg, poison_unused=False, extra_cap=gam * total_passes + 64)
+    log(f"[bench] generated {cfg.name} in {time.perf_counter() - t0:.1f}s")
+
+    bf = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(dev).view(torch.bfloat16)
+    K, V = bf(wl.K_dev), bf(wl.V_dev)
+    lens = torch.from_numpy(wl.seq_lens.copy()).to(dev)
+    pt = torch.from_numpy(wl.page_table).to(dev) if cfg.paged else None
+    kv = wm.KV(K, V, lens, page_table=pt)
+    ring = wm.Ring(B, cfg.Hkv, cfg.D, cfg.n_sink, cfg.W, device=dev)
+    ws = wm.Workspace(B, cfg.Hq, cfg.Hkv, cfg.D, device=dev)
+    q, kn, vn = bf(wl.q), bf(wl.k_new), bf(wl.v_new)
+    out_w, out_f = torch.empty_like(q), torch.empty_like(q)
+    wm.wmtp_ring_init_from_kv(ring, kv)
+    torch.cuda.synchronize()
+
+    def one_pass():
+        wm.wmtp_draft_loop_windowed(ring, q, kn, vn, out_w, ws)
+        wm.wmtp_draft_loop_full(kv, q, kn, vn, out_f, ws)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_pass()
+    barrier()
+
+    # ---- the timed region: exactly K passes, CUDA events on the launching stream
+    props = torch.cuda.get_device_properties(dev)
+    gpu_id = f"GPU-{props.uuid}" if hasattr(props, "uuid") else str(local_rank)
+    sampler = ClockSampler(gpu_id)
+    if rank == 0:
+        sampler.start()
+    launches0 = wm.wmtp_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        one_pass()
+    e1.record()
+    barrier()
+    launches = wm.wmtp_launch_count() - launches0
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = ms_per_step * 1e3 / (2 * gam) / world          # replicas: N times the draft steps in the same time
+
+    # ---- breakdown pass (outside the headline region): windowed loop and full loop timed separately
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    for k in range(args.steps):
+        ev[k][0].record()
+        wm.wmtp_draft_loop_windowed(ring, q, kn, vn, out_w, ws)
+        ev[k][1].record()
+        wm.wmtp_draft_loop_full(kv, q, kn, vn, out_f, ws)
+        ev[k][2].record()
+    torch.cuda.synchronize()
+    us_win = statistics.mean(ev[k][0].elapsed_time(ev[k][1]) for k in range(args.steps)) * 1e3 / gam
+    us_full = statistics.mean(ev[k][1].elapsed_time(ev[k][2]) for k in range(args.steps)) * 1e3 / gam
+
+    # ---- the dominant kernel alone: full-context attention call (partial + combine), events around each launch
+    reps = max(10, args.steps)
+    o1 = torch.empty((B, cfg.Hq, cfg.D), dtype=torch.bfloat16, device=dev)
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    wev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, b in kev:
+        a.record(); wm.wmtp_draft_attn_full(q[0], kv, o1, ws); b.record()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    for a, b in wev:
+        flush.fill_(1)                                      # cold L2 for the windowed call
+        a.record(); wm.wmtp_draft_attn_windowed(q[0], ring, o1, ws); b.record()
+    torch.cuda.synchronize()
+    wm.wmtp_device_status(ws)
+    us_full_call = statistics.mean(a.elapsed_time(b) for a, b in kev) * 1e3
+    us_win_call_cold = statistics.mean(a.elapsed_time(b) for a, b in wev) * 1e3
+    cur_lens = lens.cpu().numpy()
+    full_bytes = float(cur_lens.sum()) * cfg.kv_bytes_per_token
+    win_bytes = float(np.minimum(cur_lens, cfg.n_sink + cfg.W).sum()) * cfg.kv_bytes_per_token
+    peak, peak_src = measured_peaks()
+    achieved = full_bytes / (us_full_call * 1e-6) / 1e9
+
+    # ---- end to end through the host-buffer entry points (pinned host memory, copies inside the timed region)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16).pin_memory()
+    qh, kh, vh = pin(wl.q), pin(wl.k_new), pin(wl.v_new)
+    oh_w, oh_f = torch.empty_like(qh).pin_memory(), torch.empty_like(qh).pin_memory()
+    stage = torch.empty(wm.wmtp_stage_bytes(gam, B, cfg.Hq, cfg.Hkv, cfg.D), dtype=torch.uint8, device=dev)
+
+    def one_pass_host():
+        wm.wmtp_draft_loop_windowed_host(ring, qh, kh, vh, oh_w, stage, ws)
+        wm.wmtp_draft_loop_full_host(kv, qh, kh, vh, oh_f, stage, ws)
+
+    one_pass_host()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one_pass_host()
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = e2e_s / args.steps * 1e6 / (2 * gam) / world
+    h2d = 2 * (qh.numel() + kh.numel() + vh.numel()) * 2
+    d2h = 2 * oh_w.numel() * 2
+    wm.wmtp_device_status(ws)
+
+    if rank == 0:
+        cpu = None
+        if not args.no_cpu_baseline and world == 1:
+            t_win, t_full, thr = oracle_sample(wl)
+            cpu = {"value": (t_win + t_full) / 2 * 1e6, "unit": UNIT, "cores": thr, "kind": "oracle",
+                   "sample": f"1 windowed ({t_win * 1e3:.1f} ms) + 1 full-context ({t_full * 1e3:.1f} ms) draft-attention step "
+                             f"of sequence 0, all {cfg.Hq} query heads, host has {os.cpu_count()} logical cores"}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": config_dict(cfg, args),
+            "variants": {
+                "windowed": {"us_per_step": us_win, "kv_bytes_per_step": win_bytes,
+                             "algorithmic_gbs": win_bytes / (us_win * 1e-6) / 1e9,
+                             "pct_of_8tbs": win_bytes / (us_win * 1e-6) / 8e12 * 100,
+                             "us_per_call_cold_l2": us_win_call_cold},
+                "full": {"us_per_step": us_full, "kv_bytes_per_step": full_bytes,
+                         "algorithmic_gbs": full_bytes / (us_full * 1e-6) / 1e9,
+                         "pct_of_8tbs": full_bytes / (us_full * 1e-6) / 8e12 * 100,
+                         "us_per_attention_call": us_full_call},
+            },
+            "roofline": {"bound": "hbm", "kernel": "full-context draft attention (split-KV partial + combine)",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_source": peak_src, "pct_of_8tbs": achieved / 8000 * 100,
+                         "traffic": NCU_TRAFFIC_BYTES.get(args.workload)},
+            "cpu_baseline": cpu,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches,
+            "clocks": clocks,
+            "paper_context": "paper reports +28% to +44% per-decode-step gain of windowed over native MTP on one B200 "
+                             "(SGLang, NVFP4 weights, bf16 KV, 1.04M-token prompt, d=7); not the same metric",
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

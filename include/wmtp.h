@@ -1,0 +1,178 @@
+/*
+ * wmtp.h -- C ABI of the Windowed-MTP draft-attention library (single GPU, sm_100a).
+ *
+ * The library implements the draft head's GQA decode attention over its KV cache in the two
+ * forms the paper compares: windowed (attention sink + the last W tokens, kept in a compact
+ * ring buffer; Section 4 "Mechanism" and "Memory", Appendix A pseudocode) and full context
+ * (the native-MTP draft that re-reads all S keys at every draft step; Section 3).
+ *
+ * Conventions for every call
+ *  - Pointers marked "device" are CUDA device memory owned by the caller; the library
+ *    allocates nothing on the device and keeps no reference after the call's work has run.
+ *    Descriptors (wmtp_ring, wmtp_kv) are plain host structs, read during the call only.
+ *  - bf16 tensors are row-major with head_dim D contiguous; base pointers 16-byte aligned.
+ *  - `stream` is a cudaStream_t passed as void*. Calls only enqueue work on it; nothing
+ *    synchronises except wmtp_device_status and the *_host loop variants.
+ *  - Sequence lengths live in device memory (`len`), are advanced by the append kernels and
+ *    read by the attention kernels, so a chain of calls needs no host round trip.
+ *  - Return value: WMTP_OK or an error; nothing is launched when an argument is rejected.
+ *    wmtp_last_error() gives a thread-local detail string. Problems only visible on the
+ *    device (a page id out of range, an append past capacity, a bounded wait that expired)
+ *    set a sticky word in the workspace, the kernel skips the offending access, and
+ *    wmtp_device_status reports it.
+ *  - Query head h reads KV head h / (Hq / Hkv). Supported: D in {128, 256}, Hq / Hkv in [1, 8].
+ *  - sm_scale <= 0 selects 1 / sqrt(D).
+ */
+#ifndef WMTP_H_
+#define WMTP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    WMTP_OK = 0,
+    WMTP_ERR_INVALID_ARG = 1,    /* NULL / misaligned pointer, non-positive size, Hq % Hkv != 0, cap < W ... */
+    WMTP_ERR_UNSUPPORTED = 2,    /* head_dim or group size the kernels are not built for */
+    WMTP_ERR_CAPACITY = 3,       /* a length would exceed the ring / KV capacity */
+    WMTP_ERR_WORKSPACE = 4,      /* workspace missing, misaligned or too small */
+    WMTP_ERR_CUDA = 5,           /* a CUDA runtime / driver call failed (no device, launch error) */
+    WMTP_ERR_DEVICE_TIMEOUT = 6, /* a bounded device-side wait expired; outputs of that call are invalid */
+    WMTP_ERR_DEVICE_BOUNDS = 7   /* a device-side index check failed (page id, append past capacity) */
+} wmtp_status;
+
+/*
+ * Ring-buffer draft KV store (Section 4 "Memory": the draft KV is kept in a compact
+ * n_sink + W + d ring; Appendix A: slot = ring_base(r) + logical position under a modulus).
+ * Per sequence r the store has n_sink fixed sink slots followed by `cap` window slots used
+ * circularly: position p lives in slot p if p < n_sink, else n_sink + ((p - n_sink) mod cap).
+ * cap == W is the plain window; cap = W + d reserves the paper's d slots of slack. The draft
+ * attends over the sink slots and the slots holding the last W positions.
+ */
+typedef struct wmtp_ring {
+    void*    k;         /* device bf16 [batch][Hkv][n_sink + cap][D] */
+    void*    v;         /* device bf16 [batch][Hkv][n_sink + cap][D] */
+    int32_t* slot_pos;  /* device [batch][n_sink + cap]: logical position held by each slot, -1 = never written */
+    int64_t* len;       /* device [batch]: logical sequence length S (tokens appended so far) */
+    int32_t  batch, Hkv, D, n_sink, W, cap;
+} wmtp_ring;
+
+/*
+ * Full-context draft KV (the native draft's cache, Section 3).
+ * Contiguous layout (page_table == NULL): bf16 [batch][Hkv][S_cap][D].
+ * Paged layout: pool bf16 [num_pages][Hkv][page_size][D]; token p of sequence r lives in page
+ * page_table[r][p / page_size] at row p % page_size. page_size must be 64.
+ */
+typedef struct wmtp_kv {
+    void*          k;
+    void*          v;
+    const int32_t* page_table; /* device [batch][max_pages], or NULL */
+    int64_t*       len;        /* device [batch] */
+    int64_t        S_cap;      /* host-known capacity in tokens per sequence (contiguous: row count; paged: max_pages * page_size) */
+    int32_t        batch, Hkv, D, page_size, max_pages, num_pages;
+} wmtp_kv;
+
+const char* wmtp_status_string(wmtp_status s); /* static storage */
+const char* wmtp_last_error(void);             /* thread-local, valid until the thread's next failing call */
+
+/* Bytes of the ring's K (== V) tensor and of slot_pos, for the caller's allocation. Returns k_bytes. */
+size_t wmtp_ring_bytes(int batch, int Hkv, int D, int n_sink, int cap, size_t* pos_bytes);
+
+/*
+ * Workspace for the attention calls: split-KV partial results, their completion counters and
+ * the sticky device status word. Size depends only on (batch, Hq, Hkv, D). The workspace must be
+ * 256-byte aligned and initialised once with wmtp_workspace_init before its first use; after that
+ * the kernels leave it ready for the next call. Calls sharing one workspace must be ordered on
+ * one stream.
+ */
+size_t      wmtp_workspace_bytes(int batch, int Hq, int Hkv, int D);
+wmtp_status wmtp_workspace_init(void* workspace, size_t ws_bytes, void* stream);
+
+/* Synchronises `stream`, then returns (and clears) the sticky device status of the workspace. */
+wmtp_status wmtp_device_status(void* workspace, void* stream);
+
+/* ---- ring store -------------------------------------------------------------------------- */
+
+/* len = 0, every slot_pos = -1 (K/V bytes are left as they are). */
+wmtp_status wmtp_ring_reset(const wmtp_ring* ring, void* stream);
+
+/*
+ * Seeds the ring from a context KV holding S = kv->len[r] tokens per sequence: copies positions
+ * [0, min(S, n_sink)) and [max(n_sink, S - cap), S) into their slots, sets slot_pos and len = S.
+ * The result is bit-identical to S sequential wmtp_ring_append calls (Section 6, "Prefill
+ * sparsification": only O(W + n_sink) of the context is needed by the windowed draft).
+ */
+wmtp_status wmtp_ring_init_from_kv(const wmtp_ring* ring, const wmtp_kv* kv, void* stream);
+
+/*
+ * Appends one token per sequence (Appendix A, RING): p = len[r]; the K/V rows k_new, v_new
+ * (device bf16 [batch][Hkv][D]) go to the slot of position p, slot_pos[slot] = p, len[r] = p + 1.
+ */
+wmtp_status wmtp_ring_append(const wmtp_ring* ring, const void* k_new, const void* v_new, void* stream);
+
+/* Same for the full-context KV: writes position p = len[r] (through the page table if paged), len[r] = p + 1.
+ * A position beyond S_cap, or a page id outside [0, num_pages), is skipped and flagged in `workspace` (may be NULL). */
+wmtp_status wmtp_kv_append(const wmtp_kv* kv, const void* k_new, const void* v_new, void* workspace, void* stream);
+
+/* ---- draft attention --------------------------------------------------------------------- */
+
+/*
+ * Windowed draft attention (Section 4 "Mechanism"; Appendix A): for each sequence, one query
+ * per head attends over the first n_sink tokens and the last W tokens, read from the ring
+ * (all of it when S <= n_sink + W). q: device bf16 [batch][Hq][D]; out: device bf16
+ * [batch][Hq][D]; lse: device fp32 [batch][Hq] (natural-log sum of exp of the scaled logits)
+ * or NULL. Softmax in fp32; split-KV partials are merged by log-sum-exp.
+ * A sequence of length 0 yields out = 0, lse = -inf.
+ */
+wmtp_status wmtp_draft_attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm_scale,
+                                     void* out, float* lse, void* workspace, size_t ws_bytes, void* stream);
+
+/* Full-context draft attention (Section 3: the native draft re-reads all S keys): same, over positions [0, len[r]). */
+wmtp_status wmtp_draft_attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale,
+                                 void* out, float* lse, void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * gamma sequential draft steps on one stream (Section 3, Eq. 1: gamma draft forwards per decode
+ * step): for i in [0, gamma): append(k_new[i], v_new[i]) then attention(q[i]) -> out[i].
+ * q: device bf16 [gamma][batch][Hq][D]; k_new, v_new: device bf16 [gamma][batch][Hkv][D];
+ * out: device bf16 [gamma][batch][Hq][D]; lse: device fp32 [gamma][batch][Hq] or NULL.
+ */
+wmtp_status wmtp_draft_loop_windowed(const wmtp_ring* ring, int gamma, const void* q, int Hq,
+                                     const void* k_new, const void* v_new, float sm_scale,
+                                     void* out, float* lse, void* workspace, size_t ws_bytes, void* stream);
+wmtp_status wmtp_draft_loop_full(const wmtp_kv* kv, int gamma, const void* q, int Hq,
+                                 const void* k_new, const void* v_new, float sm_scale,
+                                 void* out, float* lse, void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * The same loops for a caller whose step inputs and outputs live in HOST memory (pinned memory
+ * makes the copies asynchronous): q, k_new, v_new are copied to the device staging buffer
+ * `stage` (device, at least wmtp_stage_bytes, 256-byte aligned), the loop runs, `out` (and `lse`
+ * if not NULL) are copied back to the host pointers, and the stream is synchronised before
+ * returning. The KV cache / ring stay device-resident: they are state, not step inputs.
+ */
+size_t      wmtp_stage_bytes(int gamma, int batch, int Hq, int Hkv, int D);
+wmtp_status wmtp_draft_loop_windowed_host(const wmtp_ring* ring, int gamma, const void* q_host, int Hq,
+                                          const void* k_new_host, const void* v_new_host, float sm_scale,
+                                          void* out_host, float* lse_host, void* stage,
+                                          void* workspace, size_t ws_bytes, void* stream);
+wmtp_status wmtp_draft_loop_full_host(const wmtp_kv* kv, int gamma, const void* q_host, int Hq,
+                                      const void* k_new_host, const void* v_new_host, float sm_scale,
+                                      void* out_host, float* lse_host, void* stage,
+                                      void* workspace, size_t ws_bytes, void* stream);
+
+/* ---- tuning and accounting ---------------------------------------------------------------- */
+
+/* Upper bound on the CTAs (KV splits) of the attention kernels; 0 restores the default
+ * (one CTA per SM). Process-wide; meant for tests that exercise the split/merge path. */
+void    wmtp_set_max_ctas(int max_ctas);
+/* Number of kernels this library has launched in this process (all threads). */
+int64_t wmtp_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WMTP_H_ */

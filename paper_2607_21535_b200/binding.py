@@ -1,0 +1,260 @@
+"""ctypes binding of libwmtp.so: same names as the C ABI, argument marshalling only.
+
+torch is used for device memory and streams; every step of the path runs in the
+library's kernels. There is no fallback: a missing or unloadable library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, byref, c_char_p, c_float, c_int, c_int32, c_int64, c_size_t, c_void_p
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libwmtp.so")
+
+WMTP_OK = 0
+STATUS_NAMES = {
+    0: "WMTP_OK", 1: "WMTP_ERR_INVALID_ARG", 2: "WMTP_ERR_UNSUPPORTED", 3: "WMTP_ERR_CAPACITY",
+    4: "WMTP_ERR_WORKSPACE", 5: "WMTP_ERR_CUDA", 6: "WMTP_ERR_DEVICE_TIMEOUT", 7: "WMTP_ERR_DEVICE_BOUNDS",
+}
+
+
+class wmtp_ring(ctypes.Structure):
+    _fields_ = [("k", c_void_p), ("v", c_void_p), ("slot_pos", c_void_p), ("len", c_void_p),
+                ("batch", c_int32), ("Hkv", c_int32), ("D", c_int32), ("n_sink", c_int32), ("W", c_int32),
+                ("cap", c_int32)]
+
+
+class wmtp_kv(ctypes.Structure):
+    _fields_ = [("k", c_void_p), ("v", c_void_p), ("page_table", c_void_p), ("len", c_void_p),
+                ("S_cap", c_int64), ("batch", c_int32), ("Hkv", c_int32), ("D", c_int32), ("page_size", c_int32),
+                ("max_pages", c_int32), ("num_pages", c_int32)]
+
+
+class WmtpError(RuntimeError):
+    def __init__(self, status: int, detail: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {detail}")
+        self.status = status
+
+
+# Every symbol include/wmtp.h declares, with its ctypes signature.
+_SIGNATURES = {
+    "wmtp_status_string": (c_char_p, [c_int]),
+    "wmtp_last_error": (c_char_p, []),
+    "wmtp_ring_bytes": (c_size_t, [c_int, c_int, c_int, c_int, c_int, POINTER(c_size_t)]),
+    "wmtp_workspace_bytes": (c_size_t, [c_int, c_int, c_int, c_int]),
+    "wmtp_workspace_init": (c_int, [c_void_p, c_size_t, c_void_p]),
+    "wmtp_device_status": (c_int, [c_void_p, c_void_p]),
+    "wmtp_ring_reset": (c_int, [POINTER(wmtp_ring), c_void_p]),
+    "wmtp_ring_init_from_kv": (c_int, [POINTER(wmtp_ring), POINTER(wmtp_kv), c_void_p]),
+    "wmtp_ring_append": (c_int, [POINTER(wmtp_ring), c_void_p, c_void_p, c_void_p]),
+    "wmtp_kv_append": (c_int, [POINTER(wmtp_kv), c_void_p, c_void_p, c_void_p, c_void_p]),
+    "wmtp_draft_attn_windowed": (c_int, [c_void_p, c_int, POINTER(wmtp_ring), c_float, c_void_p, c_void_p, c_void_p,
+                                         c_size_t, c_void_p]),
+    "wmtp_draft_attn_full": (c_int, [c_void_p, c_int, POINTER(wmtp_kv), c_float, c_void_p, c_void_p, c_void_p, c_size_t,
+                                     c_void_p]),
+    "wmtp_draft_loop_windowed": (c_int, [POINTER(wmtp_ring), c_int, c_void_p, c_int, c_void_p, c_void_p, c_float,
+                                         c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "wmtp_draft_loop_full": (c_int, [POINTER(wmtp_kv), c_int, c_void_p, c_int, c_void_p, c_void_p, c_float, c_void_p,
+                                     c_void_p, c_void_p, c_size_t, c_void_p]),
+    "wmtp_stage_bytes": (c_size_t, [c_int, c_int, c_int, c_int, c_int]),
+    "wmtp_draft_loop_windowed_host": (c_int, [POINTER(wmtp_ring), c_int, c_void_p, c_int, c_void_p, c_void_p, c_float,
+                                              c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "wmtp_draft_loop_full_host": (c_int, [POINTER(wmtp_kv), c_int, c_void_p, c_int, c_void_p, c_void_p, c_float,
+                                          c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "wmtp_set_max_ctas": (None, [c_int]),
+    "wmtp_launch_count": (c_int64, []),
+}
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libwmtp.so (built in-tree by ``build.py``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2607_21535_b200.build` "
+                              "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def _check(status: int) -> None:
+    if status != WMTP_OK:
+        raise WmtpError(status, lib().wmtp_last_error().decode())
+
+
+def _ptr(t) -> int | None:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+# ------------------------------------------------------------------------------------------------
+# Device-memory holders (torch allocations + the C descriptor)
+# ------------------------------------------------------------------------------------------------
+class Ring:
+    """Device ring-buffer KV store for ``batch`` sequences: n_sink sink slots + ``cap`` window slots."""
+
+    def __init__(self, batch, Hkv, D, n_sink, W, cap=None, device="cuda", guard: int = 0):
+        cap = W if cap is None else cap
+        self.batch, self.Hkv, self.D, self.n_sink, self.W, self.cap = batch, Hkv, D, n_sink, W, cap
+        slots = n_sink + cap
+        self.k = torch.zeros((batch, Hkv, slots, D), dtype=torch.bfloat16, device=device)
+        self.v = torch.zeros((batch, Hkv, slots, D), dtype=torch.bfloat16, device=device)
+        self.slot_pos = torch.full((batch, slots), -1, dtype=torch.int32, device=device)
+        self.len = torch.zeros((batch,), dtype=torch.int64, device=device)
+        self.desc = wmtp_ring(self.k.data_ptr(), self.v.data_ptr(), self.slot_pos.data_ptr(), self.len.data_ptr(),
+                              batch, Hkv, D, n_sink, W, cap)
+
+
+class KV:
+    """Full-context KV descriptor over caller-provided device tensors.
+
+    Contiguous: k, v bf16 [batch][Hkv][S_cap][D]. Paged: k, v bf16 [num_pages][Hkv][page_size][D]
+    with ``page_table`` int32 [batch][max_pages].
+    """
+
+    def __init__(self, k, v, lens, page_table=None, S_cap=None):
+        self.k, self.v, self.len, self.page_table = k, v, lens, page_table
+        if page_table is None:
+            batch, Hkv, rows, D = k.shape
+            self.S_cap = rows if S_cap is None else S_cap
+            page_size = max_pages = num_pages = 0
+        else:
+            num_pages, Hkv, page_size, D = k.shape
+            batch, max_pages = page_table.shape
+            self.S_cap = max_pages * page_size if S_cap is None else S_cap
+        self.batch, self.Hkv, self.D = batch, Hkv, D
+        self.desc = wmtp_kv(k.data_ptr(), v.data_ptr(), _ptr(page_table), lens.data_ptr(), self.S_cap, batch, Hkv, D,
+                            page_size, max_pages, num_pages)
+
+
+class Workspace:
+    def __init__(self, batch, Hq, Hkv, D, device="cuda", stream=None):
+        self.nbytes = int(lib().wmtp_workspace_bytes(batch, Hq, Hkv, D))
+        self.buf = torch.empty((self.nbytes,), dtype=torch.uint8, device=device)
+        assert self.buf.data_ptr() % 256 == 0
+        wmtp_workspace_init(self, stream=stream)
+
+    @property
+    def ptr(self) -> int:
+        return self.buf.data_ptr()
+
+
+# ------------------------------------------------------------------------------------------------
+# The C ABI, same names
+# ------------------------------------------------------------------------------------------------
+def wmtp_status_string(status: int) -> str:
+    return lib().wmtp_status_string(status).decode()
+
+
+def wmtp_last_error() -> str:
+    return lib().wmtp_last_error().decode()
+
+
+def wmtp_ring_bytes(batch, Hkv, D, n_sink, cap):
+    pos = c_size_t(0)
+    kb = lib().wmtp_ring_bytes(batch, Hkv, D, n_sink, cap, byref(pos))
+    return int(kb), int(pos.value)
+
+
+def wmtp_workspace_bytes(batch, Hq, Hkv, D) -> int:
+    return int(lib().wmtp_workspace_bytes(batch, Hq, Hkv, D))
+
+
+def wmtp_workspace_init(ws: Workspace, stream=None) -> None:
+    _check(lib().wmtp_workspace_init(ws.ptr, ws.nbytes, _stream(stream)))
+
+
+def wmtp_device_status(ws: Workspace, stream=None) -> None:
+    _check(lib().wmtp_device_status(ws.ptr, _stream(stream)))
+
+
+def wmtp_ring_reset(ring: Ring, stream=None) -> None:
+    _check(lib().wmtp_ring_reset(byref(ring.desc), _stream(stream)))
+
+
+def wmtp_ring_init_from_kv(ring: Ring, kv: KV, stream=None) -> None:
+    _check(lib().wmtp_ring_init_from_kv(byref(ring.desc), byref(kv.desc), _stream(stream)))
+
+
+def wmtp_ring_append(ring: Ring, k_new, v_new, stream=None) -> None:
+    _check(lib().wmtp_ring_append(byref(ring.desc), _ptr(k_new), _ptr(v_new), _stream(stream)))
+
+
+def wmtp_kv_append(kv: KV, k_new, v_new, ws: Workspace | None = None, stream=None) -> None:
+    _check(lib().wmtp_kv_append(byref(kv.desc), _ptr(k_new), _ptr(v_new), ws.ptr if ws is not None else None,
+                                _stream(stream)))
+
+
+def wmtp_draft_attn_windowed(q, ring: Ring, out, ws: Workspace, lse=None, sm_scale: float = 0.0, stream=None) -> None:
+    Hq = q.shape[-2]
+    _check(lib().wmtp_draft_attn_windowed(_ptr(q), Hq, byref(ring.desc), sm_scale, _ptr(out), _ptr(lse), ws.ptr,
+                                          ws.nbytes, _stream(stream)))
+
+
+def wmtp_draft_attn_full(q, kv: KV, out, ws: Workspace, lse=None, sm_scale: float = 0.0, stream=None) -> None:
+    Hq = q.shape[-2]
+    _check(lib().wmtp_draft_attn_full(_ptr(q), Hq, byref(kv.desc), sm_scale, _ptr(out), _ptr(lse), ws.ptr, ws.nbytes,
+                                      _stream(stream)))
+
+
+def wmtp_draft_loop_windowed(ring: Ring, q, k_new, v_new, out, ws: Workspace, lse=None, sm_scale: float = 0.0,
+                             stream=None) -> None:
+    gamma, Hq = q.shape[0], q.shape[-2]
+    _check(lib().wmtp_draft_loop_windowed(byref(ring.desc), gamma, _ptr(q), Hq, _ptr(k_new), _ptr(v_new), sm_scale,
+                                          _ptr(out), _ptr(lse), ws.ptr, ws.nbytes, _stream(stream)))
+
+
+def wmtp_draft_loop_full(kv: KV, q, k_new, v_new, out, ws: Workspace, lse=None, sm_scale: float = 0.0,
+                         stream=None) -> None:
+    gamma, Hq = q.shape[0], q.shape[-2]
+    _check(lib().wmtp_draft_loop_full(byref(kv.desc), gamma, _ptr(q), Hq, _ptr(k_new), _ptr(v_new), sm_scale, _ptr(out),
+                                      _ptr(lse), ws.ptr, ws.nbytes, _stream(stream)))
+
+
+def wmtp_stage_bytes(gamma, batch, Hq, Hkv, D) -> int:
+    return int(lib().wmtp_stage_bytes(gamma, batch, Hq, Hkv, D))
+
+
+def wmtp_draft_loop_windowed_host(ring: Ring, q_host, k_new_host, v_new_host, out_host, stage, ws: Workspace,
+                                  lse_host=None, sm_scale: float = 0.0, stream=None) -> None:
+    """Host tensors in, host tensors out (CPU torch tensors, ideally pinned); ``stage`` is a device byte buffer."""
+    gamma, Hq = q_host.shape[0], q_host.shape[-2]
+    _check(lib().wmtp_draft_loop_windowed_host(byref(ring.desc), gamma, _ptr(q_host), Hq, _ptr(k_new_host),
+                                               _ptr(v_new_host), sm_scale, _ptr(out_host), _ptr(lse_host), _ptr(stage),
+                                               ws.ptr, ws.nbytes, _stream(stream)))
+
+
+def wmtp_draft_loop_full_host(kv: KV, q_host, k_new_host, v_new_host, out_host, stage, ws: Workspace, lse_host=None,
+                              sm_scale: float = 0.0, stream=None) -> None:
+    gamma, Hq = q_host.shape[0], q_host.shape[-2]
+    _check(lib().wmtp_draft_loop_full_host(byref(kv.desc), gamma, _ptr(q_host), Hq, _ptr(k_new_host), _ptr(v_new_host),
+                                           sm_scale, _ptr(out_host), _ptr(lse_host), _ptr(stage), ws.ptr, ws.nbytes,
+                                           _stream(stream)))
+
+
+def wmtp_set_max_ctas(n: int) -> None:
+    lib().wmtp_set_max_ctas(int(n))
+
+
+def wmtp_launch_count() -> int:
+    return int(lib().wmtp_launch_count())

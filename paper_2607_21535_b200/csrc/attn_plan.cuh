@@ -1,0 +1,68 @@
+// Work decomposition shared by the split-KV partial kernel and the combine kernel.
+//
+// Every (sequence b, KV head g) pair is a *segment* of tiles_b = ceil(keys_b / kTileKeys) tiles;
+// segments are laid end to end on one line of n tiles in (b, g) order. CTA c of C owns the tile
+// range [c*n/C, (c+1)*n/C). A CTA emits one partial result per segment it touches; the partial of
+// (CTA c, segment s) is stored at index c + s, which is injective and makes the partials of one
+// segment contiguous. Everything is computed from the device-resident lengths in O(B) per CTA;
+// nothing is O(S) and nothing comes from the host.
+#pragma once
+
+#include "wmtp_internal.h"
+
+namespace wmtp {
+
+// Key slots the kernel scans for sequence b: the live part of the ring, or all S positions.
+__device__ __forceinline__ int64_t scan_keys(const AttnParams& p, int b) {
+    const int64_t S = p.len[b];
+    if (p.mode == kRing) {
+        const int64_t slots = (int64_t)p.n_sink + p.cap;
+        return S < slots ? S : slots;
+    }
+    return S;
+}
+
+// Is ring slot s (< scan_keys) inside sink + last-W? Always true when cap == W.
+__device__ __forceinline__ bool ring_slot_live(int s, int64_t S, int n_sink, int W, int cap) {
+    if (s < n_sink) return true;
+    const int64_t last = S - 1 - n_sink;
+    const int cur = (int)(last % cap);
+    int age = cur - (s - n_sink);
+    if (age < 0) age += cap;
+    return age < W;
+}
+
+// Fills tile_prefix[0..B] (exclusive prefix of per-sequence tile counts) in shared memory.
+// Must be called by all threads of the block; ends with a __syncthreads().
+__device__ __forceinline__ void build_tile_prefix(const AttnParams& p, int64_t* tile_prefix) {
+    for (int b = threadIdx.x; b < p.B; b += blockDim.x)
+        tile_prefix[b + 1] = (scan_keys(p, b) + kTileKeys - 1) / kTileKeys;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int64_t acc = 0;
+        tile_prefix[0] = 0;
+        for (int b = 0; b < p.B; ++b) { acc += tile_prefix[b + 1]; tile_prefix[b + 1] = acc; }
+    }
+    __syncthreads();
+}
+
+__device__ __forceinline__ int64_t cta_range_start(int c, int64_t n, int C) {
+    return ((int64_t)c * n) / C;   // c <= kMaxCtas and n < 2^40: no overflow
+}
+
+// CTA owning tile t: the largest c with cta_range_start(c) <= t.
+__device__ __forceinline__ int tile_owner(int64_t t, int64_t n, int C) {
+    return (int)(((t + 1) * (int64_t)C - 1) / n);
+}
+
+// Sequence whose segment group contains global tile t (Hkv segments per sequence).
+__device__ __forceinline__ int find_seq(const int64_t* tile_prefix, int B, int Hkv, int64_t t) {
+    int lo = 0, hi = B - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if ((int64_t)Hkv * tile_prefix[mid] <= t) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+}  // namespace wmtp

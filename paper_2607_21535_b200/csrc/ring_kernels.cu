@@ -1,0 +1,165 @@
+// Ring-buffer draft KV store and full-context KV append kernels.
+//
+// Slot rule (Section 4 "Memory"; Appendix A, RING comment, read with the sink kept fixed):
+// position p lives in slot p when p < n_sink, else in n_sink + ((p - n_sink) mod cap).
+// All of this is integer work and copies: results are bit-exact by construction.
+#include "wmtp_internal.h"
+
+namespace wmtp {
+
+namespace {
+
+constexpr int kErrBounds = WMTP_ERR_DEVICE_BOUNDS;
+
+__device__ __forceinline__ int ring_slot(int64_t p, int n_sink, int cap) {
+    return p < n_sink ? (int)p : n_sink + (int)((p - n_sink) % cap);
+}
+
+// Position held by window slot `s` (s >= n_sink) of a ring of logical length S, or -1.
+__device__ __forceinline__ int64_t ring_slot_position(int s, int64_t S, int n_sink, int cap) {
+    if (s < n_sink) return s < S ? (int64_t)s : -1;
+    if (S <= n_sink) return -1;
+    const int64_t last = S - 1 - n_sink;          // window-relative index of the newest token
+    const int cur = (int)(last % cap);
+    int age = cur - (s - n_sink);
+    if (age < 0) age += cap;
+    return (int64_t)age <= last ? S - 1 - age : -1;
+}
+
+__global__ void ring_reset_kernel(RingParams r) {
+    const int slots = r.n_sink + r.cap;
+    const int64_t n = (int64_t)r.B * slots;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        r.slot_pos[i] = -1;
+    if (blockIdx.x == 0)
+        for (int b = threadIdx.x; b < r.B; b += blockDim.x) r.len[b] = 0;
+}
+
+// One block per sequence; thread t moves 16 bytes of the token's [Hkv][D] K row and V row.
+__global__ void ring_append_kernel(RingParams r, const uint4* __restrict__ k_new, const uint4* __restrict__ v_new) {
+    const int b = blockIdx.x;
+    const int64_t p = r.len[b];
+    const int slots = r.n_sink + r.cap;
+    const int slot = ring_slot(p, r.n_sink, r.cap);
+    const int vec_per_row = r.D / 8;
+    const int n_vec = r.Hkv * vec_per_row;
+    uint4* K = reinterpret_cast<uint4*>(r.k);
+    uint4* V = reinterpret_cast<uint4*>(r.v);
+    for (int i = threadIdx.x; i < n_vec; i += blockDim.x) {
+        const int g = i / vec_per_row, c = i % vec_per_row;
+        const int64_t dst = (((int64_t)b * r.Hkv + g) * slots + slot) * vec_per_row + c;
+        const int64_t src = (int64_t)b * n_vec + i;
+        K[dst] = k_new[src];
+        V[dst] = v_new[src];
+    }
+    __syncthreads();   // every thread has read len[b] before it moves
+    if (threadIdx.x == 0) {
+        r.slot_pos[(int64_t)b * slots + slot] = (int32_t)p;
+        r.len[b] = p + 1;
+    }
+}
+
+__device__ __forceinline__ int64_t kv_row_vec(const KvParams& kv, int b, int g, int64_t p, int vec_per_row, bool* ok) {
+    if (kv.page_table == nullptr) return (((int64_t)b * kv.Hkv + g) * kv.S_cap + p) * vec_per_row;
+    const int page = kv.page_table[(int64_t)b * kv.max_pages + p / kv.page_size];
+    if (page < 0 || page >= kv.num_pages) { *ok = false; return 0; }
+    return (((int64_t)page * kv.Hkv + g) * kv.page_size + p % kv.page_size) * vec_per_row;
+}
+
+__global__ void kv_append_kernel(KvParams kv, const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, int* status) {
+    const int b = blockIdx.x;
+    const int64_t p = kv.len[b];
+    const int vec_per_row = kv.D / 8;
+    const int n_vec = kv.Hkv * vec_per_row;
+    __shared__ int bad;
+    if (threadIdx.x == 0) bad = 0;
+    __syncthreads();
+    if (p >= kv.S_cap) {
+        if (threadIdx.x == 0 && status) atomicCAS(status, 0, kErrBounds);
+        return;
+    }
+    uint4* K = reinterpret_cast<uint4*>(kv.k);
+    uint4* V = reinterpret_cast<uint4*>(kv.v);
+    for (int i = threadIdx.x; i < n_vec; i += blockDim.x) {
+        const int g = i / vec_per_row, c = i % vec_per_row;
+        bool ok = true;
+        const int64_t dst = kv_row_vec(kv, b, g, p, vec_per_row, &ok) + c;
+        if (!ok) { bad = 1; continue; }
+        const int64_t src = (int64_t)b * n_vec + i;
+        K[dst] = k_new[src];
+        V[dst] = v_new[src];
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (bad) { if (status) atomicCAS(status, 0, kErrBounds); }
+        else kv.len[b] = p + 1;
+    }
+}
+
+// grid (ceil(slots / slots_per_block), B); each warp copies whole slots.
+__global__ void ring_init_kernel(RingParams r, KvParams kv) {
+    const int b = blockIdx.y;
+    const int slots = r.n_sink + r.cap;
+    const int64_t S = kv.len[b];
+    const int vec_per_row = r.D / 8;
+    const int warps = blockDim.x / 32, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const uint4* Ksrc = reinterpret_cast<const uint4*>(kv.k);
+    const uint4* Vsrc = reinterpret_cast<const uint4*>(kv.v);
+    uint4* K = reinterpret_cast<uint4*>(r.k);
+    uint4* V = reinterpret_cast<uint4*>(r.v);
+    for (int s = blockIdx.x * warps + warp; s < slots; s += gridDim.x * warps) {
+        const int64_t p = ring_slot_position(s, S, r.n_sink, r.cap);
+        if (lane == 0) r.slot_pos[(int64_t)b * slots + s] = (int32_t)p;
+        if (p < 0) continue;
+        for (int g = 0; g < r.Hkv; ++g) {
+            bool ok = true;
+            const int64_t src = kv_row_vec(kv, b, g, p, vec_per_row, &ok);
+            if (!ok) continue;
+            const int64_t dst = (((int64_t)b * r.Hkv + g) * slots + s) * vec_per_row;
+            for (int c = lane; c < vec_per_row; c += 32) {
+                K[dst + c] = Ksrc[src + c];
+                V[dst + c] = Vsrc[src + c];
+            }
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) r.len[b] = S;
+}
+
+}  // namespace
+
+cudaError_t launch_ring_reset(const RingParams& r, cudaStream_t st) {
+    const int64_t n = (int64_t)r.B * (r.n_sink + r.cap);
+    const int blocks = (int)((n + 255) / 256 < 1 ? 1 : ((n + 255) / 256 > 1184 ? 1184 : (n + 255) / 256));
+    ring_reset_kernel<<<blocks, 256, 0, st>>>(r);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ring_append(const RingParams& r, const void* k_new, const void* v_new, cudaStream_t st) {
+    const int n_vec = r.Hkv * r.D / 8;
+    const int threads = n_vec < 32 ? 32 : (n_vec > 256 ? 256 : (n_vec + 31) / 32 * 32);
+    ring_append_kernel<<<r.B, threads, 0, st>>>(r, (const uint4*)k_new, (const uint4*)v_new);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_kv_append(const KvParams& kv, const void* k_new, const void* v_new, int* status, cudaStream_t st) {
+    const int n_vec = kv.Hkv * kv.D / 8;
+    const int threads = n_vec < 32 ? 32 : (n_vec > 256 ? 256 : (n_vec + 31) / 32 * 32);
+    kv_append_kernel<<<kv.B, threads, 0, st>>>(kv, (const uint4*)k_new, (const uint4*)v_new, status);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ring_init_from_kv(const RingParams& r, const KvParams& kv, cudaStream_t st) {
+    const int slots = r.n_sink + r.cap;
+    const int warps = 8;
+    int bx = (slots + warps - 1) / warps;
+    if (bx > 592) bx = 592;
+    dim3 grid(bx, r.B);
+    ring_init_kernel<<<grid, warps * 32, 0, st>>>(r, kv);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+}  // namespace wmtp

@@ -1,0 +1,390 @@
+// C ABI of the library: argument validation, workspace layout, launches. No device allocation.
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "wmtp_internal.h"
+
+namespace wmtp {
+
+namespace {
+thread_local char g_err[512] = "";
+std::atomic<int64_t> g_launches{0};
+std::atomic<int> g_max_ctas{0};
+
+wmtp_status fail(wmtp_status s, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return s;
+}
+
+wmtp_status cuda_fail(cudaError_t e, const char* what) {
+    return fail(WMTP_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+wmtp_status check_shape(int batch, int Hkv, int D) {
+    if (batch < 1 || Hkv < 1) return fail(WMTP_ERR_INVALID_ARG, "batch=%d, Hkv=%d must be positive", batch, Hkv);
+    if (batch > kMaxBatch) return fail(WMTP_ERR_UNSUPPORTED, "batch=%d exceeds %d", batch, kMaxBatch);
+    if (D != 128 && D != 256) return fail(WMTP_ERR_UNSUPPORTED, "head_dim=%d (supported: 128, 256)", D);
+    return WMTP_OK;
+}
+
+wmtp_status check_ring(const wmtp_ring* r) {
+    if (!r) return fail(WMTP_ERR_INVALID_ARG, "ring descriptor is NULL");
+    if (wmtp_status s = check_shape(r->batch, r->Hkv, r->D)) return s;
+    if (r->n_sink < 0 || r->W < 1 || r->cap < r->W)
+        return fail(WMTP_ERR_INVALID_ARG, "ring needs n_sink >= 0, W >= 1, cap >= W (n_sink=%d W=%d cap=%d)", r->n_sink, r->W, r->cap);
+    if ((int64_t)r->n_sink + r->cap > (1 << 30)) return fail(WMTP_ERR_INVALID_ARG, "ring of %lld slots is too large", (long long)r->n_sink + r->cap);
+    if (!r->k || !r->v || !r->slot_pos || !r->len) return fail(WMTP_ERR_INVALID_ARG, "ring has a NULL pointer");
+    if (!aligned(r->k, 16) || !aligned(r->v, 16) || !aligned(r->slot_pos, 4) || !aligned(r->len, 8))
+        return fail(WMTP_ERR_INVALID_ARG, "ring pointers must be 16-byte (k, v), 4-byte (slot_pos), 8-byte (len) aligned");
+    return WMTP_OK;
+}
+
+wmtp_status check_kv(const wmtp_kv* kv) {
+    if (!kv) return fail(WMTP_ERR_INVALID_ARG, "kv descriptor is NULL");
+    if (wmtp_status s = check_shape(kv->batch, kv->Hkv, kv->D)) return s;
+    if (!kv->k || !kv->v || !kv->len) return fail(WMTP_ERR_INVALID_ARG, "kv has a NULL pointer");
+    if (!aligned(kv->k, 16) || !aligned(kv->v, 16) || !aligned(kv->len, 8))
+        return fail(WMTP_ERR_INVALID_ARG, "kv pointers must be 16-byte (k, v), 8-byte (len) aligned");
+    if (kv->S_cap < 1) return fail(WMTP_ERR_INVALID_ARG, "S_cap=%lld must be positive", (long long)kv->S_cap);
+    if (kv->page_table) {
+        if (kv->page_size != kTileKeys) return fail(WMTP_ERR_UNSUPPORTED, "page_size=%d (supported: %d)", kv->page_size, kTileKeys);
+        if (kv->max_pages < 1 || kv->num_pages < 1) return fail(WMTP_ERR_INVALID_ARG, "max_pages, num_pages must be positive");
+        if (!aligned(kv->page_table, 4)) return fail(WMTP_ERR_INVALID_ARG, "page_table must be 4-byte aligned");
+        if (kv->S_cap > (int64_t)kv->max_pages * kv->page_size)
+            return fail(WMTP_ERR_CAPACITY, "S_cap=%lld exceeds the page table's %lld tokens", (long long)kv->S_cap,
+                        (long long)kv->max_pages * kv->page_size);
+    }
+    return WMTP_OK;
+}
+
+RingParams ring_params(const wmtp_ring* r) {
+    return RingParams{r->k, r->v, r->slot_pos, r->len, r->batch, r->Hkv, r->D, r->n_sink, r->W, r->cap};
+}
+KvParams kv_params(const wmtp_kv* kv) {
+    return KvParams{kv->k, kv->v, kv->page_table, kv->len, kv->S_cap, kv->batch, kv->Hkv, kv->D,
+                    kv->page_table ? kv->page_size : 0, kv->max_pages, kv->num_pages};
+}
+
+wmtp_status check_attn_common(const void* q, int Hq, int Hkv, int batch, int D, const void* out, const float* lse,
+                              const void* ws, size_t ws_bytes) {
+    if (!q || !out) return fail(WMTP_ERR_INVALID_ARG, "q or out is NULL");
+    if (!aligned(q, 16) || !aligned(out, 16)) return fail(WMTP_ERR_INVALID_ARG, "q and out must be 16-byte aligned");
+    if (lse && !aligned(lse, 4)) return fail(WMTP_ERR_INVALID_ARG, "lse must be 4-byte aligned");
+    if (Hq < 1 || Hq % Hkv != 0) return fail(WMTP_ERR_INVALID_ARG, "Hq=%d must be a positive multiple of Hkv=%d", Hq, Hkv);
+    if (Hq / Hkv > kMaxGroup) return fail(WMTP_ERR_UNSUPPORTED, "Hq/Hkv=%d exceeds %d", Hq / Hkv, kMaxGroup);
+    if (!ws || !aligned(ws, 256)) return fail(WMTP_ERR_WORKSPACE, "workspace is NULL or not 256-byte aligned");
+    const size_t need = wmtp_workspace_bytes(batch, Hq, Hkv, D);
+    if (ws_bytes < need) return fail(WMTP_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", ws_bytes, need);
+    return WMTP_OK;
+}
+
+int pick_ctas(int64_t max_tiles) {
+    int c = g_max_ctas.load();
+    if (c <= 0) c = sm_count();
+    if (c <= 0) return 0;
+    if (c > kMaxCtas) c = kMaxCtas;
+    if (max_tiles < c) c = (int)(max_tiles < 1 ? 1 : max_tiles);
+    return c;
+}
+
+void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, float sm_scale, void* out, float* lse,
+               void* ws) {
+    const WorkspaceLayout L = workspace_layout(batch, Hq, Hkv, D);
+    char* base = static_cast<char*>(ws);
+    p.q = q; p.out = out; p.lse = lse;
+    p.status = reinterpret_cast<int*>(base);
+    p.counters = reinterpret_cast<int*>(base + L.counters_off);
+    p.part_lse = reinterpret_cast<float*>(base + L.part_lse_off);
+    p.part_o = reinterpret_cast<float*>(base + L.part_o_off);
+    p.B = batch; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = Hq / Hkv;
+    const float s = sm_scale > 0.f ? sm_scale : 1.0f / std::sqrt((float)D);
+    p.scale_log2 = s * 1.4426950408889634f;
+}
+
+wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm_scale, void* out, float* lse,
+                          void* ws, size_t ws_bytes, cudaStream_t st, bool validate) {
+    if (validate) {
+        if (wmtp_status s = check_ring(ring)) return s;
+        if (wmtp_status s = check_attn_common(q, Hq, ring->Hkv, ring->batch, ring->D, out, lse, ws, ws_bytes)) return s;
+    }
+    AttnParams p{};
+    fill_attn(p, q, Hq, ring->Hkv, ring->batch, ring->D, sm_scale, out, lse, ws);
+    p.k = ring->k; p.v = ring->v; p.page_table = nullptr; p.len = ring->len;
+    p.mode = kRing;
+    p.rows_per_head = (int64_t)ring->n_sink + ring->cap;
+    p.n_sink = ring->n_sink; p.W = ring->W; p.cap = ring->cap;
+    const int64_t tiles = (p.rows_per_head + kTileKeys - 1) / kTileKeys * ring->batch * ring->Hkv;
+    p.num_ctas = pick_ctas(tiles);
+    if (p.num_ctas <= 0) return fail(WMTP_ERR_CUDA, "no CUDA device available");
+    cudaError_t e = launch_attention(p, st);
+    if (e != cudaSuccess) return cuda_fail(e, "windowed attention launch");
+    return WMTP_OK;
+}
+
+wmtp_status attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, void* out, float* lse, void* ws,
+                      size_t ws_bytes, cudaStream_t st, bool validate) {
+    if (validate) {
+        if (wmtp_status s = check_kv(kv)) return s;
+        if (wmtp_status s = check_attn_common(q, Hq, kv->Hkv, kv->batch, kv->D, out, lse, ws, ws_bytes)) return s;
+    }
+    AttnParams p{};
+    fill_attn(p, q, Hq, kv->Hkv, kv->batch, kv->D, sm_scale, out, lse, ws);
+    p.k = kv->k; p.v = kv->v; p.page_table = kv->page_table; p.len = kv->len;
+    p.mode = kv->page_table ? kPaged : kContiguous;
+    p.rows_per_head = kv->page_table ? kv->page_size : kv->S_cap;
+    p.page_size = kv->page_size; p.max_pages = kv->max_pages; p.num_pages = kv->num_pages;
+    const int64_t tiles = (kv->S_cap + kTileKeys - 1) / kTileKeys * kv->batch * kv->Hkv;
+    p.num_ctas = pick_ctas(tiles);
+    if (p.num_ctas <= 0) return fail(WMTP_ERR_CUDA, "no CUDA device available");
+    cudaError_t e = launch_attention(p, st);
+    if (e != cudaSuccess) return cuda_fail(e, "full attention launch");
+    return WMTP_OK;
+}
+
+wmtp_status check_loop(int gamma, const void* k_new, const void* v_new) {
+    if (gamma < 1) return fail(WMTP_ERR_INVALID_ARG, "gamma=%d must be positive", gamma);
+    if (!k_new || !v_new) return fail(WMTP_ERR_INVALID_ARG, "k_new or v_new is NULL");
+    if (!aligned(k_new, 16) || !aligned(v_new, 16)) return fail(WMTP_ERR_INVALID_ARG, "k_new and v_new must be 16-byte aligned");
+    return WMTP_OK;
+}
+
+struct StagePlan { size_t q, k, v, out, lse, total; };
+StagePlan stage_plan(int gamma, int batch, int Hq, int Hkv, int D) {
+    StagePlan s;
+    const size_t qb = (size_t)gamma * batch * Hq * D * 2, kb = (size_t)gamma * batch * Hkv * D * 2;
+    s.q = 0;
+    s.k = round_up(qb, 256);
+    s.v = s.k + round_up(kb, 256);
+    s.out = s.v + round_up(kb, 256);
+    s.lse = s.out + round_up(qb, 256);
+    s.total = s.lse + round_up((size_t)gamma * batch * Hq * 4, 256);
+    return s;
+}
+
+}  // namespace
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int sm_count() {
+    static std::atomic<int> cached{0};
+    int c = cached.load();
+    if (c > 0) return c;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    cached.store(n);
+    return n;
+}
+
+WorkspaceLayout workspace_layout(int batch, int Hq, int Hkv, int D) {
+    WorkspaceLayout L;
+    const size_t G = (size_t)(Hq / Hkv), nseg = (size_t)batch * Hkv, np = kMaxCtas + nseg;
+    L.counters_off = 256;
+    L.part_lse_off = L.counters_off + round_up(nseg * sizeof(int), 256);
+    L.part_o_off = L.part_lse_off + round_up(np * G * sizeof(float), 256);
+    L.total = L.part_o_off + round_up(np * G * D * sizeof(float), 256);
+    return L;
+}
+
+}  // namespace wmtp
+
+using namespace wmtp;
+
+extern "C" {
+
+const char* wmtp_status_string(wmtp_status s) {
+    switch (s) {
+        case WMTP_OK: return "ok";
+        case WMTP_ERR_INVALID_ARG: return "invalid argument";
+        case WMTP_ERR_UNSUPPORTED: return "unsupported shape";
+        case WMTP_ERR_CAPACITY: return "capacity exceeded";
+        case WMTP_ERR_WORKSPACE: return "bad workspace";
+        case WMTP_ERR_CUDA: return "CUDA error";
+        case WMTP_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case WMTP_ERR_DEVICE_BOUNDS: return "device-side bounds check failed";
+    }
+    return "unknown status";
+}
+
+const char* wmtp_last_error(void) { return g_err; }
+
+size_t wmtp_ring_bytes(int batch, int Hkv, int D, int n_sink, int cap, size_t* pos_bytes) {
+    if (batch < 1 || Hkv < 1 || D < 1 || n_sink < 0 || cap < 1) { if (pos_bytes) *pos_bytes = 0; return 0; }
+    const size_t slots = (size_t)n_sink + cap;
+    if (pos_bytes) *pos_bytes = (size_t)batch * slots * sizeof(int32_t);
+    return (size_t)batch * Hkv * slots * D * 2;
+}
+
+size_t wmtp_workspace_bytes(int batch, int Hq, int Hkv, int D) {
+    if (batch < 1 || Hq < 1 || Hkv < 1 || D < 1 || Hq % Hkv != 0) return 0;
+    return workspace_layout(batch, Hq, Hkv, D).total;
+}
+
+wmtp_status wmtp_workspace_init(void* workspace, size_t ws_bytes, void* stream) {
+    if (!workspace || !aligned(workspace, 256)) return fail(WMTP_ERR_WORKSPACE, "workspace is NULL or not 256-byte aligned");
+    if (ws_bytes < 512) return fail(WMTP_ERR_WORKSPACE, "workspace of %zu bytes is too small", ws_bytes);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, ws_bytes, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "workspace memset");
+    return WMTP_OK;
+}
+
+wmtp_status wmtp_device_status(void* workspace, void* stream) {
+    if (!workspace) return fail(WMTP_ERR_WORKSPACE, "workspace is NULL");
+    int word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, workspace, sizeof word, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "reading the device status");
+    if (word != 0) {
+        e = cudaMemsetAsync(workspace, 0, sizeof word, (cudaStream_t)stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(e, "clearing the device status");
+        if (word == WMTP_ERR_DEVICE_TIMEOUT) return fail(WMTP_ERR_DEVICE_TIMEOUT, "a device-side wait expired");
+        return fail(WMTP_ERR_DEVICE_BOUNDS, "a device-side bounds check failed (status word %d)", word);
+    }
+    return WMTP_OK;
+}
+
+wmtp_status wmtp_ring_reset(const wmtp_ring* ring, void* stream) {
+    if (wmtp_status s = check_ring(ring)) return s;
+    cudaError_t e = launch_ring_reset(ring_params(ring), (cudaStream_t)stream);
+    return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "ring reset launch");
+}
+
+wmtp_status wmtp_ring_init_from_kv(const wmtp_ring* ring, const wmtp_kv* kv, void* stream) {
+    if (wmtp_status s = check_ring(ring)) return s;
+    if (wmtp_status s = check_kv(kv)) return s;
+    if (ring->batch != kv->batch || ring->Hkv != kv->Hkv || ring->D != kv->D)
+        return fail(WMTP_ERR_INVALID_ARG, "ring and kv disagree on batch / Hkv / D");
+    cudaError_t e = launch_ring_init_from_kv(ring_params(ring), kv_params(kv), (cudaStream_t)stream);
+    return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "ring init launch");
+}
+
+wmtp_status wmtp_ring_append(const wmtp_ring* ring, const void* k_new, const void* v_new, void* stream) {
+    if (wmtp_status s = check_ring(ring)) return s;
+    if (wmtp_status s = check_loop(1, k_new, v_new)) return s;
+    cudaError_t e = launch_ring_append(ring_params(ring), k_new, v_new, (cudaStream_t)stream);
+    return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "ring append launch");
+}
+
+wmtp_status wmtp_kv_append(const wmtp_kv* kv, const void* k_new, const void* v_new, void* workspace, void* stream) {
+    if (wmtp_status s = check_kv(kv)) return s;
+    if (wmtp_status s = check_loop(1, k_new, v_new)) return s;
+    if (workspace && !aligned(workspace, 256)) return fail(WMTP_ERR_WORKSPACE, "workspace is not 256-byte aligned");
+    cudaError_t e = launch_kv_append(kv_params(kv), k_new, v_new, static_cast<int*>(workspace), (cudaStream_t)stream);
+    return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "kv append launch");
+}
+
+wmtp_status wmtp_draft_attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm_scale, void* out,
+                                     float* lse, void* workspace, size_t ws_bytes, void* stream) {
+    return attn_windowed(q, Hq, ring, sm_scale, out, lse, workspace, ws_bytes, (cudaStream_t)stream, true);
+}
+
+wmtp_status wmtp_draft_attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, void* out, float* lse,
+                                 void* workspace, size_t ws_bytes, void* stream) {
+    return attn_full(q, Hq, kv, sm_scale, out, lse, workspace, ws_bytes, (cudaStream_t)stream, true);
+}
+
+wmtp_status wmtp_draft_loop_windowed(const wmtp_ring* ring, int gamma, const void* q, int Hq, const void* k_new,
+                                     const void* v_new, float sm_scale, void* out, float* lse, void* workspace,
+                                     size_t ws_bytes, void* stream) {
+    if (wmtp_status s = check_ring(ring)) return s;
+    if (wmtp_status s = check_loop(gamma, k_new, v_new)) return s;
+    if (wmtp_status s = check_attn_common(q, Hq, ring->Hkv, ring->batch, ring->D, out, lse, workspace, ws_bytes)) return s;
+    const RingParams rp = ring_params(ring);
+    const size_t q_step = (size_t)ring->batch * Hq * ring->D * 2, kv_step = (size_t)ring->batch * ring->Hkv * ring->D * 2;
+    for (int i = 0; i < gamma; ++i) {
+        cudaError_t e = launch_ring_append(rp, (const char*)k_new + i * kv_step, (const char*)v_new + i * kv_step,
+                                           (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(e, "ring append launch");
+        if (wmtp_status s = attn_windowed((const char*)q + i * q_step, Hq, ring, sm_scale, (char*)out + i * q_step,
+                                          lse ? lse + (size_t)i * ring->batch * Hq : nullptr, workspace, ws_bytes,
+                                          (cudaStream_t)stream, false))
+            return s;
+    }
+    return WMTP_OK;
+}
+
+wmtp_status wmtp_draft_loop_full(const wmtp_kv* kv, int gamma, const void* q, int Hq, const void* k_new,
+                                 const void* v_new, float sm_scale, void* out, float* lse, void* workspace,
+                                 size_t ws_bytes, void* stream) {
+    if (wmtp_status s = check_kv(kv)) return s;
+    if (wmtp_status s = check_loop(gamma, k_new, v_new)) return s;
+    if (wmtp_status s = check_attn_common(q, Hq, kv->Hkv, kv->batch, kv->D, out, lse, workspace, ws_bytes)) return s;
+    const KvParams kp = kv_params(kv);
+    const size_t q_step = (size_t)kv->batch * Hq * kv->D * 2, kv_step = (size_t)kv->batch * kv->Hkv * kv->D * 2;
+    for (int i = 0; i < gamma; ++i) {
+        cudaError_t e = launch_kv_append(kp, (const char*)k_new + i * kv_step, (const char*)v_new + i * kv_step,
+                                         static_cast<int*>(workspace), (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(e, "kv append launch");
+        if (wmtp_status s = attn_full((const char*)q + i * q_step, Hq, kv, sm_scale, (char*)out + i * q_step,
+                                      lse ? lse + (size_t)i * kv->batch * Hq : nullptr, workspace, ws_bytes,
+                                      (cudaStream_t)stream, false))
+            return s;
+    }
+    return WMTP_OK;
+}
+
+size_t wmtp_stage_bytes(int gamma, int batch, int Hq, int Hkv, int D) {
+    if (gamma < 1 || batch < 1 || Hq < 1 || Hkv < 1 || D < 1) return 0;
+    return stage_plan(gamma, batch, Hq, Hkv, D).total;
+}
+
+static wmtp_status loop_host(const wmtp_ring* ring, const wmtp_kv* kv, int gamma, const void* qh, int Hq, const void* kh,
+                             const void* vh, float sm_scale, void* outh, float* lseh, void* stage, void* ws,
+                             size_t ws_bytes, void* stream) {
+    const int batch = ring ? ring->batch : kv->batch, Hkv = ring ? ring->Hkv : kv->Hkv, D = ring ? ring->D : kv->D;
+    if (!qh || !kh || !vh || !outh) return fail(WMTP_ERR_INVALID_ARG, "a host pointer is NULL");
+    if (!stage || !aligned(stage, 256)) return fail(WMTP_ERR_INVALID_ARG, "stage is NULL or not 256-byte aligned");
+    if (gamma < 1 || Hq < 1) return fail(WMTP_ERR_INVALID_ARG, "gamma and Hq must be positive");
+    const StagePlan sp = stage_plan(gamma, batch, Hq, Hkv, D);
+    const size_t qb = (size_t)gamma * batch * Hq * D * 2, kb = (size_t)gamma * batch * Hkv * D * 2;
+    char* sb = static_cast<char*>(stage);
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(sb + sp.q, qh, qb, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "H2D q");
+    if ((e = cudaMemcpyAsync(sb + sp.k, kh, kb, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "H2D k_new");
+    if ((e = cudaMemcpyAsync(sb + sp.v, vh, kb, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "H2D v_new");
+    float* lse_d = lseh ? reinterpret_cast<float*>(sb + sp.lse) : nullptr;
+    wmtp_status s = ring ? wmtp_draft_loop_windowed(ring, gamma, sb + sp.q, Hq, sb + sp.k, sb + sp.v, sm_scale, sb + sp.out,
+                                                    lse_d, ws, ws_bytes, stream)
+                         : wmtp_draft_loop_full(kv, gamma, sb + sp.q, Hq, sb + sp.k, sb + sp.v, sm_scale, sb + sp.out, lse_d,
+                                                ws, ws_bytes, stream);
+    if (s != WMTP_OK) return s;
+    if ((e = cudaMemcpyAsync(outh, sb + sp.out, qb, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "D2H out");
+    if (lseh && (e = cudaMemcpyAsync(lseh, lse_d, (size_t)gamma * batch * Hq * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+        return cuda_fail(e, "D2H lse");
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(e, "stream synchronize");
+    return WMTP_OK;
+}
+
+wmtp_status wmtp_draft_loop_windowed_host(const wmtp_ring* ring, int gamma, const void* q_host, int Hq,
+                                          const void* k_new_host, const void* v_new_host, float sm_scale, void* out_host,
+                                          float* lse_host, void* stage, void* workspace, size_t ws_bytes, void* stream) {
+    if (wmtp_status s = check_ring(ring)) return s;
+    return loop_host(ring, nullptr, gamma, q_host, Hq, k_new_host, v_new_host, sm_scale, out_host, lse_host, stage,
+                     workspace, ws_bytes, stream);
+}
+
+wmtp_status wmtp_draft_loop_full_host(const wmtp_kv* kv, int gamma, const void* q_host, int Hq, const void* k_new_host,
+                                      const void* v_new_host, float sm_scale, void* out_host, float* lse_host, void* stage,
+                                      void* workspace, size_t ws_bytes, void* stream) {
+    if (wmtp_status s = check_kv(kv)) return s;
+    return loop_host(nullptr, kv, gamma, q_host, Hq, k_new_host, v_new_host, sm_scale, out_host, lse_host, stage, workspace,
+                     ws_bytes, stream);
+}
+
+void wmtp_set_max_ctas(int max_ctas) { g_max_ctas.store(max_ctas < 0 ? 0 : max_ctas); }
+
+int64_t wmtp_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

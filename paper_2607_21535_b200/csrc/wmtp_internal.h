@@ -1,0 +1,71 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/wmtp.h"
+
+namespace wmtp {
+
+constexpr int kTileKeys = 64;       // keys per K/V tile; equals the page size of the paged layout
+constexpr int kMaxCtas = 1024;      // upper bound on attention CTAs, sizes the partial buffers
+constexpr int kMaxBatch = 1024;     // sequences per call (prefix table lives in shared memory)
+constexpr int kMaxGroup = 8;        // query heads per KV head
+
+enum KvMode : int { kContiguous = 0, kPaged = 1, kRing = 2 };
+
+// Workspace layout (all offsets from a 256-byte aligned base):
+//   [0, 256)            header: int status word at offset 0
+//   counters            int [batch * Hkv], padded to 256 bytes
+//   part_lse            float [kMaxCtas + batch * Hkv][G]
+//   part_o              float [kMaxCtas + batch * Hkv][G][D]
+struct WorkspaceLayout {
+    size_t counters_off, part_lse_off, part_o_off, total;
+};
+WorkspaceLayout workspace_layout(int batch, int Hq, int Hkv, int D);
+
+// Everything the attention kernels need; passed by value.
+struct AttnParams {
+    const void* q;            // bf16 [B][Hq][D]
+    const void* k;            // bf16, layout per mode
+    const void* v;
+    const int32_t* page_table;
+    const int64_t* len;       // [B]
+    float* part_o;
+    float* part_lse;
+    int* counters;
+    int* status;
+    void* out;                // bf16 [B][Hq][D]
+    float* lse;               // [B][Hq] or nullptr
+    int64_t rows_per_head;    // contiguous: S_cap; ring: n_sink + cap; paged: page_size
+    int B, Hq, Hkv, D, G;
+    int mode;
+    int page_size, max_pages, num_pages;
+    int n_sink, W, cap;
+    float scale_log2;         // sm_scale * log2(e)
+    int num_ctas;
+};
+
+struct RingParams {
+    void* k; void* v; int32_t* slot_pos; int64_t* len;
+    int B, Hkv, D, n_sink, W, cap;
+};
+
+struct KvParams {
+    void* k; void* v; const int32_t* page_table; int64_t* len;
+    int64_t S_cap;
+    int B, Hkv, D, page_size, max_pages, num_pages;
+};
+
+// Launchers (defined in the .cu files). Each returns the cudaError_t of its launch.
+cudaError_t launch_ring_reset(const RingParams& r, cudaStream_t st);
+cudaError_t launch_ring_append(const RingParams& r, const void* k_new, const void* v_new, cudaStream_t st);
+cudaError_t launch_ring_init_from_kv(const RingParams& r, const KvParams& kv, cudaStream_t st);
+cudaError_t launch_kv_append(const KvParams& kv, const void* k_new, const void* v_new, int* status, cudaStream_t st);
+cudaError_t launch_attention(const AttnParams& p, cudaStream_t st);   // partial + combine
+
+void count_launch(int n);
+int  sm_count();   // multiprocessors of the current device (cached), 0 on failure
+
+}  // namespace wmtp

@@ -1,0 +1,85 @@
+"""Helpers for the GPU parity tests: upload a synthetic workload, run the CUDA path through the
+C-ABI binding, run the CPU oracle on the same bits, compare."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import paper_2607_21535_b200 as wm
+import wmtp_inputs as wi
+from oracle import reference as R
+
+# Contract tolerances for bf16 outputs (differences taken in fp32/fp64 on the bf16 result) ...
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3
+# ... and the stricter per-head checks that stay meaningful when outputs are small (large S).
+REL_L2, LSE_ABS = 1e-2, 1e-3
+
+
+def to_dev_bf16(a: np.ndarray, dev="cuda"):
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(dev).view(torch.bfloat16)
+
+
+def bits(t: torch.Tensor) -> np.ndarray:
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+class DeviceWorkload:
+    """Device copies of a Workload plus ring / KV descriptors / workspace."""
+
+    def __init__(self, wl: wi.Workload, dev="cuda", cap=None):
+        cfg = wl.cfg
+        self.wl, self.cfg, self.dev = wl, cfg, dev
+        self.K, self.V = to_dev_bf16(wl.K_dev, dev), to_dev_bf16(wl.V_dev, dev)
+        self.lens = torch.from_numpy(wl.seq_lens.copy()).to(dev)
+        pt = torch.from_numpy(wl.page_table).to(dev) if cfg.paged else None
+        self.kv = wm.KV(self.K, self.V, self.lens, page_table=pt, S_cap=None if cfg.paged else wl.S_cap)
+        self.ring = wm.Ring(cfg.batch, cfg.Hkv, cfg.D, cfg.n_sink, cfg.W, cap=cap if cap is not None else cfg.W + cfg.cap_slack,
+                            device=dev)
+        self.ws = wm.Workspace(cfg.batch, cfg.Hq, cfg.Hkv, cfg.D, device=dev)
+        self.q, self.k_new, self.v_new = to_dev_bf16(wl.q, dev), to_dev_bf16(wl.k_new, dev), to_dev_bf16(wl.v_new, dev)
+        self.out_w = torch.full_like(self.q, float("nan"))
+        self.out_f = torch.full_like(self.q, float("nan"))
+        self.lse_w = torch.full(self.q.shape[:-1], float("nan"), dtype=torch.float32, device=dev)
+        self.lse_f = torch.full(self.q.shape[:-1], float("nan"), dtype=torch.float32, device=dev)
+
+    def run_loops(self, windowed=True, full=True):
+        if windowed:
+            wm.wmtp_ring_init_from_kv(self.ring, self.kv)
+            wm.wmtp_draft_loop_windowed(self.ring, self.q, self.k_new, self.v_new, self.out_w, self.ws, lse=self.lse_w)
+        if full:
+            wm.wmtp_draft_loop_full(self.kv, self.q, self.k_new, self.v_new, self.out_f, self.ws, lse=self.lse_f)
+        wm.wmtp_device_status(self.ws)
+
+
+def compare(got_bf16: torch.Tensor, got_lse: torch.Tensor | None, ref_out: np.ndarray, ref_lse: np.ndarray, what=""):
+    """got: bf16 [Hq][D] (+ fp32 lse [Hq]) from the GPU; ref: fp64 from the oracle."""
+    got = got_bf16.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    err = np.abs(got - ref_out)
+    assert err.max() <= MAX_ABS, f"{what}: max-abs {err.max():.3e}"
+    assert err.mean() <= MEAN_ABS, f"{what}: mean-abs {err.mean():.3e}"
+    num = np.linalg.norm(got - ref_out, axis=-1)
+    den = np.linalg.norm(ref_out, axis=-1)
+    rel = num / np.maximum(den, 1e-30)
+    assert (rel <= REL_L2).all(), f"{what}: per-head relative L2 {rel.max():.3e}"
+    if got_lse is not None:
+        dl = np.abs(got_lse.cpu().numpy().astype(np.float64) - ref_lse)
+        assert (dl <= LSE_ABS).all(), f"{what}: lse error {dl.max():.3e}"
+    return float(err.max()), float(rel.max())
+
+
+def check_ring_against_sim(ring: wm.Ring, b: int, sim: R.RingSim, what=""):
+    """Slot positions, length and the bf16 bit patterns of every written slot must be identical."""
+    pos = ring.slot_pos[b].cpu().numpy()
+    assert (pos == sim.slot_pos).all(), f"{what}: slot_pos differs"
+    assert int(ring.len[b]) == sim.length, f"{what}: len differs"
+    Kb, Vb = bits(ring.k[b]), bits(ring.v[b])
+    w = sim.written
+    assert (Kb[:, w] == sim.K[:, w]).all(), f"{what}: ring K bits differ"
+    assert (Vb[:, w] == sim.V[:, w]).all(), f"{what}: ring V bits differ"
+
+
+def oracle_for(wl: wi.Workload, b: int, cap=None, with_ring=True) -> R.DraftOracle:
+    cfg = wl.cfg
+    return R.DraftOracle(wl.K[b], wl.V[b], cfg.Hq, cfg.n_sink, cfg.W, cap=cap if cap is not None else cfg.W + cfg.cap_slack,
+                         reserve=cfg.gamma + 1, with_ring=with_ring)
