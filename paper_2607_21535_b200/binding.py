@@ -150,7 +150,8 @@ class KV:
 class Workspace:
     def __init__(self, batch, Hq, Hkv, D, device="cuda", stream=None):
         self.nbytes = int(lib().wmtp_workspace_bytes(batch, Hq, Hkv, D))
-        self.buf = torch.empty((self.nbytes,), dtype=torch.uint8, device=device)
+        # 0xFF bytes are NaN as floats: a partial result read before it is written cannot go unnoticed
+        self.buf = torch.full((self.nbytes,), 0xFF, dtype=torch.uint8, device=device)
         assert self.buf.data_ptr() % 256 == 0
         wmtp_workspace_init(self, stream=stream)
 

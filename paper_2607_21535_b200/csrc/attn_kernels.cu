@@ -1,8 +1,21 @@
-// Split-KV decode attention for the draft head: partial kernel + log-sum-exp combine.
+// Split-KV decode attention for the draft head: TMA-fed partial kernel + log-sum-exp combine.
 //
 // The operation is softmax attention of one query per head over a key set (Section 4
 // "Mechanism"; Appendix D: o = sum_j p_j v_j): the ring's live slots for the windowed draft,
-// all S positions for the full-context (native) draft of Section 3.
+// all S positions for the full-context (native) draft of Section 3. The work is bound by the
+// HBM read of K and V, so the kernel is organised around keeping bytes in flight:
+//
+//   * one persistent CTA per SM owns a contiguous range of 64-key tiles (attn_plan.cuh);
+//   * a producer warp streams K and V tiles into a ring of shared-memory stages with TMA
+//     (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers);
+//   * four consumer warps each take 16 keys of every tile. Scores are computed as
+//     S^T[key, head] = K[key, :] . Q^T (keys on the MMA M dimension, the G <= 8 query heads of
+//     the GQA group exactly on N = 8), the online softmax runs in fp32, and
+//     O^T[d, head] += V^T[d, key] . P^T[key, head] accumulates in registers. The 8-row problem
+//     is far too small for tcgen05 (M >= 64); mma.sync.m16n8k16 needs ~3% of tensor peak here.
+//   * every K/V byte is read once from HBM and once from shared memory, shared by all heads
+//     of the group.
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "attn_plan.cuh"
@@ -12,229 +25,531 @@ namespace wmtp {
 namespace {
 
 constexpr int kErrBounds = WMTP_ERR_DEVICE_BOUNDS;
+constexpr int kErrTimeout = WMTP_ERR_DEVICE_TIMEOUT;
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kConsumerWarps = 4;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr uint32_t kSpinLimit = 1u << 22;       // bounded mbarrier waits
+constexpr int kScratchRow = 132;                // floats per (warp, head) row of the merge scratch (128 + pad)
 
+template <int D>
+struct Cfg {
+    static constexpr int kChunks = D / 64;                    // 128-byte column chunks per row
+    static constexpr int kChunkBytes = kTileKeys * 128;       // one TMA box: 64 rows x 128 B
+    static constexpr int kTileBytes = kChunks * kChunkBytes;  // K (or V) tile
+    static constexpr int kStageBytes = 2 * kTileBytes;
+    static constexpr int kStages = (D == 256) ? 3 : 6;
+    static constexpr int kKSteps = D / 16;
+};
+
+// ---- PTX wrappers -----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kSpinLimit polls (or as soon as another thread has given up), raises
+// the CTA's abort flag and the sticky device status; the caller carries on with invalid data so that
+// every thread still follows the same control flow and nobody is left waiting.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    if (mbar_try_wait(bar, parity)) return;
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return;
+        if ((i & 1023u) == 1023u && *abort_flag) return;
+    }
+    *abort_flag = 1;
+    atomicCAS(status, 0, kErrTimeout);
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
 __device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Segment bookkeeping shared by producer and consumers.
+struct Segment {
+    int b, g, seg;
+    int64_t seg_start, t_end, nk, S;
+};
+__device__ __forceinline__ Segment locate_segment(const AttnParams& p, const int64_t* tile_prefix, int64_t t, int64_t t1) {
+    Segment s;
+    s.b = find_seq(tile_prefix, p.B, p.Hkv, t);
+    const int64_t tiles_b = tile_prefix[s.b + 1] - tile_prefix[s.b];
+    const int64_t seq_start = (int64_t)p.Hkv * tile_prefix[s.b];
+    s.g = (int)((t - seq_start) / tiles_b);
+    s.seg_start = seq_start + (int64_t)s.g * tiles_b;
+    const int64_t seg_end = s.seg_start + tiles_b;
+    s.t_end = seg_end < t1 ? seg_end : t1;
+    s.S = p.len[s.b];
+    s.nk = scan_keys(p, s.b);
+    s.seg = s.b * p.Hkv + s.g;
+    return s;
+}
 
 // ---------------------------------------------------------------------------------------------
-// Partial kernel, CUDA-core version: one warp per key row, lanes split head_dim, all G query
-// heads of the group share every K/V row that is loaded.
+// Partial kernel
 // ---------------------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(128) attn_partial_simple(AttnParams p) {
-    constexpr int EPL = D / 32;             // elements per lane (4 or 8)
-    constexpr int WPL = EPL / 2;            // 32-bit words per lane
-    constexpr int NW = 4;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    int64_t* tile_prefix = reinterpret_cast<int64_t*>(smem_raw);                 // [B + 1]
-    float* sm_m = reinterpret_cast<float*>(tile_prefix + (p.B + 1));             // [NW][8]
-    float* sm_l = sm_m + NW * kMaxGroup;                                         // [NW][8]
-    float* sm_acc = sm_l + NW * kMaxGroup;                                       // [NW][8][D]
+__global__ void __launch_bounds__(kThreads, 1)
+attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, AttnParams p) {
+    using C = Cfg<D>;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    unsigned char* stages = smem;                                                         // kStages x (K tile, V tile)
+    float* scratch = reinterpret_cast<float*>(stages + C::kStages * C::kStageBytes);      // [4][8][kScratchRow]
+    float* sm_m = scratch + kConsumerWarps * kMaxGroup * kScratchRow;                     // [4][8]
+    float* sm_l = sm_m + kConsumerWarps * kMaxGroup;                                      // [4][8]
+    float* sm_le = sm_l + kConsumerWarps * kMaxGroup;                                     // [4][8]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm_le + kConsumerWarps * kMaxGroup);     // fullK, fullV, empty
+    int* abort_flag = reinterpret_cast<int*>(bars + 3 * C::kStages);
+    int64_t* tile_prefix = reinterpret_cast<int64_t*>(abort_flag + 2);                    // [B + 1]
 
     build_tile_prefix(p, tile_prefix);
-    const int C = gridDim.x;
     const int64_t n = (int64_t)p.Hkv * tile_prefix[p.B];
-    if (n == 0) return;
-    const int64_t t0 = cta_range_start(blockIdx.x, n, C), t1 = cta_range_start(blockIdx.x + 1, n, C);
-    if (t0 >= t1) return;
+    const int Cn = effective_ctas(gridDim.x, n);
+    if ((int)blockIdx.x >= Cn) return;
+    const int64_t t0 = cta_range_start(blockIdx.x, n, Cn), t1 = cta_range_start(blockIdx.x + 1, n, Cn);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t bar_fullK = smem_u32(bars), bar_fullV = smem_u32(bars + C::kStages), bar_empty = smem_u32(bars + 2 * C::kStages);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::kStages; ++s) {
+            mbar_init(bar_fullK + 8 * s, 1);
+            mbar_init(bar_fullV + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, kConsumerWarps);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const bool slack = (p.mode == kRing) && (p.cap != p.W);
+
+    if (warp == kConsumerWarps) {
+        // =================================== producer warp ===================================
+        const uint32_t stage0 = smem_u32(stages);
+        int64_t t = t0;
+        uint32_t it = 0;
+        while (t < t1) {
+            const Segment sg = locate_segment(p, tile_prefix, t, t1);
+            const int64_t first_tile = t - sg.seg_start;
+            const int ntiles = (int)(sg.t_end - t);
+            for (int base = 0; base < ntiles; base += 32) {
+                int page = 0;
+                if (p.mode == kPaged) {        // 32 page ids at a time, one per lane
+                    const int64_t ti = first_tile + base + lane;
+                    if (base + lane < ntiles) {
+                        page = p.page_table[(int64_t)sg.b * p.max_pages + ti];
+                        if (page < 0 || page >= p.num_pages) { atomicCAS(p.status, 0, kErrBounds); page = 0; }
+                    }
+                }
+                const int cnt = ntiles - base < 32 ? ntiles - base : 32;
+                for (int j = 0; j < cnt; ++j, ++it) {
+                    const int pg = __shfl_sync(0xffffffffu, page, j);
+                    if (lane == 0) {
+                        const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+                        mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status);
+                        if (!*(volatile int*)abort_flag) {
+                            int64_t row;
+                            if (p.mode == kPaged) row = ((int64_t)pg * p.Hkv + sg.g) * kTileKeys;
+                            else row = ((int64_t)sg.b * p.Hkv + sg.g) * p.rows_per_head + (first_tile + base + j) * kTileKeys;
+                            const uint32_t dstK = stage0 + s * C::kStageBytes, dstV = dstK + C::kTileBytes;
+                            mbar_expect_tx(bar_fullK + 8 * s, C::kTileBytes);
+#pragma unroll
+                            for (int c = 0; c < C::kChunks; ++c)
+                                tma_load_2d(dstK + c * C::kChunkBytes, &mapK, c * 64, (int)row, bar_fullK + 8 * s);
+                            mbar_expect_tx(bar_fullV + 8 * s, C::kTileBytes);
+#pragma unroll
+                            for (int c = 0; c < C::kChunks; ++c)
+                                tma_load_2d(dstV + c * C::kChunkBytes, &mapV, c * 64, (int)row, bar_fullV + 8 * s);
+                        }
+                    }
+                }
+            }
+            t = sg.t_end;
+        }
+        return;
+    }
+
+    // ===================================== consumer warps =====================================
+    const int g8 = lane >> 2, t4 = lane & 3;            // MMA fragment coordinates
     const int G = p.G;
-    const __nv_bfloat16* Q = reinterpret_cast<const __nv_bfloat16*>(p.q);
+    const float scale = p.scale_log2;
+    // ldmatrix lane addressing (byte offsets inside a 64-row x 128-byte swizzled chunk)
+    const int mi = lane >> 3, rr = lane & 7;
+    const int rowK = warp * 16 + (mi & 1) * 8 + rr, halfK = mi >> 1;       // K as A operand (non-transposed)
+    const int rowV = warp * 16 + (mi >> 1) * 8 + rr, halfV = mi & 1;       // V as A operand (transposed load)
+    const uint32_t offK = rowK * 128, offV = rowV * 128;
+    const uint32_t stage0 = smem_u32(stages);
 
     int64_t t = t0;
+    uint32_t it = 0;
     while (t < t1) {
-        // ---- locate the segment (b, g) of tile t and the end of this CTA's share of it
-        const int b = find_seq(tile_prefix, p.B, p.Hkv, t);
-        const int64_t tiles_b = tile_prefix[b + 1] - tile_prefix[b];
-        const int64_t seq_start = (int64_t)p.Hkv * tile_prefix[b];
-        const int g = (int)((t - seq_start) / tiles_b);
-        const int64_t seg_start = seq_start + (int64_t)g * tiles_b;
-        const int64_t seg_end = seg_start + tiles_b;
-        const int64_t t_end = seg_end < t1 ? seg_end : t1;
-        const int64_t S = p.len[b];
-        const int64_t nk = scan_keys(p, b);
-        const int seg = b * p.Hkv + g;
-
-        // ---- query rows of this group, pre-scaled to the exp2 domain
-        float qf[kMaxGroup][EPL];
+        const Segment sg = locate_segment(p, tile_prefix, t, t1);
+        // ---- Q^T fragments (B operand: k = d, n = head); heads >= G read as zero
+        uint32_t qb[C::kKSteps][2];
+        {
+            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+                reinterpret_cast<const __nv_bfloat16*>(p.q) + ((int64_t)sg.b * p.Hq + sg.g * G + g8) * D);
 #pragma unroll
-        for (int hh = 0; hh < kMaxGroup; ++hh) {
-            if (hh < G) {
-                const __nv_bfloat16* qrow = Q + ((int64_t)b * p.Hq + g * G + hh) * D + lane * EPL;
-#pragma unroll
-                for (int e = 0; e < EPL; ++e) qf[hh][e] = __bfloat162float(qrow[e]) * p.scale_log2;
-            } else {
-#pragma unroll
-                for (int e = 0; e < EPL; ++e) qf[hh][e] = 0.f;
+            for (int ks = 0; ks < C::kKSteps; ++ks) {
+                qb[ks][0] = g8 < G ? __ldg(qrow + ks * 8 + t4) : 0u;
+                qb[ks][1] = g8 < G ? __ldg(qrow + ks * 8 + 4 + t4) : 0u;
             }
         }
-        float m[kMaxGroup], l[kMaxGroup], acc[kMaxGroup][EPL];
+        float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f}, le[2] = {0.f, 0.f};   // l: rounded weights (normaliser), le: exact (lse)
+        float o[C::kKSteps][4];
 #pragma unroll
-        for (int hh = 0; hh < kMaxGroup; ++hh) {
-            m[hh] = -INFINITY; l[hh] = 0.f;
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) acc[hh][e] = 0.f;
-        }
+        for (int mb = 0; mb < C::kKSteps; ++mb) { o[mb][0] = o[mb][1] = o[mb][2] = o[mb][3] = 0.f; }
 
-        for (int64_t tt = t; tt < t_end; ++tt) {
-            const int64_t key0 = (tt - seg_start) * kTileKeys;
-            int64_t row_base;     // element offset of the tile's first row for this KV head
-            if (p.mode == kPaged) {
-                const int page = p.page_table[(int64_t)b * p.max_pages + key0 / p.page_size];
-                if (page < 0 || page >= p.num_pages) {
-                    if (threadIdx.x == 0) atomicCAS(p.status, 0, kErrBounds);
-                    continue;
+        for (int64_t tt = t; tt < sg.t_end; ++tt, ++it) {
+            const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+            const int64_t key0 = (tt - sg.seg_start) * kTileKeys;
+            const int64_t wkey0 = key0 + warp * 16;
+            const bool tile_full = (key0 + kTileKeys <= sg.nk) && !slack;
+            const bool any_valid = wkey0 < sg.nk;
+            const uint32_t sK = stage0 + s * C::kStageBytes, sV = sK + C::kTileBytes;
+
+            mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
+            uint32_t pb0 = 0, pb1 = 0;
+            float corr0 = 1.f, corr1 = 1.f;
+            if (any_valid) {
+                // ---- S^T = K . Q^T for this warp's 16 keys (two accumulator chains)
+                float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int ks = 0; ks < C::kKSteps; ++ks) {
+                    uint32_t a[4];
+                    const uint32_t c16 = (uint32_t)((ks & 3) * 2 + halfK);
+                    ldmatrix_x4(a, sK + (ks >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
+                    if (ks & 1) mma_bf16(sb, a, qb[ks][0], qb[ks][1]);
+                    else mma_bf16(sa, a, qb[ks][0], qb[ks][1]);
                 }
-                row_base = ((int64_t)page * p.Hkv + g) * p.page_size * D;
-            } else {
-                row_base = (((int64_t)b * p.Hkv + g) * p.rows_per_head + key0) * D;
-            }
-            for (int kk = warp; kk < kTileKeys; kk += NW) {
-                const int64_t key = key0 + kk;
-                if (key >= nk) break;
-                if (p.mode == kRing && p.cap != p.W && !ring_slot_live((int)key, S, p.n_sink, p.W, p.cap)) continue;
-                const uint32_t* krow = reinterpret_cast<const uint32_t*>(
-                    reinterpret_cast<const __nv_bfloat16*>(p.k) + row_base + (int64_t)kk * D) + lane * WPL;
-                const uint32_t* vrow = reinterpret_cast<const uint32_t*>(
-                    reinterpret_cast<const __nv_bfloat16*>(p.v) + row_base + (int64_t)kk * D) + lane * WPL;
-                uint32_t kw[WPL], vw[WPL];
+                float sc[4];
 #pragma unroll
-                for (int w = 0; w < WPL; ++w) { kw[w] = __ldg(krow + w); vw[w] = __ldg(vrow + w); }
-                float s[kMaxGroup];
-#pragma unroll
-                for (int hh = 0; hh < kMaxGroup; ++hh) {
-                    float a = 0.f;
-#pragma unroll
-                    for (int w = 0; w < WPL; ++w) {
-                        a = fmaf(qf[hh][2 * w], bf16lo(kw[w]), a);
-                        a = fmaf(qf[hh][2 * w + 1], bf16hi(kw[w]), a);
+                for (int i = 0; i < 4; ++i) sc[i] = (sa[i] + sb[i]) * scale;
+                if (!tile_full) {
+                    const int64_t ka = wkey0 + g8, kb = ka + 8;
+                    bool va = ka < sg.nk, vb = kb < sg.nk;
+                    if (slack) {
+                        va = va && ring_slot_live((int)ka, sg.S, p.n_sink, p.W, p.cap);
+                        vb = vb && ring_slot_live((int)kb, sg.S, p.n_sink, p.W, p.cap);
                     }
-                    s[hh] = a;
+                    if (!va) { sc[0] = -INFINITY; sc[1] = -INFINITY; }
+                    if (!vb) { sc[2] = -INFINITY; sc[3] = -INFINITY; }
                 }
+                // ---- online softmax; this thread holds heads 2*t4, 2*t4+1 for keys g8 and g8+8
+                float mx0 = fmaxf(sc[0], sc[2]), mx1 = fmaxf(sc[1], sc[3]);
 #pragma unroll
-                for (int off = 16; off > 0; off >>= 1)
+                for (int off = 4; off <= 16; off <<= 1) {
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+                }
+                const float mn0 = fmaxf(m[0], mx0), mn1 = fmaxf(m[1], mx1);
+                const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
+                corr0 = exp2f(m[0] - mu0);
+                corr1 = exp2f(m[1] - mu1);
+                m[0] = mn0; m[1] = mn1;
+                const float p0 = exp2f(sc[0] - mu0), p1 = exp2f(sc[1] - mu1), p2 = exp2f(sc[2] - mu0), p3 = exp2f(sc[3] - mu1);
+                const uint32_t pa = pack_bf16x2(p0, p1);             // key g8   : heads 2t4, 2t4+1
+                const uint32_t pc = pack_bf16x2(p2, p3);             // key g8+8
+                le[0] = le[0] * corr0 + p0 + p2;
+                le[1] = le[1] * corr1 + p1 + p3;
+                l[0] = l[0] * corr0 + bf16lo(pa) + bf16lo(pc);      // sums of the rounded weights the MMA will use
+                l[1] = l[1] * corr1 + bf16hi(pa) + bf16hi(pc);
+                pb0 = movmatrix_trans(pa);                           // P^T as B operand: k = key, n = head
+                pb1 = movmatrix_trans(pc);
 #pragma unroll
-                    for (int hh = 0; hh < kMaxGroup; ++hh) s[hh] += __shfl_xor_sync(0xffffffffu, s[hh], off);
-#pragma unroll
-                for (int hh = 0; hh < kMaxGroup; ++hh) {
-                    const float mn = fmaxf(m[hh], s[hh]);
-                    const float corr = exp2f(m[hh] - mn);      // exp2(-inf) = 0 on the first key
-                    const float pj = exp2f(s[hh] - mn);
-                    m[hh] = mn;
-                    l[hh] = l[hh] * corr + pj;
-#pragma unroll
-                    for (int w = 0; w < WPL; ++w) {
-                        acc[hh][2 * w] = fmaf(pj, bf16lo(vw[w]), acc[hh][2 * w] * corr);
-                        acc[hh][2 * w + 1] = fmaf(pj, bf16hi(vw[w]), acc[hh][2 * w + 1] * corr);
-                    }
+                for (int mb = 0; mb < C::kKSteps; ++mb) {
+                    o[mb][0] *= corr0; o[mb][1] *= corr1; o[mb][2] *= corr0; o[mb][3] *= corr1;
                 }
             }
+            mbar_wait(bar_fullV + 8 * s, ph, abort_flag, p.status);
+            if (any_valid) {
+                if (wkey0 + 16 > sg.nk) {
+                    // rows past the sequence end were never written: they may hold NaN/Inf bit patterns,
+                    // and 0 * NaN would poison the accumulators. Zero them in shared memory.
+                    const int first_bad = (int)(sg.nk - wkey0);
+                    for (int idx = lane; idx < (16 - first_bad) * C::kChunks * 8; idx += 32) {
+                        const int r = first_bad + idx / (C::kChunks * 8), rem = idx % (C::kChunks * 8);
+                        const uint32_t addr = sV + (rem >> 3) * C::kChunkBytes + (warp * 16 + r) * 128 + ((rem & 7) << 4);
+                        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                }
+                // ---- O^T += V^T . P^T
+#pragma unroll
+                for (int mb = 0; mb < C::kKSteps; ++mb) {
+                    uint32_t a[4];
+                    const uint32_t c16 = (uint32_t)((mb & 3) * 2 + halfV);
+                    ldmatrix_x4_trans(a, sV + (mb >> 2) * C::kChunkBytes + offV + ((c16 ^ (uint32_t)rr) << 4));
+                    mma_bf16(o[mb], a, pb0, pb1);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty + 8 * s);
         }
 
         // ---- merge the four warps' states and emit the partial of (this CTA, this segment)
-        __syncthreads();
 #pragma unroll
-        for (int hh = 0; hh < kMaxGroup; ++hh) {
-            if (lane == 0) { sm_m[warp * kMaxGroup + hh] = m[hh]; sm_l[warp * kMaxGroup + hh] = l[hh]; }
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) sm_acc[(warp * kMaxGroup + hh) * D + lane * EPL + e] = acc[hh][e];
+        for (int off = 4; off <= 16; off <<= 1) {
+            l[0] += __shfl_xor_sync(0xffffffffu, l[0], off);
+            l[1] += __shfl_xor_sync(0xffffffffu, l[1], off);
+            le[0] += __shfl_xor_sync(0xffffffffu, le[0], off);
+            le[1] += __shfl_xor_sync(0xffffffffu, le[1], off);
         }
-        __syncthreads();
-        const int64_t pidx = (int64_t)blockIdx.x + seg;
-        for (int idx = threadIdx.x; idx < G * D; idx += blockDim.x) {
-            const int hh = idx / D, d = idx % D;
+        consumer_barrier();                                   // scratch / sm_m free (previous segment fully written out)
+        if (g8 == 0) {
+            sm_m[warp * kMaxGroup + 2 * t4] = m[0]; sm_m[warp * kMaxGroup + 2 * t4 + 1] = m[1];
+            sm_l[warp * kMaxGroup + 2 * t4] = l[0]; sm_l[warp * kMaxGroup + 2 * t4 + 1] = l[1];
+            sm_le[warp * kMaxGroup + 2 * t4] = le[0]; sm_le[warp * kMaxGroup + 2 * t4 + 1] = le[1];
+        }
+        consumer_barrier();
+        float f[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int h = 2 * t4 + i;
             float M = -INFINITY;
 #pragma unroll
-            for (int w = 0; w < NW; ++w) M = fmaxf(M, sm_m[w * kMaxGroup + hh]);
-            float L = 0.f, o = 0.f;
+            for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm_m[w * kMaxGroup + h]);
+            float L = 0.f, Le = 0.f;
             if (M > -INFINITY) {
 #pragma unroll
-                for (int w = 0; w < NW; ++w) {
-                    const float sc = exp2f(sm_m[w * kMaxGroup + hh] - M);
-                    L += sm_l[w * kMaxGroup + hh] * sc;
-                    o += sm_acc[(w * kMaxGroup + hh) * D + d] * sc;
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    const float e = exp2f(sm_m[w * kMaxGroup + h] - M);
+                    L += sm_l[w * kMaxGroup + h] * e;
+                    Le += sm_le[w * kMaxGroup + h] * e;
                 }
             }
-            p.part_o[(pidx * G + hh) * D + d] = L > 0.f ? o / L : 0.f;
-            if (d == 0) p.part_lse[pidx * G + hh] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+            f[i] = (L > 0.f && m[i] > -INFINITY) ? exp2f(m[i] - M) / L : 0.f;
+            if (warp == 0 && g8 == 0 && h < G)
+                p.part_lse[((int64_t)blockIdx.x + sg.seg) * G + h] = Le > 0.f ? (M + log2f(Le)) * kLn2 : -INFINITY;
         }
-        t = t_end;
+        const int64_t pidx = (int64_t)blockIdx.x + sg.seg;
+        constexpr int kPasses = D / 128;                       // 128 columns of d per pass through the scratch
+#pragma unroll
+        for (int pass = 0; pass < kPasses; ++pass) {
+            if (pass > 0) consumer_barrier();
+#pragma unroll
+            for (int mbl = 0; mbl < 8; ++mbl) {
+                const int mb = pass * 8 + mbl;
+                float* row0 = scratch + (warp * kMaxGroup + 2 * t4) * kScratchRow + mbl * 16 + g8;
+                float* row1 = row0 + kScratchRow;
+                row0[0] = o[mb][0] * f[0]; row1[0] = o[mb][1] * f[1];
+                row0[8] = o[mb][2] * f[0]; row1[8] = o[mb][3] * f[1];
+            }
+            consumer_barrier();
+            const int tid = threadIdx.x;                       // 0..127
+            for (int idx = tid; idx < G * 128; idx += 128) {
+                const int h = idx >> 7, dd = idx & 127;
+                float acc = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) acc += scratch[(w * kMaxGroup + h) * kScratchRow + dd];
+                p.part_o[(pidx * G + h) * D + pass * 128 + dd] = acc;
+            }
+        }
+        t = sg.t_end;
     }
 }
 
 // ---------------------------------------------------------------------------------------------
-// Combine: one block per segment (b, g); merges the segment's partials by log-sum-exp.
+// Combine: one block per (segment, query head); merges that head's partials by log-sum-exp:
+// lse = logsumexp_s(lse_s), out = sum_s exp(lse_s - lse) * o_s. Row groups of the block read
+// different partials with float4 loads so that all loads of a thread are in flight at once.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128) attn_combine(AttnParams p, int C) {
+constexpr int kCombineThreads = 512;
+
+__global__ void __launch_bounds__(kCombineThreads) attn_combine(AttnParams p, int launched_ctas) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    int64_t* tile_prefix = reinterpret_cast<int64_t*>(smem_raw);     // [B + 1]
-    float* w_sm = reinterpret_cast<float*>(tile_prefix + (p.B + 1)); // [kMaxGroup][np]  (np <= C)
-    __shared__ float inv_sum[kMaxGroup], lse_sm[kMaxGroup];
+    int64_t* tile_prefix = reinterpret_cast<int64_t*>(smem_raw);            // [B + 1]
+    float* w_sm = reinterpret_cast<float*>(tile_prefix + (p.B + 1));        // [np]
+    float* red = w_sm + launched_ctas;                                      // [groups][D] (16-byte aligned below)
+    red = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(red) + 15) & ~(uintptr_t)15);
+    __shared__ float warp_red[kCombineThreads / 32];
+    __shared__ float bc[2];
 
     build_tile_prefix(p, tile_prefix);
-    const int seg = blockIdx.x, b = seg / p.Hkv, g = seg % p.Hkv;
+    const int seg = blockIdx.x, hh = blockIdx.y, b = seg / p.Hkv, g = seg % p.Hkv;
     const int G = p.G, D = p.D;
     const int64_t n = (int64_t)p.Hkv * tile_prefix[p.B];
+    const int C = effective_ctas(launched_ctas, n);
     const int64_t tiles_b = tile_prefix[b + 1] - tile_prefix[b];
-    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + g * G) * D;
+    const int64_t head = (int64_t)b * p.Hq + g * G + hh;
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + head * D;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tiles_b == 0) {                       // empty sequence: out = 0, lse = -inf
-        for (int idx = threadIdx.x; idx < G * D; idx += blockDim.x) out[idx] = __float2bfloat16(0.f);
-        if (p.lse && threadIdx.x < G) p.lse[(int64_t)b * p.Hq + g * G + threadIdx.x] = -INFINITY;
+        for (int d = tid; d < D; d += blockDim.x) out[d] = __float2bfloat16(0.f);
+        if (p.lse && tid == 0) p.lse[head] = -INFINITY;
         return;
     }
     const int64_t seg_start = (int64_t)p.Hkv * tile_prefix[b] + (int64_t)g * tiles_b;
     const int c_first = tile_owner(seg_start, n, C), c_last = tile_owner(seg_start + tiles_b - 1, n, C);
     const int np = c_last - c_first + 1;
     const int64_t pbase = (int64_t)c_first + seg;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    for (int hh = warp; hh < G; hh += 4) {
-        float M = -INFINITY;
-        for (int i = lane; i < np; i += 32) M = fmaxf(M, p.part_lse[(pbase + i) * G + hh]);
+    // ---- M = max_s lse_s, then weights and their sum
+    float M = -INFINITY;
+    for (int i = tid; i < np; i += blockDim.x) M = fmaxf(M, p.part_lse[(pbase + i) * G + hh]);
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
-        float sum = 0.f;
-        for (int i = lane; i < np; i += 32) {
-            const float x = p.part_lse[(pbase + i) * G + hh];
-            const float w = (M > -INFINITY) ? __expf(x - M) : 0.f;
-            w_sm[hh * np + i] = w;
-            sum += w;
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-        if (lane == 0) {
-            inv_sum[hh] = sum > 0.f ? 1.f / sum : 0.f;
-            lse_sm[hh] = sum > 0.f ? M + __logf(sum) : -INFINITY;
-        }
+    for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+    if (lane == 0) warp_red[warp] = M;
+    __syncthreads();
+    if (tid == 0) {
+        float x = warp_red[0];
+        for (int w = 1; w < kCombineThreads / 32; ++w) x = fmaxf(x, warp_red[w]);
+        bc[0] = x;
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < G * D; idx += blockDim.x) {
-        const int hh = idx / D, d = idx % D;
-        float o = 0.f;
-        for (int i = 0; i < np; ++i) o = fmaf(w_sm[hh * np + i], p.part_o[((pbase + i) * G + hh) * D + d], o);
-        out[idx] = __float2bfloat16(o * inv_sum[hh]);
+    M = bc[0];
+    float sum = 0.f;
+    for (int i = tid; i < np; i += blockDim.x) {
+        const float w = (M > -INFINITY) ? __expf(p.part_lse[(pbase + i) * G + hh] - M) : 0.f;
+        w_sm[i] = w;
+        sum += w;
     }
-    if (p.lse && threadIdx.x < G) p.lse[(int64_t)b * p.Hq + g * G + threadIdx.x] = lse_sm[threadIdx.x];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    if (lane == 0) warp_red[warp] = sum;
+    __syncthreads();
+    if (tid == 0) {
+        float x = 0.f;
+        for (int w = 0; w < kCombineThreads / 32; ++w) x += warp_red[w];
+        bc[1] = x;
+        if (p.lse) p.lse[head] = x > 0.f ? M + __logf(x) : -INFINITY;
+    }
+    __syncthreads();
+    sum = bc[1];
+    const float inv = sum > 0.f ? 1.f / sum : 0.f;
+
+    // ---- weighted sum of the partial rows: thread = (row group, float4 column)
+    const int vec = D / 4, groups = kCombineThreads / vec;
+    const int grp = tid / vec, col = tid % vec;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const float4* rows = reinterpret_cast<const float4*>(p.part_o);
+#pragma unroll 4
+    for (int i = grp; i < np; i += groups) {
+        const float w = w_sm[i];
+        const float4 x = rows[((pbase + i) * G + hh) * vec + col];
+        acc.x = fmaf(w, x.x, acc.x); acc.y = fmaf(w, x.y, acc.y); acc.z = fmaf(w, x.z, acc.z); acc.w = fmaf(w, x.w, acc.w);
+    }
+    reinterpret_cast<float4*>(red)[grp * vec + col] = acc;
+    __syncthreads();
+    for (int d = tid; d < D; d += blockDim.x) {
+        float o = 0.f;
+        for (int gi = 0; gi < groups; ++gi) o += red[gi * D + d];
+        out[d] = __float2bfloat16(o * inv);
+    }
+}
+
+// ---- host side: tensor maps and launch --------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(f);
+    }();
+    return fn;
+}
+
+// 2-D view [rows][D] of a K or V tensor; box = 64 rows x 64 elements (128 bytes), 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int D) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTileKeys};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D>
+size_t partial_smem_bytes(int B) {
+    using C = Cfg<D>;
+    return 1024 + (size_t)C::kStages * C::kStageBytes + sizeof(float) * (kConsumerWarps * kMaxGroup * kScratchRow + 3 * kConsumerWarps * kMaxGroup) +
+           sizeof(uint64_t) * 3 * C::kStages + 2 * sizeof(int) + sizeof(int64_t) * (B + 1) + 16;
+}
+
+template <int D>
+cudaError_t launch_partial(const CUtensorMap& mk, const CUtensorMap& mv, const AttnParams& p, cudaStream_t st) {
+    const size_t smem = partial_smem_bytes<D>(p.B);
+    static bool attr_set[64] = {};          // per device: the opt-in to > 48 KB of dynamic shared memory
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(attn_partial_tma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    attn_partial_tma<D><<<p.num_ctas, kThreads, smem, st>>>(mk, mv, p);
+    return cudaGetLastError();
 }
 
 }  // namespace
 
+int64_t attention_rows(const AttnParams& p) {
+    if (p.mode == kPaged) return (int64_t)p.num_pages * p.Hkv * p.page_size;
+    return (int64_t)p.B * p.Hkv * p.rows_per_head;
+}
+
 cudaError_t launch_attention(const AttnParams& p, cudaStream_t st) {
-    const int C = p.num_ctas;
-    const size_t prefix_bytes = sizeof(int64_t) * (p.B + 1);
-    const size_t sm_partial = prefix_bytes + sizeof(float) * (4 * kMaxGroup * 2 + 4 * kMaxGroup * p.D);
-    cudaError_t e;
-    if (p.D == 128) {
-        attn_partial_simple<128><<<C, 128, sm_partial, st>>>(p);
-    } else {
-        attn_partial_simple<256><<<C, 128, sm_partial, st>>>(p);
-    }
+    const int64_t rows = attention_rows(p);
+    CUtensorMap mk, mv;
+    if (!make_map(&mk, p.k, rows, p.D) || !make_map(&mv, p.v, rows, p.D)) return cudaErrorInvalidValue;
+    cudaError_t e = p.D == 128 ? launch_partial<128>(mk, mv, p, st) : launch_partial<256>(mk, mv, p, st);
     count_launch(1);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    const size_t sm_combine = prefix_bytes + sizeof(float) * kMaxGroup * C;
-    attn_combine<<<p.B * p.Hkv, 128, sm_combine, st>>>(p, C);
+    if (e != cudaSuccess) return e;
+    const size_t sm_combine = sizeof(int64_t) * (p.B + 1) + sizeof(float) * p.num_ctas + 16 + sizeof(float) * 4 * kCombineThreads;
+    attn_combine<<<dim3(p.B * p.Hkv, p.G), kCombineThreads, sm_combine, st>>>(p, p.num_ctas);
     count_launch(1);
     return cudaGetLastError();
 }

@@ -46,6 +46,12 @@ __device__ __forceinline__ void build_tile_prefix(const AttnParams& p, int64_t* 
     __syncthreads();
 }
 
+// CTAs that take part: never more than there are tiles, so every participating CTA owns >= 1 tile
+// and the CTAs touching a segment are exactly tile_owner(first tile) .. tile_owner(last tile).
+__device__ __forceinline__ int effective_ctas(int launched, int64_t n) {
+    return n < (int64_t)launched ? (int)n : launched;
+}
+
 __device__ __forceinline__ int64_t cta_range_start(int c, int64_t n, int C) {
     return ((int64_t)c * n) / C;   // c <= kMaxCtas and n < 2^40: no overflow
 }

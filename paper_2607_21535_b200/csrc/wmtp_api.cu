@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <climits>
 #include <cstring>
 
 #include "wmtp_internal.h"
@@ -32,6 +33,7 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 wmtp_status check_shape(int batch, int Hkv, int D) {
     if (batch < 1 || Hkv < 1) return fail(WMTP_ERR_INVALID_ARG, "batch=%d, Hkv=%d must be positive", batch, Hkv);
     if (batch > kMaxBatch) return fail(WMTP_ERR_UNSUPPORTED, "batch=%d exceeds %d", batch, kMaxBatch);
+    if ((int64_t)batch * Hkv > kMaxSegments) return fail(WMTP_ERR_UNSUPPORTED, "batch*Hkv=%lld exceeds %d", (long long)batch * Hkv, kMaxSegments);
     if (D != 128 && D != 256) return fail(WMTP_ERR_UNSUPPORTED, "head_dim=%d (supported: 128, 256)", D);
     return WMTP_OK;
 }
@@ -42,6 +44,8 @@ wmtp_status check_ring(const wmtp_ring* r) {
     if (r->n_sink < 0 || r->W < 1 || r->cap < r->W)
         return fail(WMTP_ERR_INVALID_ARG, "ring needs n_sink >= 0, W >= 1, cap >= W (n_sink=%d W=%d cap=%d)", r->n_sink, r->W, r->cap);
     if ((int64_t)r->n_sink + r->cap > (1 << 30)) return fail(WMTP_ERR_INVALID_ARG, "ring of %lld slots is too large", (long long)r->n_sink + r->cap);
+    if ((int64_t)r->batch * r->Hkv * ((int64_t)r->n_sink + r->cap) > INT32_MAX)
+        return fail(WMTP_ERR_UNSUPPORTED, "ring has more than 2^31 - 1 rows in total");
     if (!r->k || !r->v || !r->slot_pos || !r->len) return fail(WMTP_ERR_INVALID_ARG, "ring has a NULL pointer");
     if (!aligned(r->k, 16) || !aligned(r->v, 16) || !aligned(r->slot_pos, 4) || !aligned(r->len, 8))
         return fail(WMTP_ERR_INVALID_ARG, "ring pointers must be 16-byte (k, v), 4-byte (slot_pos), 8-byte (len) aligned");
@@ -55,6 +59,8 @@ wmtp_status check_kv(const wmtp_kv* kv) {
     if (!aligned(kv->k, 16) || !aligned(kv->v, 16) || !aligned(kv->len, 8))
         return fail(WMTP_ERR_INVALID_ARG, "kv pointers must be 16-byte (k, v), 8-byte (len) aligned");
     if (kv->S_cap < 1) return fail(WMTP_ERR_INVALID_ARG, "S_cap=%lld must be positive", (long long)kv->S_cap);
+    const int64_t kv_rows = kv->page_table ? (int64_t)kv->num_pages * kv->Hkv * kv->page_size : (int64_t)kv->batch * kv->Hkv * kv->S_cap;
+    if (kv_rows > INT32_MAX) return fail(WMTP_ERR_UNSUPPORTED, "kv has more than 2^31 - 1 rows in total");
     if (kv->page_table) {
         if (kv->page_size != kTileKeys) return fail(WMTP_ERR_UNSUPPORTED, "page_size=%d (supported: %d)", kv->page_size, kTileKeys);
         if (kv->max_pages < 1 || kv->num_pages < 1) return fail(WMTP_ERR_INVALID_ARG, "max_pages, num_pages must be positive");
@@ -190,7 +196,7 @@ WorkspaceLayout workspace_layout(int batch, int Hq, int Hkv, int D) {
     WorkspaceLayout L;
     const size_t G = (size_t)(Hq / Hkv), nseg = (size_t)batch * Hkv, np = kMaxCtas + nseg;
     L.counters_off = 256;
-    L.part_lse_off = L.counters_off + round_up(nseg * sizeof(int), 256);
+    L.part_lse_off = kWorkspaceZeroBytes;
     L.part_o_off = L.part_lse_off + round_up(np * G * sizeof(float), 256);
     L.total = L.part_o_off + round_up(np * G * D * sizeof(float), 256);
     return L;
@@ -232,8 +238,9 @@ size_t wmtp_workspace_bytes(int batch, int Hq, int Hkv, int D) {
 
 wmtp_status wmtp_workspace_init(void* workspace, size_t ws_bytes, void* stream) {
     if (!workspace || !aligned(workspace, 256)) return fail(WMTP_ERR_WORKSPACE, "workspace is NULL or not 256-byte aligned");
-    if (ws_bytes < 512) return fail(WMTP_ERR_WORKSPACE, "workspace of %zu bytes is too small", ws_bytes);
-    cudaError_t e = cudaMemsetAsync(workspace, 0, ws_bytes, (cudaStream_t)stream);
+    if (ws_bytes < kWorkspaceZeroBytes) return fail(WMTP_ERR_WORKSPACE, "workspace of %zu bytes is too small", ws_bytes);
+    // only the status word and the completion counters must start at zero; partials are always written before read
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceZeroBytes, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(e, "workspace memset");
     return WMTP_OK;
 }

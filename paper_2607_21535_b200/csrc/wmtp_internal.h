@@ -12,12 +12,14 @@ constexpr int kTileKeys = 64;       // keys per K/V tile; equals the page size o
 constexpr int kMaxCtas = 1024;      // upper bound on attention CTAs, sizes the partial buffers
 constexpr int kMaxBatch = 1024;     // sequences per call (prefix table lives in shared memory)
 constexpr int kMaxGroup = 8;        // query heads per KV head
+constexpr int kMaxSegments = 16384; // batch * Hkv per call
+constexpr size_t kWorkspaceZeroBytes = 256 + sizeof(int) * kMaxSegments;   // header + counters
 
 enum KvMode : int { kContiguous = 0, kPaged = 1, kRing = 2 };
 
 // Workspace layout (all offsets from a 256-byte aligned base):
 //   [0, 256)            header: int status word at offset 0
-//   counters            int [batch * Hkv], padded to 256 bytes
+//   counters            int [kMaxSegments] (fixed size, so that initialisation needs no shape)
 //   part_lse            float [kMaxCtas + batch * Hkv][G]
 //   part_o              float [kMaxCtas + batch * Hkv][G][D]
 struct WorkspaceLayout {
