@@ -172,6 +172,30 @@ void    wmtp_set_max_ctas(int max_ctas);
 /* Number of kernels this library has launched in this process (all threads). */
 int64_t wmtp_launch_count(void);
 
+/* ---- for callers that cannot allocate device memory --------------------------------------------- */
+
+/*
+ * (The paper has no counterpart to this entry point; it exists for integration.)
+ * Windowed draft attention, same result as wmtp_draft_attn_windowed, for callers that cannot give the
+ * library a workspace because they cannot allocate device memory themselves: plug-ins inside a runtime
+ * that owns the allocator, processes whose device-memory budget is frozen at start-up, loops that must
+ * not allocate once they are running. The split-KV scratch is a fixed array inside the library
+ * (about 1.5 MiB, held by every GPU that loads the library until the process exits); the call, and the
+ * library on its behalf, performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *   - Limits: batch * Hkv <= 32, Hq / Hkv <= 8, D in {128, 256}; more is rejected with
+ *     WMTP_ERR_CAPACITY / WMTP_ERR_UNSUPPORTED and nothing is launched. At most 160 CTAs are used.
+ *   - The first call on each device looks up the array's device address (a one-time set-up, with that
+ *     device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the call
+ *     clears the words that must start at zero. Two calls whose GPU work can overlap (different
+ *     streams without ordering) race on it: order them on one stream or with events.
+ *   - The sticky device status lives in the array too and is cleared at the start of each call; it is
+ *     not reported (the windowed path has no page table whose ids could be out of range).
+ * Arguments as wmtp_draft_attn_windowed, without workspace.
+ */
+wmtp_status wmtp_draft_attn_windowed_noalloc(const void* q, int Hq, const wmtp_ring* ring, float sm_scale,
+                                             void* out, float* lse, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -64,6 +64,7 @@ _SIGNATURES = {
                                               c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "wmtp_draft_loop_full_host": (c_int, [POINTER(wmtp_kv), c_int, c_void_p, c_int, c_void_p, c_void_p, c_float,
                                           c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "wmtp_draft_attn_windowed_noalloc": (c_int, [c_void_p, c_int, POINTER(wmtp_ring), c_float, c_void_p, c_void_p, c_void_p]),
     "wmtp_set_max_ctas": (None, [c_int]),
     "wmtp_launch_count": (c_int64, []),
 }
@@ -251,6 +252,15 @@ def wmtp_draft_loop_full_host(kv: KV, q_host, k_new_host, v_new_host, out_host, 
     _check(lib().wmtp_draft_loop_full_host(byref(kv.desc), gamma, _ptr(q_host), Hq, _ptr(k_new_host), _ptr(v_new_host),
                                            sm_scale, _ptr(out_host), _ptr(lse_host), _ptr(stage), ws.ptr, ws.nbytes,
                                            _stream(stream)))
+
+
+def wmtp_draft_attn_windowed_noalloc(q, ring: Ring, out, lse=None, sm_scale: float = 0.0, stream=None) -> None:
+    """Windowed attention on the library's built-in scratch, for callers that cannot allocate a workspace
+    (they do not own the device allocator, or may not allocate once running). Calls sharing a device must
+    not overlap on the GPU; the first call on a device should be made outside stream capture."""
+    Hq = q.shape[-2]
+    _check(lib().wmtp_draft_attn_windowed_noalloc(_ptr(q), Hq, byref(ring.desc), sm_scale, _ptr(out), _ptr(lse),
+                                                  _stream(stream)))
 
 
 def wmtp_set_max_ctas(n: int) -> None:

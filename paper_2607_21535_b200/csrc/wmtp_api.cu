@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <climits>
 #include <cstring>
+#include <mutex>
 
 #include "wmtp_internal.h"
 
@@ -393,5 +394,85 @@ wmtp_status wmtp_draft_loop_full_host(const wmtp_kv* kv, int gamma, const void* 
 void wmtp_set_max_ctas(int max_ctas) { g_max_ctas.store(max_ctas < 0 ? 0 : max_ctas); }
 
 int64_t wmtp_launch_count(void) { return g_launches.load(); }
+
+// ---- allocation-free windowed attention ---------------------------------------------------------
+// Some callers cannot hand the library a workspace because they cannot call cudaMalloc at all: code
+// running inside a framework that owns the device allocator, a process whose memory budget is fixed
+// before start-up, a real-time loop where an allocation is forbidden after initialisation. For them
+// the split-KV scratch of the windowed attention lives in this file-scope device array instead of a
+// caller buffer. Every GPU that loads the library holds it until the process exits.
+namespace {
+constexpr int kStaticMaxCtas = 160;        // CTAs (KV splits) the static scratch has room for
+constexpr int kStaticMaxSegments = 32;     // batch * Hkv
+constexpr size_t kStaticCountersOff = 256;
+constexpr size_t kStaticPartLseOff = kStaticCountersOff + 256;                                     // 32 counters, padded
+constexpr size_t kStaticPartOOff = kStaticPartLseOff + (kStaticMaxCtas + kStaticMaxSegments) * kMaxGroup * sizeof(float);
+constexpr size_t kStaticBytes = kStaticPartOOff + (size_t)(kStaticMaxCtas + kStaticMaxSegments) * kMaxGroup * 256 * sizeof(float);
+static_assert(kStaticPartLseOff % 256 == 0 && kStaticPartOOff % 256 == 0, "static scratch regions must stay 256-byte aligned");
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];   // ~1.5 MiB
+
+// In host code the array's name is only a handle; the device address must be asked for, once per device.
+std::mutex g_static_mu;
+void* g_static_ptr[64] = {};
+
+wmtp_status static_scratch(void** ptr) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= 64) return fail(WMTP_ERR_UNSUPPORTED, "device ordinal %d is outside [0, 64)", dev);
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* a = nullptr;
+        e = cudaGetSymbolAddress(&a, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(static scratch)");
+        g_static_ptr[dev] = a;
+    }
+    *ptr = g_static_ptr[dev];
+    return WMTP_OK;
+}
+}  // namespace
+
+wmtp_status wmtp_draft_attn_windowed_noalloc(const void* q, int Hq, const wmtp_ring* ring, float sm_scale, void* out,
+                                             float* lse, void* stream) {
+    if (wmtp_status s = check_ring(ring)) return s;
+    if (!q || !out) return fail(WMTP_ERR_INVALID_ARG, "q or out is NULL");
+    if (!aligned(q, 16) || !aligned(out, 16)) return fail(WMTP_ERR_INVALID_ARG, "q and out must be 16-byte aligned");
+    if (lse && !aligned(lse, 4)) return fail(WMTP_ERR_INVALID_ARG, "lse must be 4-byte aligned");
+    if (Hq < 1 || Hq % ring->Hkv != 0) return fail(WMTP_ERR_INVALID_ARG, "Hq=%d must be a positive multiple of Hkv=%d", Hq, ring->Hkv);
+    if (Hq / ring->Hkv > kMaxGroup) return fail(WMTP_ERR_UNSUPPORTED, "Hq/Hkv=%d exceeds %d", Hq / ring->Hkv, kMaxGroup);
+    const int nseg = ring->batch * ring->Hkv;
+    if (nseg > kStaticMaxSegments)
+        return fail(WMTP_ERR_CAPACITY, "batch*Hkv=%d exceeds the %d (sequence, KV head) pairs the built-in scratch holds; "
+                    "use wmtp_draft_attn_windowed with a workspace", nseg, kStaticMaxSegments);
+    void* base_v = nullptr;
+    if (wmtp_status s = static_scratch(&base_v)) return s;
+    char* base = static_cast<char*>(base_v);
+    cudaStream_t st = (cudaStream_t)stream;
+    // status word and this call's counters must start at zero; the array keeps the previous call's contents
+    cudaError_t e = cudaMemsetAsync(base, 0, kStaticCountersOff + sizeof(int) * nseg, st);
+    if (e != cudaSuccess) return cuda_fail(e, "clearing the static scratch header");
+
+    AttnParams p{};
+    p.q = q; p.out = out; p.lse = lse;
+    p.status = reinterpret_cast<int*>(base);
+    p.counters = reinterpret_cast<int*>(base + kStaticCountersOff);
+    p.part_lse = reinterpret_cast<float*>(base + kStaticPartLseOff);
+    p.part_o = reinterpret_cast<float*>(base + kStaticPartOOff);
+    p.B = ring->batch; p.Hq = Hq; p.Hkv = ring->Hkv; p.D = ring->D; p.G = Hq / ring->Hkv;
+    const float sc = sm_scale > 0.f ? sm_scale : 1.0f / std::sqrt((float)ring->D);
+    p.scale_log2 = sc * 1.4426950408889634f;
+    p.k = ring->k; p.v = ring->v; p.page_table = nullptr; p.len = ring->len;
+    p.mode = kRing;
+    p.rows_per_head = (int64_t)ring->n_sink + ring->cap;
+    p.n_sink = ring->n_sink; p.W = ring->W; p.cap = ring->cap;
+    const int64_t tiles = (p.rows_per_head + kTileKeys - 1) / kTileKeys * ring->batch * ring->Hkv;
+    p.num_ctas = pick_ctas(tiles);
+    if (p.num_ctas <= 0) return fail(WMTP_ERR_CUDA, "no CUDA device available");
+    if (p.num_ctas > kStaticMaxCtas) p.num_ctas = kStaticMaxCtas;
+    e = launch_attention(p, st);
+    if (e != cudaSuccess) return cuda_fail(e, "windowed attention launch (static scratch)");
+    return WMTP_OK;
+}
 
 }  // extern "C"
