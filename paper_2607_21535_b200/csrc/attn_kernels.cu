@@ -1,4 +1,5 @@
-// Split-KV decode attention for the draft head: TMA-fed partial kernel + log-sum-exp combine.
+// Split-KV decode attention for the draft head: one TMA-fed kernel per draft step that appends the
+// step's K/V, computes split-KV partials and merges them by log-sum-exp.
 //
 // The operation is softmax attention of one query per head over a key set (Section 4
 // "Mechanism"; Appendix D: o = sum_j p_j v_j): the ring's live slots for the windowed draft,
@@ -14,7 +15,13 @@
 //     O^T[d, head] += V^T[d, key] . P^T[key, head] accumulates in registers. The 8-row problem
 //     is far too small for tcgen05 (M >= 64); mma.sync.m16n8k16 needs ~3% of tensor peak here.
 //   * every K/V byte is read once from HBM and once from shared memory, shared by all heads
-//     of the group.
+//     of the group;
+//   * the launch is cooperative (all CTAs co-resident): after publishing its partial a CTA waits,
+//     with a bounded spin, for the other contributors of its segment and reduces its slice of the
+//     output, so the merge needs no second launch and no single CTA serialises it;
+//   * a draft step's append (Appendix A, RING; the KV write of a draft forward) is fused: the warp
+//     that owns the new token's row patches the tile in shared memory from k_new / v_new and stores
+//     the row to the KV store; the last CTA of the grid advances len[].
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -31,6 +38,9 @@ constexpr int kConsumerWarps = 4;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr uint32_t kSpinLimit = 1u << 22;       // bounded mbarrier waits
 constexpr int kScratchRow = 132;                // floats per (warp, head) row of the merge scratch (128 + pad)
+// scratch holds either the warp merge ([4][8][kScratchRow]) or the combine's weights, inverses and reduction buffer
+constexpr int kScratchFloats = (kConsumerWarps * kMaxGroup * kScratchRow) > (kMaxGroup * kMaxCtas + 8 + 4 * 128)
+                                   ? (kConsumerWarps * kMaxGroup * kScratchRow) : (kMaxGroup * kMaxCtas + 8 + 4 * 128);
 
 template <int D>
 struct Cfg {
@@ -108,48 +118,222 @@ __device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u <
 __device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 __device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
+// Bounded spin on a global counter written by other CTAs of this (cooperative) launch.
+__device__ __forceinline__ void wait_counter(const int* ctr, int target, volatile int* abort_flag, int* status) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+        if (v >= target) return;
+        if ((i & 255u) == 255u && *abort_flag) return;
+        __nanosleep(32);
+    }
+    *abort_flag = 1;
+    atomicCAS(status, 0, kErrTimeout);
+}
+
 // Segment bookkeeping shared by producer and consumers.
 struct Segment {
     int b, g, seg;
-    int64_t seg_start, t_end, nk, S;
+    int64_t seg_start, tiles, t_end, nk, S;
 };
 __device__ __forceinline__ Segment locate_segment(const AttnParams& p, const int64_t* tile_prefix, int64_t t, int64_t t1) {
     Segment s;
     s.b = find_seq(tile_prefix, p.B, p.Hkv, t);
-    const int64_t tiles_b = tile_prefix[s.b + 1] - tile_prefix[s.b];
+    s.tiles = tile_prefix[s.b + 1] - tile_prefix[s.b];
     const int64_t seq_start = (int64_t)p.Hkv * tile_prefix[s.b];
-    s.g = (int)((t - seq_start) / tiles_b);
-    s.seg_start = seq_start + (int64_t)s.g * tiles_b;
-    const int64_t seg_end = s.seg_start + tiles_b;
+    s.g = (int)((t - seq_start) / s.tiles);
+    s.seg_start = seq_start + (int64_t)s.g * s.tiles;
+    const int64_t seg_end = s.seg_start + s.tiles;
     s.t_end = seg_end < t1 ? seg_end : t1;
-    s.S = p.len[s.b];
+    s.S = eff_len(p, s.b);
     s.nk = scan_keys(p, s.b);
     s.seg = s.b * p.Hkv + s.g;
     return s;
 }
 
+// Element offset of row `key` of (b, g) in the K / V tensor; *ok = false on a bad page id.
+__device__ __forceinline__ int64_t kv_row_offset(const AttnParams& p, int b, int g, int64_t key, bool* ok) {
+    if (p.mode == kPaged) {
+        const int page = p.page_table[(int64_t)b * p.max_pages + key / p.page_size];
+        if (page < 0 || page >= p.num_pages) { *ok = false; return 0; }
+        return (((int64_t)page * p.Hkv + g) * p.page_size + key % p.page_size) * p.D;
+    }
+    return (((int64_t)b * p.Hkv + g) * p.rows_per_head + key) * p.D;
+}
+
 // ---------------------------------------------------------------------------------------------
-// Partial kernel
+// Distributed combine of one segment (paper-independent split-KV algebra):
+// lse = logsumexp_s(lse_s), out = sum_s exp(lse_s - lse) * o_s. Called by the 128 consumer threads
+// of every CTA that contributed a partial to the segment, after the CTA has published its own.
+// CTA number j of the np contributors reduces the j-th slice of the (head, d) columns, so the
+// merge is spread over all SMs that worked on the segment instead of serialising on one.
+// ---------------------------------------------------------------------------------------------
+__device__ __noinline__ void combine_segment(const AttnParams& p, const Segment& sg, int c_first, int np, int j,
+                                             float* scratch, volatile int* abort_flag) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = p.G, D = p.D;
+    float* w_sm = scratch;                                                  // [G][np], np <= kMaxCtas
+    float* inv_sm = scratch + kMaxGroup * kMaxCtas;                         // [8]
+    float4* red = reinterpret_cast<float4*>(inv_sm + 8);                    // [128]
+    if (tid == 0) wait_counter(p.arrive + sg.seg, np, abort_flag, p.status);
+    consumer_barrier();
+    const int64_t pbase = (int64_t)c_first + sg.seg;
+
+    // ---- this CTA's slice of the (head, d) columns; the first rows are requested before the weights exist
+    constexpr int kPre = 4;
+    const int vec = D / 4, cols = G * vec;
+    const int cpc = (cols + np - 1) / np;
+    const int col_lo = j * cpc, col_hi = col_lo + cpc < cols ? col_lo + cpc : cols;
+    const float4* rows = reinterpret_cast<const float4*>(p.part_o);
+    float4 pre[kPre];
+    {
+        const int cb = col_hi - col_lo < 128 ? col_hi - col_lo : 128;
+        if (cb > 0) {
+            const int R = 128 / cb, cl = tid % cb, rg = tid / cb;
+#pragma unroll
+            for (int u = 0; u < kPre; ++u) {
+                const int i = rg + u * R;
+                pre[u] = (rg < R && i < np) ? __ldcg(rows + (pbase + i) * cols + col_lo + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+    }
+    // ---- weights: one pass over the partial lse values (<= 8 per lane)
+    for (int h = warp; h < G; h += kConsumerWarps) {
+        float x[kMaxCtas / 32];
+        float M = -INFINITY;
+#pragma unroll
+        for (int u = 0; u < kMaxCtas / 32; ++u) {
+            const int i = lane + 32 * u;
+            x[u] = i < np ? __ldcg(p.part_lse + (pbase + i) * G + h) : -INFINITY;
+            M = fmaxf(M, x[u]);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+        float sum = 0.f;
+#pragma unroll
+        for (int u = 0; u < kMaxCtas / 32; ++u) {
+            const int i = lane + 32 * u;
+            if (i < np) {
+                const float w = (M > -INFINITY) ? __expf(x[u] - M) : 0.f;
+                w_sm[h * np + i] = w;
+                sum += w;
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+        if (lane == 0) {
+            inv_sm[h] = sum > 0.f ? 1.f / sum : 0.f;
+            if (j == 0 && p.lse) p.lse[(int64_t)sg.b * p.Hq + sg.g * G + h] = sum > 0.f ? M + __logf(sum) : -INFINITY;
+        }
+    }
+    consumer_barrier();
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)sg.b * p.Hq + sg.g * G) * D;
+    for (int c0 = col_lo; c0 < col_hi; c0 += 128) {
+        const int cb = col_hi - c0 < 128 ? col_hi - c0 : 128;
+        const int R = 128 / cb, cl = tid % cb, rg = tid / cb;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (rg < R) {
+            const int col = c0 + cl, h = col / vec;
+            int i = rg;
+            if (c0 == col_lo) {
+#pragma unroll
+                for (int u = 0; u < kPre; ++u, i += R) {
+                    if (i < np) {
+                        const float w = w_sm[h * np + i];
+                        acc.x = fmaf(w, pre[u].x, acc.x); acc.y = fmaf(w, pre[u].y, acc.y);
+                        acc.z = fmaf(w, pre[u].z, acc.z); acc.w = fmaf(w, pre[u].w, acc.w);
+                    }
+                }
+            }
+#pragma unroll 4
+            for (; i < np; i += R) {
+                const float w = w_sm[h * np + i];
+                const float4 x = __ldcg(rows + (pbase + i) * cols + col);
+                acc.x = fmaf(w, x.x, acc.x); acc.y = fmaf(w, x.y, acc.y); acc.z = fmaf(w, x.z, acc.z); acc.w = fmaf(w, x.w, acc.w);
+            }
+        }
+        red[tid] = acc;
+        consumer_barrier();
+        if (tid < cb) {
+            float4 o = red[tid];
+            for (int r = 1; r < R; ++r) {
+                const float4 x = red[r * cb + tid];
+                o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
+            }
+            const int col = c0 + tid;
+            const float inv = inv_sm[col / vec];
+            uint2 packed;
+            packed.x = pack_bf16x2(o.x * inv, o.y * inv);
+            packed.y = pack_bf16x2(o.z * inv, o.w * inv);
+            *reinterpret_cast<uint2*>(out + (int64_t)col * 4) = packed;
+        }
+        consumer_barrier();
+    }
+}
+
+// End of the launch for this CTA. The last CTA of the grid (every other one has finished its combines
+// and has read every len[] by then) clears the arrival counters for the next launch and advances the
+// lengths of a fused append.
+__device__ __forceinline__ void finish_launch(const AttnParams& p, int* flag_sm, bool whole_block) {
+    if (threadIdx.x == 0) {
+        const int old = atomicAdd(p.grid_done, 1);
+        const int last = (old + 1 == (int)gridDim.x);
+        if (last) *p.grid_done = 0;
+        *flag_sm = last;
+    }
+    if (whole_block) __syncthreads(); else consumer_barrier();
+    if (*flag_sm) {
+        const int nthr = whole_block ? blockDim.x : 128;
+        for (int sgi = threadIdx.x; sgi < p.B * p.Hkv; sgi += nthr) p.arrive[sgi] = 0;
+        if (p.k_new) {
+            for (int b = threadIdx.x; b < p.B; b += nthr) {
+                if (appends_to(p, b)) p.len[b] += 1;
+                else atomicCAS(p.status, 0, kErrBounds);          // append past S_cap: skipped and flagged
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The attention kernel (one cooperative launch per draft step)
 // ---------------------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
-attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, AttnParams p) {
+attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
+               const __grid_constant__ AttnParams p) {
     using C = Cfg<D>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char* stages = smem;                                                         // kStages x (K tile, V tile)
-    float* scratch = reinterpret_cast<float*>(stages + C::kStages * C::kStageBytes);      // [4][8][kScratchRow]
-    float* sm_m = scratch + kConsumerWarps * kMaxGroup * kScratchRow;                     // [4][8]
+    float* scratch = reinterpret_cast<float*>(stages + C::kStages * C::kStageBytes);      // merge / combine scratch
+    float* sm_m = scratch + kScratchFloats;                                               // [4][8]
     float* sm_l = sm_m + kConsumerWarps * kMaxGroup;                                      // [4][8]
     float* sm_le = sm_l + kConsumerWarps * kMaxGroup;                                     // [4][8]
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm_le + kConsumerWarps * kMaxGroup);     // fullK, fullV, empty
-    int* abort_flag = reinterpret_cast<int*>(bars + 3 * C::kStages);
+    int* abort_flag = reinterpret_cast<int*>(bars + 3 * C::kStages);                      // [0] abort, [1] last-CTA flag
     int64_t* tile_prefix = reinterpret_cast<int64_t*>(abort_flag + 2);                    // [B + 1]
 
+    if (threadIdx.x == kConsumerWarps * 32) {               // descriptor fetch overlaps the len[] round trip
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapK) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&mapV) : "memory");
+    }
     build_tile_prefix(p, tile_prefix);
+    const int G = p.G;
+    const int nseg = p.B * p.Hkv;
+    // ---- sequences that hold no token: out = 0, lse = -inf (no CTA owns a tile of theirs)
+    for (int seg = blockIdx.x; seg < nseg; seg += gridDim.x) {
+        const int b = seg / p.Hkv, g = seg % p.Hkv;
+        if (tile_prefix[b + 1] != tile_prefix[b]) continue;
+        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + g * G) * D;
+        for (int idx = threadIdx.x; idx < G * D; idx += blockDim.x) o[idx] = __float2bfloat16(0.f);
+        if (p.lse && threadIdx.x < G) p.lse[(int64_t)b * p.Hq + g * G + threadIdx.x] = -INFINITY;
+    }
     const int64_t n = (int64_t)p.Hkv * tile_prefix[p.B];
     const int Cn = effective_ctas(gridDim.x, n);
-    if ((int)blockIdx.x >= Cn) return;
+    if ((int)blockIdx.x >= Cn) {
+        finish_launch(p, abort_flag + 1, true);
+        return;
+    }
     const int64_t t0 = cta_range_start(blockIdx.x, n, Cn), t1 = cta_range_start(blockIdx.x + 1, n, Cn);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -160,7 +344,7 @@ attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant
             mbar_init(bar_fullV + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, kConsumerWarps);
         }
-        *abort_flag = 0;
+        abort_flag[0] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -214,7 +398,6 @@ attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant
 
     // ===================================== consumer warps =====================================
     const int g8 = lane >> 2, t4 = lane & 3;            // MMA fragment coordinates
-    const int G = p.G;
     const float scale = p.scale_log2;
     // ldmatrix lane addressing (byte offsets inside a 64-row x 128-byte swizzled chunk)
     const int mi = lane >> 3, rr = lane & 7;
@@ -227,6 +410,16 @@ attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant
     uint32_t it = 0;
     while (t < t1) {
         const Segment sg = locate_segment(p, tile_prefix, t, t1);
+        // ---- fused append (Appendix A, RING / the KV write of a draft forward): where does the new token go?
+        int64_t new_tile = -1;                              // tile (within the segment) holding the new row
+        int new_row = 0;
+        if (appends_to(p, sg.b)) {
+            const int64_t pos = sg.S - 1;
+            const int64_t key = p.mode == kRing ? ring_slot(pos, p.n_sink, p.cap) : pos;
+            new_tile = key / kTileKeys;
+            new_row = (int)(key % kTileKeys);
+            if ((new_row >> 4) != warp || new_tile < t - sg.seg_start || new_tile >= sg.t_end - sg.seg_start) new_tile = -1;
+        }
         // ---- Q^T fragments (B operand: k = d, n = head); heads >= G read as zero
         uint32_t qb[C::kKSteps][2];
         {
@@ -249,9 +442,29 @@ attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant
             const int64_t wkey0 = key0 + warp * 16;
             const bool tile_full = (key0 + kTileKeys <= sg.nk) && !slack;
             const bool any_valid = wkey0 < sg.nk;
+            const bool has_new = (tt - sg.seg_start) == new_tile;      // this warp owns the appended row in this tile
             const uint32_t sK = stage0 + s * C::kStageBytes, sV = sK + C::kTileBytes;
+            int64_t new_off = 0;
+            bool new_ok = true;
+            if (has_new) {
+                new_off = kv_row_offset(p, sg.b, sg.g, key0 + new_row, &new_ok);
+                if (!new_ok && lane == 0) atomicCAS(p.status, 0, kErrBounds);
+            }
 
             mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
+            if (has_new && lane < D / 8) {
+                // the row TMA brought may be stale: take it from k_new, in shared memory and in the store
+                const uint4 x = __ldg(reinterpret_cast<const uint4*>(p.k_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8) + lane);
+                const uint32_t addr = sK + (lane >> 3) * C::kChunkBytes + new_row * 128 + (((lane & 7) ^ (new_row & 7)) << 4);
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
+                if (new_ok) reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.k) + new_off)[lane] = x;
+            }
+            if (has_new) {
+                if (p.mode == kRing && sg.g == 0 && lane == 0)
+                    p.slot_pos[(int64_t)sg.b * p.rows_per_head + key0 + new_row] = (int32_t)(sg.S - 1);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+            }
             uint32_t pb0 = 0, pb1 = 0;
             float corr0 = 1.f, corr1 = 1.f;
             if (any_valid) {
@@ -305,6 +518,12 @@ attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant
                 }
             }
             mbar_wait(bar_fullV + 8 * s, ph, abort_flag, p.status);
+            if (has_new && lane < D / 8) {
+                const uint4 x = __ldg(reinterpret_cast<const uint4*>(p.v_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8) + lane);
+                const uint32_t addr = sV + (lane >> 3) * C::kChunkBytes + new_row * 128 + (((lane & 7) ^ (new_row & 7)) << 4);
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
+                if (new_ok) reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.v) + new_off)[lane] = x;
+            }
             if (any_valid) {
                 if (wkey0 + 16 > sg.nk) {
                     // rows past the sequence end were never written: they may hold NaN/Inf bit patterns,
@@ -315,6 +534,8 @@ attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant
                         const uint32_t addr = sV + (rem >> 3) * C::kChunkBytes + (warp * 16 + r) * 128 + ((rem & 7) << 4);
                         asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
                     }
+                }
+                if (has_new || wkey0 + 16 > sg.nk) {
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                 }
@@ -331,7 +552,7 @@ attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant
             if (lane == 0) mbar_arrive(bar_empty + 8 * s);
         }
 
-        // ---- merge the four warps' states and emit the partial of (this CTA, this segment)
+        // ---- merge the four warps' states and publish the partial of (this CTA, this segment)
 #pragma unroll
         for (int off = 4; off <= 16; off <<= 1) {
             l[0] += __shfl_xor_sync(0xffffffffu, l[0], off);
@@ -339,13 +560,14 @@ attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant
             le[0] += __shfl_xor_sync(0xffffffffu, le[0], off);
             le[1] += __shfl_xor_sync(0xffffffffu, le[1], off);
         }
-        consumer_barrier();                                   // scratch / sm_m free (previous segment fully written out)
+        consumer_barrier();                                   // scratch / sm_m free (previous segment fully done)
         if (g8 == 0) {
             sm_m[warp * kMaxGroup + 2 * t4] = m[0]; sm_m[warp * kMaxGroup + 2 * t4 + 1] = m[1];
             sm_l[warp * kMaxGroup + 2 * t4] = l[0]; sm_l[warp * kMaxGroup + 2 * t4 + 1] = l[1];
             sm_le[warp * kMaxGroup + 2 * t4] = le[0]; sm_le[warp * kMaxGroup + 2 * t4 + 1] = le[1];
         }
         consumer_barrier();
+        const int64_t pidx = (int64_t)blockIdx.x + sg.seg;
         float f[2];
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
@@ -363,10 +585,8 @@ attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant
                 }
             }
             f[i] = (L > 0.f && m[i] > -INFINITY) ? exp2f(m[i] - M) / L : 0.f;
-            if (warp == 0 && g8 == 0 && h < G)
-                p.part_lse[((int64_t)blockIdx.x + sg.seg) * G + h] = Le > 0.f ? (M + log2f(Le)) * kLn2 : -INFINITY;
+            if (warp == 0 && g8 == 0 && h < G) p.part_lse[pidx * G + h] = Le > 0.f ? (M + log2f(Le)) * kLn2 : -INFINITY;
         }
-        const int64_t pidx = (int64_t)blockIdx.x + sg.seg;
         constexpr int kPasses = D / 128;                       // 128 columns of d per pass through the scratch
 #pragma unroll
         for (int pass = 0; pass < kPasses; ++pass) {
@@ -380,8 +600,7 @@ attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant
                 row0[8] = o[mb][2] * f[0]; row1[8] = o[mb][3] * f[1];
             }
             consumer_barrier();
-            const int tid = threadIdx.x;                       // 0..127
-            for (int idx = tid; idx < G * 128; idx += 128) {
+            for (int idx = threadIdx.x; idx < G * 128; idx += 128) {
                 const int h = idx >> 7, dd = idx & 127;
                 float acc = 0.f;
 #pragma unroll
@@ -389,97 +608,16 @@ attn_partial_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant
                 p.part_o[(pidx * G + h) * D + pass * 128 + dd] = acc;
             }
         }
+        __threadfence();                                       // partial visible device-wide before the arrival
+        consumer_barrier();
+        if (threadIdx.x == 0) atomicAdd(p.arrive + sg.seg, 1);
+
+        // ---- take part in the segment's combine
+        const int c_first = tile_owner(sg.seg_start, n, Cn), c_last = tile_owner(sg.seg_start + sg.tiles - 1, n, Cn);
+        combine_segment(p, sg, c_first, c_last - c_first + 1, (int)blockIdx.x - c_first, scratch, abort_flag);
         t = sg.t_end;
     }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Combine: one block per (segment, query head); merges that head's partials by log-sum-exp:
-// lse = logsumexp_s(lse_s), out = sum_s exp(lse_s - lse) * o_s. Row groups of the block read
-// different partials with float4 loads so that all loads of a thread are in flight at once.
-// ---------------------------------------------------------------------------------------------
-constexpr int kCombineThreads = 512;
-
-__global__ void __launch_bounds__(kCombineThreads) attn_combine(AttnParams p, int launched_ctas) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    int64_t* tile_prefix = reinterpret_cast<int64_t*>(smem_raw);            // [B + 1]
-    float* w_sm = reinterpret_cast<float*>(tile_prefix + (p.B + 1));        // [np]
-    float* red = w_sm + launched_ctas;                                      // [groups][D] (16-byte aligned below)
-    red = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(red) + 15) & ~(uintptr_t)15);
-    __shared__ float warp_red[kCombineThreads / 32];
-    __shared__ float bc[2];
-
-    build_tile_prefix(p, tile_prefix);
-    const int seg = blockIdx.x, hh = blockIdx.y, b = seg / p.Hkv, g = seg % p.Hkv;
-    const int G = p.G, D = p.D;
-    const int64_t n = (int64_t)p.Hkv * tile_prefix[p.B];
-    const int C = effective_ctas(launched_ctas, n);
-    const int64_t tiles_b = tile_prefix[b + 1] - tile_prefix[b];
-    const int64_t head = (int64_t)b * p.Hq + g * G + hh;
-    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + head * D;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tiles_b == 0) {                       // empty sequence: out = 0, lse = -inf
-        for (int d = tid; d < D; d += blockDim.x) out[d] = __float2bfloat16(0.f);
-        if (p.lse && tid == 0) p.lse[head] = -INFINITY;
-        return;
-    }
-    const int64_t seg_start = (int64_t)p.Hkv * tile_prefix[b] + (int64_t)g * tiles_b;
-    const int c_first = tile_owner(seg_start, n, C), c_last = tile_owner(seg_start + tiles_b - 1, n, C);
-    const int np = c_last - c_first + 1;
-    const int64_t pbase = (int64_t)c_first + seg;
-
-    // ---- M = max_s lse_s, then weights and their sum
-    float M = -INFINITY;
-    for (int i = tid; i < np; i += blockDim.x) M = fmaxf(M, p.part_lse[(pbase + i) * G + hh]);
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
-    if (lane == 0) warp_red[warp] = M;
-    __syncthreads();
-    if (tid == 0) {
-        float x = warp_red[0];
-        for (int w = 1; w < kCombineThreads / 32; ++w) x = fmaxf(x, warp_red[w]);
-        bc[0] = x;
-    }
-    __syncthreads();
-    M = bc[0];
-    float sum = 0.f;
-    for (int i = tid; i < np; i += blockDim.x) {
-        const float w = (M > -INFINITY) ? __expf(p.part_lse[(pbase + i) * G + hh] - M) : 0.f;
-        w_sm[i] = w;
-        sum += w;
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-    if (lane == 0) warp_red[warp] = sum;
-    __syncthreads();
-    if (tid == 0) {
-        float x = 0.f;
-        for (int w = 0; w < kCombineThreads / 32; ++w) x += warp_red[w];
-        bc[1] = x;
-        if (p.lse) p.lse[head] = x > 0.f ? M + __logf(x) : -INFINITY;
-    }
-    __syncthreads();
-    sum = bc[1];
-    const float inv = sum > 0.f ? 1.f / sum : 0.f;
-
-    // ---- weighted sum of the partial rows: thread = (row group, float4 column)
-    const int vec = D / 4, groups = kCombineThreads / vec;
-    const int grp = tid / vec, col = tid % vec;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    const float4* rows = reinterpret_cast<const float4*>(p.part_o);
-#pragma unroll 4
-    for (int i = grp; i < np; i += groups) {
-        const float w = w_sm[i];
-        const float4 x = rows[((pbase + i) * G + hh) * vec + col];
-        acc.x = fmaf(w, x.x, acc.x); acc.y = fmaf(w, x.y, acc.y); acc.z = fmaf(w, x.z, acc.z); acc.w = fmaf(w, x.w, acc.w);
-    }
-    reinterpret_cast<float4*>(red)[grp * vec + col] = acc;
-    __syncthreads();
-    for (int d = tid; d < D; d += blockDim.x) {
-        float o = 0.f;
-        for (int gi = 0; gi < groups; ++gi) o += red[gi * D + d];
-        out[d] = __float2bfloat16(o * inv);
-    }
+    finish_launch(p, abort_flag + 1, false);
 }
 
 // ---- host side: tensor maps and launch --------------------------------------------------------
@@ -515,23 +653,24 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int D) {
 template <int D>
 size_t partial_smem_bytes(int B) {
     using C = Cfg<D>;
-    return 1024 + (size_t)C::kStages * C::kStageBytes + sizeof(float) * (kConsumerWarps * kMaxGroup * kScratchRow + 3 * kConsumerWarps * kMaxGroup) +
+    return 1024 + (size_t)C::kStages * C::kStageBytes + sizeof(float) * (kScratchFloats + 3 * kConsumerWarps * kMaxGroup) +
            sizeof(uint64_t) * 3 * C::kStages + 2 * sizeof(int) + sizeof(int64_t) * (B + 1) + 16;
 }
 
 template <int D>
-cudaError_t launch_partial(const CUtensorMap& mk, const CUtensorMap& mv, const AttnParams& p, cudaStream_t st) {
+cudaError_t launch_fused(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaStream_t st) {
     const size_t smem = partial_smem_bytes<D>(p.B);
     static bool attr_set[64] = {};          // per device: the opt-in to > 48 KB of dynamic shared memory
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(attn_partial_tma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(attn_fused_tma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    attn_partial_tma<D><<<p.num_ctas, kThreads, smem, st>>>(mk, mv, p);
-    return cudaGetLastError();
+    void* args[] = {&mk, &mv, &p};
+    // cooperative: the CTAs wait on one another in the combine, so they must all be resident
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(attn_fused_tma<D>), dim3(p.num_ctas), dim3(kThreads), args, smem, st);
 }
 
 }  // namespace
@@ -541,17 +680,14 @@ int64_t attention_rows(const AttnParams& p) {
     return (int64_t)p.B * p.Hkv * p.rows_per_head;
 }
 
-cudaError_t launch_attention(const AttnParams& p, cudaStream_t st) {
+cudaError_t launch_attention(const AttnParams& p_in, cudaStream_t st) {
+    AttnParams p = p_in;
     const int64_t rows = attention_rows(p);
     CUtensorMap mk, mv;
     if (!make_map(&mk, p.k, rows, p.D) || !make_map(&mv, p.v, rows, p.D)) return cudaErrorInvalidValue;
-    cudaError_t e = p.D == 128 ? launch_partial<128>(mk, mv, p, st) : launch_partial<256>(mk, mv, p, st);
+    cudaError_t e = p.D == 128 ? launch_fused<128>(mk, mv, p, st) : launch_fused<256>(mk, mv, p, st);
     count_launch(1);
-    if (e != cudaSuccess) return e;
-    const size_t sm_combine = sizeof(int64_t) * (p.B + 1) + sizeof(float) * p.num_ctas + 16 + sizeof(float) * 4 * kCombineThreads;
-    attn_combine<<<dim3(p.B * p.Hkv, p.G), kCombineThreads, sm_combine, st>>>(p, p.num_ctas);
-    count_launch(1);
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace wmtp

@@ -1,4 +1,4 @@
-// Work decomposition shared by the split-KV partial kernel and the combine kernel.
+// Work decomposition shared by every phase of the attention kernel.
 //
 // Every (sequence b, KV head g) pair is a *segment* of tiles_b = ceil(keys_b / kTileKeys) tiles;
 // segments are laid end to end on one line of n tiles in (b, g) order. CTA c of C owns the tile
@@ -12,9 +12,24 @@
 
 namespace wmtp {
 
+// Ring slot of logical position p (Appendix A, RING): the sink is fixed, the window region circular.
+__device__ __forceinline__ int ring_slot(int64_t p, int n_sink, int cap) {
+    return p < n_sink ? (int)p : n_sink + (int)((p - n_sink) % cap);
+}
+
+// Does this launch append a token to sequence b before attending (fused draft step)?
+__device__ __forceinline__ bool appends_to(const AttnParams& p, int b) {
+    return p.k_new != nullptr && (p.mode == kRing || p.len[b] < p.S_cap);
+}
+
+// Sequence length the attention sees: the stored length, plus the token appended by this launch.
+__device__ __forceinline__ int64_t eff_len(const AttnParams& p, int b) {
+    return p.len[b] + (appends_to(p, b) ? 1 : 0);
+}
+
 // Key slots the kernel scans for sequence b: the live part of the ring, or all S positions.
 __device__ __forceinline__ int64_t scan_keys(const AttnParams& p, int b) {
-    const int64_t S = p.len[b];
+    const int64_t S = eff_len(p, b);
     if (p.mode == kRing) {
         const int64_t slots = (int64_t)p.n_sink + p.cap;
         return S < slots ? S : slots;

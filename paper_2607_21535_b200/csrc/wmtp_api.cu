@@ -96,8 +96,9 @@ wmtp_status check_attn_common(const void* q, int Hq, int Hkv, int batch, int D, 
 
 int pick_ctas(int64_t max_tiles) {
     int c = g_max_ctas.load();
-    if (c <= 0) c = sm_count();
-    if (c <= 0) return 0;
+    const int sms = sm_count();
+    if (sms <= 0) return 0;
+    if (c <= 0 || c > sms) c = sms;          // one CTA per SM: the cooperative launch needs all CTAs resident
     if (c > kMaxCtas) c = kMaxCtas;
     if (max_tiles < c) c = (int)(max_tiles < 1 ? 1 : max_tiles);
     return c;
@@ -109,7 +110,8 @@ void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, 
     char* base = static_cast<char*>(ws);
     p.q = q; p.out = out; p.lse = lse;
     p.status = reinterpret_cast<int*>(base);
-    p.counters = reinterpret_cast<int*>(base + L.counters_off);
+    p.grid_done = reinterpret_cast<int*>(base + 4);
+    p.arrive = reinterpret_cast<int*>(base + L.counters_off);
     p.part_lse = reinterpret_cast<float*>(base + L.part_lse_off);
     p.part_o = reinterpret_cast<float*>(base + L.part_o_off);
     p.B = batch; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = Hq / Hkv;
@@ -117,8 +119,10 @@ void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, 
     p.scale_log2 = s * 1.4426950408889634f;
 }
 
+// k_new / v_new non-NULL: a fused draft step (append, then attend) in one launch.
 wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm_scale, void* out, float* lse,
-                          void* ws, size_t ws_bytes, cudaStream_t st, bool validate) {
+                          void* ws, size_t ws_bytes, cudaStream_t st, bool validate, const void* k_new = nullptr,
+                          const void* v_new = nullptr) {
     if (validate) {
         if (wmtp_status s = check_ring(ring)) return s;
         if (wmtp_status s = check_attn_common(q, Hq, ring->Hkv, ring->batch, ring->D, out, lse, ws, ws_bytes)) return s;
@@ -126,6 +130,7 @@ wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm
     AttnParams p{};
     fill_attn(p, q, Hq, ring->Hkv, ring->batch, ring->D, sm_scale, out, lse, ws);
     p.k = ring->k; p.v = ring->v; p.page_table = nullptr; p.len = ring->len;
+    p.k_new = k_new; p.v_new = v_new; p.slot_pos = ring->slot_pos;
     p.mode = kRing;
     p.rows_per_head = (int64_t)ring->n_sink + ring->cap;
     p.n_sink = ring->n_sink; p.W = ring->W; p.cap = ring->cap;
@@ -138,7 +143,8 @@ wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm
 }
 
 wmtp_status attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, void* out, float* lse, void* ws,
-                      size_t ws_bytes, cudaStream_t st, bool validate) {
+                      size_t ws_bytes, cudaStream_t st, bool validate, const void* k_new = nullptr,
+                      const void* v_new = nullptr) {
     if (validate) {
         if (wmtp_status s = check_kv(kv)) return s;
         if (wmtp_status s = check_attn_common(q, Hq, kv->Hkv, kv->batch, kv->D, out, lse, ws, ws_bytes)) return s;
@@ -146,6 +152,7 @@ wmtp_status attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, 
     AttnParams p{};
     fill_attn(p, q, Hq, kv->Hkv, kv->batch, kv->D, sm_scale, out, lse, ws);
     p.k = kv->k; p.v = kv->v; p.page_table = kv->page_table; p.len = kv->len;
+    p.k_new = k_new; p.v_new = v_new; p.slot_pos = nullptr; p.S_cap = kv->S_cap;
     p.mode = kv->page_table ? kPaged : kContiguous;
     p.rows_per_head = kv->page_table ? kv->page_size : kv->S_cap;
     p.page_size = kv->page_size; p.max_pages = kv->max_pages; p.num_pages = kv->num_pages;
@@ -308,15 +315,13 @@ wmtp_status wmtp_draft_loop_windowed(const wmtp_ring* ring, int gamma, const voi
     if (wmtp_status s = check_ring(ring)) return s;
     if (wmtp_status s = check_loop(gamma, k_new, v_new)) return s;
     if (wmtp_status s = check_attn_common(q, Hq, ring->Hkv, ring->batch, ring->D, out, lse, workspace, ws_bytes)) return s;
-    const RingParams rp = ring_params(ring);
     const size_t q_step = (size_t)ring->batch * Hq * ring->D * 2, kv_step = (size_t)ring->batch * ring->Hkv * ring->D * 2;
     for (int i = 0; i < gamma; ++i) {
-        cudaError_t e = launch_ring_append(rp, (const char*)k_new + i * kv_step, (const char*)v_new + i * kv_step,
-                                           (cudaStream_t)stream);
-        if (e != cudaSuccess) return cuda_fail(e, "ring append launch");
+        // one launch per draft step: the kernel appends step i's K/V row, then attends
         if (wmtp_status s = attn_windowed((const char*)q + i * q_step, Hq, ring, sm_scale, (char*)out + i * q_step,
                                           lse ? lse + (size_t)i * ring->batch * Hq : nullptr, workspace, ws_bytes,
-                                          (cudaStream_t)stream, false))
+                                          (cudaStream_t)stream, false, (const char*)k_new + i * kv_step,
+                                          (const char*)v_new + i * kv_step))
             return s;
     }
     return WMTP_OK;
@@ -328,15 +333,12 @@ wmtp_status wmtp_draft_loop_full(const wmtp_kv* kv, int gamma, const void* q, in
     if (wmtp_status s = check_kv(kv)) return s;
     if (wmtp_status s = check_loop(gamma, k_new, v_new)) return s;
     if (wmtp_status s = check_attn_common(q, Hq, kv->Hkv, kv->batch, kv->D, out, lse, workspace, ws_bytes)) return s;
-    const KvParams kp = kv_params(kv);
     const size_t q_step = (size_t)kv->batch * Hq * kv->D * 2, kv_step = (size_t)kv->batch * kv->Hkv * kv->D * 2;
     for (int i = 0; i < gamma; ++i) {
-        cudaError_t e = launch_kv_append(kp, (const char*)k_new + i * kv_step, (const char*)v_new + i * kv_step,
-                                         static_cast<int*>(workspace), (cudaStream_t)stream);
-        if (e != cudaSuccess) return cuda_fail(e, "kv append launch");
         if (wmtp_status s = attn_full((const char*)q + i * q_step, Hq, kv, sm_scale, (char*)out + i * q_step,
                                       lse ? lse + (size_t)i * kv->batch * Hq : nullptr, workspace, ws_bytes,
-                                      (cudaStream_t)stream, false))
+                                      (cudaStream_t)stream, false, (const char*)k_new + i * kv_step,
+                                      (const char*)v_new + i * kv_step))
             return s;
     }
     return WMTP_OK;
@@ -405,7 +407,7 @@ namespace {
 constexpr int kStaticMaxCtas = 160;        // CTAs (KV splits) the static scratch has room for
 constexpr int kStaticMaxSegments = 32;     // batch * Hkv
 constexpr size_t kStaticCountersOff = 256;
-constexpr size_t kStaticPartLseOff = kStaticCountersOff + 256;                                     // 32 counters, padded
+constexpr size_t kStaticPartLseOff = kStaticCountersOff + 256;                                     // 32 arrival counters, padded
 constexpr size_t kStaticPartOOff = kStaticPartLseOff + (kStaticMaxCtas + kStaticMaxSegments) * kMaxGroup * sizeof(float);
 constexpr size_t kStaticBytes = kStaticPartOOff + (size_t)(kStaticMaxCtas + kStaticMaxSegments) * kMaxGroup * 256 * sizeof(float);
 static_assert(kStaticPartLseOff % 256 == 0 && kStaticPartOOff % 256 == 0, "static scratch regions must stay 256-byte aligned");
@@ -450,19 +452,21 @@ wmtp_status wmtp_draft_attn_windowed_noalloc(const void* q, int Hq, const wmtp_r
     char* base = static_cast<char*>(base_v);
     cudaStream_t st = (cudaStream_t)stream;
     // status word and this call's counters must start at zero; the array keeps the previous call's contents
-    cudaError_t e = cudaMemsetAsync(base, 0, kStaticCountersOff + sizeof(int) * nseg, st);
+    cudaError_t e = cudaMemsetAsync(base, 0, kStaticPartLseOff, st);
     if (e != cudaSuccess) return cuda_fail(e, "clearing the static scratch header");
 
     AttnParams p{};
     p.q = q; p.out = out; p.lse = lse;
     p.status = reinterpret_cast<int*>(base);
-    p.counters = reinterpret_cast<int*>(base + kStaticCountersOff);
+    p.grid_done = reinterpret_cast<int*>(base + 4);
+    p.arrive = reinterpret_cast<int*>(base + kStaticCountersOff);
     p.part_lse = reinterpret_cast<float*>(base + kStaticPartLseOff);
     p.part_o = reinterpret_cast<float*>(base + kStaticPartOOff);
     p.B = ring->batch; p.Hq = Hq; p.Hkv = ring->Hkv; p.D = ring->D; p.G = Hq / ring->Hkv;
     const float sc = sm_scale > 0.f ? sm_scale : 1.0f / std::sqrt((float)ring->D);
     p.scale_log2 = sc * 1.4426950408889634f;
     p.k = ring->k; p.v = ring->v; p.page_table = nullptr; p.len = ring->len;
+    p.k_new = nullptr; p.v_new = nullptr; p.slot_pos = ring->slot_pos;
     p.mode = kRing;
     p.rows_per_head = (int64_t)ring->n_sink + ring->cap;
     p.n_sink = ring->n_sink; p.W = ring->W; p.cap = ring->cap;

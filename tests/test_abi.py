@@ -39,7 +39,7 @@ def test_sizes():
     assert kb == 2 * 4100 * 256 * 2 and pb == 4100 * 4
     assert wm.wmtp_ring_bytes(0, 2, 256, 4, 4096) == (0, 0)
     ws = wm.wmtp_workspace_bytes(1, 16, 2, 256)
-    assert ws % 256 == 0 and ws > 1024 * 8 * 256 * 4
+    assert ws % 256 == 0 and ws > 148 * 8 * 257 * 4
     assert wm.wmtp_workspace_bytes(1, 15, 2, 256) == 0
     assert wm.wmtp_stage_bytes(7, 1, 16, 2, 256) >= 7 * (2 * 16 * 256 * 2 + 2 * 2 * 256 * 2)
     assert wm.wmtp_status_string(0) == "ok" and "bounds" in wm.wmtp_status_string(7)
