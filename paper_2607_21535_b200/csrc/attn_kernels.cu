@@ -37,6 +37,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kConsumerWarps = 4;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr uint32_t kSpinLimit = 1u << 22;       // bounded mbarrier waits
+constexpr uint32_t kEpochStride = 1024;         // arrival counters advance by this much per launch (> kMaxCtas)
 constexpr int kScratchRow = 132;                // floats per (warp, head) row of the merge scratch (128 + pad)
 // scratch holds either the warp merge ([4][8][kScratchRow]) or the combine's weights, inverses and reduction buffer
 constexpr int kScratchFloats = (kConsumerWarps * kMaxGroup * kScratchRow) > (kMaxGroup * kMaxCtas + 8 + 4 * 128)
@@ -51,6 +52,34 @@ struct Cfg {
     static constexpr int kStages = (D == 256) ? 3 : 6;
     static constexpr int kKSteps = D / 16;
 };
+
+// Development aid (compiled out unless WMTP_TRACE is defined): CTA 0 records %globaltimer at phase boundaries
+// into the workspace header, bytes [64, 256).
+#ifdef WMTP_TRACE
+#define WMTP_STAMP(p, i)                                                                      \
+    do {                                                                                      \
+        if (blockIdx.x == 0 && (threadIdx.x == 0)) {                                          \
+            unsigned long long t_;                                                            \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                            \
+            reinterpret_cast<unsigned long long*>(reinterpret_cast<char*>((p).status) + 64)[i] = t_; \
+        }                                                                                     \
+    } while (0)
+// per-CTA record {entry, first tile landed, tiles done, smid} right behind the partial-o area (trace builds enlarge the workspace)
+#define WMTP_CTA_STAMP(p, i)                                                                  \
+    do {                                                                                      \
+        if (threadIdx.x == 0) {                                                               \
+            unsigned long long t_;                                                            \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                            \
+            unsigned long long* rec_ = reinterpret_cast<unsigned long long*>(                 \
+                (p).part_o + (size_t)(kMaxCtas + (p).B * (p).Hkv) * (p).G * (p).D) + 4 * blockIdx.x; \
+            rec_[i] = t_;                                                                     \
+            if ((i) == 0) { unsigned sm_; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_)); rec_[3] = sm_; } \
+        }                                                                                     \
+    } while (0)
+#else
+#define WMTP_STAMP(p, i) do { } while (0)
+#define WMTP_CTA_STAMP(p, i) do { } while (0)
+#endif
 
 // ---- PTX wrappers -----------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -85,10 +114,33 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1;
     atomicCAS(status, 0, kErrTimeout);
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+#ifndef WMTP_TMA_3D
+#define WMTP_TMA_3D 1
+#endif
+#ifndef WMTP_TMA_HINT
+#define WMTP_TMA_HINT 0
+#endif
+#ifndef WMTP_L2_PROMO
+#define WMTP_L2_PROMO 3
+#endif
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t policy) {
+#if WMTP_TMA_HINT
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
+#else
+    (void)policy;
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+#endif
+}
+// Whole K (or V) tile in one instruction: box {64 elements, 64 rows, D/64 column chunks} of the 3-D view
+// [chunk][row][64] of the tensor; lands in shared memory as [chunk][row][128 B], 128-byte swizzled.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(0), "r"(y), "r"(0), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -119,11 +171,12 @@ __device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u &
 __device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Bounded spin on a global counter written by other CTAs of this (cooperative) launch.
-__device__ __forceinline__ void wait_counter(const int* ctr, int target, volatile int* abort_flag, int* status) {
+// The counter counts up from `base` (this launch's epoch * kEpochStride); wrap-around safe.
+__device__ __forceinline__ void wait_counter(const int* ctr, uint32_t base, uint32_t target, volatile int* abort_flag, int* status) {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        int v;
-        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
-        if (v >= target) return;
+        uint32_t v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+        if (v - base >= target) return;
         if ((i & 255u) == 255u && *abort_flag) return;
         __nanosleep(32);
     }
@@ -141,7 +194,8 @@ __device__ __forceinline__ Segment locate_segment(const AttnParams& p, const int
     s.b = find_seq(tile_prefix, p.B, p.Hkv, t);
     s.tiles = tile_prefix[s.b + 1] - tile_prefix[s.b];
     const int64_t seq_start = (int64_t)p.Hkv * tile_prefix[s.b];
-    s.g = (int)((t - seq_start) / s.tiles);
+    const int64_t in_seq = t - seq_start;
+    s.g = (in_seq < 0x7fffffffLL && s.tiles < 0x7fffffffLL) ? (int)((uint32_t)in_seq / (uint32_t)s.tiles) : (int)(in_seq / s.tiles);
     s.seg_start = seq_start + (int64_t)s.g * s.tiles;
     const int64_t seg_end = s.seg_start + s.tiles;
     s.t_end = seg_end < t1 ? seg_end : t1;
@@ -169,14 +223,15 @@ __device__ __forceinline__ int64_t kv_row_offset(const AttnParams& p, int b, int
 // merge is spread over all SMs that worked on the segment instead of serialising on one.
 // ---------------------------------------------------------------------------------------------
 __device__ __noinline__ void combine_segment(const AttnParams& p, const Segment& sg, int c_first, int np, int j,
-                                             float* scratch, volatile int* abort_flag) {
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+                                             float* scratch, volatile int* abort_flag, uint32_t epoch_base, bool all_arrived) {
+    const int tid = threadIdx.x;
     const int G = p.G, D = p.D;
     float* w_sm = scratch;                                                  // [G][np], np <= kMaxCtas
     float* inv_sm = scratch + kMaxGroup * kMaxCtas;                         // [8]
     float4* red = reinterpret_cast<float4*>(inv_sm + 8);                    // [128]
-    if (tid == 0) wait_counter(p.arrive + sg.seg, np, abort_flag, p.status);
+    if (tid == 0 && !all_arrived) wait_counter(p.arrive + sg.seg, epoch_base, (uint32_t)np, abort_flag, p.status);
     consumer_barrier();
+    WMTP_STAMP(p, 7);
     const int64_t pbase = (int64_t)c_first + sg.seg;
 
     // ---- this CTA's slice of the (head, d) columns; the first rows are requested before the weights exist
@@ -197,36 +252,38 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, const Segment&
             }
         }
     }
-    // ---- weights: one pass over the partial lse values (<= 8 per lane)
-    for (int h = warp; h < G; h += kConsumerWarps) {
-        float x[kMaxCtas / 32];
+    // ---- weights, all heads at once: 16 threads per head, one pass over the partial lse values
+    {
+        const int h = tid >> 4, li = tid & 15;
+        float x[kMaxCtas / 16];
         float M = -INFINITY;
 #pragma unroll
-        for (int u = 0; u < kMaxCtas / 32; ++u) {
-            const int i = lane + 32 * u;
-            x[u] = i < np ? __ldcg(p.part_lse + (pbase + i) * G + h) : -INFINITY;
+        for (int u = 0; u < kMaxCtas / 16; ++u) {
+            const int i = li + 16 * u;
+            x[u] = (h < G && i < np) ? __ldcg(p.part_lse + (pbase + i) * G + h) : -INFINITY;
             M = fmaxf(M, x[u]);
         }
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+        for (int off = 8; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
         float sum = 0.f;
 #pragma unroll
-        for (int u = 0; u < kMaxCtas / 32; ++u) {
-            const int i = lane + 32 * u;
-            if (i < np) {
+        for (int u = 0; u < kMaxCtas / 16; ++u) {
+            const int i = li + 16 * u;
+            if (h < G && i < np) {
                 const float w = (M > -INFINITY) ? __expf(x[u] - M) : 0.f;
                 w_sm[h * np + i] = w;
                 sum += w;
             }
         }
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-        if (lane == 0) {
+        for (int off = 8; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+        if (li == 0 && h < G) {
             inv_sm[h] = sum > 0.f ? 1.f / sum : 0.f;
             if (j == 0 && p.lse) p.lse[(int64_t)sg.b * p.Hq + sg.g * G + h] = sum > 0.f ? M + __logf(sum) : -INFINITY;
         }
     }
     consumer_barrier();
+    WMTP_STAMP(p, 8);
     __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)sg.b * p.Hq + sg.g * G) * D;
     for (int c0 = col_lo; c0 < col_hi; c0 += 128) {
         const int cb = col_hi - c0 < 128 ? col_hi - c0 : 128;
@@ -271,25 +328,41 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, const Segment&
     }
 }
 
-// End of the launch for this CTA. The last CTA of the grid (every other one has finished its combines
-// and has read every len[] by then) clears the arrival counters for the next launch and advances the
-// lengths of a fused append.
-__device__ __forceinline__ void finish_launch(const AttnParams& p, int* flag_sm, bool whole_block) {
-    if (threadIdx.x == 0) {
-        const int old = atomicAdd(p.grid_done, 1);
-        const int last = (old + 1 == (int)gridDim.x);
-        if (last) *p.grid_done = 0;
-        *flag_sm = last;
+// Launch-level bookkeeping lives in the workspace header and needs no reset pass and no grid barrier:
+//   epoch      every launch reads it at entry; arrival counters count up from epoch * kEpochStride, and the
+//              last arriver of a segment bumps the counter to (epoch + 1) * kEpochStride, which still
+//              satisfies every CTA that is polling it;
+//   segs_done  segments whose last partial has arrived; the CTA that completes the last segment advances
+//              the epoch and, for a fused append, the lengths. Every CTA that owns tiles has read len[]
+//              for the last time before its last arrival; CTAs without tiles check in separately.
+//   checkin    CTAs that have read len[] (entry); the length update waits until all have.
+// Called by consumer thread 0 after the segment's partial is visible. Returns true if all np partials
+// of the segment had arrived; *launch_last is set for the CTA that completed the launch's last segment.
+__device__ __forceinline__ bool publish_arrival(const AttnParams& p, int seg, int np, uint32_t epoch, int nonempty_segs,
+                                                bool* launch_last) {
+    const uint32_t old = (uint32_t)atomicAdd(p.arrive + seg, 1);
+    if (old + 1u - epoch * kEpochStride != (uint32_t)np) return false;
+    p.arrive[seg] = (int)((epoch + 1u) * kEpochStride);
+    const int old2 = atomicAdd(p.segs_done, 1);
+    if (old2 + 1 == nonempty_segs) {
+        *p.segs_done = 0;
+        *p.epoch = epoch + 1u;
+        *launch_last = true;
     }
-    if (whole_block) __syncthreads(); else consumer_barrier();
-    if (*flag_sm) {
-        const int nthr = whole_block ? blockDim.x : 128;
-        for (int sgi = threadIdx.x; sgi < p.B * p.Hkv; sgi += nthr) p.arrive[sgi] = 0;
-        if (p.k_new) {
-            for (int b = threadIdx.x; b < p.B; b += nthr) {
-                if (appends_to(p, b)) p.len[b] += 1;
-                else atomicCAS(p.status, 0, kErrBounds);          // append past S_cap: skipped and flagged
-            }
+    return true;
+}
+
+// By the CTA that completed the launch's last segment, after its own combine: advance the lengths of a fused append.
+__device__ __forceinline__ void advance_lengths(const AttnParams& p, volatile int* abort_flag) {
+    if (threadIdx.x == 0) {
+        wait_counter(p.checkin, 0u, gridDim.x, abort_flag, p.status);     // every CTA has read len[]
+        *p.checkin = 0;
+    }
+    consumer_barrier();
+    if (p.k_new) {
+        for (int b = threadIdx.x; b < p.B; b += 128) {
+            if (appends_to(p, b)) p.len[b] += 1;
+            else atomicCAS(p.status, 0, kErrBounds);          // append past S_cap: skipped and flagged
         }
     }
 }
@@ -313,11 +386,27 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     int* abort_flag = reinterpret_cast<int*>(bars + 3 * C::kStages);                      // [0] abort, [1] last-CTA flag
     int64_t* tile_prefix = reinterpret_cast<int64_t*>(abort_flag + 2);                    // [B + 1]
 
+    WMTP_STAMP(p, 0);
+    WMTP_CTA_STAMP(p, 0);
     if (threadIdx.x == kConsumerWarps * 32) {               // descriptor fetch overlaps the len[] round trip
         asm volatile("prefetch.tensormap [%0];" ::"l"(&mapK) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&mapV) : "memory");
     }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t bar_fullK = smem_u32(bars), bar_fullV = smem_u32(bars + C::kStages), bar_empty = smem_u32(bars + 2 * C::kStages);
+    if (threadIdx.x == 0) {                                  // under the shadow of the len[] round trip
+        for (int s = 0; s < C::kStages; ++s) {
+            mbar_init(bar_fullK + 8 * s, 1);
+            mbar_init(bar_fullV + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, kConsumerWarps);
+        }
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    const uint32_t epoch = *reinterpret_cast<const volatile uint32_t*>(p.epoch);
     build_tile_prefix(p, tile_prefix);
+    WMTP_STAMP(p, 1);
     const int G = p.G;
     const int nseg = p.B * p.Hkv;
     // ---- sequences that hold no token: out = 0, lse = -inf (no CTA owns a tile of theirs)
@@ -330,29 +419,31 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     }
     const int64_t n = (int64_t)p.Hkv * tile_prefix[p.B];
     const int Cn = effective_ctas(gridDim.x, n);
-    if ((int)blockIdx.x >= Cn) {
-        finish_launch(p, abort_flag + 1, true);
-        return;
-    }
-    const int64_t t0 = cta_range_start(blockIdx.x, n, Cn), t1 = cta_range_start(blockIdx.x + 1, n, Cn);
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t bar_fullK = smem_u32(bars), bar_fullV = smem_u32(bars + C::kStages), bar_empty = smem_u32(bars + 2 * C::kStages);
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < C::kStages; ++s) {
-            mbar_init(bar_fullK + 8 * s, 1);
-            mbar_init(bar_fullV + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, kConsumerWarps);
+    if (threadIdx.x == 0) {                                  // check in: this CTA has read len[] (see publish_arrival)
+        if (n > 0) {
+            atomicAdd(p.checkin, 1);
+        } else if (atomicAdd(p.checkin, 1) + 1 == (int)gridDim.x) {   // nothing to attend over at all
+            *p.checkin = 0;
+            if (p.k_new) atomicCAS(p.status, 0, kErrBounds);
         }
-        abort_flag[0] = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    __syncthreads();
+    if ((int)blockIdx.x >= Cn) return;
+    const int64_t t0 = cta_range_start(blockIdx.x, n, Cn), t1 = cta_range_start(blockIdx.x + 1, n, Cn);
+    int nonempty_segs = 0;                                   // used by consumer thread 0 only
+    if (threadIdx.x == 0)
+        for (int b = 0; b < p.B; ++b) nonempty_segs += (tile_prefix[b + 1] != tile_prefix[b]) ? p.Hkv : 0;
+    WMTP_STAMP(p, 2);
     const bool slack = (p.mode == kRing) && (p.cap != p.W);
 
     if (warp == kConsumerWarps) {
         // =================================== producer warp ===================================
         const uint32_t stage0 = smem_u32(stages);
+        uint64_t policy = 0;
+#if WMTP_TMA_HINT == 1
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+#elif WMTP_TMA_HINT == 2
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
+#endif
         int64_t t = t0;
         uint32_t it = 0;
         while (t < t1) {
@@ -380,13 +471,21 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                             else row = ((int64_t)sg.b * p.Hkv + sg.g) * p.rows_per_head + (first_tile + base + j) * kTileKeys;
                             const uint32_t dstK = stage0 + s * C::kStageBytes, dstV = dstK + C::kTileBytes;
                             mbar_expect_tx(bar_fullK + 8 * s, C::kTileBytes);
+#if WMTP_TMA_3D
+                            tma_load_3d(dstK, &mapK, (int)row, bar_fullK + 8 * s);
+#else
 #pragma unroll
                             for (int c = 0; c < C::kChunks; ++c)
-                                tma_load_2d(dstK + c * C::kChunkBytes, &mapK, c * 64, (int)row, bar_fullK + 8 * s);
+                                tma_load_2d(dstK + c * C::kChunkBytes, &mapK, c * 64, (int)row, bar_fullK + 8 * s, policy);
+#endif
                             mbar_expect_tx(bar_fullV + 8 * s, C::kTileBytes);
+#if WMTP_TMA_3D
+                            tma_load_3d(dstV, &mapV, (int)row, bar_fullV + 8 * s);
+#else
 #pragma unroll
                             for (int c = 0; c < C::kChunks; ++c)
-                                tma_load_2d(dstV + c * C::kChunkBytes, &mapV, c * 64, (int)row, bar_fullV + 8 * s);
+                                tma_load_2d(dstV + c * C::kChunkBytes, &mapV, c * 64, (int)row, bar_fullV + 8 * s, policy);
+#endif
                         }
                     }
                 }
@@ -408,6 +507,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 
     int64_t t = t0;
     uint32_t it = 0;
+    bool launch_last = false;                            // consumer thread 0: did this CTA complete the launch's last segment?
     while (t < t1) {
         const Segment sg = locate_segment(p, tile_prefix, t, t1);
         // ---- fused append (Appendix A, RING / the KV write of a draft forward): where does the new token go?
@@ -452,6 +552,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             }
 
             mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
+            if (tt == t0) { WMTP_STAMP(p, 3); WMTP_CTA_STAMP(p, 1); }
             if (has_new && lane < D / 8) {
                 // the row TMA brought may be stale: take it from k_new, in shared memory and in the store
                 const uint4 x = __ldg(reinterpret_cast<const uint4*>(p.k_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8) + lane);
@@ -518,6 +619,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 }
             }
             mbar_wait(bar_fullV + 8 * s, ph, abort_flag, p.status);
+            if (tt == t0) WMTP_STAMP(p, 4);
             if (has_new && lane < D / 8) {
                 const uint4 x = __ldg(reinterpret_cast<const uint4*>(p.v_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8) + lane);
                 const uint32_t addr = sV + (lane >> 3) * C::kChunkBytes + new_row * 128 + (((lane & 7) ^ (new_row & 7)) << 4);
@@ -552,6 +654,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             if (lane == 0) mbar_arrive(bar_empty + 8 * s);
         }
 
+        WMTP_STAMP(p, 5);
+        WMTP_CTA_STAMP(p, 2);
         // ---- merge the four warps' states and publish the partial of (this CTA, this segment)
 #pragma unroll
         for (int off = 4; off <= 16; off <<= 1) {
@@ -610,14 +714,21 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         }
         __threadfence();                                       // partial visible device-wide before the arrival
         consumer_barrier();
-        if (threadIdx.x == 0) atomicAdd(p.arrive + sg.seg, 1);
+        const int c_first = tile_owner(sg.seg_start, n, Cn), c_last = tile_owner(sg.seg_start + sg.tiles - 1, n, Cn);
+        const int np = c_last - c_first + 1;
+        bool all_arrived = false;
+        if (threadIdx.x == 0) all_arrived = publish_arrival(p, sg.seg, np, epoch, nonempty_segs, &launch_last);
+        WMTP_STAMP(p, 6);
 
         // ---- take part in the segment's combine
-        const int c_first = tile_owner(sg.seg_start, n, Cn), c_last = tile_owner(sg.seg_start + sg.tiles - 1, n, Cn);
-        combine_segment(p, sg, c_first, c_last - c_first + 1, (int)blockIdx.x - c_first, scratch, abort_flag);
+        combine_segment(p, sg, c_first, np, (int)blockIdx.x - c_first, scratch, abort_flag, epoch * kEpochStride, all_arrived);
+        WMTP_STAMP(p, 9);
         t = sg.t_end;
     }
-    finish_launch(p, abort_flag + 1, false);
+    if (threadIdx.x == 0) abort_flag[1] = launch_last ? 1 : 0;
+    consumer_barrier();
+    if (abort_flag[1]) advance_lengths(p, abort_flag);
+    WMTP_STAMP(p, 10);
 }
 
 // ---- host side: tensor maps and launch --------------------------------------------------------
@@ -637,16 +748,26 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// 2-D view [rows][D] of a K or V tensor; box = 64 rows x 64 elements (128 bytes), 128-byte swizzle.
+// View of a K or V tensor [rows][D] for TMA, 128-byte swizzle.
+//   3-D (default): dims {64, rows, D/64} with strides {2 D, 128} bytes, box {64, 64, D/64}: one copy per tile.
+//   2-D: dims {D, rows}, box {64, 64}: D/64 copies per tile.
 bool make_map(CUtensorMap* map, const void* base, int64_t rows, int D) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
+    const cuuint32_t estr[3] = {1, 1, 1};
+#if WMTP_TMA_3D
+    const cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(D / 64)};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kTileKeys, (cuuint32_t)(D / 64)};
+    const cuuint32_t rank = 3;
+#else
     const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
     const cuuint32_t box[2] = {64, (cuuint32_t)kTileKeys};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    const cuuint32_t rank = 2;
+#endif
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, (CUtensorMapL2promotion)WMTP_L2_PROMO,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

@@ -14,7 +14,10 @@ namespace wmtp {
 
 // Ring slot of logical position p (Appendix A, RING): the sink is fixed, the window region circular.
 __device__ __forceinline__ int ring_slot(int64_t p, int n_sink, int cap) {
-    return p < n_sink ? (int)p : n_sink + (int)((p - n_sink) % cap);
+    if (p < n_sink) return (int)p;
+    const int64_t w = p - n_sink;
+    // 64-bit division is a long dependent instruction chain on the GPU: take the 32-bit path when it is exact
+    return n_sink + (w < 0x7fffffffLL ? (int)((uint32_t)w % (uint32_t)cap) : (int)(w % cap));
 }
 
 // Does this launch append a token to sequence b before attending (fused draft step)?
@@ -41,7 +44,7 @@ __device__ __forceinline__ int64_t scan_keys(const AttnParams& p, int b) {
 __device__ __forceinline__ bool ring_slot_live(int s, int64_t S, int n_sink, int W, int cap) {
     if (s < n_sink) return true;
     const int64_t last = S - 1 - n_sink;
-    const int cur = (int)(last % cap);
+    const int cur = last < 0x7fffffffLL ? (int)((uint32_t)last % (uint32_t)cap) : (int)(last % cap);
     int age = cur - (s - n_sink);
     if (age < 0) age += cap;
     return age < W;
@@ -67,12 +70,16 @@ __device__ __forceinline__ int effective_ctas(int launched, int64_t n) {
     return n < (int64_t)launched ? (int)n : launched;
 }
 
+// (Tile counts below 2^23 keep c * n and (t + 1) * C inside 32 bits for C <= kMaxCtas = 256; 64-bit division
+// costs hundreds of dependent cycles on one thread, which the short windowed launches would feel.)
 __device__ __forceinline__ int64_t cta_range_start(int c, int64_t n, int C) {
+    if (n < (1 << 23)) return (int64_t)(((uint32_t)c * (uint32_t)n) / (uint32_t)C);
     return ((int64_t)c * n) / C;   // c <= kMaxCtas and n < 2^40: no overflow
 }
 
 // CTA owning tile t: the largest c with cta_range_start(c) <= t.
 __device__ __forceinline__ int tile_owner(int64_t t, int64_t n, int C) {
+    if (n < (1 << 23)) return (int)((((uint32_t)t + 1u) * (uint32_t)C - 1u) / (uint32_t)n);
     return (int)(((t + 1) * (int64_t)C - 1) / n);
 }
 

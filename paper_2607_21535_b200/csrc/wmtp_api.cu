@@ -110,7 +110,9 @@ void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, 
     char* base = static_cast<char*>(ws);
     p.q = q; p.out = out; p.lse = lse;
     p.status = reinterpret_cast<int*>(base);
-    p.grid_done = reinterpret_cast<int*>(base + 4);
+    p.epoch = reinterpret_cast<uint32_t*>(base + 4);
+    p.segs_done = reinterpret_cast<int*>(base + 8);
+    p.checkin = reinterpret_cast<int*>(base + 12);
     p.arrive = reinterpret_cast<int*>(base + L.counters_off);
     p.part_lse = reinterpret_cast<float*>(base + L.part_lse_off);
     p.part_o = reinterpret_cast<float*>(base + L.part_o_off);
@@ -207,6 +209,9 @@ WorkspaceLayout workspace_layout(int batch, int Hq, int Hkv, int D) {
     L.part_lse_off = kWorkspaceZeroBytes;
     L.part_o_off = L.part_lse_off + round_up(np * G * sizeof(float), 256);
     L.total = L.part_o_off + round_up(np * G * D * sizeof(float), 256);
+#ifdef WMTP_TRACE
+    L.total += 32 * kMaxCtas;     // per-CTA trace records
+#endif
     return L;
 }
 
@@ -458,7 +463,9 @@ wmtp_status wmtp_draft_attn_windowed_noalloc(const void* q, int Hq, const wmtp_r
     AttnParams p{};
     p.q = q; p.out = out; p.lse = lse;
     p.status = reinterpret_cast<int*>(base);
-    p.grid_done = reinterpret_cast<int*>(base + 4);
+    p.epoch = reinterpret_cast<uint32_t*>(base + 4);
+    p.segs_done = reinterpret_cast<int*>(base + 8);
+    p.checkin = reinterpret_cast<int*>(base + 12);
     p.arrive = reinterpret_cast<int*>(base + kStaticCountersOff);
     p.part_lse = reinterpret_cast<float*>(base + kStaticPartLseOff);
     p.part_o = reinterpret_cast<float*>(base + kStaticPartOOff);

@@ -18,7 +18,7 @@ constexpr size_t kWorkspaceZeroBytes = 256 + sizeof(int) * kMaxSegments;   // he
 enum KvMode : int { kContiguous = 0, kPaged = 1, kRing = 2 };
 
 // Workspace layout (all offsets from a 256-byte aligned base):
-//   [0, 256)            header: int status word at offset 0, int grid_done at offset 4
+//   [0, 256)            header: int status @0, uint epoch @4, int segs_done @8, int checkin @12
 //   counters            int arrive[kMaxSegments] (fixed size: initialisation needs no shape)
 //   part_lse            float [kMaxCtas + batch * Hkv][G]
 //   part_o              float [kMaxCtas + batch * Hkv][G][D]
@@ -40,7 +40,9 @@ struct AttnParams {
     float* part_o;
     float* part_lse;
     int* arrive;              // [segments]: CTAs that have published their partial of the segment
-    int* grid_done;           // CTAs that have finished the launch
+    uint32_t* epoch;          // launch counter (header); arrival counters count from epoch * stride
+    int* segs_done;           // segments whose last partial has arrived (header)
+    int* checkin;             // CTAs of this launch that have read len[] (header)
     int* status;
     void* out;                // bf16 [B][Hq][D]
     float* lse;               // [B][Hq] or nullptr
