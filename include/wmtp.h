@@ -169,6 +169,10 @@ wmtp_status wmtp_draft_loop_full_host(const wmtp_kv* kv, int gamma, const void* 
 /* Upper bound on the CTAs (KV splits) of the attention kernels; 0 restores the default
  * (one CTA per SM). Process-wide; meant for tests that exercise the split/merge path. */
 void    wmtp_set_max_ctas(int max_ctas);
+/* Tile-level work stealing between CTAs (default on): SMs that stream faster take tiles from slower ones, which
+ * shortens long launches by several percent but makes the low bits of the result depend on timing. 0 selects a
+ * fixed partition: bit-reproducible results. Process-wide. */
+void    wmtp_set_work_stealing(int enabled);
 /* Number of kernels this library has launched in this process (all threads). */
 int64_t wmtp_launch_count(void);
 
@@ -180,7 +184,7 @@ int64_t wmtp_launch_count(void);
  * library a workspace because they cannot allocate device memory themselves: plug-ins inside a runtime
  * that owns the allocator, processes whose device-memory budget is frozen at start-up, loops that must
  * not allocate once they are running. The split-KV scratch is a fixed array inside the library
- * (about 1.5 MiB, held by every GPU that loads the library until the process exits); the call, and the
+ * (about 1.8 MiB, held by every GPU that loads the library until the process exits); the call, and the
  * library on its behalf, performs no cudaMalloc / cudaFree and calls no allocating routine.
  *   - Limits: batch * Hkv <= 32, Hq / Hkv <= 8, D in {128, 256}; more is rejected with
  *     WMTP_ERR_CAPACITY / WMTP_ERR_UNSUPPORTED and nothing is launched. At most 160 CTAs are used.

@@ -66,6 +66,7 @@ _SIGNATURES = {
                                           c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "wmtp_draft_attn_windowed_noalloc": (c_int, [c_void_p, c_int, POINTER(wmtp_ring), c_float, c_void_p, c_void_p, c_void_p]),
     "wmtp_set_max_ctas": (None, [c_int]),
+    "wmtp_set_work_stealing": (None, [c_int]),
     "wmtp_launch_count": (c_int64, []),
 }
 
@@ -265,6 +266,10 @@ def wmtp_draft_attn_windowed_noalloc(q, ring: Ring, out, lse=None, sm_scale: flo
 
 def wmtp_set_max_ctas(n: int) -> None:
     lib().wmtp_set_max_ctas(int(n))
+
+
+def wmtp_set_work_stealing(enabled: bool) -> None:
+    lib().wmtp_set_work_stealing(1 if enabled else 0)
 
 
 def wmtp_launch_count() -> int:

@@ -37,7 +37,6 @@ constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kConsumerWarps = 4;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr uint32_t kSpinLimit = 1u << 22;       // bounded mbarrier waits
-constexpr uint32_t kEpochStride = 1024;         // arrival counters advance by this much per launch (> kMaxCtas)
 constexpr int kScratchRow = 132;                // floats per (warp, head) row of the merge scratch (128 + pad)
 // scratch holds either the warp merge ([4][8][kScratchRow]) or the combine's weights, inverses and reduction buffer
 constexpr int kScratchFloats = (kConsumerWarps * kMaxGroup * kScratchRow) > (kMaxGroup * kMaxCtas + 8 + 4 * 128)
@@ -71,7 +70,7 @@ struct Cfg {
             unsigned long long t_;                                                            \
             asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                            \
             unsigned long long* rec_ = reinterpret_cast<unsigned long long*>(                 \
-                (p).part_o + (size_t)(kMaxCtas + (p).B * (p).Hkv) * (p).G * (p).D) + 4 * blockIdx.x; \
+                (p).part_o + (size_t)(kMaxCtas + ((512 / ((p).B * (p).Hkv) > kStealSlotsMax ? kStealSlotsMax : 512 / ((p).B * (p).Hkv)) + 3) * (p).B * (p).Hkv) * (p).G * (p).D) + 4 * blockIdx.x; \
             rec_[i] = t_;                                                                     \
             if ((i) == 0) { unsigned sm_; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_)); rec_[3] = sm_; } \
         }                                                                                     \
@@ -123,7 +122,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
 #ifndef WMTP_L2_PROMO
 #define WMTP_L2_PROMO 3
 #endif
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t policy) {
+[[maybe_unused]] __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t policy) {
 #if WMTP_TMA_HINT
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
@@ -137,7 +136,7 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 }
 // Whole K (or V) tile in one instruction: box {64 elements, 64 rows, D/64 column chunks} of the 3-D view
 // [chunk][row][64] of the tensor; lands in shared memory as [chunk][row][128 B], 128-byte swizzled.
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int y, uint32_t bar) {
+[[maybe_unused]] __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(map), "r"(0), "r"(y), "r"(0), "r"(bar) : "memory");
@@ -170,13 +169,27 @@ __device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u <
 __device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 __device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// Bounded spin on a global counter written by other CTAs of this (cooperative) launch.
-// The counter counts up from `base` (this launch's epoch * kEpochStride); wrap-around safe.
-__device__ __forceinline__ void wait_counter(const int* ctr, uint32_t base, uint32_t target, volatile int* abort_flag, int* status) {
+// Bounded spin on a global word written by other CTAs of this (cooperative) launch: waits until
+// (value - base) >= target in wrap-around arithmetic.
+__device__ __forceinline__ uint32_t wait_word(const void* word, uint32_t base, uint32_t target, volatile int* abort_flag, int* status) {
+    uint32_t v = 0;
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(word) : "memory");
+        if (v - base >= target) return v;
+        if ((i & 255u) == 255u && *abort_flag) return v;
+        __nanosleep(32);
+    }
+    *abort_flag = 1;
+    atomicCAS(status, 0, kErrTimeout);
+    return v;
+}
+
+// Bounded spin until a global word equals `want` (an epoch tag: stale values never match).
+__device__ __forceinline__ void wait_equal(const uint32_t* word, uint32_t want, volatile int* abort_flag, int* status) {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         uint32_t v;
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
-        if (v - base >= target) return;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(word) : "memory");
+        if (v == want) return;
         if ((i & 255u) == 255u && *abort_flag) return;
         __nanosleep(32);
     }
@@ -184,12 +197,13 @@ __device__ __forceinline__ void wait_counter(const int* ctr, uint32_t base, uint
     atomicCAS(status, 0, kErrTimeout);
 }
 
-// Segment bookkeeping shared by producer and consumers.
+// One (sequence, KV head) segment as seen by a CTA.
 struct Segment {
     int b, g, seg;
-    int64_t seg_start, tiles, t_end, nk, S;
+    int64_t seg_start, tiles, nk, S;
+    int64_t slot_base;          // first partial slot of the segment
 };
-__device__ __forceinline__ Segment locate_segment(const AttnParams& p, const int64_t* tile_prefix, int64_t t, int64_t t1) {
+__device__ __forceinline__ Segment locate_segment(const AttnParams& p, const int64_t* tile_prefix, const int* cap_prefix, int64_t t) {
     Segment s;
     s.b = find_seq(tile_prefix, p.B, p.Hkv, t);
     s.tiles = tile_prefix[s.b + 1] - tile_prefix[s.b];
@@ -197,11 +211,10 @@ __device__ __forceinline__ Segment locate_segment(const AttnParams& p, const int
     const int64_t in_seq = t - seq_start;
     s.g = (in_seq < 0x7fffffffLL && s.tiles < 0x7fffffffLL) ? (int)((uint32_t)in_seq / (uint32_t)s.tiles) : (int)(in_seq / s.tiles);
     s.seg_start = seq_start + (int64_t)s.g * s.tiles;
-    const int64_t seg_end = s.seg_start + s.tiles;
-    s.t_end = seg_end < t1 ? seg_end : t1;
     s.S = eff_len(p, s.b);
     s.nk = scan_keys(p, s.b);
     s.seg = s.b * p.Hkv + s.g;
+    s.slot_base = (int64_t)p.Hkv * cap_prefix[s.b] + (int64_t)s.g * (cap_prefix[s.b + 1] - cap_prefix[s.b]);
     return s;
 }
 
@@ -216,23 +229,18 @@ __device__ __forceinline__ int64_t kv_row_offset(const AttnParams& p, int b, int
 }
 
 // ---------------------------------------------------------------------------------------------
-// Distributed combine of one segment (paper-independent split-KV algebra):
-// lse = logsumexp_s(lse_s), out = sum_s exp(lse_s - lse) * o_s. Called by the 128 consumer threads
-// of every CTA that contributed a partial to the segment, after the CTA has published its own.
-// CTA number j of the np contributors reduces the j-th slice of the (head, d) columns, so the
-// merge is spread over all SMs that worked on the segment instead of serialising on one.
+// Distributed combine of one segment (split-KV algebra): lse = logsumexp_s(lse_s),
+// out = sum_s exp(lse_s - lse) * o_s. Called by the 128 consumer threads of every CTA that contributed
+// a partial to the segment. Contributor number j of the np contributors reduces the j-th slice of the
+// (head, d) columns, so the merge is spread over all SMs that worked on the segment.
 // ---------------------------------------------------------------------------------------------
-__device__ __noinline__ void combine_segment(const AttnParams& p, const Segment& sg, int c_first, int np, int j,
-                                             float* scratch, volatile int* abort_flag, uint32_t epoch_base, bool all_arrived) {
+__device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, int64_t pbase, int np, int j, float* scratch) {
     const int tid = threadIdx.x;
     const int G = p.G, D = p.D;
     float* w_sm = scratch;                                                  // [G][np], np <= kMaxCtas
     float* inv_sm = scratch + kMaxGroup * kMaxCtas;                         // [8]
     float4* red = reinterpret_cast<float4*>(inv_sm + 8);                    // [128]
-    if (tid == 0 && !all_arrived) wait_counter(p.arrive + sg.seg, epoch_base, (uint32_t)np, abort_flag, p.status);
-    consumer_barrier();
     WMTP_STAMP(p, 7);
-    const int64_t pbase = (int64_t)c_first + sg.seg;
 
     // ---- this CTA's slice of the (head, d) columns; the first rows are requested before the weights exist
     constexpr int kPre = 4;
@@ -255,10 +263,10 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, const Segment&
     // ---- weights, all heads at once: 16 threads per head, one pass over the partial lse values
     {
         const int h = tid >> 4, li = tid & 15;
-        float x[kMaxCtas / 16];
+        float x[(kMaxCtas + 15) / 16];
         float M = -INFINITY;
 #pragma unroll
-        for (int u = 0; u < kMaxCtas / 16; ++u) {
+        for (int u = 0; u < (kMaxCtas + 15) / 16; ++u) {
             const int i = li + 16 * u;
             x[u] = (h < G && i < np) ? __ldcg(p.part_lse + (pbase + i) * G + h) : -INFINITY;
             M = fmaxf(M, x[u]);
@@ -267,7 +275,7 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, const Segment&
         for (int off = 8; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
         float sum = 0.f;
 #pragma unroll
-        for (int u = 0; u < kMaxCtas / 16; ++u) {
+        for (int u = 0; u < (kMaxCtas + 15) / 16; ++u) {
             const int i = li + 16 * u;
             if (h < G && i < np) {
                 const float w = (M > -INFINITY) ? __expf(x[u] - M) : 0.f;
@@ -279,12 +287,12 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, const Segment&
         for (int off = 8; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
         if (li == 0 && h < G) {
             inv_sm[h] = sum > 0.f ? 1.f / sum : 0.f;
-            if (j == 0 && p.lse) p.lse[(int64_t)sg.b * p.Hq + sg.g * G + h] = sum > 0.f ? M + __logf(sum) : -INFINITY;
+            if (j == 0 && p.lse) p.lse[(int64_t)b * p.Hq + g * G + h] = sum > 0.f ? M + __logf(sum) : -INFINITY;
         }
     }
     consumer_barrier();
     WMTP_STAMP(p, 8);
-    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)sg.b * p.Hq + sg.g * G) * D;
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + g * G) * D;
     for (int c0 = col_lo; c0 < col_hi; c0 += 128) {
         const int cb = col_hi - c0 < 128 ? col_hi - c0 : 128;
         const int R = 128 / cb, cl = tid % cb, rg = tid / cb;
@@ -328,44 +336,21 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, const Segment&
     }
 }
 
-// Launch-level bookkeeping lives in the workspace header and needs no reset pass and no grid barrier:
-//   epoch      every launch reads it at entry; arrival counters count up from epoch * kEpochStride, and the
-//              last arriver of a segment bumps the counter to (epoch + 1) * kEpochStride, which still
-//              satisfies every CTA that is polling it;
-//   segs_done  segments whose last partial has arrived; the CTA that completes the last segment advances
-//              the epoch and, for a fused append, the lengths. Every CTA that owns tiles has read len[]
-//              for the last time before its last arrival; CTAs without tiles check in separately.
-//   checkin    CTAs that have read len[] (entry); the length update waits until all have.
-// Called by consumer thread 0 after the segment's partial is visible. Returns true if all np partials
-// of the segment had arrived; *launch_last is set for the CTA that completed the launch's last segment.
-__device__ __forceinline__ bool publish_arrival(const AttnParams& p, int seg, int np, uint32_t epoch, int nonempty_segs,
-                                                bool* launch_last) {
-    const uint32_t old = (uint32_t)atomicAdd(p.arrive + seg, 1);
-    if (old + 1u - epoch * kEpochStride != (uint32_t)np) return false;
-    p.arrive[seg] = (int)((epoch + 1u) * kEpochStride);
-    const int old2 = atomicAdd(p.segs_done, 1);
-    if (old2 + 1 == nonempty_segs) {
-        *p.segs_done = 0;
-        *p.epoch = epoch + 1u;
-        *launch_last = true;
-    }
-    return true;
-}
-
-// By the CTA that completed the launch's last segment, after its own combine: advance the lengths of a fused append.
-__device__ __forceinline__ void advance_lengths(const AttnParams& p, volatile int* abort_flag) {
-    if (threadIdx.x == 0) {
-        wait_counter(p.checkin, 0u, gridDim.x, abort_flag, p.status);     // every CTA has read len[]
-        *p.checkin = 0;
-    }
-    consumer_barrier();
-    if (p.k_new) {
-        for (int b = threadIdx.x; b < p.B; b += 128) {
-            if (appends_to(p, b)) p.len[b] += 1;
-            else atomicCAS(p.status, 0, kErrBounds);          // append past S_cap: skipped and flagged
-        }
-    }
-}
+// Launch-level bookkeeping (workspace header and per-segment words), with no reset pass and no grid barrier:
+//   cur[c]       tiles of CTA c's dynamic part already handed out (to the owner or to thieves);
+//   nparts[s]    partial slots handed out for segment s (a CTA takes one whenever it enters s);
+//   nthief[s]    CTAs admitted into s from another segment;
+//   arrive[s]    tiles of s whose result is in a published partial; the contributor that completes the
+//                segment resets nparts/arrive, stores the partial count in ready_np[s] and releases
+//                ready[s] = epoch + 1;
+//   ready[s]     polled by the contributors before they combine; a value left by an earlier launch never
+//                equals this launch's tag;
+//   segs_done    completed segments; the CTA that completes the last one advances the epoch and, after every
+//                CTA has stopped taking tiles (grab_done, which also means it has read len[] for the last
+//                time), resets the cursors and advances the lengths of a fused append.
+constexpr int kMaxContrib = 32;     // segments a CTA may have outstanding before it combines them
+constexpr int kStealChunk = 2;      // tiles handed out per cursor step
+constexpr int kStealMinTiles = 16;  // ranges shorter than this are streamed statically
 
 // ---------------------------------------------------------------------------------------------
 // The attention kernel (one cooperative launch per draft step)
@@ -383,8 +368,14 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     float* sm_l = sm_m + kConsumerWarps * kMaxGroup;                                      // [4][8]
     float* sm_le = sm_l + kConsumerWarps * kMaxGroup;                                     // [4][8]
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm_le + kConsumerWarps * kMaxGroup);     // fullK, fullV, empty
-    int* abort_flag = reinterpret_cast<int*>(bars + 3 * C::kStages);                      // [0] abort, [1] last-CTA flag
-    int64_t* tile_prefix = reinterpret_cast<int64_t*>(abort_flag + 2);                    // [B + 1]
+    int64_t* stage_tile = reinterpret_cast<int64_t*>(bars + 3 * C::kStages);              // [kStages] global tile index, -1 = end
+    int* flags = reinterpret_cast<int*>(stage_tile + C::kStages);                         // [0] abort, [1] launch-last, [2] spare, [3] broadcast word
+    int* contrib = flags + 4;                                                             // [kMaxContrib][4]: seg, b, g, slot index k
+    volatile int* reg_k = flags + 4 + 4 * kMaxContrib;                                    // [kMaxContrib] slot index of the CTA's i-th contribution (producer -> consumers)
+    int64_t* contrib_base = reinterpret_cast<int64_t*>(contrib + 5 * kMaxContrib);        // [kMaxContrib] slot base
+    int64_t* tile_prefix = contrib_base + kMaxContrib;                                    // [B + 1]
+    int* cap_prefix = reinterpret_cast<int*>(tile_prefix + (p.B + 1));                    // [B + 1]
+    volatile int* abort_flag = flags;
 
     WMTP_STAMP(p, 0);
     WMTP_CTA_STAMP(p, 0);
@@ -400,15 +391,41 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             mbar_init(bar_fullV + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, kConsumerWarps);
         }
-        abort_flag[0] = 0;
-        abort_flag[1] = 0;
+        flags[0] = 0;
+        flags[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     const uint32_t epoch = *reinterpret_cast<const volatile uint32_t*>(p.epoch);
-    build_tile_prefix(p, tile_prefix);
+
+    // ---- plan: tiles per sequence and partial-slot capacity per sequence (all from len[], O(B))
+    for (int b = threadIdx.x; b < p.B; b += blockDim.x)
+        tile_prefix[b + 1] = (scan_keys(p, b) + kTileKeys - 1) / kTileKeys;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int64_t acc = 0;
+        tile_prefix[0] = 0;
+        for (int b = 0; b < p.B; ++b) { acc += tile_prefix[b + 1]; tile_prefix[b + 1] = acc; }
+        const int64_t n_ = acc * p.Hkv;
+        const int cn_ = effective_ctas(gridDim.x, n_);
+        int cacc = 0;
+        cap_prefix[0] = 0;
+        for (int b = 0; b < p.B; ++b) {
+            // contributors of a segment: the CTAs whose static range meets it (<= T * Cn / n + 2), thieves
+            // admitted from other segments (<= steal_slots) and one chunk that straddles into it
+            const int64_t tb = tile_prefix[b + 1] - tile_prefix[b];
+            int64_t own = tb == 0 ? 0 : (n_ < (1 << 23) ? (int64_t)(((uint32_t)tb * (uint32_t)cn_) / (uint32_t)n_) : tb * cn_ / n_) + 2;
+            if (own > tb) own = tb;
+            cacc += tb == 0 ? 0 : (int)own + p.steal_slots + 1;
+            cap_prefix[b + 1] = cacc;
+        }
+    }
+    __syncthreads();
     WMTP_STAMP(p, 1);
     const int G = p.G;
     const int nseg = p.B * p.Hkv;
+    const int64_t n = (int64_t)p.Hkv * tile_prefix[p.B];
+    const int Cg = gridDim.x;
+    const int Cn = effective_ctas(Cg, n);
     // ---- sequences that hold no token: out = 0, lse = -inf (no CTA owns a tile of theirs)
     for (int seg = blockIdx.x; seg < nseg; seg += gridDim.x) {
         const int b = seg / p.Hkv, g = seg % p.Hkv;
@@ -417,26 +434,23 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         for (int idx = threadIdx.x; idx < G * D; idx += blockDim.x) o[idx] = __float2bfloat16(0.f);
         if (p.lse && threadIdx.x < G) p.lse[(int64_t)b * p.Hq + g * G + threadIdx.x] = -INFINITY;
     }
-    const int64_t n = (int64_t)p.Hkv * tile_prefix[p.B];
-    const int Cn = effective_ctas(gridDim.x, n);
-    if (threadIdx.x == 0) {                                  // check in: this CTA has read len[] (see publish_arrival)
-        if (n > 0) {
-            atomicAdd(p.checkin, 1);
-        } else if (atomicAdd(p.checkin, 1) + 1 == (int)gridDim.x) {   // nothing to attend over at all
-            *p.checkin = 0;
+    if (n == 0) {                                            // nothing to attend over at all
+        if (threadIdx.x == 0 && atomicAdd(p.grab_done, 1) + 1 == Cg) {
+            *p.grab_done = 0;
             if (p.k_new) atomicCAS(p.status, 0, kErrBounds);
         }
+        return;
     }
-    if ((int)blockIdx.x >= Cn) return;
-    const int64_t t0 = cta_range_start(blockIdx.x, n, Cn), t1 = cta_range_start(blockIdx.x + 1, n, Cn);
-    int nonempty_segs = 0;                                   // used by consumer thread 0 only
-    if (threadIdx.x == 0)
-        for (int b = 0; b < p.B; ++b) nonempty_segs += (tile_prefix[b + 1] != tile_prefix[b]) ? p.Hkv : 0;
     WMTP_STAMP(p, 2);
     const bool slack = (p.mode == kRing) && (p.cap != p.W);
 
     if (warp == kConsumerWarps) {
         // =================================== producer warp ===================================
+        // CTA c < Cn owns the tile range [c n / Cn, (c+1) n / Cn). It streams the first part of it without any
+        // bookkeeping; the rest is handed out in small chunks through the per-CTA cursor cur[c], to the owner
+        // and, once they run dry, to other CTAs: SMs do not all stream at the same rate, and the slowest one
+        // would otherwise set the launch time. A thief prefers a victim inside the segment it is already in
+        // (no new partial); moving into another segment is admitted steal_slots times per segment.
         const uint32_t stage0 = smem_u32(stages);
         uint64_t policy = 0;
 #if WMTP_TMA_HINT == 1
@@ -444,53 +458,158 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 #elif WMTP_TMA_HINT == 2
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
 #endif
-        int64_t t = t0;
+        (void)policy;
         uint32_t it = 0;
-        while (t < t1) {
-            const Segment sg = locate_segment(p, tile_prefix, t, t1);
-            const int64_t first_tile = t - sg.seg_start;
-            const int ntiles = (int)(sg.t_end - t);
-            for (int base = 0; base < ntiles; base += 32) {
-                int page = 0;
-                if (p.mode == kPaged) {        // 32 page ids at a time, one per lane
-                    const int64_t ti = first_tile + base + lane;
-                    if (base + lane < ntiles) {
-                        page = p.page_table[(int64_t)sg.b * p.max_pages + ti];
-                        if (page < 0 || page >= p.num_pages) { atomicCAS(p.status, 0, kErrBounds); page = 0; }
-                    }
+        int cur_seg = -1;                    // segment of the last issued tile
+        int64_t cur_lo = 0, cur_hi = 0;      // its tile range
+        int ord = 0;                         // contributions (segment entries) so far
+        const bool is_owner = (int)blockIdx.x < Cn;
+
+        // tiles [a, e) of the global line (may cross segment boundaries); page ids fetched 32 at a time
+        auto issue_range = [&](int64_t a, int64_t e) {
+            int64_t t = a;
+            while (t < e) {
+                const Segment sg = locate_segment(p, tile_prefix, cap_prefix, t);
+                const int64_t seg_end = sg.seg_start + sg.tiles;
+                const int64_t t_end = seg_end < e ? seg_end : e;
+                const int64_t first_tile = t - sg.seg_start;
+                const int ntiles = (int)(t_end - t);
+                int slot_k = 0;
+                const bool entering = sg.seg != cur_seg;
+                if (entering && lane == 0) {
+                    // fixed partition: the contributors of a segment are known, so slots follow the CTA order and the
+                    // result is bit-reproducible; with stealing they are handed out first come, first served
+                    if (p.steal_slots_enabled) slot_k = atomicAdd(p.nparts + sg.seg, 1);   // consumed after the tiles are issued
+                    else slot_k = (int)blockIdx.x - tile_owner(sg.seg_start, n, Cn);
                 }
-                const int cnt = ntiles - base < 32 ? ntiles - base : 32;
-                for (int j = 0; j < cnt; ++j, ++it) {
-                    const int pg = __shfl_sync(0xffffffffu, page, j);
-                    if (lane == 0) {
-                        const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
-                        mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status);
-                        if (!*(volatile int*)abort_flag) {
-                            int64_t row;
-                            if (p.mode == kPaged) row = ((int64_t)pg * p.Hkv + sg.g) * kTileKeys;
-                            else row = ((int64_t)sg.b * p.Hkv + sg.g) * p.rows_per_head + (first_tile + base + j) * kTileKeys;
-                            const uint32_t dstK = stage0 + s * C::kStageBytes, dstV = dstK + C::kTileBytes;
-                            mbar_expect_tx(bar_fullK + 8 * s, C::kTileBytes);
+                for (int base = 0; base < ntiles; base += 32) {
+                    int page = 0;
+                    if (p.mode == kPaged) {
+                        const int64_t ti = first_tile + base + lane;
+                        if (base + lane < ntiles) {
+                            page = p.page_table[(int64_t)sg.b * p.max_pages + ti];
+                            if (page < 0 || page >= p.num_pages) { atomicCAS(p.status, 0, kErrBounds); page = 0; }
+                        }
+                    }
+                    const int cnt = ntiles - base < 32 ? ntiles - base : 32;
+                    for (int j = 0; j < cnt; ++j, ++it) {
+                        const int pg = __shfl_sync(0xffffffffu, page, j);
+                        if (lane == 0) {
+                            const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+                            mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status);
+                            if (!*abort_flag) {
+                                int64_t row;
+                                if (p.mode == kPaged) row = ((int64_t)pg * p.Hkv + sg.g) * kTileKeys;
+                                else row = ((int64_t)sg.b * p.Hkv + sg.g) * p.rows_per_head + (first_tile + base + j) * kTileKeys;
+                                const uint32_t dstK = stage0 + s * C::kStageBytes, dstV = dstK + C::kTileBytes;
+                                stage_tile[s] = t + base + j;          // ordered before the consumers' wait by the arrive below
+                                mbar_expect_tx(bar_fullK + 8 * s, C::kTileBytes);
 #if WMTP_TMA_3D
-                            tma_load_3d(dstK, &mapK, (int)row, bar_fullK + 8 * s);
+                                tma_load_3d(dstK, &mapK, (int)row, bar_fullK + 8 * s);
 #else
 #pragma unroll
-                            for (int c = 0; c < C::kChunks; ++c)
-                                tma_load_2d(dstK + c * C::kChunkBytes, &mapK, c * 64, (int)row, bar_fullK + 8 * s, policy);
+                                for (int c = 0; c < C::kChunks; ++c)
+                                    tma_load_2d(dstK + c * C::kChunkBytes, &mapK, c * 64, (int)row, bar_fullK + 8 * s, policy);
 #endif
-                            mbar_expect_tx(bar_fullV + 8 * s, C::kTileBytes);
+                                mbar_expect_tx(bar_fullV + 8 * s, C::kTileBytes);
 #if WMTP_TMA_3D
-                            tma_load_3d(dstV, &mapV, (int)row, bar_fullV + 8 * s);
+                                tma_load_3d(dstV, &mapV, (int)row, bar_fullV + 8 * s);
 #else
 #pragma unroll
-                            for (int c = 0; c < C::kChunks; ++c)
-                                tma_load_2d(dstV + c * C::kChunkBytes, &mapV, c * 64, (int)row, bar_fullV + 8 * s, policy);
+                                for (int c = 0; c < C::kChunks; ++c)
+                                    tma_load_2d(dstV + c * C::kChunkBytes, &mapV, c * 64, (int)row, bar_fullV + 8 * s, policy);
 #endif
+                            }
                         }
                     }
                 }
+                if (entering) {
+                    // the consumers read this at their flush of the segment, which follows a later arrive of ours
+                    if (lane == 0) reg_k[ord % kMaxContrib] = slot_k;
+                    ++ord;
+                    cur_seg = sg.seg; cur_lo = sg.seg_start; cur_hi = seg_end;
+                }
+                t = t_end;
             }
-            t = sg.t_end;
+        };
+        auto range_of = [&](int c, int64_t* lo, int64_t* len, int64_t* first) {
+            *lo = cta_range_start(c, n, Cn);
+            *len = cta_range_start(c + 1, n, Cn) - *lo;
+            *first = (!p.steal_slots_enabled || *len < kStealMinTiles) ? *len : *len - *len / 4;
+        };
+
+        if (is_owner) {
+            int64_t lo, len, first;
+            range_of(blockIdx.x, &lo, &len, &first);
+            issue_range(lo, lo + first);
+            // the rest of the own range, chunk by chunk through the cursor (thieves may be taking from it too)
+            const int64_t dyn = len - first;
+            if (dyn > 0) {
+                int k = 0;
+                if (lane == 0) k = atomicAdd(p.cur + blockIdx.x, kStealChunk);
+                k = __shfl_sync(0xffffffffu, k, 0);
+                while (k < dyn) {
+                    int k_next = 0;
+                    if (lane == 0) k_next = atomicAdd(p.cur + blockIdx.x, kStealChunk);       // overlaps the issue below
+                    const int64_t a = lo + first + k;
+                    issue_range(a, a + kStealChunk < lo + len ? a + kStealChunk : lo + len);
+                    k = __shfl_sync(0xffffffffu, k_next, 0);
+                }
+            }
+        }
+        if (p.steal_slots_enabled && n >= (int64_t)kStealMinTiles * Cn) {
+            // ---- steal: look at every cursor, take from the range with the most left
+            for (int round = 0; round < 4096; ++round) {
+                int64_t best_rem = 0;
+                int best_v = -1;
+                for (int v = lane; v < Cn; v += 32) {
+                    if (v == (int)blockIdx.x) continue;
+                    int64_t lo, len, first;
+                    range_of(v, &lo, &len, &first);
+                    const int64_t used = __ldcg(p.cur + v);
+                    int64_t rem = len - first - used;
+                    if (rem <= 0) continue;
+                    const int64_t tv = lo + first + used;
+                    if (cur_seg >= 0 && tv >= cur_lo && tv < cur_hi) rem += (int64_t)1 << 40;     // same segment: preferred
+                    if (rem > best_rem) { best_rem = rem; best_v = v; }
+                }
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) {
+                    const int64_t r2 = __shfl_xor_sync(0xffffffffu, best_rem, off);
+                    const int v2 = __shfl_xor_sync(0xffffffffu, best_v, off);
+                    if (r2 > best_rem || (r2 == best_rem && v2 > best_v)) { best_rem = r2; best_v = v2; }
+                }
+                if (best_v < 0 || *abort_flag) break;
+                int64_t lo, len, first;
+                range_of(best_v, &lo, &len, &first);
+                int ok = 1;
+                if (best_rem < ((int64_t)1 << 40)) {
+                    // another segment: needs a partial slot there, admitted steal_slots times per segment
+                    int admitted = 0;
+                    if (lane == 0) {
+                        const int64_t tv = lo + first + __ldcg(p.cur + best_v);
+                        const Segment vs = locate_segment(p, tile_prefix, cap_prefix, tv < lo + len ? tv : lo + len - 1);
+                        admitted = atomicAdd(p.nthief + vs.seg, 1) < p.steal_slots;
+                    }
+                    ok = __shfl_sync(0xffffffffu, admitted, 0);
+                }
+                if (!ok) break;                   // no slot for us elsewhere: stop stealing
+                int k = 0;
+                if (lane == 0) k = atomicAdd(p.cur + best_v, kStealChunk);
+                k = __shfl_sync(0xffffffffu, k, 0);
+                if (k >= len - first) continue;    // somebody else got there first: look again
+                const int64_t a = lo + first + k;
+                issue_range(a, a + kStealChunk < lo + len ? a + kStealChunk : lo + len);
+            }
+        }
+        if (lane == 0) {
+            // end marker for the consumers, then: this CTA takes no more tiles
+            const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+            mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status);
+            stage_tile[s] = -1;
+            mbar_arrive(bar_fullK + 8 * s);
+            mbar_arrive(bar_fullV + 8 * s);
+            atomicAdd(p.grab_done, 1);
         }
         return;
     }
@@ -505,39 +624,168 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     const uint32_t offK = rowK * 128, offV = rowV * 128;
     const uint32_t stage0 = smem_u32(stages);
 
-    int64_t t = t0;
-    uint32_t it = 0;
+    int nonempty_segs = 0;                               // consumer thread 0 only
+    if (threadIdx.x == 0)
+        for (int b = 0; b < p.B; ++b) nonempty_segs += (tile_prefix[b + 1] != tile_prefix[b]) ? p.Hkv : 0;
     bool launch_last = false;                            // consumer thread 0: did this CTA complete the launch's last segment?
-    while (t < t1) {
-        const Segment sg = locate_segment(p, tile_prefix, t, t1);
-        // ---- fused append (Appendix A, RING / the KV write of a draft forward): where does the new token go?
-        int64_t new_tile = -1;                              // tile (within the segment) holding the new row
-        int new_row = 0;
+    int ncontrib = 0;                                    // uniform across the consumer threads
+    int ord = 0;                                         // segment entries so far (mirrors the producer's count)
+
+    Segment sg;
+    sg.seg = -1; sg.seg_start = 0; sg.tiles = 0; sg.b = 0; sg.g = 0; sg.nk = 0; sg.S = 0; sg.slot_base = 0;
+    int64_t new_tile = -1;                               // tile (within the segment) whose row this warp must patch (fused append)
+    int new_row = 0;
+    int seg_tiles_done = 0;                              // tiles of the current segment this CTA has processed
+    uint32_t qb[C::kKSteps][2];
+    float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f}, le[2] = {0.f, 0.f};   // l: rounded weights (normaliser), le: exact (lse)
+    float o[C::kKSteps][4];
+
+    // Combine every segment this CTA has contributed to (waits for their last partial), then forget them.
+    auto combine_outstanding = [&]() {
+        for (int i = 0; i < ncontrib; ++i) {
+            const int seg = contrib[4 * i], b = contrib[4 * i + 1], g = contrib[4 * i + 2], k = contrib[4 * i + 3];
+            if (threadIdx.x == 0) {
+                wait_equal(p.ready + seg, epoch + 1u, abort_flag, p.status);
+                flags[3] = *reinterpret_cast<volatile int*>(p.ready_np + seg);
+            }
+            consumer_barrier();
+            const int np = flags[3];
+            if (np >= 1 && np <= kMaxCtas && k < np) combine_segment(p, b, g, contrib_base[i], np, k, scratch);
+            consumer_barrier();
+        }
+        ncontrib = 0;
+    };
+
+    // Merge the four warps' states, publish the partial of (this CTA, current segment), note the contribution.
+    auto flush_segment = [&]() {
+        WMTP_STAMP(p, 5);
+        WMTP_CTA_STAMP(p, 2);
+#pragma unroll
+        for (int off = 4; off <= 16; off <<= 1) {
+            l[0] += __shfl_xor_sync(0xffffffffu, l[0], off);
+            l[1] += __shfl_xor_sync(0xffffffffu, l[1], off);
+            le[0] += __shfl_xor_sync(0xffffffffu, le[0], off);
+            le[1] += __shfl_xor_sync(0xffffffffu, le[1], off);
+        }
+        consumer_barrier();                                   // scratch / sm_m free
+        if (g8 == 0) {
+            sm_m[warp * kMaxGroup + 2 * t4] = m[0]; sm_m[warp * kMaxGroup + 2 * t4 + 1] = m[1];
+            sm_l[warp * kMaxGroup + 2 * t4] = l[0]; sm_l[warp * kMaxGroup + 2 * t4 + 1] = l[1];
+            sm_le[warp * kMaxGroup + 2 * t4] = le[0]; sm_le[warp * kMaxGroup + 2 * t4 + 1] = le[1];
+        }
+        consumer_barrier();
+        const int k = reg_k[ord % kMaxContrib];               // slot the producer took when it entered the segment
+        if (threadIdx.x == 0) contrib[4 * ncontrib + 3] = k;
+        ++ord;
+        const int64_t pidx = sg.slot_base + k;
+        float f[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int h = 2 * t4 + i;
+            float M = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm_m[w * kMaxGroup + h]);
+            float L = 0.f, Le = 0.f;
+            if (M > -INFINITY) {
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    const float e = exp2f(sm_m[w * kMaxGroup + h] - M);
+                    L += sm_l[w * kMaxGroup + h] * e;
+                    Le += sm_le[w * kMaxGroup + h] * e;
+                }
+            }
+            f[i] = (L > 0.f && m[i] > -INFINITY) ? exp2f(m[i] - M) / L : 0.f;
+            if (warp == 0 && g8 == 0 && h < G) p.part_lse[pidx * G + h] = Le > 0.f ? (M + log2f(Le)) * kLn2 : -INFINITY;
+        }
+        constexpr int kPasses = D / 128;                       // 128 columns of d per pass through the scratch
+#pragma unroll
+        for (int pass = 0; pass < kPasses; ++pass) {
+            if (pass > 0) consumer_barrier();
+#pragma unroll
+            for (int mbl = 0; mbl < 8; ++mbl) {
+                const int mb = pass * 8 + mbl;
+                float* row0 = scratch + (warp * kMaxGroup + 2 * t4) * kScratchRow + mbl * 16 + g8;
+                float* row1 = row0 + kScratchRow;
+                row0[0] = o[mb][0] * f[0]; row1[0] = o[mb][1] * f[1];
+                row0[8] = o[mb][2] * f[0]; row1[8] = o[mb][3] * f[1];
+            }
+            consumer_barrier();
+            for (int idx = threadIdx.x; idx < G * 128; idx += 128) {
+                const int h = idx >> 7, dd = idx & 127;
+                float acc = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) acc += scratch[(w * kMaxGroup + h) * kScratchRow + dd];
+                p.part_o[(pidx * G + h) * D + pass * 128 + dd] = acc;
+            }
+        }
+        consumer_barrier();
+        if (threadIdx.x == 0) {
+            __threadfence();                                   // the CTA's partial is visible device-wide before the arrival
+            const int old = atomicAdd(p.arrive + sg.seg, seg_tiles_done);
+            if ((int64_t)old + seg_tiles_done == sg.tiles) {   // this contribution completes the segment
+                __threadfence();
+                const int np = p.steal_slots_enabled ? *reinterpret_cast<volatile int*>(p.nparts + sg.seg)
+                                                     : tile_owner(sg.seg_start + sg.tiles - 1, n, Cn) - tile_owner(sg.seg_start, n, Cn) + 1;
+                p.nparts[sg.seg] = 0;
+                p.nthief[sg.seg] = 0;
+                p.arrive[sg.seg] = 0;
+                p.ready_np[sg.seg] = np;
+                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.ready + sg.seg), "r"(epoch + 1u) : "memory");
+                if (atomicAdd(p.segs_done, 1) + 1 == nonempty_segs) {
+                    *p.segs_done = 0;
+                    *p.epoch = epoch + 1u;
+                    launch_last = true;
+                }
+            }
+        }
+        WMTP_STAMP(p, 6);
+        ++ncontrib;
+        if (ncontrib == kMaxContrib) combine_outstanding();
+    };
+
+    // Start work on the segment that holds tile tt: partial bookkeeping, append target, query fragments, fresh state.
+    auto enter_segment = [&](int64_t tt) {
+        sg = locate_segment(p, tile_prefix, cap_prefix, tt);
+        if (threadIdx.x == 0) {
+            contrib[4 * ncontrib] = sg.seg; contrib[4 * ncontrib + 1] = sg.b; contrib[4 * ncontrib + 2] = sg.g;
+            contrib_base[ncontrib] = sg.slot_base;
+        }
+        seg_tiles_done = 0;
+        // fused append (Appendix A, RING / the KV write of a draft forward): where does the new token go?
+        new_tile = -1;
         if (appends_to(p, sg.b)) {
             const int64_t pos = sg.S - 1;
             const int64_t key = p.mode == kRing ? ring_slot(pos, p.n_sink, p.cap) : pos;
-            new_tile = key / kTileKeys;
             new_row = (int)(key % kTileKeys);
-            if ((new_row >> 4) != warp || new_tile < t - sg.seg_start || new_tile >= sg.t_end - sg.seg_start) new_tile = -1;
+            if ((new_row >> 4) == warp) new_tile = key / kTileKeys;
         }
-        // ---- Q^T fragments (B operand: k = d, n = head); heads >= G read as zero
-        uint32_t qb[C::kKSteps][2];
-        {
-            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
-                reinterpret_cast<const __nv_bfloat16*>(p.q) + ((int64_t)sg.b * p.Hq + sg.g * G + g8) * D);
+        // Q^T fragments (B operand: k = d, n = head); heads >= G read as zero
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+            reinterpret_cast<const __nv_bfloat16*>(p.q) + ((int64_t)sg.b * p.Hq + sg.g * G + g8) * D);
 #pragma unroll
-            for (int ks = 0; ks < C::kKSteps; ++ks) {
-                qb[ks][0] = g8 < G ? __ldg(qrow + ks * 8 + t4) : 0u;
-                qb[ks][1] = g8 < G ? __ldg(qrow + ks * 8 + 4 + t4) : 0u;
-            }
+        for (int ks = 0; ks < C::kKSteps; ++ks) {
+            qb[ks][0] = g8 < G ? __ldg(qrow + ks * 8 + t4) : 0u;
+            qb[ks][1] = g8 < G ? __ldg(qrow + ks * 8 + 4 + t4) : 0u;
         }
-        float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f}, le[2] = {0.f, 0.f};   // l: rounded weights (normaliser), le: exact (lse)
-        float o[C::kKSteps][4];
+        m[0] = m[1] = -INFINITY; l[0] = l[1] = 0.f; le[0] = le[1] = 0.f;
 #pragma unroll
         for (int mb = 0; mb < C::kKSteps; ++mb) { o[mb][0] = o[mb][1] = o[mb][2] = o[mb][3] = 0.f; }
+    };
+    // an owner knows its first tile: fetch the query while that tile is still in flight
+    if ((int)blockIdx.x < Cn) enter_segment(cta_range_start(blockIdx.x, n, Cn));
 
-        for (int64_t tt = t; tt < sg.t_end; ++tt, ++it) {
-            const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+    for (uint32_t it = 0;; ++it) {
+        const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+        mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
+        if (it == 0) { WMTP_STAMP(p, 3); WMTP_CTA_STAMP(p, 1); }
+        const int64_t tt = *reinterpret_cast<volatile int64_t*>(stage_tile + s);
+        if (tt < 0 || *abort_flag) break;
+        if (sg.seg < 0 || tt < sg.seg_start || tt >= sg.seg_start + sg.tiles) {
+            if (sg.seg >= 0) flush_segment();
+            enter_segment(tt);
+        }
+        ++seg_tiles_done;
+        {
             const int64_t key0 = (tt - sg.seg_start) * kTileKeys;
             const int64_t wkey0 = key0 + warp * 16;
             const bool tile_full = (key0 + kTileKeys <= sg.nk) && !slack;
@@ -550,9 +798,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 new_off = kv_row_offset(p, sg.b, sg.g, key0 + new_row, &new_ok);
                 if (!new_ok && lane == 0) atomicCAS(p.status, 0, kErrBounds);
             }
-
-            mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
-            if (tt == t0) { WMTP_STAMP(p, 3); WMTP_CTA_STAMP(p, 1); }
             if (has_new && lane < D / 8) {
                 // the row TMA brought may be stale: take it from k_new, in shared memory and in the store
                 const uint4 x = __ldg(reinterpret_cast<const uint4*>(p.k_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8) + lane);
@@ -619,7 +864,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 }
             }
             mbar_wait(bar_fullV + 8 * s, ph, abort_flag, p.status);
-            if (tt == t0) WMTP_STAMP(p, 4);
+            if (it == 0) WMTP_STAMP(p, 4);
             if (has_new && lane < D / 8) {
                 const uint4 x = __ldg(reinterpret_cast<const uint4*>(p.v_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8) + lane);
                 const uint32_t addr = sV + (lane >> 3) * C::kChunkBytes + new_row * 128 + (((lane & 7) ^ (new_row & 7)) << 4);
@@ -653,81 +898,28 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty + 8 * s);
         }
-
-        WMTP_STAMP(p, 5);
-        WMTP_CTA_STAMP(p, 2);
-        // ---- merge the four warps' states and publish the partial of (this CTA, this segment)
-#pragma unroll
-        for (int off = 4; off <= 16; off <<= 1) {
-            l[0] += __shfl_xor_sync(0xffffffffu, l[0], off);
-            l[1] += __shfl_xor_sync(0xffffffffu, l[1], off);
-            le[0] += __shfl_xor_sync(0xffffffffu, le[0], off);
-            le[1] += __shfl_xor_sync(0xffffffffu, le[1], off);
-        }
-        consumer_barrier();                                   // scratch / sm_m free (previous segment fully done)
-        if (g8 == 0) {
-            sm_m[warp * kMaxGroup + 2 * t4] = m[0]; sm_m[warp * kMaxGroup + 2 * t4 + 1] = m[1];
-            sm_l[warp * kMaxGroup + 2 * t4] = l[0]; sm_l[warp * kMaxGroup + 2 * t4 + 1] = l[1];
-            sm_le[warp * kMaxGroup + 2 * t4] = le[0]; sm_le[warp * kMaxGroup + 2 * t4 + 1] = le[1];
-        }
-        consumer_barrier();
-        const int64_t pidx = (int64_t)blockIdx.x + sg.seg;
-        float f[2];
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const int h = 2 * t4 + i;
-            float M = -INFINITY;
-#pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm_m[w * kMaxGroup + h]);
-            float L = 0.f, Le = 0.f;
-            if (M > -INFINITY) {
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) {
-                    const float e = exp2f(sm_m[w * kMaxGroup + h] - M);
-                    L += sm_l[w * kMaxGroup + h] * e;
-                    Le += sm_le[w * kMaxGroup + h] * e;
-                }
-            }
-            f[i] = (L > 0.f && m[i] > -INFINITY) ? exp2f(m[i] - M) / L : 0.f;
-            if (warp == 0 && g8 == 0 && h < G) p.part_lse[pidx * G + h] = Le > 0.f ? (M + log2f(Le)) * kLn2 : -INFINITY;
-        }
-        constexpr int kPasses = D / 128;                       // 128 columns of d per pass through the scratch
-#pragma unroll
-        for (int pass = 0; pass < kPasses; ++pass) {
-            if (pass > 0) consumer_barrier();
-#pragma unroll
-            for (int mbl = 0; mbl < 8; ++mbl) {
-                const int mb = pass * 8 + mbl;
-                float* row0 = scratch + (warp * kMaxGroup + 2 * t4) * kScratchRow + mbl * 16 + g8;
-                float* row1 = row0 + kScratchRow;
-                row0[0] = o[mb][0] * f[0]; row1[0] = o[mb][1] * f[1];
-                row0[8] = o[mb][2] * f[0]; row1[8] = o[mb][3] * f[1];
-            }
-            consumer_barrier();
-            for (int idx = threadIdx.x; idx < G * 128; idx += 128) {
-                const int h = idx >> 7, dd = idx & 127;
-                float acc = 0.f;
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) acc += scratch[(w * kMaxGroup + h) * kScratchRow + dd];
-                p.part_o[(pidx * G + h) * D + pass * 128 + dd] = acc;
-            }
-        }
-        __threadfence();                                       // partial visible device-wide before the arrival
-        consumer_barrier();
-        const int c_first = tile_owner(sg.seg_start, n, Cn), c_last = tile_owner(sg.seg_start + sg.tiles - 1, n, Cn);
-        const int np = c_last - c_first + 1;
-        bool all_arrived = false;
-        if (threadIdx.x == 0) all_arrived = publish_arrival(p, sg.seg, np, epoch, nonempty_segs, &launch_last);
-        WMTP_STAMP(p, 6);
-
-        // ---- take part in the segment's combine
-        combine_segment(p, sg, c_first, np, (int)blockIdx.x - c_first, scratch, abort_flag, epoch * kEpochStride, all_arrived);
-        WMTP_STAMP(p, 9);
-        t = sg.t_end;
     }
-    if (threadIdx.x == 0) abort_flag[1] = launch_last ? 1 : 0;
+    if (sg.seg >= 0 && seg_tiles_done > 0) flush_segment();
+    combine_outstanding();
+    WMTP_STAMP(p, 9);
+
+    // ---- the CTA that completed the launch's last segment closes the launch
+    if (threadIdx.x == 0) flags[1] = launch_last ? 1 : 0;
     consumer_barrier();
-    if (abort_flag[1]) advance_lengths(p, abort_flag);
+    if (flags[1]) {
+        if (threadIdx.x == 0) {
+            wait_word(p.grab_done, 0u, (uint32_t)Cg, abort_flag, p.status);   // nobody takes tickets or reads len[] any more
+            *p.grab_done = 0;
+        }
+        consumer_barrier();
+        for (int c = threadIdx.x; c < Cg; c += 128) p.cur[c] = 0;
+        if (p.k_new) {
+            for (int b = threadIdx.x; b < p.B; b += 128) {
+                if (appends_to(p, b)) p.len[b] += 1;
+                else atomicCAS(p.status, 0, kErrBounds);      // append past S_cap: skipped and flagged
+            }
+        }
+    }
     WMTP_STAMP(p, 10);
 }
 
@@ -775,7 +967,8 @@ template <int D>
 size_t partial_smem_bytes(int B) {
     using C = Cfg<D>;
     return 1024 + (size_t)C::kStages * C::kStageBytes + sizeof(float) * (kScratchFloats + 3 * kConsumerWarps * kMaxGroup) +
-           sizeof(uint64_t) * 3 * C::kStages + 2 * sizeof(int) + sizeof(int64_t) * (B + 1) + 16;
+           sizeof(uint64_t) * 3 * C::kStages + sizeof(int64_t) * C::kStages + sizeof(int) * (4 + 5 * kMaxContrib) +
+           sizeof(int64_t) * kMaxContrib + (sizeof(int64_t) + sizeof(int)) * (B + 1) + 16;
 }
 
 template <int D>

@@ -15,6 +15,7 @@ namespace {
 thread_local char g_err[512] = "";
 std::atomic<int64_t> g_launches{0};
 std::atomic<int> g_max_ctas{0};
+std::atomic<int> g_stealing{1};
 
 wmtp_status fail(wmtp_status s, const char* fmt, ...) {
     va_list ap;
@@ -112,8 +113,15 @@ void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, 
     p.status = reinterpret_cast<int*>(base);
     p.epoch = reinterpret_cast<uint32_t*>(base + 4);
     p.segs_done = reinterpret_cast<int*>(base + 8);
-    p.checkin = reinterpret_cast<int*>(base + 12);
+    p.grab_done = reinterpret_cast<int*>(base + 12);
+    p.cur = reinterpret_cast<int*>(base + 256);
     p.arrive = reinterpret_cast<int*>(base + L.counters_off);
+    p.nparts = p.arrive + kMaxSegments;
+    p.nthief = p.nparts + kMaxSegments;
+    p.ready = reinterpret_cast<uint32_t*>(p.nthief + kMaxSegments);
+    p.ready_np = reinterpret_cast<int*>(p.ready + kMaxSegments);
+    p.steal_slots_enabled = g_stealing.load() ? 1 : 0;
+    p.steal_slots = p.steal_slots_enabled ? steal_slots_for(batch * Hkv) : 0;
     p.part_lse = reinterpret_cast<float*>(base + L.part_lse_off);
     p.part_o = reinterpret_cast<float*>(base + L.part_o_off);
     p.B = batch; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = Hq / Hkv;
@@ -190,6 +198,11 @@ StagePlan stage_plan(int gamma, int batch, int Hq, int Hkv, int D) {
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+int steal_slots_for(int nseg) {
+    int x = 512 / (nseg < 1 ? 1 : nseg);
+    return x > kStealSlotsMax ? kStealSlotsMax : x;
+}
+
 int sm_count() {
     static std::atomic<int> cached{0};
     int c = cached.load();
@@ -204,8 +217,8 @@ int sm_count() {
 
 WorkspaceLayout workspace_layout(int batch, int Hq, int Hkv, int D) {
     WorkspaceLayout L;
-    const size_t G = (size_t)(Hq / Hkv), nseg = (size_t)batch * Hkv, np = kMaxCtas + nseg;
-    L.counters_off = 256;
+    const size_t G = (size_t)(Hq / Hkv), nseg = (size_t)batch * Hkv, np = (size_t)kMaxCtas + (size_t)(steal_slots_for((int)nseg) + 3) * nseg;
+    L.counters_off = 256 + kCursorBytes;
     L.part_lse_off = kWorkspaceZeroBytes;
     L.part_o_off = L.part_lse_off + round_up(np * G * sizeof(float), 256);
     L.total = L.part_o_off + round_up(np * G * D * sizeof(float), 256);
@@ -400,6 +413,8 @@ wmtp_status wmtp_draft_loop_full_host(const wmtp_kv* kv, int gamma, const void* 
 
 void wmtp_set_max_ctas(int max_ctas) { g_max_ctas.store(max_ctas < 0 ? 0 : max_ctas); }
 
+void wmtp_set_work_stealing(int enabled) { g_stealing.store(enabled ? 1 : 0); }
+
 int64_t wmtp_launch_count(void) { return g_launches.load(); }
 
 // ---- allocation-free windowed attention ---------------------------------------------------------
@@ -411,13 +426,13 @@ int64_t wmtp_launch_count(void) { return g_launches.load(); }
 namespace {
 constexpr int kStaticMaxCtas = 160;        // CTAs (KV splits) the static scratch has room for
 constexpr int kStaticMaxSegments = 32;     // batch * Hkv
-constexpr size_t kStaticCountersOff = 256;
-constexpr size_t kStaticPartLseOff = kStaticCountersOff + 256;                                     // 32 arrival counters, padded
-constexpr size_t kStaticPartOOff = kStaticPartLseOff + (kStaticMaxCtas + kStaticMaxSegments) * kMaxGroup * sizeof(float);
-constexpr size_t kStaticBytes = kStaticPartOOff + (size_t)(kStaticMaxCtas + kStaticMaxSegments) * kMaxGroup * 256 * sizeof(float);
+constexpr size_t kStaticCountersOff = 256 + kCursorBytes;
+constexpr size_t kStaticPartLseOff = kStaticCountersOff + 5 * sizeof(int) * kStaticMaxSegments + 128; // five per-segment arrays, padded to 256
+constexpr size_t kStaticPartOOff = kStaticPartLseOff + (kStaticMaxCtas + 3 * kStaticMaxSegments) * kMaxGroup * sizeof(float);
+constexpr size_t kStaticBytes = kStaticPartOOff + (size_t)(kStaticMaxCtas + 3 * kStaticMaxSegments) * kMaxGroup * 256 * sizeof(float);
 static_assert(kStaticPartLseOff % 256 == 0 && kStaticPartOOff % 256 == 0, "static scratch regions must stay 256-byte aligned");
 
-static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];   // ~1.5 MiB
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];   // ~1.8 MiB
 
 // In host code the array's name is only a handle; the device address must be asked for, once per device.
 std::mutex g_static_mu;
@@ -465,8 +480,15 @@ wmtp_status wmtp_draft_attn_windowed_noalloc(const void* q, int Hq, const wmtp_r
     p.status = reinterpret_cast<int*>(base);
     p.epoch = reinterpret_cast<uint32_t*>(base + 4);
     p.segs_done = reinterpret_cast<int*>(base + 8);
-    p.checkin = reinterpret_cast<int*>(base + 12);
+    p.grab_done = reinterpret_cast<int*>(base + 12);
+    p.cur = reinterpret_cast<int*>(base + 256);
     p.arrive = reinterpret_cast<int*>(base + kStaticCountersOff);
+    p.nparts = p.arrive + kStaticMaxSegments;
+    p.nthief = p.nparts + kStaticMaxSegments;
+    p.ready = reinterpret_cast<uint32_t*>(p.nthief + kStaticMaxSegments);
+    p.ready_np = reinterpret_cast<int*>(p.ready + kStaticMaxSegments);
+    p.steal_slots_enabled = 0;                 // static partition: deterministic and the smallest partial pool
+    p.steal_slots = 0;
     p.part_lse = reinterpret_cast<float*>(base + kStaticPartLseOff);
     p.part_o = reinterpret_cast<float*>(base + kStaticPartOOff);
     p.B = ring->batch; p.Hq = Hq; p.Hkv = ring->Hkv; p.D = ring->D; p.G = Hq / ring->Hkv;

@@ -9,23 +9,28 @@
 namespace wmtp {
 
 constexpr int kTileKeys = 64;       // keys per K/V tile; equals the page size of the paged layout
-constexpr int kMaxCtas = 256;       // upper bound on attention CTAs (one per SM), sizes the partial buffers
+constexpr int kMaxCtas = 160;       // upper bound on attention CTAs (one per SM; a B200 has 148)
+constexpr int kStealSlotsMax = 16;   // thieves a segment admits from other segments (fewer when there are many segments)
 constexpr int kMaxBatch = 1024;     // sequences per call (prefix table lives in shared memory)
 constexpr int kMaxGroup = 8;        // query heads per KV head
 constexpr int kMaxSegments = 16384; // batch * Hkv per call
-constexpr size_t kWorkspaceZeroBytes = 256 + sizeof(int) * kMaxSegments;   // header + arrival counters
+constexpr size_t kCursorBytes = 1024;                                          // int cur[kMaxCtas], padded
+constexpr size_t kWorkspaceZeroBytes = 256 + kCursorBytes + 5 * sizeof(int) * kMaxSegments;   // header + cursors + per-segment arrays
 
 enum KvMode : int { kContiguous = 0, kPaged = 1, kRing = 2 };
 
 // Workspace layout (all offsets from a 256-byte aligned base):
-//   [0, 256)            header: int status @0, uint epoch @4, int segs_done @8, int checkin @12
-//   counters            int arrive[kMaxSegments] (fixed size: initialisation needs no shape)
-//   part_lse            float [kMaxCtas + batch * Hkv][G]
-//   part_o              float [kMaxCtas + batch * Hkv][G][D]
+//   [0, 256)            header: int status @0, uint epoch @4, int segs_done @8, int grab_done @12
+//   [256, 1280)         int cur[kMaxCtas]: per-CTA cursors of the work-stealing scheme
+//   counters            int arrive[kMaxSegments], nparts[..], nthief[..], uint ready[..], int ready_np[..]
+//                       (fixed size: initialisation needs no shape)
+//   part_lse            float [slots][G]        slots = kMaxCtas + (steal_slots + 3) * batch * Hkv
+//   part_o              float [slots][G][D]
 struct WorkspaceLayout {
     size_t counters_off, part_lse_off, part_o_off, total;
 };
 WorkspaceLayout workspace_layout(int batch, int Hq, int Hkv, int D);
+int steal_slots_for(int nseg);   // kStealSlotsMax for few segments, fewer as batch * Hkv grows
 
 // Everything the attention kernel needs; passed by value.
 struct AttnParams {
@@ -39,10 +44,17 @@ struct AttnParams {
     int32_t* slot_pos;        // ring only: [B][n_sink + cap]
     float* part_o;
     float* part_lse;
-    int* arrive;              // [segments]: CTAs that have published their partial of the segment
-    uint32_t* epoch;          // launch counter (header); arrival counters count from epoch * stride
-    int* segs_done;           // segments whose last partial has arrived (header)
-    int* checkin;             // CTAs of this launch that have read len[] (header)
+    int* arrive;              // [segments]: tiles of the segment covered by published partials
+    int* nparts;              // [segments]: partial slots handed out
+    uint32_t* ready;          // [segments]: epoch tag released when the segment's last partial is in
+    int* ready_np;            // [segments]: number of partials, valid once ready matches
+    uint32_t* epoch;          // launch counter (header)
+    int* segs_done;           // completed segments (header)
+    int* grab_done;           // CTAs that take no more tickets (header)
+    int* cur;                 // [CTAs]: tiles of each CTA's dynamic part handed out so far
+    int* nthief;              // [segments]: CTAs admitted from other segments
+    int steal_slots;          // thieves a segment admits from other segments
+    int steal_slots_enabled;  // 0: purely static partition (deterministic, smallest partial pool)
     int* status;
     void* out;                // bf16 [B][Hq][D]
     float* lse;               // [B][Hq] or nullptr

@@ -23,8 +23,10 @@ pytestmark = pytest.mark.gpu
 @pytest.fixture(autouse=True)
 def _default_ctas():
     wm.wmtp_set_max_ctas(0)
+    wm.wmtp_set_work_stealing(True)
     yield
     wm.wmtp_set_max_ctas(0)
+    wm.wmtp_set_work_stealing(True)
 
 
 def _cfg(**kw):
@@ -253,15 +255,31 @@ def test_host_buffer_loop_matches_device_loop():
     lh = torch.empty(qh.shape[:-1], dtype=torch.float32).pin_memory()
     wm.wmtp_ring_init_from_kv(dw2.ring, dw2.kv)
     wm.wmtp_draft_loop_windowed_host(dw2.ring, qh, kh, vh, oh_w, stage, dw2.ws, lse_host=lh)
-    assert torch.equal(oh_w.view(torch.int16), dw.out_w.cpu().view(torch.int16))
-    assert torch.equal(lh, dw.lse_w.cpu())
+    # same kernels on the same bits; equal up to the order in which split-KV partials are summed
+    assert (oh_w.float() - dw.out_w.cpu().float()).abs().max().item() <= 4e-3
+    assert (lh - dw.lse_w.cpu()).abs().max().item() <= 1e-4
     wm.wmtp_draft_loop_full_host(dw2.kv, qh, kh, vh, oh_f, stage, dw2.ws)
-    assert torch.equal(oh_f.view(torch.int16), dw.out_f.cpu().view(torch.int16))
+    assert (oh_f.float() - dw.out_f.cpu().float()).abs().max().item() <= 4e-3
 
 
 # ------------------------------------------------------------------------------------------ benchmark configurations
 def test_config_tiny_full_gamma_loop():
     _run_and_check(wi.CONFIGS[0])
+
+
+def test_fixed_partition_is_bit_reproducible_and_stealing_agrees():
+    cfg = wi.scaled(wi.CONFIGS[1], S0=40000, gamma=2, name="repro")
+    wl = wi.make_workload(cfg)
+    outs = []
+    for stealing in (False, False, True):
+        wm.wmtp_set_work_stealing(stealing)
+        dw = DeviceWorkload(wl)
+        dw.run_loops()
+        outs.append((dw.out_f.clone(), dw.lse_f.clone(), dw.out_w.clone()))
+    assert torch.equal(outs[0][0].view(torch.int16), outs[1][0].view(torch.int16))
+    assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2].view(torch.int16), outs[1][2].view(torch.int16))
+    assert (outs[0][0].float() - outs[2][0].float()).abs().max().item() <= 4e-3
+    assert (outs[0][1] - outs[2][1]).abs().max().item() <= 1e-4
 
 
 def test_config_s128k():

@@ -48,8 +48,8 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row(D):
         d = (got.float() - ref.float()).abs()
         assert d.max().item() <= 2e-2 and d.mean().item() <= 2e-3          # the tolerance of the parity tests
         assert (got_lse - ref_lse).abs().max().item() <= 1e-3
-        # same kernels, same split: in fact identical
-        assert torch.equal(got.view(torch.int16), ref.view(torch.int16))
+        # same kernels on the same bits: equal up to the order in which split-KV partials are summed
+        assert d.max().item() <= 4e-3
 
 
 def test_noalloc_rejects_shapes_beyond_its_scratch():
