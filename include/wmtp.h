@@ -184,7 +184,7 @@ int64_t wmtp_launch_count(void);
  * library a workspace because they cannot allocate device memory themselves: plug-ins inside a runtime
  * that owns the allocator, processes whose device-memory budget is frozen at start-up, loops that must
  * not allocate once they are running. The split-KV scratch is a fixed array inside the library
- * (about 1.8 MiB, held by every GPU that loads the library until the process exits); the call, and the
+ * (about 4 MiB, held by every GPU that loads the library until the process exits); the call, and the
  * library on its behalf, performs no cudaMalloc / cudaFree and calls no allocating routine.
  *   - Limits: batch * Hkv <= 32, Hq / Hkv <= 8, D in {128, 256}; more is rejected with
  *     WMTP_ERR_CAPACITY / WMTP_ERR_UNSUPPORTED and nothing is launched. At most 160 CTAs are used.

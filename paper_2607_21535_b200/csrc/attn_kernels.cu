@@ -6,22 +6,27 @@
 // all S positions for the full-context (native) draft of Section 3. The work is bound by the
 // HBM read of K and V, so the kernel is organised around keeping bytes in flight:
 //
-//   * one persistent CTA per SM owns a contiguous range of 64-key tiles (attn_plan.cuh);
+//   * one persistent CTA per SM; the tile line (attn_plan.cuh) is split into one contiguous range per
+//     CTA, and the tail of every range can be taken over by CTAs that finish early (SMs do not all
+//     stream at the same rate);
 //   * a producer warp streams K and V tiles into a ring of shared-memory stages with TMA
-//     (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers);
-//   * four consumer warps each take 16 keys of every tile. Scores are computed as
-//     S^T[key, head] = K[key, :] . Q^T (keys on the MMA M dimension, the G <= 8 query heads of
-//     the GQA group exactly on N = 8), the online softmax runs in fp32, and
-//     O^T[d, head] += V^T[d, key] . P^T[key, head] accumulates in registers. The 8-row problem
-//     is far too small for tcgen05 (M >= 64); mma.sync.m16n8k16 needs ~3% of tensor peak here.
+//     (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers) and tells the consumers
+//     which tile each stage holds;
+//   * consumer groups of four warps take whole tiles in turn (one group for head_dim 256, two for
+//     head_dim 128, where a tile carries half the bytes for the same softmax work); each warp of a
+//     group takes 16 keys of the tile. Scores are computed as S^T[key, head] = K[key, :] . Q^T (keys
+//     on the MMA M dimension, the G <= 8 query heads of the GQA group exactly on N = 8), the online
+//     softmax runs in fp32, and O^T[d, head] += V^T[d, key] . P^T[key, head] accumulates in
+//     registers. The 8-row problem is far too small for tcgen05 (M >= 64); mma.sync.m16n8k16 needs a
+//     few percent of tensor peak here;
 //   * every K/V byte is read once from HBM and once from shared memory, shared by all heads
 //     of the group;
-//   * the launch is cooperative (all CTAs co-resident): after publishing its partial a CTA waits,
+//   * the launch is cooperative (all CTAs co-resident): after publishing its partial a group waits,
 //     with a bounded spin, for the other contributors of its segment and reduces its slice of the
 //     output, so the merge needs no second launch and no single CTA serialises it;
 //   * a draft step's append (Appendix A, RING; the KV write of a draft forward) is fused: the warp
 //     that owns the new token's row patches the tile in shared memory from k_new / v_new and stores
-//     the row to the KV store; the last CTA of the grid advances len[].
+//     the row to the KV store; the group that completes the launch's last segment advances len[].
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -34,13 +39,22 @@ namespace {
 constexpr int kErrBounds = WMTP_ERR_DEVICE_BOUNDS;
 constexpr int kErrTimeout = WMTP_ERR_DEVICE_TIMEOUT;
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr int kConsumerWarps = 4;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
-constexpr uint32_t kSpinLimit = 1u << 22;       // bounded mbarrier waits
+constexpr int kGroupWarps = 4;                  // warps per consumer group: 4 x 16 keys = one tile
+constexpr int kGroupThreads = kGroupWarps * 32;
+constexpr int kMaxGroups = 2;
+constexpr int kMaxParts = kMaxGroups * kMaxCtas; // partials one segment can receive
+constexpr uint32_t kSpinLimit = 1u << 22;       // bounded waits
 constexpr int kScratchRow = 132;                // floats per (warp, head) row of the merge scratch (128 + pad)
-// scratch holds either the warp merge ([4][8][kScratchRow]) or the combine's weights, inverses and reduction buffer
-constexpr int kScratchFloats = (kConsumerWarps * kMaxGroup * kScratchRow) > (kMaxGroup * kMaxCtas + 8 + 4 * 128)
-                                   ? (kConsumerWarps * kMaxGroup * kScratchRow) : (kMaxGroup * kMaxCtas + 8 + 4 * 128);
+// per-group scratch: either the warp merge ([4][8][kScratchRow]) or the combine's weights, inverses, ranks and reduction buffer
+constexpr int kCombineFloats = kMaxGroup * kMaxParts + 8 + 4 * kGroupThreads + kMaxParts;
+constexpr int kMergeFloats = kGroupWarps * kMaxGroup * kScratchRow;
+constexpr int kScratchFloats = kMergeFloats > kCombineFloats ? kMergeFloats : kCombineFloats;
+constexpr int kMaxContrib = 32;     // segments a group may have outstanding before it combines them
+constexpr int kStealChunk = 2;      // tiles handed out per cursor step
+constexpr int kStealMinTiles = 16;  // ranges shorter than this are streamed statically
+// per-group bookkeeping in shared memory (ints): [0] launch-last flag, [1] broadcast word, then
+// contrib[kMaxContrib][4] = {seg, b, g, slot}, reg_k[kMaxContrib] (slot of the group's i-th contribution, producer -> group)
+constexpr int kGroupInts = 4 + 5 * kMaxContrib;
 
 template <int D>
 struct Cfg {
@@ -48,8 +62,15 @@ struct Cfg {
     static constexpr int kChunkBytes = kTileKeys * 128;       // one TMA box: 64 rows x 128 B
     static constexpr int kTileBytes = kChunks * kChunkBytes;  // K (or V) tile
     static constexpr int kStageBytes = 2 * kTileBytes;
-    static constexpr int kStages = (D == 256) ? 3 : 6;
+    static constexpr int kGroups = (D == 256) ? 1 : 2;        // consumer groups
+    static constexpr int kStages = (D == 256) ? 3 : 5;
+    static constexpr int kConsumerWarps = kGroups * kGroupWarps;
+    static constexpr int kThreads = (kConsumerWarps + 1) * 32;
     static constexpr int kKSteps = D / 16;
+    static constexpr int kBarriers = (1 + 2 * kGroups) * kStages;
+    // iterations between two uses of the same stage by the same group: lcm(kStages, kGroups)
+    static constexpr int kUsePeriod = (kStages % kGroups == 0) ? kStages : kStages * kGroups;
+    static_assert(kGroups == 1 || kGroups == 2, "kUsePeriod assumes one or two groups");
 };
 
 // Development aid (compiled out unless WMTP_TRACE is defined): CTA 0 records %globaltimer at phase boundaries
@@ -70,7 +91,7 @@ struct Cfg {
             unsigned long long t_;                                                            \
             asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                            \
             unsigned long long* rec_ = reinterpret_cast<unsigned long long*>(                 \
-                (p).part_o + (size_t)(kMaxCtas + ((512 / ((p).B * (p).Hkv) > kStealSlotsMax ? kStealSlotsMax : 512 / ((p).B * (p).Hkv)) + 3) * (p).B * (p).Hkv) * (p).G * (p).D) + 4 * blockIdx.x; \
+                (p).part_o + pool_slots((p).B * (p).Hkv) * (p).G * (p).D) + 4 * blockIdx.x; \
             rec_[i] = t_;                                                                     \
             if ((i) == 0) { unsigned sm_; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_)); rec_[3] = sm_; } \
         }                                                                                     \
@@ -167,7 +188,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 __device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
-__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void group_barrier(int grp) { asm volatile("bar.sync %0, 128;" ::"r"(grp + 1) : "memory"); }
 
 // Bounded spin on a global word written by other CTAs of this (cooperative) launch: waits until
 // (value - base) >= target in wrap-around arithmetic.
@@ -202,6 +223,7 @@ struct Segment {
     int b, g, seg;
     int64_t seg_start, tiles, nk, S;
     int64_t slot_base;          // first partial slot of the segment
+    int cap;                    // partial slots the segment has
 };
 __device__ __forceinline__ Segment locate_segment(const AttnParams& p, const int64_t* tile_prefix, const int* cap_prefix, int64_t t) {
     Segment s;
@@ -214,7 +236,8 @@ __device__ __forceinline__ Segment locate_segment(const AttnParams& p, const int
     s.S = eff_len(p, s.b);
     s.nk = scan_keys(p, s.b);
     s.seg = s.b * p.Hkv + s.g;
-    s.slot_base = (int64_t)p.Hkv * cap_prefix[s.b] + (int64_t)s.g * (cap_prefix[s.b + 1] - cap_prefix[s.b]);
+    s.cap = cap_prefix[s.b + 1] - cap_prefix[s.b];
+    s.slot_base = (int64_t)p.Hkv * cap_prefix[s.b] + (int64_t)s.g * s.cap;
     return s;
 }
 
@@ -230,19 +253,38 @@ __device__ __forceinline__ int64_t kv_row_offset(const AttnParams& p, int b, int
 
 // ---------------------------------------------------------------------------------------------
 // Distributed combine of one segment (split-KV algebra): lse = logsumexp_s(lse_s),
-// out = sum_s exp(lse_s - lse) * o_s. Called by the 128 consumer threads of every CTA that contributed
+// out = sum_s exp(lse_s - lse) * o_s. Called by the 128 threads of every consumer group that contributed
 // a partial to the segment. Contributor number j of the np contributors reduces the j-th slice of the
 // (head, d) columns, so the merge is spread over all SMs that worked on the segment.
+// With the fixed partition the partials are visited in the order of their keys (CTA, group), which makes
+// the result independent of the order in which the slots were handed out: bit-reproducible.
 // ---------------------------------------------------------------------------------------------
-__device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, int64_t pbase, int np, int j, float* scratch) {
-    const int tid = threadIdx.x;
+__device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, int64_t pbase, int np, int j, float* scratch,
+                                             int tid, int grp) {
     const int G = p.G, D = p.D;
-    float* w_sm = scratch;                                                  // [G][np], np <= kMaxCtas
-    float* inv_sm = scratch + kMaxGroup * kMaxCtas;                         // [8]
+    float* w_sm = scratch;                                                  // [G][np], np <= kMaxParts
+    float* inv_sm = scratch + kMaxGroup * kMaxParts;                        // [8]
     float4* red = reinterpret_cast<float4*>(inv_sm + 8);                    // [128]
+    int* perm = reinterpret_cast<int*>(inv_sm + 8 + 4 * kGroupThreads);     // [np] visiting order
     WMTP_STAMP(p, 7);
 
-    // ---- this CTA's slice of the (head, d) columns; the first rows are requested before the weights exist
+    // ---- visiting order
+    if (p.steal_slots_enabled) {
+        for (int i = tid; i < np; i += kGroupThreads) perm[i] = i;
+    } else {
+        int* keys = reinterpret_cast<int*>(red);                            // borrowed until the first barrier below
+        for (int i = tid; i < np; i += kGroupThreads) keys[i] = __ldcg(p.part_key + pbase + i);
+        group_barrier(grp);
+        for (int i = tid; i < np; i += kGroupThreads) {
+            const int ki = keys[i];
+            int r = 0;
+            for (int q = 0; q < np; ++q) r += keys[q] < ki;
+            perm[r] = i;
+        }
+    }
+    group_barrier(grp);
+
+    // ---- this group's slice of the (head, d) columns; the first rows are requested before the weights exist
     constexpr int kPre = 4;
     const int vec = D / 4, cols = G * vec;
     const int cpc = (cols + np - 1) / np;
@@ -250,32 +292,33 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
     const float4* rows = reinterpret_cast<const float4*>(p.part_o);
     float4 pre[kPre];
     {
-        const int cb = col_hi - col_lo < 128 ? col_hi - col_lo : 128;
+        const int cb = col_hi - col_lo < kGroupThreads ? col_hi - col_lo : kGroupThreads;
         if (cb > 0) {
-            const int R = 128 / cb, cl = tid % cb, rg = tid / cb;
+            const int R = kGroupThreads / cb, cl = tid % cb, rg = tid / cb;
 #pragma unroll
             for (int u = 0; u < kPre; ++u) {
                 const int i = rg + u * R;
-                pre[u] = (rg < R && i < np) ? __ldcg(rows + (pbase + i) * cols + col_lo + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
+                pre[u] = (rg < R && i < np) ? __ldcg(rows + (pbase + perm[i]) * cols + col_lo + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
     }
     // ---- weights, all heads at once: 16 threads per head, one pass over the partial lse values
     {
         const int h = tid >> 4, li = tid & 15;
-        float x[(kMaxCtas + 15) / 16];
+        constexpr int kPer = (kMaxParts + 15) / 16;
+        float x[kPer];
         float M = -INFINITY;
 #pragma unroll
-        for (int u = 0; u < (kMaxCtas + 15) / 16; ++u) {
+        for (int u = 0; u < kPer; ++u) {
             const int i = li + 16 * u;
-            x[u] = (h < G && i < np) ? __ldcg(p.part_lse + (pbase + i) * G + h) : -INFINITY;
+            x[u] = (h < G && i < np) ? __ldcg(p.part_lse + (pbase + perm[i]) * G + h) : -INFINITY;
             M = fmaxf(M, x[u]);
         }
 #pragma unroll
         for (int off = 8; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
         float sum = 0.f;
 #pragma unroll
-        for (int u = 0; u < (kMaxCtas + 15) / 16; ++u) {
+        for (int u = 0; u < kPer; ++u) {
             const int i = li + 16 * u;
             if (h < G && i < np) {
                 const float w = (M > -INFINITY) ? __expf(x[u] - M) : 0.f;
@@ -290,12 +333,12 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
             if (j == 0 && p.lse) p.lse[(int64_t)b * p.Hq + g * G + h] = sum > 0.f ? M + __logf(sum) : -INFINITY;
         }
     }
-    consumer_barrier();
+    group_barrier(grp);
     WMTP_STAMP(p, 8);
     __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + g * G) * D;
-    for (int c0 = col_lo; c0 < col_hi; c0 += 128) {
-        const int cb = col_hi - c0 < 128 ? col_hi - c0 : 128;
-        const int R = 128 / cb, cl = tid % cb, rg = tid / cb;
+    for (int c0 = col_lo; c0 < col_hi; c0 += kGroupThreads) {
+        const int cb = col_hi - c0 < kGroupThreads ? col_hi - c0 : kGroupThreads;
+        const int R = kGroupThreads / cb, cl = tid % cb, rg = tid / cb;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (rg < R) {
             const int col = c0 + cl, h = col / vec;
@@ -313,12 +356,12 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
 #pragma unroll 4
             for (; i < np; i += R) {
                 const float w = w_sm[h * np + i];
-                const float4 x = __ldcg(rows + (pbase + i) * cols + col);
+                const float4 x = __ldcg(rows + (pbase + perm[i]) * cols + col);
                 acc.x = fmaf(w, x.x, acc.x); acc.y = fmaf(w, x.y, acc.y); acc.z = fmaf(w, x.z, acc.z); acc.w = fmaf(w, x.w, acc.w);
             }
         }
         red[tid] = acc;
-        consumer_barrier();
+        group_barrier(grp);
         if (tid < cb) {
             float4 o = red[tid];
             for (int r = 1; r < R; ++r) {
@@ -332,67 +375,65 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
             packed.y = pack_bf16x2(o.z * inv, o.w * inv);
             *reinterpret_cast<uint2*>(out + (int64_t)col * 4) = packed;
         }
-        consumer_barrier();
+        group_barrier(grp);
     }
 }
 
 // Launch-level bookkeeping (workspace header and per-segment words), with no reset pass and no grid barrier:
 //   cur[c]       tiles of CTA c's dynamic part already handed out (to the owner or to thieves);
-//   nparts[s]    partial slots handed out for segment s (a CTA takes one whenever it enters s);
+//   nparts[s]    partial slots handed out for segment s (a consumer group takes one whenever it enters s);
 //   nthief[s]    CTAs admitted into s from another segment;
 //   arrive[s]    tiles of s whose result is in a published partial; the contributor that completes the
-//                segment resets nparts/arrive, stores the partial count in ready_np[s] and releases
+//                segment resets nparts/nthief/arrive, stores the partial count in ready_np[s] and releases
 //                ready[s] = epoch + 1;
 //   ready[s]     polled by the contributors before they combine; a value left by an earlier launch never
 //                equals this launch's tag;
-//   segs_done    completed segments; the CTA that completes the last one advances the epoch and, after every
+//   segs_done    completed segments; the group that completes the last one advances the epoch and, after every
 //                CTA has stopped taking tiles (grab_done, which also means it has read len[] for the last
 //                time), resets the cursors and advances the lengths of a fused append.
-constexpr int kMaxContrib = 32;     // segments a CTA may have outstanding before it combines them
-constexpr int kStealChunk = 2;      // tiles handed out per cursor step
-constexpr int kStealMinTiles = 16;  // ranges shorter than this are streamed statically
 
 // ---------------------------------------------------------------------------------------------
 // The attention kernel (one cooperative launch per draft step)
 // ---------------------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(Cfg<D>::kThreads, 1)
 attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                const __grid_constant__ AttnParams p) {
     using C = Cfg<D>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char* stages = smem;                                                         // kStages x (K tile, V tile)
-    float* scratch = reinterpret_cast<float*>(stages + C::kStages * C::kStageBytes);      // merge / combine scratch
-    float* sm_m = scratch + kScratchFloats;                                               // [4][8]
-    float* sm_l = sm_m + kConsumerWarps * kMaxGroup;                                      // [4][8]
-    float* sm_le = sm_l + kConsumerWarps * kMaxGroup;                                     // [4][8]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sm_le + kConsumerWarps * kMaxGroup);     // fullK, fullV, empty
-    int64_t* stage_tile = reinterpret_cast<int64_t*>(bars + 3 * C::kStages);              // [kStages] global tile index, -1 = end
-    int* flags = reinterpret_cast<int*>(stage_tile + C::kStages);                         // [0] abort, [1] launch-last, [2] spare, [3] broadcast word
-    int* contrib = flags + 4;                                                             // [kMaxContrib][4]: seg, b, g, slot index k
-    volatile int* reg_k = flags + 4 + 4 * kMaxContrib;                                    // [kMaxContrib] slot index of the CTA's i-th contribution (producer -> consumers)
-    int64_t* contrib_base = reinterpret_cast<int64_t*>(contrib + 5 * kMaxContrib);        // [kMaxContrib] slot base
-    int64_t* tile_prefix = contrib_base + kMaxContrib;                                    // [B + 1]
+    float* scratch_all = reinterpret_cast<float*>(stages + C::kStages * C::kStageBytes);  // [kGroups][kScratchFloats]
+    float* sm_stats = scratch_all + C::kGroups * kScratchFloats;                          // [kGroups][3][4][8]: m, l, le per warp and head
+    // Barriers: empty[stage] (the producer observes every use of a stage) and, per consumer group, fullK / fullV[stage].
+    // A group only sees the uses of a stage that are its own, and a parity wait can only tell consecutive phases
+    // apart, so the "full" barriers must not be shared between groups.
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm_stats + C::kGroups * 3 * kGroupWarps * kMaxGroup);
+    int64_t* stage_tile = reinterpret_cast<int64_t*>(bars + C::kBarriers);                // [kStages] global tile index, -1 = end
+    int64_t* contrib_base_all = stage_tile + C::kStages;                                  // [kGroups][kMaxContrib] slot base
+    int64_t* tile_prefix = contrib_base_all + C::kGroups * kMaxContrib;                   // [B + 1]
     int* cap_prefix = reinterpret_cast<int*>(tile_prefix + (p.B + 1));                    // [B + 1]
-    volatile int* abort_flag = flags;
+    int* group_ints = cap_prefix + (p.B + 1);                                             // [kGroups][kGroupInts]
+    int* cta_flags = group_ints + C::kGroups * kGroupInts;                                // [0] abort
+    volatile int* abort_flag = cta_flags;
 
     WMTP_STAMP(p, 0);
     WMTP_CTA_STAMP(p, 0);
-    if (threadIdx.x == kConsumerWarps * 32) {               // descriptor fetch overlaps the len[] round trip
+    if (threadIdx.x == C::kConsumerWarps * 32) {            // descriptor fetch overlaps the len[] round trip
         asm volatile("prefetch.tensormap [%0];" ::"l"(&mapK) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&mapV) : "memory");
     }
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t bar_fullK = smem_u32(bars), bar_fullV = smem_u32(bars + C::kStages), bar_empty = smem_u32(bars + 2 * C::kStages);
+    const int lane = threadIdx.x & 31;
+    const uint32_t bar_empty = smem_u32(bars), bar_fullK0 = smem_u32(bars + C::kStages), bar_fullV0 = smem_u32(bars + (1 + C::kGroups) * C::kStages);
     if (threadIdx.x == 0) {                                  // under the shadow of the len[] round trip
         for (int s = 0; s < C::kStages; ++s) {
-            mbar_init(bar_fullK + 8 * s, 1);
-            mbar_init(bar_fullV + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, kConsumerWarps);
+            mbar_init(bar_empty + 8 * s, kGroupWarps);
+            for (int q = 0; q < C::kGroups; ++q) {
+                mbar_init(bar_fullK0 + 8 * (q * C::kStages + s), 1);
+                mbar_init(bar_fullV0 + 8 * (q * C::kStages + s), 1);
+            }
         }
-        flags[0] = 0;
-        flags[1] = 0;
+        cta_flags[0] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     const uint32_t epoch = *reinterpret_cast<const volatile uint32_t*>(p.epoch);
@@ -410,12 +451,12 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         int cacc = 0;
         cap_prefix[0] = 0;
         for (int b = 0; b < p.B; ++b) {
-            // contributors of a segment: the CTAs whose static range meets it (<= T * Cn / n + 2), thieves
-            // admitted from other segments (<= steal_slots) and one chunk that straddles into it
+            // contributors of a segment: per CTA whose static range meets it (<= T * Cn / n + 2 of them), per thief
+            // admitted from another segment (<= steal_slots) and per chunk straddling into it, one partial per group
             const int64_t tb = tile_prefix[b + 1] - tile_prefix[b];
             int64_t own = tb == 0 ? 0 : (n_ < (1 << 23) ? (int64_t)(((uint32_t)tb * (uint32_t)cn_) / (uint32_t)n_) : tb * cn_ / n_) + 2;
             if (own > tb) own = tb;
-            cacc += tb == 0 ? 0 : (int)own + p.steal_slots + 1;
+            cacc += tb == 0 ? 0 : kMaxGroups * ((int)own + p.steal_slots + 1);
             cap_prefix[b + 1] = cacc;
         }
     }
@@ -444,13 +485,14 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     WMTP_STAMP(p, 2);
     const bool slack = (p.mode == kRing) && (p.cap != p.W);
 
-    if (warp == kConsumerWarps) {
+    if ((threadIdx.x >> 5) == C::kConsumerWarps) {
         // =================================== producer warp ===================================
         // CTA c < Cn owns the tile range [c n / Cn, (c+1) n / Cn). It streams the first part of it without any
         // bookkeeping; the rest is handed out in small chunks through the per-CTA cursor cur[c], to the owner
         // and, once they run dry, to other CTAs: SMs do not all stream at the same rate, and the slowest one
         // would otherwise set the launch time. A thief prefers a victim inside the segment it is already in
         // (no new partial); moving into another segment is admitted steal_slots times per segment.
+        // Tile number `it` of this CTA goes to stage it % kStages and to consumer group it % kGroups.
         const uint32_t stage0 = smem_u32(stages);
         uint64_t policy = 0;
 #if WMTP_TMA_HINT == 1
@@ -462,9 +504,20 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         uint32_t it = 0;
         int cur_seg = -1;                    // segment of the last issued tile
         int64_t cur_lo = 0, cur_hi = 0;      // its tile range
-        int ord = 0;                         // contributions (segment entries) so far
+        int grp_seg[kMaxGroups], grp_ord[kMaxGroups], pend_k[kMaxGroups];
+        bool pend[kMaxGroups];
+#pragma unroll
+        for (int q = 0; q < kMaxGroups; ++q) { grp_seg[q] = -1; grp_ord[q] = 0; pend_k[q] = 0; pend[q] = false; }
         const bool is_owner = (int)blockIdx.x < Cn;
 
+        // hand the slot number of group gq's latest segment entry over (the group reads it at its flush of that
+        // segment, which follows a later arrive of ours on one of its stages)
+        auto settle = [&](int gq) {
+            if (pend[gq]) {
+                if (lane == 0) group_ints[gq * kGroupInts + 4 + 4 * kMaxContrib + (grp_ord[gq] - 1) % kMaxContrib] = pend_k[gq];
+                pend[gq] = false;
+            }
+        };
         // tiles [a, e) of the global line (may cross segment boundaries); page ids fetched 32 at a time
         auto issue_range = [&](int64_t a, int64_t e) {
             int64_t t = a;
@@ -474,14 +527,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 const int64_t t_end = seg_end < e ? seg_end : e;
                 const int64_t first_tile = t - sg.seg_start;
                 const int ntiles = (int)(t_end - t);
-                int slot_k = 0;
-                const bool entering = sg.seg != cur_seg;
-                if (entering && lane == 0) {
-                    // fixed partition: the contributors of a segment are known, so slots follow the CTA order and the
-                    // result is bit-reproducible; with stealing they are handed out first come, first served
-                    if (p.steal_slots_enabled) slot_k = atomicAdd(p.nparts + sg.seg, 1);   // consumed after the tiles are issued
-                    else slot_k = (int)blockIdx.x - tile_owner(sg.seg_start, n, Cn);
-                }
                 for (int base = 0; base < ntiles; base += 32) {
                     int page = 0;
                     if (p.mode == kPaged) {
@@ -494,8 +539,18 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                     const int cnt = ntiles - base < 32 ? ntiles - base : 32;
                     for (int j = 0; j < cnt; ++j, ++it) {
                         const int pg = __shfl_sync(0xffffffffu, page, j);
+                        const int gq = (int)(it % C::kGroups);
+                        settle(gq);
+                        if (grp_seg[gq] != sg.seg) {
+                            // group gq enters the segment: it needs a partial slot there (result used at the next settle)
+                            if (lane == 0) pend_k[gq] = atomicAdd(p.nparts + sg.seg, 1);
+                            pend[gq] = true;
+                            grp_seg[gq] = sg.seg;
+                            ++grp_ord[gq];
+                        }
                         if (lane == 0) {
                             const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+                            const uint32_t bar_fullK = bar_fullK0 + 8 * (gq * C::kStages), bar_fullV = bar_fullV0 + 8 * (gq * C::kStages);
                             mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status);
                             if (!*abort_flag) {
                                 int64_t row;
@@ -523,12 +578,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         }
                     }
                 }
-                if (entering) {
-                    // the consumers read this at their flush of the segment, which follows a later arrive of ours
-                    if (lane == 0) reg_k[ord % kMaxContrib] = slot_k;
-                    ++ord;
-                    cur_seg = sg.seg; cur_lo = sg.seg_start; cur_hi = seg_end;
-                }
+                cur_seg = sg.seg; cur_lo = sg.seg_start; cur_hi = seg_end;
                 t = t_end;
             }
         };
@@ -584,7 +634,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 range_of(best_v, &lo, &len, &first);
                 int ok = 1;
                 if (best_rem < ((int64_t)1 << 40)) {
-                    // another segment: needs a partial slot there, admitted steal_slots times per segment
+                    // another segment: needs partial slots there, admitted steal_slots times per segment
                     int admitted = 0;
                     if (lane == 0) {
                         const int64_t tv = lo + first + __ldcg(p.cur + best_v);
@@ -602,19 +652,34 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 issue_range(a, a + kStealChunk < lo + len ? a + kStealChunk : lo + len);
             }
         }
+#pragma unroll
+        for (int q = 0; q < C::kGroups; ++q) settle(q);
         if (lane == 0) {
-            // end marker for the consumers, then: this CTA takes no more tiles
-            const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
-            mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status);
-            stage_tile[s] = -1;
-            mbar_arrive(bar_fullK + 8 * s);
-            mbar_arrive(bar_fullV + 8 * s);
+            // one end marker per consumer group, then: this CTA takes no more tiles
+            for (int q = 0; q < C::kGroups; ++q, ++it) {
+                const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+                const uint32_t gq = it % C::kGroups;
+                mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status);
+                stage_tile[s] = -1;
+                mbar_arrive(bar_fullK0 + 8 * (gq * C::kStages + s));
+                mbar_arrive(bar_fullV0 + 8 * (gq * C::kStages + s));
+            }
             atomicAdd(p.grab_done, 1);
         }
         return;
     }
 
-    // ===================================== consumer warps =====================================
+    // ===================================== consumer groups =====================================
+    const int grp = threadIdx.x / kGroupThreads, tid = threadIdx.x % kGroupThreads;   // group, thread within the group
+    const int warp = tid >> 5;                           // warp within the group: owns keys [16 warp, 16 warp + 16) of a tile
+    float* scratch = scratch_all + grp * kScratchFloats;
+    float* sm_m = sm_stats + grp * 3 * kGroupWarps * kMaxGroup;
+    float* sm_l = sm_m + kGroupWarps * kMaxGroup;
+    float* sm_le = sm_l + kGroupWarps * kMaxGroup;
+    int* gints = group_ints + grp * kGroupInts;          // [0] launch-last, [1] broadcast
+    int* contrib = gints + 4;                            // [kMaxContrib][4]
+    volatile int* reg_k = gints + 4 + 4 * kMaxContrib;   // [kMaxContrib]
+    int64_t* contrib_base = contrib_base_all + grp * kMaxContrib;
     const int g8 = lane >> 2, t4 = lane & 3;            // MMA fragment coordinates
     const float scale = p.scale_log2;
     // ldmatrix lane addressing (byte offsets inside a 64-row x 128-byte swizzled chunk)
@@ -623,40 +688,41 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     const int rowV = warp * 16 + (mi >> 1) * 8 + rr, halfV = mi & 1;       // V as A operand (transposed load)
     const uint32_t offK = rowK * 128, offV = rowV * 128;
     const uint32_t stage0 = smem_u32(stages);
+    const uint32_t bar_fullK = bar_fullK0 + 8 * (grp * C::kStages), bar_fullV = bar_fullV0 + 8 * (grp * C::kStages);
 
-    int nonempty_segs = 0;                               // consumer thread 0 only
-    if (threadIdx.x == 0)
+    int nonempty_segs = 0;                               // group thread 0 only
+    if (tid == 0)
         for (int b = 0; b < p.B; ++b) nonempty_segs += (tile_prefix[b + 1] != tile_prefix[b]) ? p.Hkv : 0;
-    bool launch_last = false;                            // consumer thread 0: did this CTA complete the launch's last segment?
-    int ncontrib = 0;                                    // uniform across the consumer threads
-    int ord = 0;                                         // segment entries so far (mirrors the producer's count)
+    bool launch_last = false;                            // group thread 0: did this group complete the launch's last segment?
+    int ncontrib = 0;                                    // uniform across the group
+    int ord = 0;                                         // segment entries so far (mirrors the producer's count for this group)
 
     Segment sg;
-    sg.seg = -1; sg.seg_start = 0; sg.tiles = 0; sg.b = 0; sg.g = 0; sg.nk = 0; sg.S = 0; sg.slot_base = 0;
+    sg.seg = -1; sg.seg_start = 0; sg.tiles = 0; sg.b = 0; sg.g = 0; sg.nk = 0; sg.S = 0; sg.slot_base = 0; sg.cap = 0;
     int64_t new_tile = -1;                               // tile (within the segment) whose row this warp must patch (fused append)
     int new_row = 0;
-    int seg_tiles_done = 0;                              // tiles of the current segment this CTA has processed
+    int seg_tiles_done = 0;                              // tiles of the current segment this group has processed
     uint32_t qb[C::kKSteps][2];
     float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f}, le[2] = {0.f, 0.f};   // l: rounded weights (normaliser), le: exact (lse)
     float o[C::kKSteps][4];
 
-    // Combine every segment this CTA has contributed to (waits for their last partial), then forget them.
+    // Combine every segment this group has contributed to (waits for their last partial), then forget them.
     auto combine_outstanding = [&]() {
         for (int i = 0; i < ncontrib; ++i) {
             const int seg = contrib[4 * i], b = contrib[4 * i + 1], g = contrib[4 * i + 2], k = contrib[4 * i + 3];
-            if (threadIdx.x == 0) {
+            if (tid == 0) {
                 wait_equal(p.ready + seg, epoch + 1u, abort_flag, p.status);
-                flags[3] = *reinterpret_cast<volatile int*>(p.ready_np + seg);
+                gints[1] = *reinterpret_cast<volatile int*>(p.ready_np + seg);
             }
-            consumer_barrier();
-            const int np = flags[3];
-            if (np >= 1 && np <= kMaxCtas && k < np) combine_segment(p, b, g, contrib_base[i], np, k, scratch);
-            consumer_barrier();
+            group_barrier(grp);
+            const int np = gints[1];
+            if (np >= 1 && np <= kMaxParts && k < np) combine_segment(p, b, g, contrib_base[i], np, k, scratch, tid, grp);
+            group_barrier(grp);
         }
         ncontrib = 0;
     };
 
-    // Merge the four warps' states, publish the partial of (this CTA, current segment), note the contribution.
+    // Merge the four warps' states, publish the partial of (this group, current segment), note the contribution.
     auto flush_segment = [&]() {
         WMTP_STAMP(p, 5);
         WMTP_CTA_STAMP(p, 2);
@@ -667,15 +733,27 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             le[0] += __shfl_xor_sync(0xffffffffu, le[0], off);
             le[1] += __shfl_xor_sync(0xffffffffu, le[1], off);
         }
-        consumer_barrier();                                   // scratch / sm_m free
+        group_barrier(grp);                                   // scratch / sm_m free
         if (g8 == 0) {
             sm_m[warp * kMaxGroup + 2 * t4] = m[0]; sm_m[warp * kMaxGroup + 2 * t4 + 1] = m[1];
             sm_l[warp * kMaxGroup + 2 * t4] = l[0]; sm_l[warp * kMaxGroup + 2 * t4 + 1] = l[1];
             sm_le[warp * kMaxGroup + 2 * t4] = le[0]; sm_le[warp * kMaxGroup + 2 * t4 + 1] = le[1];
         }
-        consumer_barrier();
-        const int k = reg_k[ord % kMaxContrib];               // slot the producer took when it entered the segment
-        if (threadIdx.x == 0) contrib[4 * ncontrib + 3] = k;
+        group_barrier(grp);
+        int k = reg_k[ord % kMaxContrib];                     // slot the producer took when this group entered the segment
+        if (k < 0 || k >= sg.cap) {
+            // cannot happen while the admission rules hold; never write outside the segment's slots
+            if (tid == 0) {
+                atomicCAS(p.status, 0, kErrBounds);
+                int* dbg = p.status + 8;                       // header bytes [32, 64): diagnostic record
+                dbg[0] = k; dbg[1] = sg.cap; dbg[2] = sg.seg; dbg[3] = (int)blockIdx.x * kMaxGroups + grp; dbg[4] = ord; dbg[5] = seg_tiles_done;
+            }
+            k = sg.cap - 1;
+        }
+        if (tid == 0) {
+            contrib[4 * ncontrib + 3] = k;
+            p.part_key[sg.slot_base + k] = (int)blockIdx.x * kMaxGroups + grp;
+        }
         ++ord;
         const int64_t pidx = sg.slot_base + k;
         float f[2];
@@ -684,11 +762,11 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             const int h = 2 * t4 + i;
             float M = -INFINITY;
 #pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm_m[w * kMaxGroup + h]);
+            for (int w = 0; w < kGroupWarps; ++w) M = fmaxf(M, sm_m[w * kMaxGroup + h]);
             float L = 0.f, Le = 0.f;
             if (M > -INFINITY) {
 #pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) {
+                for (int w = 0; w < kGroupWarps; ++w) {
                     const float e = exp2f(sm_m[w * kMaxGroup + h] - M);
                     L += sm_l[w * kMaxGroup + h] * e;
                     Le += sm_le[w * kMaxGroup + h] * e;
@@ -700,7 +778,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         constexpr int kPasses = D / 128;                       // 128 columns of d per pass through the scratch
 #pragma unroll
         for (int pass = 0; pass < kPasses; ++pass) {
-            if (pass > 0) consumer_barrier();
+            if (pass > 0) group_barrier(grp);
 #pragma unroll
             for (int mbl = 0; mbl < 8; ++mbl) {
                 const int mb = pass * 8 + mbl;
@@ -709,23 +787,22 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 row0[0] = o[mb][0] * f[0]; row1[0] = o[mb][1] * f[1];
                 row0[8] = o[mb][2] * f[0]; row1[8] = o[mb][3] * f[1];
             }
-            consumer_barrier();
-            for (int idx = threadIdx.x; idx < G * 128; idx += 128) {
+            group_barrier(grp);
+            for (int idx = tid; idx < G * 128; idx += kGroupThreads) {
                 const int h = idx >> 7, dd = idx & 127;
                 float acc = 0.f;
 #pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) acc += scratch[(w * kMaxGroup + h) * kScratchRow + dd];
+                for (int w = 0; w < kGroupWarps; ++w) acc += scratch[(w * kMaxGroup + h) * kScratchRow + dd];
                 p.part_o[(pidx * G + h) * D + pass * 128 + dd] = acc;
             }
         }
-        consumer_barrier();
-        if (threadIdx.x == 0) {
-            __threadfence();                                   // the CTA's partial is visible device-wide before the arrival
+        group_barrier(grp);
+        if (tid == 0) {
+            __threadfence();                                   // the group's partial is visible device-wide before the arrival
             const int old = atomicAdd(p.arrive + sg.seg, seg_tiles_done);
             if ((int64_t)old + seg_tiles_done == sg.tiles) {   // this contribution completes the segment
                 __threadfence();
-                const int np = p.steal_slots_enabled ? *reinterpret_cast<volatile int*>(p.nparts + sg.seg)
-                                                     : tile_owner(sg.seg_start + sg.tiles - 1, n, Cn) - tile_owner(sg.seg_start, n, Cn) + 1;
+                const int np = *reinterpret_cast<volatile int*>(p.nparts + sg.seg);
                 p.nparts[sg.seg] = 0;
                 p.nthief[sg.seg] = 0;
                 p.arrive[sg.seg] = 0;
@@ -746,7 +823,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     // Start work on the segment that holds tile tt: partial bookkeeping, append target, query fragments, fresh state.
     auto enter_segment = [&](int64_t tt) {
         sg = locate_segment(p, tile_prefix, cap_prefix, tt);
-        if (threadIdx.x == 0) {
+        if (tid == 0) {
             contrib[4 * ncontrib] = sg.seg; contrib[4 * ncontrib + 1] = sg.b; contrib[4 * ncontrib + 2] = sg.g;
             contrib_base[ncontrib] = sg.slot_base;
         }
@@ -771,17 +848,21 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 #pragma unroll
         for (int mb = 0; mb < C::kKSteps; ++mb) { o[mb][0] = o[mb][1] = o[mb][2] = o[mb][3] = 0.f; }
     };
-    // an owner knows its first tile: fetch the query while that tile is still in flight
-    if ((int)blockIdx.x < Cn) enter_segment(cta_range_start(blockIdx.x, n, Cn));
+    // an owner knows its first tiles: fetch the query while they are still in flight
+    if ((int)blockIdx.x < Cn) {
+        const int64_t first = cta_range_start(blockIdx.x, n, Cn) + grp;
+        if (first < cta_range_start(blockIdx.x + 1, n, Cn)) enter_segment(first);
+    }
 
-    for (uint32_t it = 0;; ++it) {
-        const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+    for (uint32_t it = grp;; it += C::kGroups) {
+        // this group's uses of stage s are kUsePeriod iterations apart: that is what its "full" barriers count
+        const uint32_t s = it % C::kStages, ph = (it / C::kUsePeriod) & 1u;
         mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
         if (it == 0) { WMTP_STAMP(p, 3); WMTP_CTA_STAMP(p, 1); }
         const int64_t tt = *reinterpret_cast<volatile int64_t*>(stage_tile + s);
         if (tt < 0 || *abort_flag) break;
         if (sg.seg < 0 || tt < sg.seg_start || tt >= sg.seg_start + sg.tiles) {
-            if (sg.seg >= 0) flush_segment();
+            if (sg.seg >= 0 && seg_tiles_done > 0) flush_segment();
             enter_segment(tt);
         }
         ++seg_tiles_done;
@@ -813,7 +894,11 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             }
             uint32_t pb0 = 0, pb1 = 0;
             float corr0 = 1.f, corr1 = 1.f;
+#ifdef WMTP_SKIP_COMPUTE
+            if (false) {
+#else
             if (any_valid) {
+#endif
                 // ---- S^T = K . Q^T for this warp's 16 keys (two accumulator chains)
                 float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -871,7 +956,11 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
                 if (new_ok) reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.v) + new_off)[lane] = x;
             }
+#ifdef WMTP_SKIP_COMPUTE
+            if (false) {
+#else
             if (any_valid) {
+#endif
                 if (wkey0 + 16 > sg.nk) {
                     // rows past the sequence end were never written: they may hold NaN/Inf bit patterns,
                     // and 0 * NaN would poison the accumulators. Zero them in shared memory.
@@ -903,18 +992,18 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     combine_outstanding();
     WMTP_STAMP(p, 9);
 
-    // ---- the CTA that completed the launch's last segment closes the launch
-    if (threadIdx.x == 0) flags[1] = launch_last ? 1 : 0;
-    consumer_barrier();
-    if (flags[1]) {
-        if (threadIdx.x == 0) {
-            wait_word(p.grab_done, 0u, (uint32_t)Cg, abort_flag, p.status);   // nobody takes tickets or reads len[] any more
+    // ---- the group that completed the launch's last segment closes the launch
+    if (tid == 0) gints[0] = launch_last ? 1 : 0;
+    group_barrier(grp);
+    if (gints[0]) {
+        if (tid == 0) {
+            wait_word(p.grab_done, 0u, (uint32_t)Cg, abort_flag, p.status);   // nobody takes tiles or reads len[] any more
             *p.grab_done = 0;
         }
-        consumer_barrier();
-        for (int c = threadIdx.x; c < Cg; c += 128) p.cur[c] = 0;
+        group_barrier(grp);
+        for (int c = tid; c < Cg; c += kGroupThreads) p.cur[c] = 0;
         if (p.k_new) {
-            for (int b = threadIdx.x; b < p.B; b += 128) {
+            for (int b = tid; b < p.B; b += kGroupThreads) {
                 if (appends_to(p, b)) p.len[b] += 1;
                 else atomicCAS(p.status, 0, kErrBounds);      // append past S_cap: skipped and flagged
             }
@@ -966,9 +1055,10 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int D) {
 template <int D>
 size_t partial_smem_bytes(int B) {
     using C = Cfg<D>;
-    return 1024 + (size_t)C::kStages * C::kStageBytes + sizeof(float) * (kScratchFloats + 3 * kConsumerWarps * kMaxGroup) +
-           sizeof(uint64_t) * 3 * C::kStages + sizeof(int64_t) * C::kStages + sizeof(int) * (4 + 5 * kMaxContrib) +
-           sizeof(int64_t) * kMaxContrib + (sizeof(int64_t) + sizeof(int)) * (B + 1) + 16;
+    return 1024 + (size_t)C::kStages * C::kStageBytes +
+           sizeof(float) * C::kGroups * (kScratchFloats + 3 * kGroupWarps * kMaxGroup) +
+           sizeof(uint64_t) * C::kBarriers + sizeof(int64_t) * C::kStages + sizeof(int64_t) * C::kGroups * kMaxContrib +
+           (sizeof(int64_t) + sizeof(int)) * (B + 1) + sizeof(int) * (C::kGroups * kGroupInts + 4) + 16;
 }
 
 template <int D>
@@ -984,7 +1074,7 @@ cudaError_t launch_fused(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaSt
     }
     void* args[] = {&mk, &mv, &p};
     // cooperative: the CTAs wait on one another in the combine, so they must all be resident
-    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(attn_fused_tma<D>), dim3(p.num_ctas), dim3(kThreads), args, smem, st);
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(attn_fused_tma<D>), dim3(p.num_ctas), dim3(Cfg<D>::kThreads), args, smem, st);
 }
 
 }  // namespace

@@ -122,6 +122,7 @@ void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, 
     p.ready_np = reinterpret_cast<int*>(p.ready + kMaxSegments);
     p.steal_slots_enabled = g_stealing.load() ? 1 : 0;
     p.steal_slots = p.steal_slots_enabled ? steal_slots_for(batch * Hkv) : 0;
+    p.part_key = reinterpret_cast<int*>(base + L.part_key_off);
     p.part_lse = reinterpret_cast<float*>(base + L.part_lse_off);
     p.part_o = reinterpret_cast<float*>(base + L.part_o_off);
     p.B = batch; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = Hq / Hkv;
@@ -198,10 +199,6 @@ StagePlan stage_plan(int gamma, int batch, int Hq, int Hkv, int D) {
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
-int steal_slots_for(int nseg) {
-    int x = 512 / (nseg < 1 ? 1 : nseg);
-    return x > kStealSlotsMax ? kStealSlotsMax : x;
-}
 
 int sm_count() {
     static std::atomic<int> cached{0};
@@ -217,9 +214,10 @@ int sm_count() {
 
 WorkspaceLayout workspace_layout(int batch, int Hq, int Hkv, int D) {
     WorkspaceLayout L;
-    const size_t G = (size_t)(Hq / Hkv), nseg = (size_t)batch * Hkv, np = (size_t)kMaxCtas + (size_t)(steal_slots_for((int)nseg) + 3) * nseg;
+    const size_t G = (size_t)(Hq / Hkv), nseg = (size_t)batch * Hkv, np = pool_slots((int)nseg);
     L.counters_off = 256 + kCursorBytes;
-    L.part_lse_off = kWorkspaceZeroBytes;
+    L.part_key_off = kWorkspaceZeroBytes;
+    L.part_lse_off = L.part_key_off + round_up(np * sizeof(int), 256);
     L.part_o_off = L.part_lse_off + round_up(np * G * sizeof(float), 256);
     L.total = L.part_o_off + round_up(np * G * D * sizeof(float), 256);
 #ifdef WMTP_TRACE
@@ -428,11 +426,14 @@ constexpr int kStaticMaxCtas = 160;        // CTAs (KV splits) the static scratc
 constexpr int kStaticMaxSegments = 32;     // batch * Hkv
 constexpr size_t kStaticCountersOff = 256 + kCursorBytes;
 constexpr size_t kStaticPartLseOff = kStaticCountersOff + 5 * sizeof(int) * kStaticMaxSegments + 128; // five per-segment arrays, padded to 256
-constexpr size_t kStaticPartOOff = kStaticPartLseOff + (kStaticMaxCtas + 3 * kStaticMaxSegments) * kMaxGroup * sizeof(float);
-constexpr size_t kStaticBytes = kStaticPartOOff + (size_t)(kStaticMaxCtas + 3 * kStaticMaxSegments) * kMaxGroup * 256 * sizeof(float);
+constexpr size_t kStaticSlots = (size_t)kMaxGroups * (kStaticMaxCtas + 3 * kStaticMaxSegments);
+constexpr size_t kStaticPartKeyOff = kStaticPartLseOff;                      // int [kStaticSlots]
+constexpr size_t kStaticPartLse2Off = kStaticPartKeyOff + kStaticSlots * sizeof(int);
+constexpr size_t kStaticPartOOff = kStaticPartLse2Off + kStaticSlots * kMaxGroup * sizeof(float);
+constexpr size_t kStaticBytes = kStaticPartOOff + kStaticSlots * kMaxGroup * 256 * sizeof(float);
 static_assert(kStaticPartLseOff % 256 == 0 && kStaticPartOOff % 256 == 0, "static scratch regions must stay 256-byte aligned");
 
-static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];   // ~1.8 MiB
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];   // ~4 MiB
 
 // In host code the array's name is only a handle; the device address must be asked for, once per device.
 std::mutex g_static_mu;
@@ -489,7 +490,8 @@ wmtp_status wmtp_draft_attn_windowed_noalloc(const void* q, int Hq, const wmtp_r
     p.ready_np = reinterpret_cast<int*>(p.ready + kStaticMaxSegments);
     p.steal_slots_enabled = 0;                 // static partition: deterministic and the smallest partial pool
     p.steal_slots = 0;
-    p.part_lse = reinterpret_cast<float*>(base + kStaticPartLseOff);
+    p.part_key = reinterpret_cast<int*>(base + kStaticPartKeyOff);
+    p.part_lse = reinterpret_cast<float*>(base + kStaticPartLse2Off);
     p.part_o = reinterpret_cast<float*>(base + kStaticPartOOff);
     p.B = ring->batch; p.Hq = Hq; p.Hkv = ring->Hkv; p.D = ring->D; p.G = Hq / ring->Hkv;
     const float sc = sm_scale > 0.f ? sm_scale : 1.0f / std::sqrt((float)ring->D);

@@ -11,6 +11,7 @@ namespace wmtp {
 constexpr int kTileKeys = 64;       // keys per K/V tile; equals the page size of the paged layout
 constexpr int kMaxCtas = 160;       // upper bound on attention CTAs (one per SM; a B200 has 148)
 constexpr int kStealSlotsMax = 16;   // thieves a segment admits from other segments (fewer when there are many segments)
+constexpr int kMaxGroups = 2;        // consumer groups per CTA (each contributes its own partial)
 constexpr int kMaxBatch = 1024;     // sequences per call (prefix table lives in shared memory)
 constexpr int kMaxGroup = 8;        // query heads per KV head
 constexpr int kMaxSegments = 16384; // batch * Hkv per call
@@ -24,13 +25,22 @@ enum KvMode : int { kContiguous = 0, kPaged = 1, kRing = 2 };
 //   [256, 1280)         int cur[kMaxCtas]: per-CTA cursors of the work-stealing scheme
 //   counters            int arrive[kMaxSegments], nparts[..], nthief[..], uint ready[..], int ready_np[..]
 //                       (fixed size: initialisation needs no shape)
-//   part_lse            float [slots][G]        slots = kMaxCtas + (steal_slots + 3) * batch * Hkv
+//   part_key            int   [slots]           slots = pool_slots(batch * Hkv)
+//   part_lse            float [slots][G]
 //   part_o              float [slots][G][D]
 struct WorkspaceLayout {
-    size_t counters_off, part_lse_off, part_o_off, total;
+    size_t counters_off, part_key_off, part_lse_off, part_o_off, total;
 };
 WorkspaceLayout workspace_layout(int batch, int Hq, int Hkv, int D);
-int steal_slots_for(int nseg);   // kStealSlotsMax for few segments, fewer as batch * Hkv grows
+// kStealSlotsMax for few segments, fewer as batch * Hkv grows
+__host__ __device__ inline int steal_slots_for(int nseg) {
+    const int x = 512 / (nseg < 1 ? 1 : nseg);
+    return x > kStealSlotsMax ? kStealSlotsMax : x;
+}
+// Partial slots the workspace holds: per CTA or admitted thief or straddling chunk, one per consumer group.
+__host__ __device__ inline size_t pool_slots(int nseg) {
+    return (size_t)kMaxGroups * ((size_t)kMaxCtas + (size_t)(steal_slots_for(nseg) + 3) * (size_t)nseg);
+}
 
 // Everything the attention kernel needs; passed by value.
 struct AttnParams {
@@ -44,6 +54,7 @@ struct AttnParams {
     int32_t* slot_pos;        // ring only: [B][n_sink + cap]
     float* part_o;
     float* part_lse;
+    int* part_key;            // [slots]: (CTA, group) that wrote the partial; orders the fixed-partition combine
     int* arrive;              // [segments]: tiles of the segment covered by published partials
     int* nparts;              // [segments]: partial slots handed out
     uint32_t* ready;          // [segments]: epoch tag released when the segment's last partial is in
