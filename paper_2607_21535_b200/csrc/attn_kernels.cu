@@ -205,18 +205,21 @@ __device__ __forceinline__ uint32_t wait_word(const void* word, uint32_t base, u
     return v;
 }
 
-// Bounded spin until a global word equals `want` (an epoch tag: stale values never match).
-__device__ __forceinline__ void wait_equal(const uint32_t* word, uint32_t want, volatile int* abort_flag, int* status) {
+// Bounded spin on a segment's arrival word until its tile count (low half) reaches `tiles`; returns the number of
+// published partials (high half).
+__device__ __forceinline__ int wait_tiles(const unsigned long long* word, uint32_t tiles, volatile int* abort_flag, int* status) {
+    unsigned long long v = 0;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        uint32_t v;
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(word) : "memory");
-        if (v == want) return;
-        if ((i & 255u) == 255u && *abort_flag) return;
+        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(word) : "memory");
+        if ((uint32_t)v >= tiles) return (int)(v >> 32);
+        if ((i & 255u) == 255u && *abort_flag) return 0;
         __nanosleep(32);
     }
     *abort_flag = 1;
     atomicCAS(status, 0, kErrTimeout);
+    return 0;
 }
+__device__ __forceinline__ int kMaxSegmentsPadded(const AttnParams& p) { return p.seg_stride; }
 
 // One (sequence, KV head) segment as seen by a CTA.
 struct Segment {
@@ -285,7 +288,7 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
     group_barrier(grp);
 
     // ---- this group's slice of the (head, d) columns; the first rows are requested before the weights exist
-    constexpr int kPre = 4;
+    constexpr int kPre = 6;
     const int vec = D / 4, cols = G * vec;
     const int cpc = (cols + np - 1) / np;
     const int col_lo = j * cpc, col_hi = col_lo + cpc < cols ? col_lo + cpc : cols;
@@ -379,18 +382,18 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
     }
 }
 
-// Launch-level bookkeeping (workspace header and per-segment words), with no reset pass and no grid barrier:
+// Launch-level bookkeeping (workspace header and per-segment words), with no reset pass and no grid barrier.
+// The per-segment words exist twice; a launch uses the copy selected by the parity of the launch epoch and,
+// at its very end, clears the other copy for the next launch (nobody can be using that one).
 //   cur[c]       tiles of CTA c's dynamic part already handed out (to the owner or to thieves);
 //   nparts[s]    partial slots handed out for segment s (a consumer group takes one whenever it enters s);
 //   nthief[s]    CTAs admitted into s from another segment;
-//   arrive[s]    tiles of s whose result is in a published partial; the contributor that completes the
-//                segment resets nparts/nthief/arrive, stores the partial count in ready_np[s] and releases
-//                ready[s] = epoch + 1;
-//   ready[s]     polled by the contributors before they combine; a value left by an earlier launch never
-//                equals this launch's tag;
+//   arrive[s]    64 bits: (published partials << 32) | tiles covered by them. Contributors add to it after their
+//                partial is visible and then poll it: when the tile count equals the segment's tiles, the high
+//                half is the number of partials to combine. One hop, no "ready" flag;
 //   segs_done    completed segments; the group that completes the last one advances the epoch and, after every
 //                CTA has stopped taking tiles (grab_done, which also means it has read len[] for the last
-//                time), resets the cursors and advances the lengths of a fused append.
+//                time), resets the cursors, clears the other copy and advances the lengths of a fused append.
 
 // ---------------------------------------------------------------------------------------------
 // The attention kernel (one cooperative launch per draft step)
@@ -410,8 +413,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     // apart, so the "full" barriers must not be shared between groups.
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm_stats + C::kGroups * 3 * kGroupWarps * kMaxGroup);
     int64_t* stage_tile = reinterpret_cast<int64_t*>(bars + C::kBarriers);                // [kStages] global tile index, -1 = end
-    int64_t* contrib_base_all = stage_tile + C::kStages;                                  // [kGroups][kMaxContrib] slot base
-    int64_t* tile_prefix = contrib_base_all + C::kGroups * kMaxContrib;                   // [B + 1]
+    int64_t* contrib_base_all = stage_tile + C::kStages;                                  // [kGroups][2][kMaxContrib]
+    int64_t* tile_prefix = contrib_base_all + C::kGroups * 2 * kMaxContrib;               // [B + 1]
     int* cap_prefix = reinterpret_cast<int*>(tile_prefix + (p.B + 1));                    // [B + 1]
     int* group_ints = cap_prefix + (p.B + 1);                                             // [kGroups][kGroupInts]
     int* cta_flags = group_ints + C::kGroups * kGroupInts;                                // [0] abort
@@ -437,6 +440,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     const uint32_t epoch = *reinterpret_cast<const volatile uint32_t*>(p.epoch);
+    const int par_off = (epoch & 1u) ? kMaxSegmentsPadded(p) : 0;        // which copy of the per-segment words this launch uses
 
     // ---- plan: tiles per sequence and partial-slot capacity per sequence (all from len[], O(B))
     for (int b = threadIdx.x; b < p.B; b += blockDim.x)
@@ -543,7 +547,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         settle(gq);
                         if (grp_seg[gq] != sg.seg) {
                             // group gq enters the segment: it needs a partial slot there (result used at the next settle)
-                            if (lane == 0) pend_k[gq] = atomicAdd(p.nparts + sg.seg, 1);
+                            if (lane == 0) pend_k[gq] = atomicAdd(p.nparts + par_off + sg.seg, 1);
                             pend[gq] = true;
                             grp_seg[gq] = sg.seg;
                             ++grp_ord[gq];
@@ -639,7 +643,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                     if (lane == 0) {
                         const int64_t tv = lo + first + __ldcg(p.cur + best_v);
                         const Segment vs = locate_segment(p, tile_prefix, cap_prefix, tv < lo + len ? tv : lo + len - 1);
-                        admitted = atomicAdd(p.nthief + vs.seg, 1) < p.steal_slots;
+                        admitted = atomicAdd(p.nthief + par_off + vs.seg, 1) < p.steal_slots;
                     }
                     ok = __shfl_sync(0xffffffffu, admitted, 0);
                 }
@@ -679,7 +683,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     int* gints = group_ints + grp * kGroupInts;          // [0] launch-last, [1] broadcast
     int* contrib = gints + 4;                            // [kMaxContrib][4]
     volatile int* reg_k = gints + 4 + 4 * kMaxContrib;   // [kMaxContrib]
-    int64_t* contrib_base = contrib_base_all + grp * kMaxContrib;
+    int64_t* contrib_base = contrib_base_all + grp * 2 * kMaxContrib;       // [kMaxContrib] slot base, then [kMaxContrib] segment tiles
+    int64_t* contrib_tiles = contrib_base + kMaxContrib;
     const int g8 = lane >> 2, t4 = lane & 3;            // MMA fragment coordinates
     const float scale = p.scale_log2;
     // ldmatrix lane addressing (byte offsets inside a 64-row x 128-byte swizzled chunk)
@@ -711,8 +716,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         for (int i = 0; i < ncontrib; ++i) {
             const int seg = contrib[4 * i], b = contrib[4 * i + 1], g = contrib[4 * i + 2], k = contrib[4 * i + 3];
             if (tid == 0) {
-                wait_equal(p.ready + seg, epoch + 1u, abort_flag, p.status);
-                gints[1] = *reinterpret_cast<volatile int*>(p.ready_np + seg);
+                gints[1] = wait_tiles(p.arrive + par_off + seg, (uint32_t)contrib_tiles[i], abort_flag, p.status);
             }
             group_barrier(grp);
             const int np = gints[1];
@@ -799,15 +803,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         group_barrier(grp);
         if (tid == 0) {
             __threadfence();                                   // the group's partial is visible device-wide before the arrival
-            const int old = atomicAdd(p.arrive + sg.seg, seg_tiles_done);
-            if ((int64_t)old + seg_tiles_done == sg.tiles) {   // this contribution completes the segment
-                __threadfence();
-                const int np = *reinterpret_cast<volatile int*>(p.nparts + sg.seg);
-                p.nparts[sg.seg] = 0;
-                p.nthief[sg.seg] = 0;
-                p.arrive[sg.seg] = 0;
-                p.ready_np[sg.seg] = np;
-                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.ready + sg.seg), "r"(epoch + 1u) : "memory");
+            const unsigned long long old = atomicAdd(p.arrive + par_off + sg.seg, (1ull << 32) | (unsigned long long)seg_tiles_done);
+            if ((int64_t)(uint32_t)old + seg_tiles_done == sg.tiles) {   // this contribution completes the segment
                 if (atomicAdd(p.segs_done, 1) + 1 == nonempty_segs) {
                     *p.segs_done = 0;
                     *p.epoch = epoch + 1u;
@@ -826,6 +823,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         if (tid == 0) {
             contrib[4 * ncontrib] = sg.seg; contrib[4 * ncontrib + 1] = sg.b; contrib[4 * ncontrib + 2] = sg.g;
             contrib_base[ncontrib] = sg.slot_base;
+            contrib_tiles[ncontrib] = sg.tiles;
         }
         seg_tiles_done = 0;
         // fused append (Appendix A, RING / the KV write of a draft forward): where does the new token go?
@@ -1002,6 +1000,10 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         }
         group_barrier(grp);
         for (int c = tid; c < Cg; c += kGroupThreads) p.cur[c] = 0;
+        const int other = (epoch & 1u) ? 0 : kMaxSegmentsPadded(p);
+        for (int sgi = tid; sgi < nseg; sgi += kGroupThreads) {               // the next launch's copy
+            p.arrive[other + sgi] = 0ull; p.nparts[other + sgi] = 0; p.nthief[other + sgi] = 0;
+        }
         if (p.k_new) {
             for (int b = tid; b < p.B; b += kGroupThreads) {
                 if (appends_to(p, b)) p.len[b] += 1;
@@ -1057,7 +1059,7 @@ size_t partial_smem_bytes(int B) {
     using C = Cfg<D>;
     return 1024 + (size_t)C::kStages * C::kStageBytes +
            sizeof(float) * C::kGroups * (kScratchFloats + 3 * kGroupWarps * kMaxGroup) +
-           sizeof(uint64_t) * C::kBarriers + sizeof(int64_t) * C::kStages + sizeof(int64_t) * C::kGroups * kMaxContrib +
+           sizeof(uint64_t) * C::kBarriers + sizeof(int64_t) * C::kStages + sizeof(int64_t) * C::kGroups * 2 * kMaxContrib +
            (sizeof(int64_t) + sizeof(int)) * (B + 1) + sizeof(int) * (C::kGroups * kGroupInts + 4) + 16;
 }
 

@@ -115,11 +115,10 @@ void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, 
     p.segs_done = reinterpret_cast<int*>(base + 8);
     p.grab_done = reinterpret_cast<int*>(base + 12);
     p.cur = reinterpret_cast<int*>(base + 256);
-    p.arrive = reinterpret_cast<int*>(base + L.counters_off);
-    p.nparts = p.arrive + kMaxSegments;
-    p.nthief = p.nparts + kMaxSegments;
-    p.ready = reinterpret_cast<uint32_t*>(p.nthief + kMaxSegments);
-    p.ready_np = reinterpret_cast<int*>(p.ready + kMaxSegments);
+    p.arrive = reinterpret_cast<unsigned long long*>(base + L.counters_off);
+    p.nparts = reinterpret_cast<int*>(p.arrive + 2 * kMaxSegments);
+    p.nthief = p.nparts + 2 * kMaxSegments;
+    p.seg_stride = kMaxSegments;
     p.steal_slots_enabled = g_stealing.load() ? 1 : 0;
     p.steal_slots = p.steal_slots_enabled ? steal_slots_for(batch * Hkv) : 0;
     p.part_key = reinterpret_cast<int*>(base + L.part_key_off);
@@ -425,7 +424,7 @@ namespace {
 constexpr int kStaticMaxCtas = 160;        // CTAs (KV splits) the static scratch has room for
 constexpr int kStaticMaxSegments = 32;     // batch * Hkv
 constexpr size_t kStaticCountersOff = 256 + kCursorBytes;
-constexpr size_t kStaticPartLseOff = kStaticCountersOff + 5 * sizeof(int) * kStaticMaxSegments + 128; // five per-segment arrays, padded to 256
+constexpr size_t kStaticPartLseOff = kStaticCountersOff + 2 * (8 + 4 + 4) * kStaticMaxSegments;       // two copies of the per-segment words
 constexpr size_t kStaticSlots = (size_t)kMaxGroups * (kStaticMaxCtas + 3 * kStaticMaxSegments);
 constexpr size_t kStaticPartKeyOff = kStaticPartLseOff;                      // int [kStaticSlots]
 constexpr size_t kStaticPartLse2Off = kStaticPartKeyOff + kStaticSlots * sizeof(int);
@@ -483,11 +482,10 @@ wmtp_status wmtp_draft_attn_windowed_noalloc(const void* q, int Hq, const wmtp_r
     p.segs_done = reinterpret_cast<int*>(base + 8);
     p.grab_done = reinterpret_cast<int*>(base + 12);
     p.cur = reinterpret_cast<int*>(base + 256);
-    p.arrive = reinterpret_cast<int*>(base + kStaticCountersOff);
-    p.nparts = p.arrive + kStaticMaxSegments;
-    p.nthief = p.nparts + kStaticMaxSegments;
-    p.ready = reinterpret_cast<uint32_t*>(p.nthief + kStaticMaxSegments);
-    p.ready_np = reinterpret_cast<int*>(p.ready + kStaticMaxSegments);
+    p.arrive = reinterpret_cast<unsigned long long*>(base + kStaticCountersOff);
+    p.nparts = reinterpret_cast<int*>(p.arrive + 2 * kStaticMaxSegments);
+    p.nthief = p.nparts + 2 * kStaticMaxSegments;
+    p.seg_stride = kStaticMaxSegments;
     p.steal_slots_enabled = 0;                 // static partition: deterministic and the smallest partial pool
     p.steal_slots = 0;
     p.part_key = reinterpret_cast<int*>(base + kStaticPartKeyOff);

@@ -16,14 +16,14 @@ constexpr int kMaxBatch = 1024;     // sequences per call (prefix table lives in
 constexpr int kMaxGroup = 8;        // query heads per KV head
 constexpr int kMaxSegments = 16384; // batch * Hkv per call
 constexpr size_t kCursorBytes = 1024;                                          // int cur[kMaxCtas], padded
-constexpr size_t kWorkspaceZeroBytes = 256 + kCursorBytes + 5 * sizeof(int) * kMaxSegments;   // header + cursors + per-segment arrays
+constexpr size_t kWorkspaceZeroBytes = 256 + kCursorBytes + 2 * (8 + 4 + 4) * kMaxSegments;   // header + cursors + two copies of the per-segment words
 
 enum KvMode : int { kContiguous = 0, kPaged = 1, kRing = 2 };
 
 // Workspace layout (all offsets from a 256-byte aligned base):
 //   [0, 256)            header: int status @0, uint epoch @4, int segs_done @8, int grab_done @12
 //   [256, 1280)         int cur[kMaxCtas]: per-CTA cursors of the work-stealing scheme
-//   counters            int arrive[kMaxSegments], nparts[..], nthief[..], uint ready[..], int ready_np[..]
+//   counters            u64 arrive[2][kMaxSegments], int nparts[2][..], int nthief[2][..]
 //                       (fixed size: initialisation needs no shape)
 //   part_key            int   [slots]           slots = pool_slots(batch * Hkv)
 //   part_lse            float [slots][G]
@@ -55,15 +55,14 @@ struct AttnParams {
     float* part_o;
     float* part_lse;
     int* part_key;            // [slots]: (CTA, group) that wrote the partial; orders the fixed-partition combine
-    int* arrive;              // [segments]: tiles of the segment covered by published partials
-    int* nparts;              // [segments]: partial slots handed out
-    uint32_t* ready;          // [segments]: epoch tag released when the segment's last partial is in
-    int* ready_np;            // [segments]: number of partials, valid once ready matches
+    unsigned long long* arrive;   // [2][seg_stride]: (published partials << 32) | tiles covered by them
+    int* nparts;              // [2][seg_stride]: partial slots handed out
+    int seg_stride;           // elements between the two copies of the per-segment words (selected by epoch parity)
     uint32_t* epoch;          // launch counter (header)
     int* segs_done;           // completed segments (header)
     int* grab_done;           // CTAs that take no more tickets (header)
     int* cur;                 // [CTAs]: tiles of each CTA's dynamic part handed out so far
-    int* nthief;              // [segments]: CTAs admitted from other segments
+    int* nthief;              // [2][seg_stride]: CTAs admitted from other segments
     int steal_slots;          // thieves a segment admits from other segments
     int steal_slots_enabled;  // 0: purely static partition (deterministic, smallest partial pool)
     int* status;
