@@ -592,28 +592,32 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             *first = (!p.steal_slots_enabled || *len < kStealMinTiles) ? *len : *len - *len / 4;
         };
 
-        if (is_owner) {
-            int64_t lo, len, first;
-            range_of(blockIdx.x, &lo, &len, &first);
-            issue_range(lo, lo + first);
-            // the rest of the own range, chunk by chunk through the cursor (thieves may be taking from it too)
-            const int64_t dyn = len - first;
-            if (dyn > 0) {
-                int k = 0;
-                if (lane == 0) k = atomicAdd(p.cur + blockIdx.x, kStealChunk);
-                k = __shfl_sync(0xffffffffu, k, 0);
-                while (k < dyn) {
-                    int k_next = 0;
-                    if (lane == 0) k_next = atomicAdd(p.cur + blockIdx.x, kStealChunk);       // overlaps the issue below
-                    const int64_t a = lo + first + k;
-                    issue_range(a, a + kStealChunk < lo + len ? a + kStealChunk : lo + len);
-                    k = __shfl_sync(0xffffffffu, k_next, 0);
+        // One loop, three sources of work in turn: the static part of the own range, the rest of the own range chunk
+        // by chunk through the cursor (thieves may be taking from it too), then other CTAs' cursors.
+        const bool may_steal = p.steal_slots_enabled && n >= (int64_t)kStealMinTiles * Cn;
+        int phase = is_owner ? 0 : 2;
+        int64_t own_lo = 0, own_len = 0, own_first = 0;
+        int k_own = 0;                       // own cursor value for the next chunk (phase 1), fetched one chunk ahead
+        if (is_owner) range_of(blockIdx.x, &own_lo, &own_len, &own_first);
+        for (int round = 0; round < (1 << 20); ++round) {
+            int64_t a = 0, e = 0;            // next tiles to issue
+            if (phase == 0) {
+                a = own_lo; e = own_lo + own_first;
+                phase = 1;
+                if (own_len > own_first) {
+                    if (lane == 0) k_own = atomicAdd(p.cur + blockIdx.x, kStealChunk);
+                } else {
+                    k_own = 0x7fffffff;
                 }
-            }
-        }
-        if (p.steal_slots_enabled && n >= (int64_t)kStealMinTiles * Cn) {
-            // ---- steal: look at every cursor, take from the range with the most left
-            for (int round = 0; round < 4096; ++round) {
+            } else if (phase == 1) {
+                const int k = __shfl_sync(0xffffffffu, k_own, 0);
+                if (k >= own_len - own_first) { phase = 2; continue; }
+                if (lane == 0) k_own = atomicAdd(p.cur + blockIdx.x, kStealChunk);     // overlaps the issue below
+                a = own_lo + own_first + k;
+                e = a + kStealChunk < own_lo + own_len ? a + kStealChunk : own_lo + own_len;
+            } else {
+                if (!may_steal || *abort_flag) break;
+                // ---- steal: look at every cursor, take from the range with the most left
                 int64_t best_rem = 0;
                 int best_v = -1;
                 for (int v = lane; v < Cn; v += 32) {
@@ -633,7 +637,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                     const int v2 = __shfl_xor_sync(0xffffffffu, best_v, off);
                     if (r2 > best_rem || (r2 == best_rem && v2 > best_v)) { best_rem = r2; best_v = v2; }
                 }
-                if (best_v < 0 || *abort_flag) break;
+                if (best_v < 0) break;
                 int64_t lo, len, first;
                 range_of(best_v, &lo, &len, &first);
                 int ok = 1;
@@ -652,9 +656,10 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 if (lane == 0) k = atomicAdd(p.cur + best_v, kStealChunk);
                 k = __shfl_sync(0xffffffffu, k, 0);
                 if (k >= len - first) continue;    // somebody else got there first: look again
-                const int64_t a = lo + first + k;
-                issue_range(a, a + kStealChunk < lo + len ? a + kStealChunk : lo + len);
+                a = lo + first + k;
+                e = a + kStealChunk < lo + len ? a + kStealChunk : lo + len;
             }
+            issue_range(a, e);
         }
 #pragma unroll
         for (int q = 0; q < C::kGroups; ++q) settle(q);
@@ -814,7 +819,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         }
         WMTP_STAMP(p, 6);
         ++ncontrib;
-        if (ncontrib == kMaxContrib) combine_outstanding();
     };
 
     // Start work on the segment that holds tile tt: partial bookkeeping, append target, query fragments, fresh state.
@@ -846,23 +850,34 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 #pragma unroll
         for (int mb = 0; mb < C::kKSteps; ++mb) { o[mb][0] = o[mb][1] = o[mb][2] = o[mb][3] = 0.f; }
     };
-    // an owner knows its first tiles: fetch the query while they are still in flight
+    // The loop is written so that enter / flush / tile processing each appear once in the code (the kernel's
+    // tail runs once per launch, from a cold instruction cache: code size is latency there).
+    int64_t tt = -1;                                     // tile in hand
+    bool have_tile = false, need_enter = false;
     if ((int)blockIdx.x < Cn) {
+        // an owner knows its first tiles: fetch the query while they are still in flight
         const int64_t first = cta_range_start(blockIdx.x, n, Cn) + grp;
-        if (first < cta_range_start(blockIdx.x + 1, n, Cn)) enter_segment(first);
+        if (first < cta_range_start(blockIdx.x + 1, n, Cn)) { tt = first; need_enter = true; }
     }
-
-    for (uint32_t it = grp;; it += C::kGroups) {
-        // this group's uses of stage s are kUsePeriod iterations apart: that is what its "full" barriers count
-        const uint32_t s = it % C::kStages, ph = (it / C::kUsePeriod) & 1u;
-        mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
-        if (it == 0) { WMTP_STAMP(p, 3); WMTP_CTA_STAMP(p, 1); }
-        const int64_t tt = *reinterpret_cast<volatile int64_t*>(stage_tile + s);
-        if (tt < 0 || *abort_flag) break;
-        if (sg.seg < 0 || tt < sg.seg_start || tt >= sg.seg_start + sg.tiles) {
-            if (sg.seg >= 0 && seg_tiles_done > 0) flush_segment();
-            enter_segment(tt);
+    uint32_t it = grp;
+    for (;;) {
+        if (need_enter) { enter_segment(tt); need_enter = false; }
+        const uint32_t s = it % C::kStages, ph = (it / C::kUsePeriod) & 1u;   // this group's uses of stage s are kUsePeriod iterations apart
+        if (!have_tile) {
+            mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
+            if (it == 0) { WMTP_STAMP(p, 3); WMTP_CTA_STAMP(p, 1); }
+            tt = *reinterpret_cast<volatile int64_t*>(stage_tile + s);
+            const bool end = tt < 0 || *abort_flag;
+            const bool outside = sg.seg < 0 || tt < sg.seg_start || tt >= sg.seg_start + sg.tiles;
+            if ((end || outside) && sg.seg >= 0 && seg_tiles_done > 0) flush_segment();
+            if (end || ncontrib == kMaxContrib) {
+                combine_outstanding();           // every segment this group contributed to (normally: once, at the end)
+                if (end) break;
+            }
+            have_tile = true;
+            if (outside) { need_enter = true; continue; }
         }
+        have_tile = false;
         ++seg_tiles_done;
         {
             const int64_t key0 = (tt - sg.seg_start) * kTileKeys;
@@ -985,9 +1000,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty + 8 * s);
         }
+        it += C::kGroups;
     }
-    if (sg.seg >= 0 && seg_tiles_done > 0) flush_segment();
-    combine_outstanding();
     WMTP_STAMP(p, 9);
 
     // ---- the group that completed the launch's last segment closes the launch
