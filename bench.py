@@ -31,9 +31,10 @@ METRIC = "us_per_draft_attention_step"
 UNIT = "us"
 WORKLOADS = {"tiny": 0, "s128k": 1, "million": 2, "batched": 3, "sweep": 4}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (full-context partial
-# kernel), from the ncu capture summarised under profiles/; keyed by workload. None = not captured.
-NCU_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (attn_fused_tma on the full
+# context). Captured with ncu on the s128k workload (profiles/attn_fused_tma_D256_s128k_ncu_full.md: 272.8 MB
+# for 131,075 keys = 2081.3 B per key, against 2048 algorithmic) and scaled by the keys one launch scans.
+NCU_TRAFFIC_BYTES_PER_KEY = {256: 2081.3}
 
 
 def log(*a):
@@ -64,7 +65,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -95,6 +96,23 @@ class ClockSampler:
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
         return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def max_over_ranks(x: float) -> float:
+    """MAX of a host scalar over the ranks of the default process group (no-op without one)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    dev = torch.device("cuda", torch.cuda.current_device()) if dist.get_backend() == "nccl" else torch.device("cpu")
+    t = torch.tensor([x], device=dev, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_value(ms_per_step_max: float, gamma: int, world: int) -> float:
+    """us per draft-attention step of the whole job: N replicas run N times the draft steps in the slowest rank's time."""
+    return ms_per_step_max * 1e3 / (2 * gamma) / world
 
 
 def pick_config(name: str, steps_total: int):
@@ -245,12 +263,9 @@ def main():
     launches = wm.wmtp_launch_count() - launches0
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total)
     ms_per_step = ms_total / args.steps
-    value = ms_per_step * 1e3 / (2 * gam) / world          # replicas: N times the draft steps in the same time
+    value = replica_value(ms_per_step, gam, world)
 
     # ---- breakdown pass (outside the headline region): windowed loop and full loop timed separately
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
@@ -264,22 +279,48 @@ def main():
     us_win = statistics.mean(ev[k][0].elapsed_time(ev[k][1]) for k in range(args.steps)) * 1e3 / gam
     us_full = statistics.mean(ev[k][1].elapsed_time(ev[k][2]) for k in range(args.steps)) * 1e3 / gam
 
-    # ---- the dominant kernel alone: full-context attention call (partial + combine), events around each launch
+    # ---- the dominant kernel alone: `reps` launches of the full-context attention kernel back to back between one
+    #      pair of events on the launching stream (average launch duration, inter-launch gap included)
     reps = max(10, args.steps)
     o1 = torch.empty((B, cfg.Hq, cfg.D), dtype=torch.bfloat16, device=dev)
-    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wm.wmtp_draft_attn_full(q[0], kv, o1, ws)
+    k0.record()
+    for _ in range(reps):
+        wm.wmtp_draft_attn_full(q[0], kv, o1, ws)
+    k1.record()
     wev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
-    for a, b in kev:
-        a.record(); wm.wmtp_draft_attn_full(q[0], kv, o1, ws); b.record()
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     for a, b in wev:
         flush.fill_(1)                                      # cold L2 for the windowed call
         a.record(); wm.wmtp_draft_attn_windowed(q[0], ring, o1, ws); b.record()
     torch.cuda.synchronize()
     wm.wmtp_device_status(ws)
-    us_full_call = statistics.mean(a.elapsed_time(b) for a, b in kev) * 1e3
+    us_full_call = k0.elapsed_time(k1) * 1e3 / reps
     us_win_call_cold = statistics.mean(a.elapsed_time(b) for a, b in wev) * 1e3
     cur_lens = lens.cpu().numpy()
+
+    # ---- windowed step time against context length: same ring shape, ring re-seeded at other lengths
+    flat = None
+    if B == 1 and not cfg.paged:
+        flat = {"S": [], "us_per_step": []}
+        S_now = int(cur_lens[0])
+        for S_try in sorted({min(S_now, max(cfg.n_sink + cfg.W + 1, S_now // d)) for d in (16, 4, 1)}):
+            lens.fill_(S_try)
+            wm.wmtp_ring_init_from_kv(ring, kv)
+            for _ in range(2):
+                wm.wmtp_draft_loop_windowed(ring, q, kn, vn, out_w, ws)
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            f0.record()
+            for _ in range(reps):
+                wm.wmtp_draft_loop_windowed(ring, q, kn, vn, out_w, ws)
+            f1.record()
+            torch.cuda.synchronize()
+            flat["S"].append(S_try)
+            flat["us_per_step"].append(f0.elapsed_time(f1) * 1e3 / reps / gam)
+        lens.copy_(torch.from_numpy(cur_lens).to(dev))
+        wm.wmtp_ring_init_from_kv(ring, kv)
+        torch.cuda.synchronize()
     full_bytes = float(cur_lens.sum()) * cfg.kv_bytes_per_token
     win_bytes = float(np.minimum(cur_lens, cfg.n_sink + cfg.W).sum()) * cfg.kv_bytes_per_token
     peak, peak_src = measured_peaks()
@@ -302,11 +343,8 @@ def main():
         one_pass_host()
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = e2e_s / args.steps * 1e6 / (2 * gam) / world
+    e2e_s = max_over_ranks(e2e_s)
+    e2e_value = replica_value(e2e_s / args.steps * 1e3, gam, world)
     h2d = 2 * (qh.numel() + kh.numel() + vh.numel()) * 2
     d2h = 2 * oh_w.numel() * 2
     wm.wmtp_device_status(ws)
@@ -332,10 +370,13 @@ def main():
                          "pct_of_8tbs": full_bytes / (us_full * 1e-6) / 8e12 * 100,
                          "us_per_attention_call": us_full_call},
             },
-            "roofline": {"bound": "hbm", "kernel": "full-context draft attention (split-KV partial + combine)",
+            "windowed_flatness": flat,
+            "roofline": {"bound": "hbm", "kernel": "attn_fused_tma (full-context draft attention: split-KV partials + in-kernel combine)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": peak_src, "pct_of_8tbs": achieved / 8000 * 100,
-                         "traffic": NCU_TRAFFIC_BYTES.get(args.workload)},
+                         "traffic": (NCU_TRAFFIC_BYTES_PER_KEY[cfg.D] * float(cur_lens.sum())
+                                     if cfg.D in NCU_TRAFFIC_BYTES_PER_KEY and cfg.Hkv == 2 else None),
+                         "algorithmic_bytes": full_bytes},
             "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": launches,
