@@ -598,6 +598,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         int phase = is_owner ? 0 : 2;
         int64_t own_lo = 0, own_len = 0, own_first = 0;
         int k_own = 0;                       // own cursor value for the next chunk (phase 1), fetched one chunk ahead
+        int64_t adm_lo = 0, adm_hi = 0;      // lane 0: tile range of the segment this CTA was last admitted to as a thief
         if (is_owner) range_of(blockIdx.x, &own_lo, &own_len, &own_first);
         for (int round = 0; round < (1 << 20); ++round) {
             int64_t a = 0, e = 0;            // next tiles to issue
@@ -640,24 +641,37 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 if (best_v < 0) break;
                 int64_t lo, len, first;
                 range_of(best_v, &lo, &len, &first);
-                int ok = 1;
-                if (best_rem < ((int64_t)1 << 40)) {
-                    // another segment: needs partial slots there, admitted steal_slots times per segment
-                    int admitted = 0;
-                    if (lane == 0) {
-                        const int64_t tv = lo + first + __ldcg(p.cur + best_v);
-                        const Segment vs = locate_segment(p, tile_prefix, cap_prefix, tv < lo + len ? tv : lo + len - 1);
-                        admitted = atomicAdd(p.nthief + par_off + vs.seg, 1) < p.steal_slots;
+                // Take tiles from the victim's cursor with a compare-and-swap, clipped to the segment we are in or have
+                // been admitted to: a thief never lands in a segment where it holds no right to a partial slot, and a
+                // stolen chunk never straddles a segment boundary.
+                int got = 0;                       // 1: tiles [a, e) are ours; 0: look again; -1: stop stealing
+                if (lane == 0) {
+                    for (int tries = 0; tries < 8 && got == 0; ++tries) {
+                        const int used = __ldcg(p.cur + best_v);
+                        const int64_t rem = len - first - used;
+                        if (rem <= 0) break;
+                        const int64_t tv = lo + first + used;
+                        int64_t alo = cur_lo, ahi = cur_hi;
+                        if (!(cur_seg >= 0 && tv >= cur_lo && tv < cur_hi)) {
+                            if (tv >= adm_lo && tv < adm_hi) {
+                                alo = adm_lo; ahi = adm_hi;
+                            } else {
+                                // another segment: needs partial slots there, admitted steal_slots times per segment
+                                const Segment vs = locate_segment(p, tile_prefix, cap_prefix, tv);
+                                if (atomicAdd(p.nthief + par_off + vs.seg, 1) >= p.steal_slots) { got = -1; break; }
+                                adm_lo = alo = vs.seg_start; adm_hi = ahi = vs.seg_start + vs.tiles;
+                            }
+                        }
+                        int64_t take = rem < kStealChunk ? rem : kStealChunk;
+                        if (tv + take > ahi) take = ahi - tv;
+                        if (atomicCAS(p.cur + best_v, used, used + (int)take) == used) { a = tv; e = tv + take; got = 1; }
                     }
-                    ok = __shfl_sync(0xffffffffu, admitted, 0);
                 }
-                if (!ok) break;                   // no slot for us elsewhere: stop stealing
-                int k = 0;
-                if (lane == 0) k = atomicAdd(p.cur + best_v, kStealChunk);
-                k = __shfl_sync(0xffffffffu, k, 0);
-                if (k >= len - first) continue;    // somebody else got there first: look again
-                a = lo + first + k;
-                e = a + kStealChunk < lo + len ? a + kStealChunk : lo + len;
+                got = __shfl_sync(0xffffffffu, got, 0);
+                if (got < 0) break;                // no slot for us elsewhere: stop stealing
+                if (got == 0) continue;            // somebody else got there first: look again
+                a = __shfl_sync(0xffffffffu, a, 0);
+                e = __shfl_sync(0xffffffffu, e, 0);
             }
             issue_range(a, e);
         }
