@@ -164,6 +164,21 @@ wmtp_status wmtp_draft_loop_full_host(const wmtp_kv* kv, int gamma, const void* 
                                       void* out_host, float* lse_host, void* stage,
                                       void* workspace, size_t ws_bytes, void* stream);
 
+/* ---- diagnostics ------------------------------------------------------------------------------ */
+
+/*
+ * Attention-mass diagnostics of a windowed against a full-context read-out of the same queries (Appendix D, the
+ * attention-mass table), from the outputs of wmtp_draft_attn_windowed and wmtp_draft_attn_full. Per row
+ * (sequence, query head), rows = batch * Hq:
+ *   mass[r]    = exp(lse_win - lse_full)                 share of the softmax mass inside sink + window
+ *   perturb[r] = ||o_full - o_win|| / ||o_full||           relative L2 change of the read-out when the far keys are dropped
+ *   tail[r]    = ||o_full - mass * o_win|| / ||o_full||    share of the read-out norm contributed by the far keys
+ *                (o_full = mass * o_win + (1 - mass) * o_far)
+ * out_*: device bf16 [rows][D]; lse_*: device fp32 [rows]; mass / perturb / tail: device fp32 [rows], any may be NULL.
+ */
+wmtp_status wmtp_attn_mass_diagnostics(const void* out_win, const float* lse_win, const void* out_full, const float* lse_full,
+                                       int rows, int D, float* mass, float* perturb, float* tail, void* stream);
+
 /* ---- tuning and accounting ---------------------------------------------------------------- */
 
 /* Upper bound on the CTAs (KV splits) of the attention kernels; 0 restores the default

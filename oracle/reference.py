@@ -229,6 +229,14 @@ def in_window_mass(lse_win, lse_full):
     return np.exp(np.asarray(lse_win) - np.asarray(lse_full))
 
 
+def tail_out_frac(o_full, o_win, lse_win, lse_full):
+    """Share of the read-out norm contributed by the far keys (Appendix D): ||(1 - mu) o_far|| / ||o_full||,
+    with (1 - mu) o_far = o_full - mu o_win."""
+    o_full, o_win = np.asarray(o_full), np.asarray(o_win)
+    mu = in_window_mass(lse_win, lse_full)[..., None]
+    return np.linalg.norm(o_full - mu * o_win, axis=-1) / np.linalg.norm(o_full, axis=-1)
+
+
 def win_perturb(o_full, o_win):
     """Relative L2 change of the read-out when the far keys are dropped (Appendix D)."""
     o_full, o_win = np.asarray(o_full), np.asarray(o_win)

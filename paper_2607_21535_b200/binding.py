@@ -65,6 +65,8 @@ _SIGNATURES = {
     "wmtp_draft_loop_full_host": (c_int, [POINTER(wmtp_kv), c_int, c_void_p, c_int, c_void_p, c_void_p, c_float,
                                           c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "wmtp_draft_attn_windowed_noalloc": (c_int, [c_void_p, c_int, POINTER(wmtp_ring), c_float, c_void_p, c_void_p, c_void_p]),
+    "wmtp_attn_mass_diagnostics": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p,
+                                           c_void_p]),
     "wmtp_set_max_ctas": (None, [c_int]),
     "wmtp_set_work_stealing": (None, [c_int]),
     "wmtp_launch_count": (c_int64, []),
@@ -262,6 +264,13 @@ def wmtp_draft_attn_windowed_noalloc(q, ring: Ring, out, lse=None, sm_scale: flo
     Hq = q.shape[-2]
     _check(lib().wmtp_draft_attn_windowed_noalloc(_ptr(q), Hq, byref(ring.desc), sm_scale, _ptr(out), _ptr(lse),
                                                   _stream(stream)))
+
+
+def wmtp_attn_mass_diagnostics(out_win, lse_win, out_full, lse_full, mass=None, perturb=None, tail=None, stream=None) -> None:
+    D = out_win.shape[-1]
+    rows = out_win.numel() // D
+    _check(lib().wmtp_attn_mass_diagnostics(_ptr(out_win), _ptr(lse_win), _ptr(out_full), _ptr(lse_full), rows, D, _ptr(mass),
+                                            _ptr(perturb), _ptr(tail), _stream(stream)))
 
 
 def wmtp_set_max_ctas(n: int) -> None:

@@ -125,6 +125,40 @@ __global__ void ring_init_kernel(RingParams r, KvParams kv) {
     if (blockIdx.x == 0 && threadIdx.x == 0) r.len[b] = S;
 }
 
+
+__device__ __forceinline__ float bf16_bits_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_bits_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// One warp per (sequence, query head) row: attention-mass diagnostics of a windowed against a full read-out
+// (Appendix D): mu = exp(lse_win - lse_full), ||o_full - o_win|| / ||o_full||, ||o_full - mu o_win|| / ||o_full||.
+__global__ void mass_diagnostics_kernel(const uint32_t* __restrict__ o_win, const float* __restrict__ lse_win,
+                                        const uint32_t* __restrict__ o_full, const float* __restrict__ lse_full, int rows,
+                                        int D, float* __restrict__ mass, float* __restrict__ perturb, float* __restrict__ tail) {
+    const int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32, lane = threadIdx.x % 32;
+    if (row >= rows) return;
+    const float lw = lse_win[row], lf = lse_full[row];
+    const float mu = (lf == -INFINITY) ? 0.f : __expf(lw - lf);
+    float n_full = 0.f, n_diff = 0.f, n_far = 0.f;
+    for (int w = lane; w < D / 2; w += 32) {
+        const uint32_t a = o_win[(int64_t)row * (D / 2) + w], b = o_full[(int64_t)row * (D / 2) + w];
+        const float w0 = bf16_bits_lo(a), w1 = bf16_bits_hi(a), f0 = bf16_bits_lo(b), f1 = bf16_bits_hi(b);
+        n_full += f0 * f0 + f1 * f1;
+        n_diff += (f0 - w0) * (f0 - w0) + (f1 - w1) * (f1 - w1);
+        n_far += (f0 - mu * w0) * (f0 - mu * w0) + (f1 - mu * w1) * (f1 - mu * w1);
+    }
+    for (int off = 16; off > 0; off >>= 1) {
+        n_full += __shfl_xor_sync(0xffffffffu, n_full, off);
+        n_diff += __shfl_xor_sync(0xffffffffu, n_diff, off);
+        n_far += __shfl_xor_sync(0xffffffffu, n_far, off);
+    }
+    if (lane == 0) {
+        const float inv = n_full > 0.f ? rsqrtf(n_full) : 0.f;
+        if (mass) mass[row] = mu;
+        if (perturb) perturb[row] = sqrtf(n_diff) * inv;
+        if (tail) tail[row] = sqrtf(n_far) * inv;
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_ring_reset(const RingParams& r, cudaStream_t st) {
@@ -158,6 +192,15 @@ cudaError_t launch_ring_init_from_kv(const RingParams& r, const KvParams& kv, cu
     if (bx > 592) bx = 592;
     dim3 grid(bx, r.B);
     ring_init_kernel<<<grid, warps * 32, 0, st>>>(r, kv);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mass_diagnostics(const void* o_win, const float* lse_win, const void* o_full, const float* lse_full, int rows,
+                                    int D, float* mass, float* perturb, float* tail, cudaStream_t st) {
+    const int warps = 4;
+    mass_diagnostics_kernel<<<(rows + warps - 1) / warps, warps * 32, 0, st>>>((const uint32_t*)o_win, lse_win, (const uint32_t*)o_full,
+                                                                             lse_full, rows, D, mass, perturb, tail);
     count_launch(1);
     return cudaGetLastError();
 }

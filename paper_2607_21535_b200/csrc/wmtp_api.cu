@@ -408,6 +408,16 @@ wmtp_status wmtp_draft_loop_full_host(const wmtp_kv* kv, int gamma, const void* 
                      ws_bytes, stream);
 }
 
+wmtp_status wmtp_attn_mass_diagnostics(const void* out_win, const float* lse_win, const void* out_full, const float* lse_full,
+                                       int rows, int D, float* mass, float* perturb, float* tail, void* stream) {
+    if (!out_win || !lse_win || !out_full || !lse_full) return fail(WMTP_ERR_INVALID_ARG, "an input pointer is NULL");
+    if (!mass && !perturb && !tail) return fail(WMTP_ERR_INVALID_ARG, "no output requested");
+    if (rows < 1 || D < 2 || D % 2 != 0) return fail(WMTP_ERR_INVALID_ARG, "rows=%d must be positive and D=%d even", rows, D);
+    if (!aligned(out_win, 4) || !aligned(out_full, 4)) return fail(WMTP_ERR_INVALID_ARG, "outputs of attention must be 4-byte aligned");
+    cudaError_t e = launch_mass_diagnostics(out_win, lse_win, out_full, lse_full, rows, D, mass, perturb, tail, (cudaStream_t)stream);
+    return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "mass diagnostics launch");
+}
+
 void wmtp_set_max_ctas(int max_ctas) { g_max_ctas.store(max_ctas < 0 ? 0 : max_ctas); }
 
 void wmtp_set_work_stealing(int enabled) { g_stealing.store(enabled ? 1 : 0); }

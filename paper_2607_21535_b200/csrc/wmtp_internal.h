@@ -97,6 +97,9 @@ cudaError_t launch_kv_append(const KvParams& kv, const void* k_new, const void* 
 // One cooperative launch: optional append of (k_new, v_new), split-KV partials, distributed LSE combine.
 cudaError_t launch_attention(const AttnParams& p, cudaStream_t st);
 
+cudaError_t launch_mass_diagnostics(const void* o_win, const float* lse_win, const void* o_full, const float* lse_full, int rows,
+                                    int D, float* mass, float* perturb, float* tail, cudaStream_t st);
+
 void count_launch(int n);
 int  sm_count();   // multiprocessors of the current device (cached), 0 on failure
 

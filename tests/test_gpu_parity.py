@@ -231,6 +231,27 @@ def test_planted_needle_full_finds_it_windowed_does_not():
     assert mass < 1e-3
 
 
+def test_attention_mass_diagnostics_match_oracle():
+    cfg = _cfg(S0=3000, D=128, W=256, gamma=2, seed=33, key_scale=(1.5, 2.5))     # peaked softmax: O(0.1..1) read-outs
+    wl = wi.make_workload(cfg)
+    dw = DeviceWorkload(wl)
+    dw.run_loops()
+    rows = cfg.gamma * cfg.Hq
+    mass, perturb, tail = (torch.full((rows,), float("nan"), device="cuda") for _ in range(3))
+    wm.wmtp_attn_mass_diagnostics(dw.out_w, dw.lse_w, dw.out_f, dw.lse_f, mass=mass, perturb=perturb, tail=tail)
+    orc = oracle_for(wl, 0)
+    for i in range(cfg.gamma):
+        r = orc.step(wl.q[i, 0], wl.k_new[i, 0], wl.v_new[i, 0])
+        (ow, lw), (of, lf) = r["win"], r["full"]
+        sl = slice(i * cfg.Hq, (i + 1) * cfg.Hq)
+        np.testing.assert_allclose(mass[sl].cpu().numpy(), R.in_window_mass(lw, lf), rtol=2e-3, atol=1e-6)
+        # the device works from the bf16 outputs: allow their rounding (2^-9 relative per element on both vectors)
+        np.testing.assert_allclose(perturb[sl].cpu().numpy(), R.win_perturb(of, ow), atol=1e-2, rtol=1e-2)
+        np.testing.assert_allclose(tail[sl].cpu().numpy(), R.tail_out_frac(of, ow, lw, lf), atol=1e-2, rtol=1e-2)
+    m = mass.cpu().numpy()
+    assert ((m > 0) & (m <= 1 + 1e-6)).all()
+
+
 def test_explicit_softmax_scale():
     cfg = _cfg(S0=700, D=128, gamma=1)
     wl = wi.make_workload(cfg)

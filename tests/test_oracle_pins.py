@@ -282,3 +282,20 @@ def test_mass_identity_and_needle():
     assert np.abs(of[0] - needle_v).max() < 1e-2
     assert np.abs(ow[0] - needle_v).max() > 0.5
     assert R.win_perturb(of, ow)[0] > 0.5
+
+
+def test_tail_out_frac_matches_far_key_contribution():
+    cfg = _small_cfg(S0=200, W=24, n_sink=3, D=16)
+    wl = wi.make_workload(cfg, threads=1)
+    o = R.DraftOracle(wl.K[0], wl.V[0], cfg.Hq, cfg.n_sink, cfg.W)
+    r = o.step(wl.q[0, 0], wl.k_new[0, 0], wl.v_new[0, 0])
+    (ow, lw), (of, lf) = r["win"], r["full"]
+    keep = set(R.keep_set(o.S, cfg.n_sink, cfg.W))
+    far = [p for p in range(o.S) if p not in keep]
+    ofar, lfar = R.attention(wl.q[0, 0], o.Kfull[:, :o.S], o.Vfull[:, :o.S], keys=far)
+    far_share = np.exp(lfar - lf)[:, None] * ofar                 # the far keys' part of the full read-out, computed directly
+    want = np.linalg.norm(far_share, axis=-1) / np.linalg.norm(of, axis=-1)
+    np.testing.assert_allclose(R.tail_out_frac(of, ow, lw, lf), want, rtol=1e-10)
+    # dropping nothing changes nothing
+    np.testing.assert_allclose(R.tail_out_frac(of, of, lf, lf), 0.0, atol=1e-15)
+    np.testing.assert_allclose(R.win_perturb(of, of), 0.0, atol=1e-15)
