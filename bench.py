@@ -289,6 +289,13 @@ def main():
     for _ in range(reps):
         wm.wmtp_draft_attn_full(q[0], kv, o1, ws)
     k1.record()
+    # windowed attention read straight from the KV store through the sink + last-W tiles (no ring), same launches
+    v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wm.wmtp_draft_attn_windowed_kv(q[0], kv, cfg.n_sink, cfg.W, o1, ws)
+    v0.record()
+    for _ in range(reps):
+        wm.wmtp_draft_attn_windowed_kv(q[0], kv, cfg.n_sink, cfg.W, o1, ws)
+    v1.record()
     wev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     for a, b in wev:
@@ -297,6 +304,7 @@ def main():
     torch.cuda.synchronize()
     wm.wmtp_device_status(ws)
     us_full_call = k0.elapsed_time(k1) * 1e3 / reps
+    us_win_kv_call = v0.elapsed_time(v1) * 1e3 / reps
     us_win_call_cold = statistics.mean(a.elapsed_time(b) for a, b in wev) * 1e3
     cur_lens = lens.cpu().numpy()
 
@@ -365,6 +373,8 @@ def main():
                              "algorithmic_gbs": win_bytes / (us_win * 1e-6) / 1e9,
                              "pct_of_8tbs": win_bytes / (us_win * 1e-6) / 8e12 * 100,
                              "us_per_call_cold_l2": us_win_call_cold},
+                "windowed_kv_view": {"us_per_attention_call": us_win_kv_call,
+                                     "note": "sink + last-W tiles read from the KV store through its page table / rows"},
                 "full": {"us_per_step": us_full, "kv_bytes_per_step": full_bytes,
                          "algorithmic_gbs": full_bytes / (us_full * 1e-6) / 1e9,
                          "pct_of_8tbs": full_bytes / (us_full * 1e-6) / 8e12 * 100,

@@ -164,6 +164,26 @@ wmtp_status wmtp_draft_loop_full_host(const wmtp_kv* kv, int gamma, const void* 
                                       void* out_host, float* lse_host, void* stage,
                                       void* workspace, size_t ws_bytes, void* stream);
 
+/* ---- windowed attention straight from the KV store (no ring) ----------------------------------- */
+
+/*
+ * The paper's own realisation of the window (Section 4 "Mechanism"; Appendix A pseudocode): the draft keeps its
+ * full-length KV, and each draft step attends over a reduced key set taken from it -- the first n_sink positions and
+ * the last W positions, [0, S) when S <= n_sink + W -- which in a paged store is the per-request block table reduced
+ * to [sink blocks] || [recent-W blocks]. Here the reduced table is never materialised: the kernel walks the sink
+ * tiles and the tiles of the last W tokens through the page table (or the contiguous rows) arithmetically, O(W) per
+ * step, and masks the ragged ends row by row, so the window is token-granular whatever the page size. Same result as
+ * wmtp_draft_attn_windowed on a ring that holds the same tokens; arguments as wmtp_draft_attn_full plus n_sink >= 0,
+ * W >= 1.
+ */
+wmtp_status wmtp_draft_attn_windowed_kv(const void* q, int Hq, const wmtp_kv* kv, int n_sink, int W, float sm_scale,
+                                        void* out, float* lse, void* workspace, size_t ws_bytes, void* stream);
+
+/* gamma draft steps on the KV store: append (k_new[i], v_new[i]) at position len, then attend over sink + last W. */
+wmtp_status wmtp_draft_loop_windowed_kv(const wmtp_kv* kv, int n_sink, int W, int gamma, const void* q, int Hq,
+                                        const void* k_new, const void* v_new, float sm_scale, void* out, float* lse,
+                                        void* workspace, size_t ws_bytes, void* stream);
+
 /* ---- diagnostics ------------------------------------------------------------------------------ */
 
 /*

@@ -65,6 +65,10 @@ _SIGNATURES = {
     "wmtp_draft_loop_full_host": (c_int, [POINTER(wmtp_kv), c_int, c_void_p, c_int, c_void_p, c_void_p, c_float,
                                           c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "wmtp_draft_attn_windowed_noalloc": (c_int, [c_void_p, c_int, POINTER(wmtp_ring), c_float, c_void_p, c_void_p, c_void_p]),
+    "wmtp_draft_attn_windowed_kv": (c_int, [c_void_p, c_int, POINTER(wmtp_kv), c_int, c_int, c_float, c_void_p, c_void_p,
+                                            c_void_p, c_size_t, c_void_p]),
+    "wmtp_draft_loop_windowed_kv": (c_int, [POINTER(wmtp_kv), c_int, c_int, c_int, c_void_p, c_int, c_void_p, c_void_p,
+                                            c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "wmtp_attn_mass_diagnostics": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p,
                                            c_void_p]),
     "wmtp_set_max_ctas": (None, [c_int]),
@@ -264,6 +268,20 @@ def wmtp_draft_attn_windowed_noalloc(q, ring: Ring, out, lse=None, sm_scale: flo
     Hq = q.shape[-2]
     _check(lib().wmtp_draft_attn_windowed_noalloc(_ptr(q), Hq, byref(ring.desc), sm_scale, _ptr(out), _ptr(lse),
                                                   _stream(stream)))
+
+
+def wmtp_draft_attn_windowed_kv(q, kv: KV, n_sink: int, W: int, out, ws: Workspace, lse=None, sm_scale: float = 0.0,
+                                stream=None) -> None:
+    Hq = q.shape[-2]
+    _check(lib().wmtp_draft_attn_windowed_kv(_ptr(q), Hq, byref(kv.desc), n_sink, W, sm_scale, _ptr(out), _ptr(lse), ws.ptr,
+                                             ws.nbytes, _stream(stream)))
+
+
+def wmtp_draft_loop_windowed_kv(kv: KV, n_sink: int, W: int, q, k_new, v_new, out, ws: Workspace, lse=None,
+                                sm_scale: float = 0.0, stream=None) -> None:
+    gamma, Hq = q.shape[0], q.shape[-2]
+    _check(lib().wmtp_draft_loop_windowed_kv(byref(kv.desc), n_sink, W, gamma, _ptr(q), Hq, _ptr(k_new), _ptr(v_new),
+                                             sm_scale, _ptr(out), _ptr(lse), ws.ptr, ws.nbytes, _stream(stream)))
 
 
 def wmtp_attn_mass_diagnostics(out_win, lse_win, out_full, lse_full, mass=None, perturb=None, tail=None, stream=None) -> None:

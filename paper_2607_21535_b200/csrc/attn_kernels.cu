@@ -225,6 +225,7 @@ __device__ __forceinline__ int kMaxSegmentsPadded(const AttnParams& p) { return 
 struct Segment {
     int b, g, seg;
     int64_t seg_start, tiles, nk, S;
+    int64_t ns, lo, sink_tiles, win_first;   // tile -> row mapping of the sequence (SeqView)
     int64_t slot_base;          // first partial slot of the segment
     int cap;                    // partial slots the segment has
 };
@@ -236,8 +237,8 @@ __device__ __forceinline__ Segment locate_segment(const AttnParams& p, const int
     const int64_t in_seq = t - seq_start;
     s.g = (in_seq < 0x7fffffffLL && s.tiles < 0x7fffffffLL) ? (int)((uint32_t)in_seq / (uint32_t)s.tiles) : (int)(in_seq / s.tiles);
     s.seg_start = seq_start + (int64_t)s.g * s.tiles;
-    s.S = eff_len(p, s.b);
-    s.nk = scan_keys(p, s.b);
+    const SeqView v = seq_view(p, s.b);
+    s.S = v.S; s.nk = v.nk; s.ns = v.ns; s.lo = v.lo; s.sink_tiles = v.sink_tiles; s.win_first = v.win_first;
     s.seg = s.b * p.Hkv + s.g;
     s.cap = cap_prefix[s.b + 1] - cap_prefix[s.b];
     s.slot_base = (int64_t)p.Hkv * cap_prefix[s.b] + (int64_t)s.g * s.cap;
@@ -444,7 +445,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 
     // ---- plan: tiles per sequence and partial-slot capacity per sequence (all from len[], O(B))
     for (int b = threadIdx.x; b < p.B; b += blockDim.x)
-        tile_prefix[b + 1] = (scan_keys(p, b) + kTileKeys - 1) / kTileKeys;
+        tile_prefix[b + 1] = seq_view(p, b).tiles;
     __syncthreads();
     if (threadIdx.x == 0) {
         int64_t acc = 0;
@@ -534,7 +535,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 for (int base = 0; base < ntiles; base += 32) {
                     int page = 0;
                     if (p.mode == kPaged) {
-                        const int64_t ti = first_tile + base + lane;
+                        const int64_t tj = first_tile + base + lane;
+                        const int64_t ti = tj < sg.sink_tiles ? tj : sg.win_first + tj - sg.sink_tiles;   // source tile = page index
                         if (base + lane < ntiles) {
                             page = p.page_table[(int64_t)sg.b * p.max_pages + ti];
                             if (page < 0 || page >= p.num_pages) { atomicCAS(p.status, 0, kErrBounds); page = 0; }
@@ -559,7 +561,11 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                             if (!*abort_flag) {
                                 int64_t row;
                                 if (p.mode == kPaged) row = ((int64_t)pg * p.Hkv + sg.g) * kTileKeys;
-                                else row = ((int64_t)sg.b * p.Hkv + sg.g) * p.rows_per_head + (first_tile + base + j) * kTileKeys;
+                                else {
+                                    const int64_t tj = first_tile + base + j;
+                                    const int64_t src = tj < sg.sink_tiles ? tj : sg.win_first + tj - sg.sink_tiles;
+                                    row = ((int64_t)sg.b * p.Hkv + sg.g) * p.rows_per_head + src * kTileKeys;
+                                }
                                 const uint32_t dstK = stage0 + s * C::kStageBytes, dstV = dstK + C::kTileBytes;
                                 stage_tile[s] = t + base + j;          // ordered before the consumers' wait by the arrive below
                                 mbar_expect_tx(bar_fullK + 8 * s, C::kTileBytes);
@@ -723,6 +729,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 
     Segment sg;
     sg.seg = -1; sg.seg_start = 0; sg.tiles = 0; sg.b = 0; sg.g = 0; sg.nk = 0; sg.S = 0; sg.slot_base = 0; sg.cap = 0;
+    sg.ns = 0; sg.lo = 0; sg.sink_tiles = 0; sg.win_first = 0;
     int64_t new_tile = -1;                               // tile (within the segment) whose row this warp must patch (fused append)
     int new_row = 0;
     int seg_tiles_done = 0;                              // tiles of the current segment this group has processed
@@ -850,7 +857,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             const int64_t pos = sg.S - 1;
             const int64_t key = p.mode == kRing ? ring_slot(pos, p.n_sink, p.cap) : pos;
             new_row = (int)(key % kTileKeys);
-            if ((new_row >> 4) == warp) new_tile = key / kTileKeys;
+            // tile of the segment that holds the row: with a window view, the last tile unless the token is a sink token
+            if ((new_row >> 4) == warp) new_tile = (p.window_view && sg.S > sg.ns) ? sg.tiles - 1 : key / kTileKeys;
         }
         // Q^T fragments (B operand: k = d, n = head); heads >= G read as zero
         const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
@@ -894,11 +902,14 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         have_tile = false;
         ++seg_tiles_done;
         {
-            const int64_t key0 = (tt - sg.seg_start) * kTileKeys;
+            const int64_t tj = tt - sg.seg_start;                      // tile within the segment
+            const bool sink_part = tj < sg.sink_tiles;
+            const int64_t key0 = (sink_part ? tj : sg.win_first + tj - sg.sink_tiles) * kTileKeys;   // first row of the tile
+            const int64_t vlo = sink_part ? 0 : sg.lo, vhi = sink_part ? sg.ns : sg.S;              // rows of it that count
             const int64_t wkey0 = key0 + warp * 16;
-            const bool tile_full = (key0 + kTileKeys <= sg.nk) && !slack;
-            const bool any_valid = wkey0 < sg.nk;
-            const bool has_new = (tt - sg.seg_start) == new_tile;      // this warp owns the appended row in this tile
+            const bool tile_full = key0 >= vlo && key0 + kTileKeys <= vhi && !slack;
+            const bool any_valid = wkey0 < vhi && wkey0 + 16 > vlo;
+            const bool has_new = tj == new_tile;                       // this warp owns the appended row in this tile
             const uint32_t sK = stage0 + s * C::kStageBytes, sV = sK + C::kTileBytes;
             int64_t new_off = 0;
             bool new_ok = true;
@@ -941,7 +952,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 for (int i = 0; i < 4; ++i) sc[i] = (sa[i] + sb[i]) * scale;
                 if (!tile_full) {
                     const int64_t ka = wkey0 + g8, kb = ka + 8;
-                    bool va = ka < sg.nk, vb = kb < sg.nk;
+                    bool va = ka >= vlo && ka < vhi, vb = kb >= vlo && kb < vhi;
                     if (slack) {
                         va = va && ring_slot_live((int)ka, sg.S, p.n_sink, p.W, p.cap);
                         vb = vb && ring_slot_live((int)kb, sg.S, p.n_sink, p.W, p.cap);
@@ -988,17 +999,17 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 #else
             if (any_valid) {
 #endif
-                if (wkey0 + 16 > sg.nk) {
-                    // rows past the sequence end were never written: they may hold NaN/Inf bit patterns,
-                    // and 0 * NaN would poison the accumulators. Zero them in shared memory.
-                    const int first_bad = (int)(sg.nk - wkey0);
+                if (wkey0 + 16 > vhi) {
+                    // rows past the end were never written (or, in a sink tile of a window view, may be): they can hold
+                    // NaN/Inf bit patterns, and 0 * NaN would poison the accumulators. Zero them in shared memory.
+                    const int first_bad = vhi > wkey0 ? (int)(vhi - wkey0) : 0;
                     for (int idx = lane; idx < (16 - first_bad) * C::kChunks * 8; idx += 32) {
                         const int r = first_bad + idx / (C::kChunks * 8), rem = idx % (C::kChunks * 8);
                         const uint32_t addr = sV + (rem >> 3) * C::kChunkBytes + (warp * 16 + r) * 128 + ((rem & 7) << 4);
                         asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
                     }
                 }
-                if (has_new || wkey0 + 16 > sg.nk) {
+                if (has_new || wkey0 + 16 > vhi) {
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                 }

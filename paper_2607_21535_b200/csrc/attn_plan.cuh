@@ -40,6 +40,35 @@ __device__ __forceinline__ int64_t scan_keys(const AttnParams& p, int b) {
     return S;
 }
 
+// How the tiles of one sequence map onto its K/V rows. A sequence contributes `tiles` tiles per KV head: first
+// `sink_tiles` tiles covering rows [0, ns) (source tile j = j), then tiles covering rows [lo, S) (source tile
+// win_first + j - sink_tiles). Without a window view everything is the first kind: ns = keys scanned, no second part.
+// With a window view (the paper's own mechanism, Section 4: the draft's block table is reduced to the sink blocks and
+// the blocks of the last W tokens) the rows are those of the full KV store and ns = min(S, n_sink),
+// lo = max(ns, S - W); a 64-row tile that straddles lo, ns or S is masked row by row, so the ends are token-granular
+// whatever the page size.
+struct SeqView {
+    int64_t S, nk, ns, lo, sink_tiles, win_first, tiles;
+};
+__device__ __forceinline__ SeqView seq_view(const AttnParams& p, int b) {
+    SeqView v;
+    v.S = eff_len(p, b);
+    v.nk = scan_keys(p, b);
+    if (!p.window_view) {
+        v.ns = v.nk; v.lo = v.nk;
+        v.sink_tiles = (v.nk + kTileKeys - 1) / kTileKeys;
+        v.win_first = 0;
+        v.tiles = v.sink_tiles;
+    } else {
+        v.ns = v.S < p.n_sink ? v.S : p.n_sink;
+        v.lo = v.S - p.W > v.ns ? v.S - p.W : v.ns;
+        v.sink_tiles = (v.ns + kTileKeys - 1) / kTileKeys;
+        v.win_first = v.lo / kTileKeys;
+        v.tiles = v.sink_tiles + (v.S > v.ns ? (v.S - 1) / kTileKeys - v.win_first + 1 : 0);
+    }
+    return v;
+}
+
 // Is ring slot s (< scan_keys) inside sink + last-W? Always true when cap == W.
 __device__ __forceinline__ bool ring_slot_live(int s, int64_t S, int n_sink, int W, int cap) {
     if (s < n_sink) return true;

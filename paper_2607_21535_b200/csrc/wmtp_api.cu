@@ -152,9 +152,10 @@ wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm
     return WMTP_OK;
 }
 
+// W > 0: window view (attend over the first n_sink and the last W positions of the KV store); W == 0: all positions.
 wmtp_status attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, void* out, float* lse, void* ws,
                       size_t ws_bytes, cudaStream_t st, bool validate, const void* k_new = nullptr,
-                      const void* v_new = nullptr) {
+                      const void* v_new = nullptr, int n_sink = 0, int W = 0) {
     if (validate) {
         if (wmtp_status s = check_kv(kv)) return s;
         if (wmtp_status s = check_attn_common(q, Hq, kv->Hkv, kv->batch, kv->D, out, lse, ws, ws_bytes)) return s;
@@ -166,11 +167,16 @@ wmtp_status attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, 
     p.mode = kv->page_table ? kPaged : kContiguous;
     p.rows_per_head = kv->page_table ? kv->page_size : kv->S_cap;
     p.page_size = kv->page_size; p.max_pages = kv->max_pages; p.num_pages = kv->num_pages;
-    const int64_t tiles = (kv->S_cap + kTileKeys - 1) / kTileKeys * kv->batch * kv->Hkv;
-    p.num_ctas = pick_ctas(tiles);
+    int64_t tiles_per_seg = (kv->S_cap + kTileKeys - 1) / kTileKeys;
+    if (W > 0) {
+        p.window_view = 1; p.n_sink = n_sink; p.W = W;
+        const int64_t view_tiles = ((int64_t)n_sink + kTileKeys - 1) / kTileKeys + ((int64_t)W + kTileKeys - 1) / kTileKeys + 1;
+        if (view_tiles < tiles_per_seg) tiles_per_seg = view_tiles;
+    }
+    p.num_ctas = pick_ctas(tiles_per_seg * kv->batch * kv->Hkv);
     if (p.num_ctas <= 0) return fail(WMTP_ERR_CUDA, "no CUDA device available");
     cudaError_t e = launch_attention(p, st);
-    if (e != cudaSuccess) return cuda_fail(e, "full attention launch");
+    if (e != cudaSuccess) return cuda_fail(e, W > 0 ? "windowed (KV view) attention launch" : "full attention launch");
     return WMTP_OK;
 }
 
@@ -354,6 +360,35 @@ wmtp_status wmtp_draft_loop_full(const wmtp_kv* kv, int gamma, const void* q, in
                                       lse ? lse + (size_t)i * kv->batch * Hq : nullptr, workspace, ws_bytes,
                                       (cudaStream_t)stream, false, (const char*)k_new + i * kv_step,
                                       (const char*)v_new + i * kv_step))
+            return s;
+    }
+    return WMTP_OK;
+}
+
+static wmtp_status check_window(int n_sink, int W) {
+    if (n_sink < 0 || W < 1) return fail(WMTP_ERR_INVALID_ARG, "window view needs n_sink >= 0 and W >= 1 (n_sink=%d W=%d)", n_sink, W);
+    return WMTP_OK;
+}
+
+wmtp_status wmtp_draft_attn_windowed_kv(const void* q, int Hq, const wmtp_kv* kv, int n_sink, int W, float sm_scale,
+                                        void* out, float* lse, void* workspace, size_t ws_bytes, void* stream) {
+    if (wmtp_status s = check_window(n_sink, W)) return s;
+    return attn_full(q, Hq, kv, sm_scale, out, lse, workspace, ws_bytes, (cudaStream_t)stream, true, nullptr, nullptr, n_sink, W);
+}
+
+wmtp_status wmtp_draft_loop_windowed_kv(const wmtp_kv* kv, int n_sink, int W, int gamma, const void* q, int Hq,
+                                        const void* k_new, const void* v_new, float sm_scale, void* out, float* lse,
+                                        void* workspace, size_t ws_bytes, void* stream) {
+    if (wmtp_status s = check_window(n_sink, W)) return s;
+    if (wmtp_status s = check_kv(kv)) return s;
+    if (wmtp_status s = check_loop(gamma, k_new, v_new)) return s;
+    if (wmtp_status s = check_attn_common(q, Hq, kv->Hkv, kv->batch, kv->D, out, lse, workspace, ws_bytes)) return s;
+    const size_t q_step = (size_t)kv->batch * Hq * kv->D * 2, kv_step = (size_t)kv->batch * kv->Hkv * kv->D * 2;
+    for (int i = 0; i < gamma; ++i) {
+        if (wmtp_status s = attn_full((const char*)q + i * q_step, Hq, kv, sm_scale, (char*)out + i * q_step,
+                                      lse ? lse + (size_t)i * kv->batch * Hq : nullptr, workspace, ws_bytes,
+                                      (cudaStream_t)stream, false, (const char*)k_new + i * kv_step,
+                                      (const char*)v_new + i * kv_step, n_sink, W))
             return s;
     }
     return WMTP_OK;

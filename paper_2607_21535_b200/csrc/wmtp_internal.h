@@ -74,6 +74,7 @@ struct AttnParams {
     int mode;
     int page_size, max_pages, num_pages;
     int n_sink, W, cap;
+    int window_view;          // contiguous / paged only: attend over the first n_sink and the last W positions of the KV store
     float scale_log2;         // sm_scale * log2(e)
     int num_ctas;
 };
