@@ -224,24 +224,28 @@ __device__ __forceinline__ int kMaxSegmentsPadded(const AttnParams& p) { return 
 // One (sequence, KV head) segment as seen by a CTA.
 struct Segment {
     int b, g, seg;
-    int64_t seg_start, tiles, nk, S;
-    int64_t ns, lo, sink_tiles, win_first;   // tile -> row mapping of the sequence (SeqView)
-    int64_t slot_base;          // first partial slot of the segment
+    // Tile indices and row counts fit 32 bits: the K/V tensors are limited to 2^31 - 1 rows (TMA coordinates), so the
+    // tile line has fewer than 2^25 tiles. Only the logical length of a ring can be larger.
+    int seg_start, tiles, nk;
+    int ns, lo, hi, sink_tiles, win_first;   // tile -> row mapping of the sequence (SeqView); hi = rows end of the second part
+    int slot_base;              // first partial slot of the segment
+    int64_t S;
     int cap;                    // partial slots the segment has
 };
 __device__ __forceinline__ Segment locate_segment(const AttnParams& p, const int64_t* tile_prefix, const int* cap_prefix, int64_t t) {
     Segment s;
     s.b = find_seq(tile_prefix, p.B, p.Hkv, t);
-    s.tiles = tile_prefix[s.b + 1] - tile_prefix[s.b];
-    const int64_t seq_start = (int64_t)p.Hkv * tile_prefix[s.b];
-    const int64_t in_seq = t - seq_start;
-    s.g = (in_seq < 0x7fffffffLL && s.tiles < 0x7fffffffLL) ? (int)((uint32_t)in_seq / (uint32_t)s.tiles) : (int)(in_seq / s.tiles);
-    s.seg_start = seq_start + (int64_t)s.g * s.tiles;
+    s.tiles = (int)(tile_prefix[s.b + 1] - tile_prefix[s.b]);
+    const int seq_start = p.Hkv * (int)tile_prefix[s.b];
+    const int in_seq = (int)t - seq_start;
+    s.g = (int)((uint32_t)in_seq / (uint32_t)s.tiles);
+    s.seg_start = seq_start + s.g * s.tiles;
     const SeqView v = seq_view(p, s.b);
-    s.S = v.S; s.nk = v.nk; s.ns = v.ns; s.lo = v.lo; s.sink_tiles = v.sink_tiles; s.win_first = v.win_first;
+    s.S = v.S; s.nk = (int)v.nk; s.ns = (int)v.ns; s.lo = (int)v.lo; s.sink_tiles = (int)v.sink_tiles; s.win_first = (int)v.win_first;
+    s.hi = (int)(v.S < 0x7fffffffLL ? v.S : 0x7fffffffLL);
     s.seg = s.b * p.Hkv + s.g;
     s.cap = cap_prefix[s.b + 1] - cap_prefix[s.b];
-    s.slot_base = (int64_t)p.Hkv * cap_prefix[s.b] + (int64_t)s.g * s.cap;
+    s.slot_base = p.Hkv * cap_prefix[s.b] + s.g * s.cap;
     return s;
 }
 
@@ -626,7 +630,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 if (!may_steal || *abort_flag) break;
                 // ---- steal: look at every cursor, take from the range with the most left
                 int64_t best_rem = 0;
-                int best_v = -1;
+                int best_v = -1, best_used = 0;
                 for (int v = lane; v < Cn; v += 32) {
                     if (v == (int)blockIdx.x) continue;
                     int64_t lo, len, first;
@@ -636,13 +640,14 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                     if (rem <= 0) continue;
                     const int64_t tv = lo + first + used;
                     if (cur_seg >= 0 && tv >= cur_lo && tv < cur_hi) rem += (int64_t)1 << 40;     // same segment: preferred
-                    if (rem > best_rem) { best_rem = rem; best_v = v; }
+                    if (rem > best_rem) { best_rem = rem; best_v = v; best_used = (int)used; }
                 }
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) {
                     const int64_t r2 = __shfl_xor_sync(0xffffffffu, best_rem, off);
                     const int v2 = __shfl_xor_sync(0xffffffffu, best_v, off);
-                    if (r2 > best_rem || (r2 == best_rem && v2 > best_v)) { best_rem = r2; best_v = v2; }
+                    const int u2 = __shfl_xor_sync(0xffffffffu, best_used, off);
+                    if (r2 > best_rem || (r2 == best_rem && v2 > best_v)) { best_rem = r2; best_v = v2; best_used = u2; }
                 }
                 if (best_v < 0) break;
                 int64_t lo, len, first;
@@ -652,8 +657,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 // stolen chunk never straddles a segment boundary.
                 int got = 0;                       // 1: tiles [a, e) are ours; 0: look again; -1: stop stealing
                 if (lane == 0) {
+                    int used = best_used;          // cursor value seen by the scan; a failed swap returns the current one
                     for (int tries = 0; tries < 8 && got == 0; ++tries) {
-                        const int used = __ldcg(p.cur + best_v);
                         const int64_t rem = len - first - used;
                         if (rem <= 0) break;
                         const int64_t tv = lo + first + used;
@@ -668,9 +673,14 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                                 adm_lo = alo = vs.seg_start; adm_hi = ahi = vs.seg_start + vs.tiles;
                             }
                         }
-                        int64_t take = rem < kStealChunk ? rem : kStealChunk;
+                        int64_t take = rem / 8;            // larger bites while much is left: a steal costs two round trips
+                        if (take < kStealChunk) take = kStealChunk;
+                        if (take > 8) take = 8;
+                        if (take > rem) take = rem;
                         if (tv + take > ahi) take = ahi - tv;
-                        if (atomicCAS(p.cur + best_v, used, used + (int)take) == used) { a = tv; e = tv + take; got = 1; }
+                        const int prev = atomicCAS(p.cur + best_v, used, used + (int)take);
+                        if (prev == used) { a = tv; e = tv + take; got = 1; }
+                        else used = prev;
                     }
                 }
                 got = __shfl_sync(0xffffffffu, got, 0);
@@ -729,8 +739,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 
     Segment sg;
     sg.seg = -1; sg.seg_start = 0; sg.tiles = 0; sg.b = 0; sg.g = 0; sg.nk = 0; sg.S = 0; sg.slot_base = 0; sg.cap = 0;
-    sg.ns = 0; sg.lo = 0; sg.sink_tiles = 0; sg.win_first = 0;
-    int64_t new_tile = -1;                               // tile (within the segment) whose row this warp must patch (fused append)
+    sg.ns = 0; sg.lo = 0; sg.hi = 0; sg.sink_tiles = 0; sg.win_first = 0;
+    int new_tile = -1;                                   // tile (within the segment) whose row this warp must patch (fused append)
     int new_row = 0;
     int seg_tiles_done = 0;                              // tiles of the current segment this group has processed
     uint32_t qb[C::kKSteps][2];
@@ -785,7 +795,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             p.part_key[sg.slot_base + k] = (int)blockIdx.x * kMaxGroups + grp;
         }
         ++ord;
-        const int64_t pidx = sg.slot_base + k;
+        const int64_t pidx = (int64_t)sg.slot_base + k;
         float f[2];
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
@@ -830,7 +840,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         if (tid == 0) {
             __threadfence();                                   // the group's partial is visible device-wide before the arrival
             const unsigned long long old = atomicAdd(p.arrive + par_off + sg.seg, (1ull << 32) | (unsigned long long)seg_tiles_done);
-            if ((int64_t)(uint32_t)old + seg_tiles_done == sg.tiles) {   // this contribution completes the segment
+            if ((int)(uint32_t)old + seg_tiles_done == sg.tiles) {        // this contribution completes the segment
                 if (atomicAdd(p.segs_done, 1) + 1 == nonempty_segs) {
                     *p.segs_done = 0;
                     *p.epoch = epoch + 1u;
@@ -858,7 +868,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             const int64_t key = p.mode == kRing ? ring_slot(pos, p.n_sink, p.cap) : pos;
             new_row = (int)(key % kTileKeys);
             // tile of the segment that holds the row: with a window view, the last tile unless the token is a sink token
-            if ((new_row >> 4) == warp) new_tile = (p.window_view && sg.S > sg.ns) ? sg.tiles - 1 : key / kTileKeys;
+            if ((new_row >> 4) == warp) new_tile = (p.window_view && sg.S > sg.ns) ? sg.tiles - 1 : (int)(key / kTileKeys);
         }
         // Q^T fragments (B operand: k = d, n = head); heads >= G read as zero
         const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
@@ -902,11 +912,11 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         have_tile = false;
         ++seg_tiles_done;
         {
-            const int64_t tj = tt - sg.seg_start;                      // tile within the segment
+            const int tj = (int)tt - sg.seg_start;                     // tile within the segment
             const bool sink_part = tj < sg.sink_tiles;
-            const int64_t key0 = (sink_part ? tj : sg.win_first + tj - sg.sink_tiles) * kTileKeys;   // first row of the tile
-            const int64_t vlo = sink_part ? 0 : sg.lo, vhi = sink_part ? sg.ns : sg.S;              // rows of it that count
-            const int64_t wkey0 = key0 + warp * 16;
+            const int key0 = (sink_part ? tj : sg.win_first + tj - sg.sink_tiles) * kTileKeys;   // first row of the tile
+            const int vlo = sink_part ? 0 : sg.lo, vhi = sink_part ? sg.ns : sg.hi;             // rows of it that count
+            const int wkey0 = key0 + warp * 16;
             const bool tile_full = key0 >= vlo && key0 + kTileKeys <= vhi && !slack;
             const bool any_valid = wkey0 < vhi && wkey0 + 16 > vlo;
             const bool has_new = tj == new_tile;                       // this warp owns the appended row in this tile
@@ -951,11 +961,11 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 #pragma unroll
                 for (int i = 0; i < 4; ++i) sc[i] = (sa[i] + sb[i]) * scale;
                 if (!tile_full) {
-                    const int64_t ka = wkey0 + g8, kb = ka + 8;
+                    const int ka = wkey0 + g8, kb = ka + 8;
                     bool va = ka >= vlo && ka < vhi, vb = kb >= vlo && kb < vhi;
                     if (slack) {
-                        va = va && ring_slot_live((int)ka, sg.S, p.n_sink, p.W, p.cap);
-                        vb = vb && ring_slot_live((int)kb, sg.S, p.n_sink, p.W, p.cap);
+                        va = va && ring_slot_live(ka, sg.S, p.n_sink, p.W, p.cap);
+                        vb = vb && ring_slot_live(kb, sg.S, p.n_sink, p.W, p.cap);
                     }
                     if (!va) { sc[0] = -INFINITY; sc[1] = -INFINITY; }
                     if (!vb) { sc[2] = -INFINITY; sc[3] = -INFINITY; }
@@ -1002,7 +1012,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 if (wkey0 + 16 > vhi) {
                     // rows past the end were never written (or, in a sink tile of a window view, may be): they can hold
                     // NaN/Inf bit patterns, and 0 * NaN would poison the accumulators. Zero them in shared memory.
-                    const int first_bad = vhi > wkey0 ? (int)(vhi - wkey0) : 0;
+                    const int first_bad = vhi > wkey0 ? vhi - wkey0 : 0;
                     for (int idx = lane; idx < (16 - first_bad) * C::kChunks * 8; idx += 32) {
                         const int r = first_bad + idx / (C::kChunks * 8), rem = idx % (C::kChunks * 8);
                         const uint32_t addr = sV + (rem >> 3) * C::kChunkBytes + (warp * 16 + r) * 128 + ((rem & 7) << 4);
