@@ -82,4 +82,4 @@ def check_ring_against_sim(ring: wm.Ring, b: int, sim: R.RingSim, what=""):
 def oracle_for(wl: wi.Workload, b: int, cap=None, with_ring=True) -> R.DraftOracle:
     cfg = wl.cfg
     return R.DraftOracle(wl.K[b], wl.V[b], cfg.Hq, cfg.n_sink, cfg.W, cap=cap if cap is not None else cfg.W + cfg.cap_slack,
-                         reserve=cfg.gamma + 1, with_ring=with_ring)
+                         reserve=4 * cfg.gamma + 4, with_ring=with_ring)

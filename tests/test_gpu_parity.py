@@ -155,6 +155,20 @@ def test_batched_ragged_lengths(paged, max_ctas):
     _run_and_check(cfg, max_ctas=max_ctas)
 
 
+@pytest.mark.parametrize("max_ctas", [1, 2, 0])
+@pytest.mark.parametrize("D", [128, 256])
+def test_many_short_sequences_one_cta_touches_many_segments(max_ctas, D):
+    # 48 sequences x 2 KV heads = 96 segments: with one or two CTAs a consumer group contributes to more segments than
+    # it can keep outstanding, so it has to combine part-way through its range
+    cfg = _cfg(batch=48, S0=0, S0_range=(1, 400), D=D, W=64, n_sink=4, gamma=2, seed=4242)
+    _run_and_check(cfg, max_ctas=max_ctas, check_ring=False)
+
+
+def test_large_batch_of_short_sequences():
+    cfg = _cfg(batch=300, S0=0, S0_range=(1, 150), D=128, W=32, n_sink=2, gamma=1, seed=99, paged=True)
+    _run_and_check(cfg, check_ring=False, seqs=[0, 1, 57, 150, 298, 299])
+
+
 def test_batch_with_empty_sequences():
     cfg = _cfg(batch=4, S0=0, S0_range=(1, 300), gamma=1, seed=5)
     wl = wi.make_workload(cfg)
@@ -261,6 +275,33 @@ def test_explicit_softmax_scale():
     wm.wmtp_draft_attn_full(dw.q[0], dw.kv, out, dw.ws, lse=lse, sm_scale=0.25)
     ro, rl = R.attention(wl.q[0, 0], np.ascontiguousarray(wl.K[0]), np.ascontiguousarray(wl.V[0]), sm_scale=0.25)
     compare(out[0], lse[0], ro, rl, what="scale 0.25")
+
+
+def test_draft_loops_replay_from_a_cuda_graph():
+    # lengths live on the device and are advanced by the kernels, so a captured loop can be replayed as is
+    cfg = _cfg(S0=3000, D=256, W=256, gamma=3, seed=61)
+    wl = wi.make_workload(cfg, extra_cap=16)
+    dw = DeviceWorkload(wl)
+    wm.wmtp_ring_init_from_kv(dw.ring, dw.kv)
+    torch.cuda.synchronize()
+    g, s = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            wm.wmtp_draft_loop_windowed(dw.ring, dw.q, dw.k_new, dw.v_new, dw.out_w, dw.ws, lse=dw.lse_w)
+            wm.wmtp_draft_loop_full(dw.kv, dw.q, dw.k_new, dw.v_new, dw.out_f, dw.ws, lse=dw.lse_f)
+    orc = oracle_for(wl, 0)
+    orc_reserve = orc.Kfull.shape[1]
+    assert orc_reserve >= cfg.S0 + 2 * cfg.gamma
+    for replay in range(2):
+        g.replay()
+        torch.cuda.synchronize()
+        wm.wmtp_device_status(dw.ws)
+        for i in range(cfg.gamma):
+            r = orc.step(wl.q[i, 0], wl.k_new[i, 0], wl.v_new[i, 0])
+            compare(dw.out_w[i, 0], dw.lse_w[i, 0], *r["win"], what=f"graph replay {replay} step {i} windowed")
+            compare(dw.out_f[i, 0], dw.lse_f[i, 0], *r["full"], what=f"graph replay {replay} step {i} full")
+        assert int(dw.lens[0]) == orc.S and int(dw.ring.len[0]) == orc.S
+    check_ring_against_sim(dw.ring, 0, orc.ring, "after two graph replays")
 
 
 def test_host_buffer_loop_matches_device_loop():
