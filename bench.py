@@ -329,6 +329,41 @@ def main():
         lens.copy_(torch.from_numpy(cur_lens).to(dev))
         wm.wmtp_ring_init_from_kv(ring, kv)
         torch.cuda.synchronize()
+    # ---- draft-extend after a verify step: q_len = 4 tokens per sequence (3 accepted + the bonus token) appended to
+    #      a ring with slack slots and to the KV store, then attended in one launch each
+    ext = None
+    ql = 4
+    if B * ql <= 1024:
+        ring_x = wm.Ring(B, cfg.Hkv, cfg.D, cfg.n_sink, cfg.W, cap=cfg.W + 8, device=dev)
+        ws_x = wm.Workspace(B * ql, cfg.Hq, cfg.Hkv, cfg.D, device=dev)
+        wm.wmtp_ring_init_from_kv(ring_x, kv)
+        per_seq = lambda t: t[:ql].transpose(0, 1).contiguous()
+        qx, kx, vx = per_seq(q), per_seq(kn), per_seq(vn)
+        ox = torch.empty_like(qx)
+        drop = torch.full((B,), ql, dtype=torch.int32, device=dev)
+
+        def extend_windowed():
+            wm.wmtp_ring_append_many(ring_x, kx, vx)
+            wm.wmtp_draft_extend_windowed(qx, ring_x, ox, ws_x)
+            wm.wmtp_ring_rewind(ring_x, drop, ws_x)          # keeps the ring at the same length for the next repeat
+
+        extend_windowed()
+        wm.wmtp_draft_extend_full(qx, kv, ox, ws_x)
+        x0, x1, x2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        x0.record()
+        for _ in range(reps):
+            extend_windowed()
+        x1.record()
+        for _ in range(reps):
+            wm.wmtp_draft_extend_full(qx, kv, ox, ws_x)      # the last q_len tokens of the store, re-attended
+        x2.record()
+        torch.cuda.synchronize()
+        wm.wmtp_device_status(ws_x)
+        ext = {"q_len": ql,
+               "windowed_us_per_iteration": x0.elapsed_time(x1) * 1e3 / reps,
+               "full_us_per_call": x1.elapsed_time(x2) * 1e3 / reps,
+               "note": "windowed: append q_len tokens to a ring with 8 slack slots + one multi-query attention launch + "
+                       "rollback (3 launches); full: one multi-query attention launch over the whole KV store"}
     full_bytes = float(cur_lens.sum()) * cfg.kv_bytes_per_token
     win_bytes = float(np.minimum(cur_lens, cfg.n_sink + cfg.W).sum()) * cfg.kv_bytes_per_token
     peak, peak_src = measured_peaks()
@@ -379,6 +414,7 @@ def main():
                          "algorithmic_gbs": full_bytes / (us_full * 1e-6) / 1e9,
                          "pct_of_8tbs": full_bytes / (us_full * 1e-6) / 8e12 * 100,
                          "us_per_attention_call": us_full_call},
+                "draft_extend": ext,
             },
             "windowed_flatness": flat,
             "roofline": {"bound": "hbm", "kernel": "attn_fused_tma (full-context draft attention: split-KV partials + in-kernel combine)",

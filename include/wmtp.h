@@ -184,6 +184,39 @@ wmtp_status wmtp_draft_loop_windowed_kv(const wmtp_kv* kv, int n_sink, int W, in
                                         const void* k_new, const void* v_new, float sm_scale, void* out, float* lse,
                                         void* workspace, size_t ws_bytes, void* stream);
 
+/* ---- after verification: rollback and draft-extend -------------------------------------------- */
+
+/*
+ * A decode step ends with the target accepting some of the proposed tokens. The draft then (a) discards the K/V of the
+ * rejected ones -- the ring reserves d slots of slack for exactly this (Section 4 "Memory"; Section 6 "Compatibility
+ * with tree speculation": n_sink + W + d) -- and (b) re-processes the accepted tokens in one "draft-extend" pass,
+ * several new tokens per sequence at once, each attending causally up to itself (Section 5 "The backend is not the
+ * confound"; Appendix B, per-kernel table).
+ *
+ * wmtp_ring_rewind: drops the last n_drop[r] tokens of every sequence (device int32 [batch]): len shrinks and the
+ *   slots of the dropped positions get slot_pos = -1. Requires 0 <= n_drop[r] <= min(len[r], cap - W): the rows those
+ *   tokens overwrote are then outside every later window. A violation is flagged in `workspace` (may be NULL) and the
+ *   sequence is left unchanged. The bound is on the distance below the longest length the sequence has reached:
+ *   the kernel checks each call by itself, so a caller that rewinds twice without appending in between keeps the
+ *   sum within cap - W.
+ * wmtp_ring_append_many / wmtp_kv_append_many: n_tok tokens per sequence in one launch; k_new, v_new are device bf16
+ *   [batch][n_tok][Hkv][D]; token j goes to position len + j; len += n_tok (all or nothing for the KV store).
+ * wmtp_draft_extend_windowed / _full: q is device bf16 [batch][q_len][Hq][D]; the q_len tokens must already be in the
+ *   store. Query i of a sequence attends as a decode step would have at length len - (q_len - 1 - i): over sink + last W
+ *   of that length (windowed; needs cap >= W + q_len - 1) or over all positions below it (full). out: device bf16
+ *   [batch][q_len][Hq][D]; lse: device fp32 [batch][q_len][Hq] or NULL. The workspace must be sized for
+ *   batch * q_len sequences: wmtp_workspace_bytes(batch * q_len, Hq, Hkv, D). One launch; K/V are read once per
+ *   query from L2/HBM.
+ */
+wmtp_status wmtp_ring_rewind(const wmtp_ring* ring, const int32_t* n_drop, void* workspace, void* stream);
+wmtp_status wmtp_ring_append_many(const wmtp_ring* ring, int n_tok, const void* k_new, const void* v_new, void* stream);
+wmtp_status wmtp_kv_append_many(const wmtp_kv* kv, int n_tok, const void* k_new, const void* v_new, void* workspace,
+                                void* stream);
+wmtp_status wmtp_draft_extend_windowed(const void* q, int q_len, int Hq, const wmtp_ring* ring, float sm_scale, void* out,
+                                       float* lse, void* workspace, size_t ws_bytes, void* stream);
+wmtp_status wmtp_draft_extend_full(const void* q, int q_len, int Hq, const wmtp_kv* kv, float sm_scale, void* out,
+                                   float* lse, void* workspace, size_t ws_bytes, void* stream);
+
 /* ---- diagnostics ------------------------------------------------------------------------------ */
 
 /*

@@ -174,6 +174,20 @@ class RingSim:
         return slot
 
 
+    def rewind(self, n_drop: int):
+        """Discard the last n_drop tokens (rejected speculative tokens): their slots become empty."""
+        assert 0 <= n_drop <= self.length
+        for _ in range(n_drop):
+            p = self.length - 1
+            slot = p if p < self.n_sink else (self.cursor - 1 if self.cursor > self.n_sink else self.n_sink + self.cap - 1)
+            assert self.slot_pos[slot] == p
+            self.slot_pos[slot] = -1
+            self.written[slot] = False
+            if p >= self.n_sink:
+                self.cursor = slot
+            self.length = p
+
+
 class DraftOracle:
     """One sequence's draft state: full KV, list store and ring simulation, stepped together."""
 

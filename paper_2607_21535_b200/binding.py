@@ -69,6 +69,13 @@ _SIGNATURES = {
                                             c_void_p, c_size_t, c_void_p]),
     "wmtp_draft_loop_windowed_kv": (c_int, [POINTER(wmtp_kv), c_int, c_int, c_int, c_void_p, c_int, c_void_p, c_void_p,
                                             c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "wmtp_ring_rewind": (c_int, [POINTER(wmtp_ring), c_void_p, c_void_p, c_void_p]),
+    "wmtp_ring_append_many": (c_int, [POINTER(wmtp_ring), c_int, c_void_p, c_void_p, c_void_p]),
+    "wmtp_kv_append_many": (c_int, [POINTER(wmtp_kv), c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "wmtp_draft_extend_windowed": (c_int, [c_void_p, c_int, c_int, POINTER(wmtp_ring), c_float, c_void_p, c_void_p, c_void_p,
+                                           c_size_t, c_void_p]),
+    "wmtp_draft_extend_full": (c_int, [c_void_p, c_int, c_int, POINTER(wmtp_kv), c_float, c_void_p, c_void_p, c_void_p,
+                                       c_size_t, c_void_p]),
     "wmtp_attn_mass_diagnostics": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p,
                                            c_void_p]),
     "wmtp_set_max_ctas": (None, [c_int]),
@@ -282,6 +289,33 @@ def wmtp_draft_loop_windowed_kv(kv: KV, n_sink: int, W: int, q, k_new, v_new, ou
     gamma, Hq = q.shape[0], q.shape[-2]
     _check(lib().wmtp_draft_loop_windowed_kv(byref(kv.desc), n_sink, W, gamma, _ptr(q), Hq, _ptr(k_new), _ptr(v_new),
                                              sm_scale, _ptr(out), _ptr(lse), ws.ptr, ws.nbytes, _stream(stream)))
+
+
+def wmtp_ring_rewind(ring: Ring, n_drop, ws: Workspace | None = None, stream=None) -> None:
+    _check(lib().wmtp_ring_rewind(byref(ring.desc), _ptr(n_drop), ws.ptr if ws is not None else None, _stream(stream)))
+
+
+def wmtp_ring_append_many(ring: Ring, k_new, v_new, stream=None) -> None:
+    """k_new, v_new: [batch][n_tok][Hkv][D]."""
+    _check(lib().wmtp_ring_append_many(byref(ring.desc), k_new.shape[1], _ptr(k_new), _ptr(v_new), _stream(stream)))
+
+
+def wmtp_kv_append_many(kv: KV, k_new, v_new, ws: Workspace | None = None, stream=None) -> None:
+    _check(lib().wmtp_kv_append_many(byref(kv.desc), k_new.shape[1], _ptr(k_new), _ptr(v_new),
+                                     ws.ptr if ws is not None else None, _stream(stream)))
+
+
+def wmtp_draft_extend_windowed(q, ring: Ring, out, ws: Workspace, lse=None, sm_scale: float = 0.0, stream=None) -> None:
+    """q, out: [batch][q_len][Hq][D]; the workspace must be sized for batch * q_len sequences."""
+    q_len, Hq = q.shape[1], q.shape[2]
+    _check(lib().wmtp_draft_extend_windowed(_ptr(q), q_len, Hq, byref(ring.desc), sm_scale, _ptr(out), _ptr(lse), ws.ptr,
+                                            ws.nbytes, _stream(stream)))
+
+
+def wmtp_draft_extend_full(q, kv: KV, out, ws: Workspace, lse=None, sm_scale: float = 0.0, stream=None) -> None:
+    q_len, Hq = q.shape[1], q.shape[2]
+    _check(lib().wmtp_draft_extend_full(_ptr(q), q_len, Hq, byref(kv.desc), sm_scale, _ptr(out), _ptr(lse), ws.ptr,
+                                        ws.nbytes, _stream(stream)))
 
 
 def wmtp_attn_mass_diagnostics(out_win, lse_win, out_full, lse_full, mass=None, perturb=None, tail=None, stream=None) -> None:

@@ -542,7 +542,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         const int64_t tj = first_tile + base + lane;
                         const int64_t ti = tj < sg.sink_tiles ? tj : sg.win_first + tj - sg.sink_tiles;   // source tile = page index
                         if (base + lane < ntiles) {
-                            page = p.page_table[(int64_t)sg.b * p.max_pages + ti];
+                            page = p.page_table[(int64_t)kv_seq(p, sg.b) * p.max_pages + ti];
                             if (page < 0 || page >= p.num_pages) { atomicCAS(p.status, 0, kErrBounds); page = 0; }
                         }
                     }
@@ -568,7 +568,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                                 else {
                                     const int64_t tj = first_tile + base + j;
                                     const int64_t src = tj < sg.sink_tiles ? tj : sg.win_first + tj - sg.sink_tiles;
-                                    row = ((int64_t)sg.b * p.Hkv + sg.g) * p.rows_per_head + src * kTileKeys;
+                                    row = ((int64_t)kv_seq(p, sg.b) * p.Hkv + sg.g) * p.rows_per_head + src * kTileKeys;
                                 }
                                 const uint32_t dstK = stage0 + s * C::kStageBytes, dstV = dstK + C::kTileBytes;
                                 stage_tile[s] = t + base + j;          // ordered before the consumers' wait by the arrive below
@@ -1132,7 +1132,9 @@ cudaError_t launch_fused(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaSt
 
 int64_t attention_rows(const AttnParams& p) {
     if (p.mode == kPaged) return (int64_t)p.num_pages * p.Hkv * p.page_size;
-    return (int64_t)p.B * p.Hkv * p.rows_per_head;
+    // p.B counts queries; the store holds p.B / q_len sequences. The extent must be exact: rows of the last tile that
+    // lie beyond it are filled by TMA instead of being read from memory the caller may not own.
+    return (int64_t)(p.B / (p.q_len > 1 ? p.q_len : 1)) * p.Hkv * p.rows_per_head;
 }
 
 cudaError_t launch_attention(const AttnParams& p_in, cudaStream_t st) {

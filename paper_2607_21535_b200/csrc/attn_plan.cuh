@@ -20,13 +20,23 @@ __device__ __forceinline__ int ring_slot(int64_t p, int n_sink, int cap) {
     return n_sink + (w < 0x7fffffffLL ? (int)((uint32_t)w % (uint32_t)cap) : (int)(w % cap));
 }
 
-// Does this launch append a token to sequence b before attending (fused draft step)?
+// Does this launch append a token to sequence b before attending (fused draft step)? (Only with one query per sequence.)
 __device__ __forceinline__ bool appends_to(const AttnParams& p, int b) {
     return p.k_new != nullptr && (p.mode == kRing || p.len[b] < p.S_cap);
 }
 
-// Sequence length the attention sees: the stored length, plus the token appended by this launch.
+// The batch index b of the kernel counts *queries*: with q_len queries per sequence (draft-extend: the last q_len
+// tokens of a sequence re-processed in one launch, each attending causally up to itself), query b belongs to
+// sequence b / q_len and is its (b % q_len)-th new token.
+__device__ __forceinline__ int kv_seq(const AttnParams& p, int b) { return p.q_len > 1 ? b / p.q_len : b; }
+
+// Sequence length the attention of query b sees: the stored length, plus the token appended by this launch; for
+// draft-extend, the length at which that query's own token was the newest.
 __device__ __forceinline__ int64_t eff_len(const AttnParams& p, int b) {
+    if (p.q_len > 1) {
+        const int64_t S = p.len[b / p.q_len] - (p.q_len - 1 - b % p.q_len);
+        return S > 0 ? S : 0;
+    }
     return p.len[b] + (appends_to(p, b) ? 1 : 0);
 }
 

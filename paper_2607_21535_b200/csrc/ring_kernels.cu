@@ -126,6 +126,82 @@ __global__ void ring_init_kernel(RingParams r, KvParams kv) {
 }
 
 
+// n_tok tokens per sequence in one launch (the accepted tokens of a decode step, re-processed by the draft):
+// token j goes to position len + j. One block per sequence; k_new / v_new are [B][n_tok][Hkv][D].
+__global__ void ring_append_many_kernel(RingParams r, int n_tok, const uint4* __restrict__ k_new, const uint4* __restrict__ v_new) {
+    const int b = blockIdx.x;
+    const int64_t p0 = r.len[b];
+    const int slots = r.n_sink + r.cap;
+    const int vec_per_row = r.D / 8;
+    const int n_vec = r.Hkv * vec_per_row;
+    uint4* K = reinterpret_cast<uint4*>(r.k);
+    uint4* V = reinterpret_cast<uint4*>(r.v);
+    for (int idx = threadIdx.x; idx < n_tok * n_vec; idx += blockDim.x) {
+        const int j = idx / n_vec, i = idx % n_vec;
+        const int g = i / vec_per_row, c = i % vec_per_row;
+        const int slot = ring_slot(p0 + j, r.n_sink, r.cap);
+        const int64_t dst = (((int64_t)b * r.Hkv + g) * slots + slot) * vec_per_row + c;
+        const int64_t src = ((int64_t)b * n_tok + j) * n_vec + i;
+        K[dst] = k_new[src];
+        V[dst] = v_new[src];
+    }
+    __syncthreads();   // every thread has read len[b] before it moves
+    for (int j = threadIdx.x; j < n_tok; j += blockDim.x)
+        r.slot_pos[(int64_t)b * slots + ring_slot(p0 + j, r.n_sink, r.cap)] = (int32_t)(p0 + j);
+    if (threadIdx.x == 0) r.len[b] = p0 + n_tok;
+}
+
+__global__ void kv_append_many_kernel(KvParams kv, int n_tok, const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                                      int* status) {
+    const int b = blockIdx.x;
+    const int64_t p0 = kv.len[b];
+    const int vec_per_row = kv.D / 8;
+    const int n_vec = kv.Hkv * vec_per_row;
+    __shared__ int bad;
+    if (threadIdx.x == 0) bad = 0;
+    __syncthreads();
+    if (p0 + n_tok > kv.S_cap) {                     // all or nothing: a partial append would leave len ambiguous
+        if (threadIdx.x == 0 && status) atomicCAS(status, 0, kErrBounds);
+        return;
+    }
+    uint4* K = reinterpret_cast<uint4*>(kv.k);
+    uint4* V = reinterpret_cast<uint4*>(kv.v);
+    for (int idx = threadIdx.x; idx < n_tok * n_vec; idx += blockDim.x) {
+        const int j = idx / n_vec, i = idx % n_vec;
+        const int g = i / vec_per_row, c = i % vec_per_row;
+        bool ok = true;
+        const int64_t dst = kv_row_vec(kv, b, g, p0 + j, vec_per_row, &ok) + c;
+        if (!ok) { bad = 1; continue; }
+        const int64_t src = ((int64_t)b * n_tok + j) * n_vec + i;
+        K[dst] = k_new[src];
+        V[dst] = v_new[src];
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (bad) { if (status) atomicCAS(status, 0, kErrBounds); }
+        else kv.len[b] = p0 + n_tok;
+    }
+}
+
+// Discards the last n_drop[b] tokens of every sequence (speculative tokens the target rejected; Section 4 "Memory" and
+// Section 6: the ring reserves d extra slots for them). Only the bookkeeping moves: len shrinks and the slots of the
+// dropped positions are marked empty; the rows they overwrote lie outside every future window as long as no more than
+// cap - W tokens are dropped, which is checked.
+__global__ void ring_rewind_kernel(RingParams r, const int32_t* __restrict__ n_drop, int* status) {
+    const int b = blockIdx.x;
+    const int64_t S = r.len[b];
+    const int slots = r.n_sink + r.cap;
+    const int n = n_drop[b];
+    if (n < 0 || n > S || n > r.cap - r.W) {
+        if (threadIdx.x == 0 && status) atomicCAS(status, 0, kErrBounds);
+        return;
+    }
+    for (int j = threadIdx.x; j < n; j += blockDim.x)
+        r.slot_pos[(int64_t)b * slots + ring_slot(S - 1 - j, r.n_sink, r.cap)] = -1;
+    __syncthreads();
+    if (threadIdx.x == 0) r.len[b] = S - n;
+}
+
 __device__ __forceinline__ float bf16_bits_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_bits_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
@@ -201,6 +277,24 @@ cudaError_t launch_mass_diagnostics(const void* o_win, const float* lse_win, con
     const int warps = 4;
     mass_diagnostics_kernel<<<(rows + warps - 1) / warps, warps * 32, 0, st>>>((const uint32_t*)o_win, lse_win, (const uint32_t*)o_full,
                                                                              lse_full, rows, D, mass, perturb, tail);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ring_append_many(const RingParams& r, int n_tok, const void* k_new, const void* v_new, cudaStream_t st) {
+    ring_append_many_kernel<<<r.B, 256, 0, st>>>(r, n_tok, (const uint4*)k_new, (const uint4*)v_new);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_kv_append_many(const KvParams& kv, int n_tok, const void* k_new, const void* v_new, int* status, cudaStream_t st) {
+    kv_append_many_kernel<<<kv.B, 256, 0, st>>>(kv, n_tok, (const uint4*)k_new, (const uint4*)v_new, status);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ring_rewind(const RingParams& r, const int32_t* n_drop, int* status, cudaStream_t st) {
+    ring_rewind_kernel<<<r.B, 32, 0, st>>>(r, n_drop, status);
     count_launch(1);
     return cudaGetLastError();
 }

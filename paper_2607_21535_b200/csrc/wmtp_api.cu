@@ -125,6 +125,7 @@ void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, 
     p.part_lse = reinterpret_cast<float*>(base + L.part_lse_off);
     p.part_o = reinterpret_cast<float*>(base + L.part_o_off);
     p.B = batch; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.G = Hq / Hkv;
+    p.q_len = 1;
     const float s = sm_scale > 0.f ? sm_scale : 1.0f / std::sqrt((float)D);
     p.scale_log2 = s * 1.4426950408889634f;
 }
@@ -132,19 +133,20 @@ void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, 
 // k_new / v_new non-NULL: a fused draft step (append, then attend) in one launch.
 wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm_scale, void* out, float* lse,
                           void* ws, size_t ws_bytes, cudaStream_t st, bool validate, const void* k_new = nullptr,
-                          const void* v_new = nullptr) {
+                          const void* v_new = nullptr, int q_len = 1) {
     if (validate) {
         if (wmtp_status s = check_ring(ring)) return s;
-        if (wmtp_status s = check_attn_common(q, Hq, ring->Hkv, ring->batch, ring->D, out, lse, ws, ws_bytes)) return s;
+        if (wmtp_status s = check_attn_common(q, Hq, ring->Hkv, ring->batch * q_len, ring->D, out, lse, ws, ws_bytes)) return s;
     }
     AttnParams p{};
-    fill_attn(p, q, Hq, ring->Hkv, ring->batch, ring->D, sm_scale, out, lse, ws);
+    fill_attn(p, q, Hq, ring->Hkv, ring->batch * q_len, ring->D, sm_scale, out, lse, ws);
+    p.q_len = q_len;
     p.k = ring->k; p.v = ring->v; p.page_table = nullptr; p.len = ring->len;
     p.k_new = k_new; p.v_new = v_new; p.slot_pos = ring->slot_pos;
     p.mode = kRing;
     p.rows_per_head = (int64_t)ring->n_sink + ring->cap;
     p.n_sink = ring->n_sink; p.W = ring->W; p.cap = ring->cap;
-    const int64_t tiles = (p.rows_per_head + kTileKeys - 1) / kTileKeys * ring->batch * ring->Hkv;
+    const int64_t tiles = (p.rows_per_head + kTileKeys - 1) / kTileKeys * ring->batch * q_len * ring->Hkv;
     p.num_ctas = pick_ctas(tiles);
     if (p.num_ctas <= 0) return fail(WMTP_ERR_CUDA, "no CUDA device available");
     cudaError_t e = launch_attention(p, st);
@@ -155,13 +157,14 @@ wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm
 // W > 0: window view (attend over the first n_sink and the last W positions of the KV store); W == 0: all positions.
 wmtp_status attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, void* out, float* lse, void* ws,
                       size_t ws_bytes, cudaStream_t st, bool validate, const void* k_new = nullptr,
-                      const void* v_new = nullptr, int n_sink = 0, int W = 0) {
+                      const void* v_new = nullptr, int n_sink = 0, int W = 0, int q_len = 1) {
     if (validate) {
         if (wmtp_status s = check_kv(kv)) return s;
-        if (wmtp_status s = check_attn_common(q, Hq, kv->Hkv, kv->batch, kv->D, out, lse, ws, ws_bytes)) return s;
+        if (wmtp_status s = check_attn_common(q, Hq, kv->Hkv, kv->batch * q_len, kv->D, out, lse, ws, ws_bytes)) return s;
     }
     AttnParams p{};
-    fill_attn(p, q, Hq, kv->Hkv, kv->batch, kv->D, sm_scale, out, lse, ws);
+    fill_attn(p, q, Hq, kv->Hkv, kv->batch * q_len, kv->D, sm_scale, out, lse, ws);
+    p.q_len = q_len;
     p.k = kv->k; p.v = kv->v; p.page_table = kv->page_table; p.len = kv->len;
     p.k_new = k_new; p.v_new = v_new; p.slot_pos = nullptr; p.S_cap = kv->S_cap;
     p.mode = kv->page_table ? kPaged : kContiguous;
@@ -173,7 +176,7 @@ wmtp_status attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, 
         const int64_t view_tiles = ((int64_t)n_sink + kTileKeys - 1) / kTileKeys + ((int64_t)W + kTileKeys - 1) / kTileKeys + 1;
         if (view_tiles < tiles_per_seg) tiles_per_seg = view_tiles;
     }
-    p.num_ctas = pick_ctas(tiles_per_seg * kv->batch * kv->Hkv);
+    p.num_ctas = pick_ctas(tiles_per_seg * kv->batch * q_len * kv->Hkv);
     if (p.num_ctas <= 0) return fail(WMTP_ERR_CUDA, "no CUDA device available");
     cudaError_t e = launch_attention(p, st);
     if (e != cudaSuccess) return cuda_fail(e, W > 0 ? "windowed (KV view) attention launch" : "full attention launch");
@@ -363,6 +366,55 @@ wmtp_status wmtp_draft_loop_full(const wmtp_kv* kv, int gamma, const void* q, in
             return s;
     }
     return WMTP_OK;
+}
+
+/* ---- draft-extend: several new tokens per sequence in one launch ---- */
+
+static wmtp_status check_extend(int q_len, int batch) {
+    if (q_len < 1 || q_len > 64) return fail(WMTP_ERR_INVALID_ARG, "q_len=%d must be in [1, 64]", q_len);
+    if ((int64_t)batch * q_len > kMaxBatch) return fail(WMTP_ERR_UNSUPPORTED, "batch*q_len=%lld exceeds %d", (long long)batch * q_len, kMaxBatch);
+    return WMTP_OK;
+}
+
+wmtp_status wmtp_ring_append_many(const wmtp_ring* ring, int n_tok, const void* k_new, const void* v_new, void* stream) {
+    if (wmtp_status s = check_ring(ring)) return s;
+    if (wmtp_status s = check_loop(n_tok, k_new, v_new)) return s;
+    if (n_tok > ring->cap) return fail(WMTP_ERR_CAPACITY, "n_tok=%d exceeds the ring's %d window slots", n_tok, ring->cap);
+    cudaError_t e = launch_ring_append_many(ring_params(ring), n_tok, k_new, v_new, (cudaStream_t)stream);
+    return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "ring append launch");
+}
+
+wmtp_status wmtp_kv_append_many(const wmtp_kv* kv, int n_tok, const void* k_new, const void* v_new, void* workspace, void* stream) {
+    if (wmtp_status s = check_kv(kv)) return s;
+    if (wmtp_status s = check_loop(n_tok, k_new, v_new)) return s;
+    if (workspace && !aligned(workspace, 256)) return fail(WMTP_ERR_WORKSPACE, "workspace is not 256-byte aligned");
+    cudaError_t e = launch_kv_append_many(kv_params(kv), n_tok, k_new, v_new, static_cast<int*>(workspace), (cudaStream_t)stream);
+    return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "kv append launch");
+}
+
+wmtp_status wmtp_ring_rewind(const wmtp_ring* ring, const int32_t* n_drop, void* workspace, void* stream) {
+    if (wmtp_status s = check_ring(ring)) return s;
+    if (!n_drop || !aligned(n_drop, 4)) return fail(WMTP_ERR_INVALID_ARG, "n_drop is NULL or misaligned");
+    if (workspace && !aligned(workspace, 256)) return fail(WMTP_ERR_WORKSPACE, "workspace is not 256-byte aligned");
+    cudaError_t e = launch_ring_rewind(ring_params(ring), n_drop, static_cast<int*>(workspace), (cudaStream_t)stream);
+    return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "ring rewind launch");
+}
+
+wmtp_status wmtp_draft_extend_windowed(const void* q, int q_len, int Hq, const wmtp_ring* ring, float sm_scale, void* out,
+                                       float* lse, void* workspace, size_t ws_bytes, void* stream) {
+    if (wmtp_status s = check_ring(ring)) return s;
+    if (wmtp_status s = check_extend(q_len, ring->batch)) return s;
+    if (ring->cap < ring->W + q_len - 1)
+        return fail(WMTP_ERR_CAPACITY, "draft-extend of %d tokens needs cap >= W + %d slots (cap=%d, W=%d): the oldest query's "
+                    "window would already be overwritten", q_len, q_len - 1, ring->cap, ring->W);
+    return attn_windowed(q, Hq, ring, sm_scale, out, lse, workspace, ws_bytes, (cudaStream_t)stream, true, nullptr, nullptr, q_len);
+}
+
+wmtp_status wmtp_draft_extend_full(const void* q, int q_len, int Hq, const wmtp_kv* kv, float sm_scale, void* out, float* lse,
+                                   void* workspace, size_t ws_bytes, void* stream) {
+    if (wmtp_status s = check_kv(kv)) return s;
+    if (wmtp_status s = check_extend(q_len, kv->batch)) return s;
+    return attn_full(q, Hq, kv, sm_scale, out, lse, workspace, ws_bytes, (cudaStream_t)stream, true, nullptr, nullptr, 0, 0, q_len);
 }
 
 static wmtp_status check_window(int n_sink, int W) {

@@ -74,6 +74,7 @@ struct AttnParams {
     int mode;
     int page_size, max_pages, num_pages;
     int n_sink, W, cap;
+    int q_len;                // queries per sequence (1: decode; > 1: draft-extend, B then counts queries)
     int window_view;          // contiguous / paged only: attend over the first n_sink and the last W positions of the KV store
     float scale_log2;         // sm_scale * log2(e)
     int num_ctas;
@@ -95,6 +96,9 @@ cudaError_t launch_ring_reset(const RingParams& r, cudaStream_t st);
 cudaError_t launch_ring_append(const RingParams& r, const void* k_new, const void* v_new, cudaStream_t st);
 cudaError_t launch_ring_init_from_kv(const RingParams& r, const KvParams& kv, cudaStream_t st);
 cudaError_t launch_kv_append(const KvParams& kv, const void* k_new, const void* v_new, int* status, cudaStream_t st);
+cudaError_t launch_ring_append_many(const RingParams& r, int n_tok, const void* k_new, const void* v_new, cudaStream_t st);
+cudaError_t launch_kv_append_many(const KvParams& kv, int n_tok, const void* k_new, const void* v_new, int* status, cudaStream_t st);
+cudaError_t launch_ring_rewind(const RingParams& r, const int32_t* n_drop, int* status, cudaStream_t st);
 // One cooperative launch: optional append of (k_new, v_new), split-KV partials, distributed LSE combine.
 cudaError_t launch_attention(const AttnParams& p, cudaStream_t st);
 

@@ -100,3 +100,24 @@ def test_attention_arguments_rejected_on_host():
     assert L.wmtp_ring_init_from_kv(ctypes.byref(r), ctypes.byref(_kv_desc(Hkv=4)), None) == 1
     with pytest.raises(wm.WmtpError):
         binding._check(1)
+
+
+def test_extend_and_rollback_arguments_rejected_on_host():
+    L = wm.lib()
+    r, kv = _ring_desc(cap=12), _kv_desc()
+    big = 1 << 30
+    rb, kb = ctypes.byref(r), ctypes.byref(kv)
+    assert L.wmtp_draft_extend_windowed(4096, 0, 16, rb, 0.0, 4096, None, 4096, big, None) == 1       # q_len < 1
+    assert L.wmtp_draft_extend_windowed(4096, 65, 16, rb, 0.0, 4096, None, 4096, big, None) == 1      # q_len > 64
+    assert L.wmtp_draft_extend_windowed(4096, 6, 16, rb, 0.0, 4096, None, 4096, big, None) == 3       # cap 12 < W + 5
+    assert L.wmtp_draft_extend_windowed(None, 5, 16, rb, 0.0, 4096, None, 4096, big, None) == 1
+    assert L.wmtp_draft_extend_windowed(4096, 5, 16, rb, 0.0, 4096, None, 4096, 1000, None) == 4      # workspace too small
+    assert L.wmtp_draft_extend_full(4096, 0, 16, kb, 0.0, 4096, None, 4096, big, None) == 1
+    assert L.wmtp_draft_extend_full(4096, 4, 16, ctypes.byref(_kv_desc(batch=512)), 0.0, 4096, None, 4096, big, None) == 2
+    assert L.wmtp_draft_extend_full(4096, 4, 16, kb, 0.0, None, None, 4096, big, None) == 1
+    assert L.wmtp_ring_append_many(rb, 0, 4096, 4096, None) == 1
+    assert L.wmtp_ring_append_many(rb, 3, None, 4096, None) == 1
+    assert L.wmtp_kv_append_many(kb, 0, 4096, 4096, None, None) == 1
+    assert L.wmtp_kv_append_many(kb, 2, 4096, None, None, None) == 1
+    assert L.wmtp_ring_rewind(rb, None, None, None) == 1
+    assert L.wmtp_ring_rewind(ctypes.byref(_ring_desc(W=0)), 4096, None, None) == 1

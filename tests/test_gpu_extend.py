@@ -1,0 +1,192 @@
+"""Rollback of rejected tokens and draft-extend (several new tokens per sequence in one launch), against the oracle's
+sequential decode steps and its slot-level ring simulation."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2607_21535_b200 as wm
+import wmtp_inputs as wi
+from oracle import reference as R
+
+from harness import DeviceWorkload, bits, check_ring_against_sim, compare, oracle_for, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def _defaults():
+    wm.wmtp_set_max_ctas(0)
+    wm.wmtp_set_work_stealing(True)
+    yield
+    wm.wmtp_set_max_ctas(0)
+
+
+def _cfg(**kw):
+    base = dict(name="ext", batch=1, S0=300, Hq=16, Hkv=2, D=128, W=64, n_sink=4, gamma=5, seed=808)
+    base.update(kw)
+    return wi.DraftConfig(**base)
+
+
+def _per_seq(a):
+    """[gamma][B][...] -> contiguous [B][gamma][...] (the layout of the *_many / extend calls)."""
+    return np.ascontiguousarray(np.swapaxes(a, 0, 1))
+
+
+# ------------------------------------------------------------------------------------------ store operations
+@pytest.mark.parametrize("n_sink,W,slack", [(4, 8, 3), (0, 5, 7), (2, 16, 16)])
+def test_ring_rewind_then_append_bit_exact(n_sink, W, slack):
+    B, Hkv, D, cap = 2, 2, 128, W + slack
+    n = 4 * (n_sink + cap)
+    k = wi.normal_bf16(5, (1, n_sink, W), (n, B, Hkv, D))
+    v = wi.normal_bf16(5, (2, n_sink, W), (n, B, Hkv, D))
+    kd, vd = to_dev_bf16(k), to_dev_bf16(v)
+    ring = wm.Ring(B, Hkv, D, n_sink, W, cap=cap)
+    wm.wmtp_ring_reset(ring)
+    sims = [R.RingSim(n_sink, cap, Hkv, D) for _ in range(B)]
+    rng = np.random.RandomState(n_sink + W)
+    i = 0
+    while i < n - (slack + 2):
+        burst = int(rng.randint(1, slack + 2))
+        for _ in range(burst):
+            wm.wmtp_ring_append(ring, kd[i], vd[i])
+            for b in range(B):
+                sims[b].append(k[i, b], v[i, b])
+            i += 1
+        drops = np.array([int(rng.randint(0, min(burst, slack) + 1)) for _ in range(B)], dtype=np.int32)
+        wm.wmtp_ring_rewind(ring, torch.from_numpy(drops).cuda())
+        for b in range(B):
+            sims[b].rewind(int(drops[b]))
+            check_ring_against_sim(ring, b, sims[b], f"after rewind at {i}")
+        # the sequences now differ in length: re-align them so that one append call serves both
+        catch_up = int(drops.max())
+        for b in range(B):
+            for _ in range(catch_up - int(drops[b])):
+                sims[b].rewind(1)
+        wm.wmtp_ring_rewind(ring, torch.from_numpy((catch_up - drops).astype(np.int32)).cuda())
+        i -= catch_up
+        assert all(s.length == i for s in sims)
+
+
+def test_ring_rewind_beyond_slack_is_flagged_and_ignored():
+    ring = wm.Ring(1, 2, 128, 4, 8, cap=10)
+    ws = wm.Workspace(1, 16, 2, 128)
+    wm.wmtp_ring_reset(ring)
+    k = to_dev_bf16(wi.normal_bf16(1, 1, (20, 1, 2, 128)))
+    for i in range(20):
+        wm.wmtp_ring_append(ring, k[i], k[i])
+    before = ring.slot_pos.clone()
+    wm.wmtp_ring_rewind(ring, torch.tensor([3], dtype=torch.int32, device="cuda"), ws)      # slack is 2
+    with pytest.raises(wm.WmtpError) as ei:
+        wm.wmtp_device_status(ws)
+    assert ei.value.status == 7 and int(ring.len[0]) == 20 and torch.equal(ring.slot_pos, before)
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_append_many_equals_sequential_appends(paged):
+    cfg = _cfg(batch=3, S0=0, S0_range=(50, 400), paged=paged, gamma=6, cap_slack=6)
+    wl = wi.make_workload(cfg)
+    a, b_ = DeviceWorkload(wl), DeviceWorkload(wl)
+    for dw in (a, b_):
+        wm.wmtp_ring_init_from_kv(dw.ring, dw.kv)
+    for i in range(cfg.gamma):
+        wm.wmtp_ring_append(a.ring, a.k_new[i], a.v_new[i])
+        wm.wmtp_kv_append(a.kv, a.k_new[i], a.v_new[i], a.ws)
+    km, vm = to_dev_bf16(_per_seq(wl.k_new)), to_dev_bf16(_per_seq(wl.v_new))
+    wm.wmtp_ring_append_many(b_.ring, km, vm)
+    wm.wmtp_kv_append_many(b_.kv, km, vm, b_.ws)
+    wm.wmtp_device_status(a.ws); wm.wmtp_device_status(b_.ws)
+    for x, y in ((a.ring.k, b_.ring.k), (a.ring.v, b_.ring.v), (a.K, b_.K), (a.V, b_.V)):
+        assert (bits(x) == bits(y)).all()
+    assert torch.equal(a.ring.slot_pos, b_.ring.slot_pos) and torch.equal(a.ring.len, b_.ring.len) and torch.equal(a.lens, b_.lens)
+
+
+# ------------------------------------------------------------------------------------------ draft-extend attention
+def _extend_and_check(cfg, max_ctas=0, seqs=None):
+    wl = wi.make_workload(cfg)
+    dw = DeviceWorkload(wl)
+    wm.wmtp_set_max_ctas(max_ctas)
+    qlen = cfg.gamma
+    ws = wm.Workspace(cfg.batch * qlen, cfg.Hq, cfg.Hkv, cfg.D)
+    wm.wmtp_ring_init_from_kv(dw.ring, dw.kv)
+    km, vm, qm = to_dev_bf16(_per_seq(wl.k_new)), to_dev_bf16(_per_seq(wl.v_new)), to_dev_bf16(_per_seq(wl.q))
+    wm.wmtp_ring_append_many(dw.ring, km, vm)
+    wm.wmtp_kv_append_many(dw.kv, km, vm, ws)
+    out_w, out_f = torch.full_like(qm, float("nan")), torch.full_like(qm, float("nan"))
+    lse_w = torch.full(qm.shape[:-1], float("nan"), dtype=torch.float32, device="cuda")
+    lse_f = torch.full_like(lse_w, float("nan"))
+    wm.wmtp_draft_extend_windowed(qm, dw.ring, out_w, ws, lse=lse_w)
+    wm.wmtp_draft_extend_full(qm, dw.kv, out_f, ws, lse=lse_f)
+    wm.wmtp_device_status(ws)
+    for b in (range(cfg.batch) if seqs is None else seqs):
+        orc = oracle_for(wl, b, with_ring=False)
+        for i in range(qlen):
+            r = orc.step(wl.q[i, b], wl.k_new[i, b], wl.v_new[i, b])
+            tag = f"{cfg.name} ctas={max_ctas} seq={b} token={i}"
+            compare(out_w[b, i], lse_w[b, i], *r["win"], what=tag + " extend windowed")
+            compare(out_f[b, i], lse_f[b, i], *r["full"], what=tag + " extend full")
+
+
+@pytest.mark.parametrize("D", [128, 256])
+@pytest.mark.parametrize("S0", [0, 2, 60, 66, 70, 300, 2000])
+@pytest.mark.parametrize("max_ctas", [1, 0])
+def test_extend_matches_sequential_steps(D, S0, max_ctas):
+    # n_sink + W = 68 and five new tokens: the queries straddle sink-filling, window-filling and sliding states
+    _extend_and_check(_cfg(S0=S0, D=D, cap_slack=4, seed=900 + S0), max_ctas=max_ctas)
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_extend_batched_ragged(paged):
+    _extend_and_check(_cfg(batch=4, S0=0, S0_range=(10, 3000), paged=paged, gamma=7, cap_slack=8, W=128, seed=31))
+
+
+def test_extend_at_long_context():
+    _extend_and_check(wi.scaled(wi.CONFIGS[1], gamma=7, cap_slack=6, name="ext_s128k"))
+
+
+def test_extend_needs_slack_slots():
+    cfg = _cfg(S0=200, gamma=3, cap_slack=1)             # 3 tokens need cap >= W + 2
+    wl = wi.make_workload(cfg)
+    dw = DeviceWorkload(wl)
+    ws = wm.Workspace(3, cfg.Hq, cfg.Hkv, cfg.D)
+    qm = to_dev_bf16(_per_seq(wl.q))
+    with pytest.raises(wm.WmtpError) as ei:
+        wm.wmtp_draft_extend_windowed(qm, dw.ring, torch.empty_like(qm), ws)
+    assert ei.value.status == 3
+
+
+def test_speculative_cycle_draft_rewind_extend():
+    """gamma speculative draft steps, the target accepts `a` of them plus its own bonus token, the draft rolls back
+    and re-processes the accepted tokens: the ring ends up exactly as if only those tokens had ever been appended."""
+    cfg = _cfg(S0=500, D=256, W=128, gamma=6, cap_slack=7, seed=77)
+    wl = wi.make_workload(cfg)
+    dw = DeviceWorkload(wl)
+    dw.run_loops(full=False)                              # 6 speculative tokens in the ring
+    accepted = 2
+    wm.wmtp_ring_rewind(dw.ring, torch.tensor([cfg.gamma - accepted], dtype=torch.int32, device="cuda"), dw.ws)
+    # the target's verified tokens: the two accepted ones plus a bonus token with its own K/V
+    bonus_k = wi.normal_bf16(cfg.seed, 91, (1, 1, cfg.Hkv, cfg.D))
+    bonus_v = wi.normal_bf16(cfg.seed, 92, (1, 1, cfg.Hkv, cfg.D))
+    bonus_q = wi.normal_bf16(cfg.seed, 93, (1, 1, cfg.Hq, cfg.D))
+    wm.wmtp_ring_append_many(dw.ring, to_dev_bf16(bonus_k), to_dev_bf16(bonus_v))
+    qd = to_dev_bf16(bonus_q)
+    out = torch.empty_like(qd)
+    lse = torch.empty(qd.shape[:-1], dtype=torch.float32, device="cuda")
+    wm.wmtp_draft_extend_windowed(qd, dw.ring, out, dw.ws, lse=lse)
+    wm.wmtp_device_status(dw.ws)
+    orc = oracle_for(wl, 0)
+    for i in range(accepted):
+        orc.step(wl.q[i, 0], wl.k_new[i, 0], wl.v_new[i, 0], full=False)
+    r = orc.step(bonus_q[0, 0], bonus_k[0, 0], bonus_v[0, 0], full=False)
+    compare(out[0, 0], lse[0, 0], *r["win"], what="bonus token after rollback")
+    assert int(dw.ring.len[0]) == orc.S
+    # every position of the kept set sits in the slot the oracle's ring has it in, with the same bits; no slot
+    # claims a position at or beyond the new length
+    pos = dw.ring.slot_pos[0].cpu().numpy()
+    keep = set(R.keep_set(orc.S, cfg.n_sink, cfg.W))
+    Kb = bits(dw.ring.k[0])
+    seen = 0
+    for s, p in enumerate(orc.ring.slot_pos):
+        if int(p) in keep:
+            assert pos[s] == p and (Kb[:, s] == orc.ring.K[:, s]).all()
+            seen += 1
+    assert seen == len(keep) and (pos < orc.S).all()
