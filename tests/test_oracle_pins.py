@@ -95,6 +95,34 @@ def test_ring_sim_holds_sink_and_last_W(n_sink, W, slack):
                 assert not ring.written[s]
 
 
+@pytest.mark.parametrize("n_sink,W,d", [(4, 8, 3), (0, 5, 7), (2, 3, 1), (3, 6, 6)])
+def test_ring_sim_rollback_within_slack_keeps_the_window(n_sink, W, d):
+    """With d slack slots (Section 4 "Memory", Section 6 tree speculation: n_sink + W + d) up to d speculative tokens
+    can be written and discarded: afterwards the ring still holds every position of sink + last W, with the rows the
+    positions were first given, and appending again behaves as if the discarded tokens had never been written."""
+    cap, Hkv, D = W + d, 1, 2
+    rng = np.random.RandomState(n_sink * 100 + W)
+    ring, clean = R.RingSim(n_sink, cap, Hkv, D), R.RingSim(n_sink, cap, Hkv, D)
+    row = lambda p, gen: np.full((Hkv, D), (p * 7 + gen * 3 + 1) % 65521, dtype=np.uint16)
+    S = 0
+    for it in range(60):
+        n_acc, n_rej = int(rng.randint(0, 4)), int(rng.randint(0, d + 1))
+        for _ in range(n_acc):                                 # tokens that stay: both rings get them
+            ring.append(row(S, 0), row(S, 0)); clean.append(row(S, 0), row(S, 0)); S += 1
+        for j in range(n_rej):                                 # speculative tokens: only the ring with rollback sees them
+            ring.append(row(S + j, it + 1), row(S + j, it + 1))
+        ring.rewind(n_rej)
+        assert ring.length == clean.length == S
+        held = {int(p): s for s, p in enumerate(ring.slot_pos) if p >= 0}
+        assert all(p < S for p in held)                        # no slot claims a discarded position
+        for p in R.keep_set(S, n_sink, W):                     # brute force over what the draft reads
+            s = held[p]
+            assert s == (p if p < n_sink else n_sink + (p - n_sink) % cap)
+            assert ring.written[s] and (ring.K[:, s] == row(p, 0)).all() and (ring.V[:, s] == row(p, 0)).all()
+        # the next append lands where it would have without the speculation
+        assert ring.append(row(S, 0), row(S, 0)) == clean.append(row(S, 0), row(S, 0)); S += 1
+
+
 # ---------------------------------------------------------------- softmax attention, closed forms
 def test_uniform_keys_give_mean_of_values():
     Hq, Hkv, D, n = 8, 2, 16, 37
