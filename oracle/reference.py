@@ -16,6 +16,11 @@ What is here, and the passage each part restates:
 * ``DraftOracle``   -- gamma sequential draft steps: append the step's K/V, then attend,
                        in the windowed and in the full-context form (Section 3, Eq. 1:
                        gamma draft forwards per decode step).
+* ``e4m3_decode`` / ``e4m3_encode`` / ``quantize_rows`` and the uint8 branch of ``attention``
+                    -- the fp8-KV variant (Section 6, "Robustness to KV-cache quantization":
+                       the KV dtype only sets the bytes per entry): e4m3 codes with one fp32
+                       scale per KV head, value = code value * scale; new rows are quantised
+                       on append with round-to-nearest-even and saturation at 448.
 
 Readings of points the paper leaves open are listed in the repository's design notes;
 the ones that matter here: the window includes the token appended in the same step; sink
@@ -26,7 +31,9 @@ scale defaults to 1/sqrt(D).
 Pins (tests/test_oracle_*.py): closed forms of softmax attention, brute force against a
 pure-Python twin on tiny inputs, torch's scaled_dot_product_attention in fp64, the
 windowed == full identity for S <= n_sink + W, the mass identity, hand-written key sets
-under tests/golden/.  No function here is "parity unpinned".
+under tests/golden/; for fp8: hand-worked codes of the format, torch's float8_e4m3fn cast,
+brute-force nearest-code search, equality with the bf16 read-out on exactly representable
+values.  No function here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -61,6 +68,11 @@ def lib():
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
             ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_double,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int]
+        L.wmtp_oracle_attention_f8.restype = ctypes.c_int
+        L.wmtp_oracle_attention_f8.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
+            ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_double,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int]
         L.wmtp_oracle_threads.restype = ctypes.c_int
         _lib = L
     return _lib
@@ -70,21 +82,24 @@ def threads() -> int:
     return int(lib().wmtp_oracle_threads())
 
 
-def attention(q, K, V, keys=None, sm_scale=None, heads=None):
+def attention(q, K, V, keys=None, sm_scale=None, heads=None, k_scale=None, v_scale=None):
     """Softmax attention of one decode query per head over a key set, in fp64.
 
-    q: uint16 [Hq][D] (bf16 bits); K, V: uint16 [Hkv][rows][D] (the two inner dimensions
-    contiguous; heads may be strided).  ``keys`` selects rows (default: all rows).
-    Returns (out float64 [Hq][D], lse float64 [Hq]).  ``heads=(lo, hi)`` computes only
-    that range of query heads (other rows of the result are NaN).
+    q: uint16 [Hq][D] (bf16 bits); K, V: [Hkv][rows][D] (the two inner dimensions contiguous; heads
+    may be strided), either uint16 (bf16 bits) or uint8 (e4m3 codes; the value of an entry of KV head
+    g is the code's value times k_scale[g] / v_scale[g], fp32 [Hkv]).  ``keys`` selects rows
+    (default: all rows).  Returns (out float64 [Hq][D], lse float64 [Hq]).  ``heads=(lo, hi)``
+    computes only that range of query heads (other rows of the result are NaN).
     """
     q = np.ascontiguousarray(q, dtype=np.uint16)
     Hq, D = q.shape
     Hkv, rows, D2 = K.shape
-    assert D2 == D and V.shape == K.shape and K.dtype == np.uint16 and V.dtype == np.uint16
+    f8 = K.dtype == np.uint8
+    esz = 1 if f8 else 2
+    assert D2 == D and V.shape == K.shape and K.dtype in (np.uint16, np.uint8) and V.dtype == K.dtype
     if rows > 0:
-        assert K.strides[2] == 2 and K.strides[1] == 2 * D and V.strides == K.strides
-    head_stride = K.strides[0] // 2 if (Hkv > 1 and rows > 0) else rows * D
+        assert K.strides[2] == esz and K.strides[1] == esz * D and V.strides == K.strides
+    head_stride = K.strides[0] // esz if (Hkv > 1 and rows > 0) else rows * D
     if keys is None:
         n, kptr, kref = rows, None, None
     else:
@@ -97,11 +112,60 @@ def attention(q, K, V, keys=None, sm_scale=None, heads=None):
     out = np.full((Hq, D), np.nan, dtype=np.float64)
     lse = np.full((Hq,), np.nan, dtype=np.float64)
     lo, hi = (0, Hq) if heads is None else heads
-    rc = lib().wmtp_oracle_attention(q.ctypes.data, K.ctypes.data, V.ctypes.data, head_stride, kptr, n,
-                                     Hq, Hkv, D, float(sm_scale), out.ctypes.data, lse.ctypes.data, lo, hi)
+    if f8:
+        ks = np.ascontiguousarray(k_scale, dtype=np.float32)
+        vs = np.ascontiguousarray(v_scale, dtype=np.float32)
+        assert ks.shape == (Hkv,) and vs.shape == (Hkv,)
+        rc = lib().wmtp_oracle_attention_f8(q.ctypes.data, K.ctypes.data, V.ctypes.data, head_stride, kptr, n,
+                                            Hq, Hkv, D, float(sm_scale), ks.ctypes.data, vs.ctypes.data,
+                                            out.ctypes.data, lse.ctypes.data, lo, hi)
+    else:
+        assert k_scale is None and v_scale is None
+        rc = lib().wmtp_oracle_attention(q.ctypes.data, K.ctypes.data, V.ctypes.data, head_stride, kptr, n,
+                                         Hq, Hkv, D, float(sm_scale), out.ctypes.data, lse.ctypes.data, lo, hi)
     if rc != 0:
         raise RuntimeError("wmtp_oracle_attention failed")
     return out, lse
+
+
+# ---- fp8 (e4m3) KV entries (Section 6, "Robustness to KV-cache quantization") ----------------------
+def e4m3_decode(codes):
+    """Value of e4m3 codes as float64: 1 sign, 4 exponent (bias 7), 3 mantissa bits; exponent 0 is
+    subnormal; 0x7f / 0xff are NaN; no infinities; largest finite value 448."""
+    b = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    s, e, m = b >> 7, (b >> 3) & 15, b & 7
+    mag = np.where(e == 0, (m / 8.0) * 2.0 ** -6, (1.0 + m / 8.0) * np.exp2((e - 7).astype(np.float64)))
+    mag = np.where((e == 15) & (m == 7), np.nan, mag)
+    return np.where(s == 1, -mag, mag)
+
+
+def e4m3_encode(x):
+    """Nearest e4m3 code of fp32 values: round to nearest, ties to the even mantissa, magnitudes that
+    would round beyond 448 saturate to 448 (no infinities in the format), NaN stays NaN."""
+    x = np.asarray(x, dtype=np.float32)
+    a = np.abs(x.astype(np.float64))
+    sign = np.signbit(x).astype(np.int64) << 7
+    with np.errstate(invalid="ignore", divide="ignore"):
+        e = np.floor(np.log2(np.where(a > 0, a, 1.0))).astype(np.int64)     # exact: a is an fp32 value
+        e = np.clip(e, -6, 8)                                                  # below 2^-6 the spacing stays 2^-9
+        steps = np.rint(a / np.exp2((e - 3).astype(np.float64))).astype(np.int64)   # multiples of the spacing, ties to even
+    # steps in [0, 16]: 16 means the next binade (mantissa 0 there); subnormals (e = -6, steps < 8) have exponent field 0
+    code = np.where(steps < 8, steps, ((e + 7) << 3) + (steps - 8))            # carries propagate into the exponent field
+    code = np.where((a >= 448.0) | (code > 0x7e), 0x7e, code)
+    code = np.where(np.isnan(a), 0x7f, code)
+    return (code | sign).astype(np.uint8)
+
+
+def bf16_bits_to_f32(bits):
+    return (np.asarray(bits, dtype=np.uint16).astype(np.uint32) << 16).view(np.float32)
+
+
+def quantize_rows(rows_bf16, scale):
+    """Store-side quantisation of new K or V rows [Hkv][D] (bf16 bits): code = e4m3(x / scale[g]), the
+    division in fp32 (so that value ~ code * scale[g], the dequantisation the attention applies)."""
+    x = bf16_bits_to_f32(rows_bf16)
+    sc = np.asarray(scale, dtype=np.float32).reshape(-1, 1)
+    return e4m3_encode((x / sc).astype(np.float32))
 
 
 def keep_set(S: int, n_sink: int, W: int) -> list:
@@ -148,11 +212,11 @@ class WindowStore:
 class RingSim:
     """Slot-level ring: n_sink fixed slots, then `cap` window slots written by a wrapping cursor."""
 
-    def __init__(self, n_sink: int, cap: int, Hkv: int, D: int):
+    def __init__(self, n_sink: int, cap: int, Hkv: int, D: int, dtype=np.uint16):
         self.n_sink, self.cap = n_sink, cap
         self.slot_pos = np.full(n_sink + cap, -1, dtype=np.int32)
-        self.K = np.zeros((Hkv, n_sink + cap, D), dtype=np.uint16)
-        self.V = np.zeros((Hkv, n_sink + cap, D), dtype=np.uint16)
+        self.K = np.zeros((Hkv, n_sink + cap, D), dtype=dtype)
+        self.V = np.zeros((Hkv, n_sink + cap, D), dtype=dtype)
         self.written = np.zeros(n_sink + cap, dtype=bool)
         self.cursor = n_sink
         self.length = 0
@@ -192,18 +256,24 @@ class DraftOracle:
     """One sequence's draft state: full KV, list store and ring simulation, stepped together."""
 
     def __init__(self, K0, V0, Hq: int, n_sink: int, W: int, cap: int | None = None,
-                 sm_scale=None, reserve: int = 16, with_ring: bool = True):
+                 sm_scale=None, reserve: int = 16, with_ring: bool = True, k_scale=None, v_scale=None):
+        """K0, V0: [Hkv][S0][D] bf16 bits (uint16), or e4m3 codes (uint8) with per-KV-head scales: the
+        stores then hold codes, and the K/V rows of a step (always bf16) are quantised on append."""
         Hkv, S0, D = K0.shape
         self.Hq, self.Hkv, self.D = Hq, Hkv, D
         self.n_sink, self.W = n_sink, W
         self.sm_scale = sm_scale
-        self.Kfull = np.zeros((Hkv, S0 + reserve, D), dtype=np.uint16)
-        self.Vfull = np.zeros((Hkv, S0 + reserve, D), dtype=np.uint16)
+        self.f8 = K0.dtype == np.uint8
+        assert self.f8 == (k_scale is not None) == (v_scale is not None) and V0.dtype == K0.dtype
+        self.k_scale = None if k_scale is None else np.asarray(k_scale, dtype=np.float32)
+        self.v_scale = None if v_scale is None else np.asarray(v_scale, dtype=np.float32)
+        self.Kfull = np.zeros((Hkv, S0 + reserve, D), dtype=K0.dtype)
+        self.Vfull = np.zeros((Hkv, S0 + reserve, D), dtype=K0.dtype)
         self.Kfull[:, :S0] = K0
         self.Vfull[:, :S0] = V0
         self.S = S0
         self.store = WindowStore(n_sink, W)
-        self.ring = RingSim(n_sink, W if cap is None else cap, Hkv, D) if with_ring else None
+        self.ring = RingSim(n_sink, W if cap is None else cap, Hkv, D, dtype=K0.dtype) if with_ring else None
         for p in range(S0):
             k, v = self.Kfull[:, p, :], self.Vfull[:, p, :]
             self.store.append(k, v)
@@ -212,6 +282,8 @@ class DraftOracle:
 
     def append(self, k_row, v_row):
         assert self.S < self.Kfull.shape[1]
+        if self.f8:
+            k_row, v_row = quantize_rows(k_row, self.k_scale), quantize_rows(v_row, self.v_scale)
         self.Kfull[:, self.S, :] = k_row
         self.Vfull[:, self.S, :] = v_row
         k, v = self.Kfull[:, self.S, :], self.Vfull[:, self.S, :]
@@ -222,10 +294,11 @@ class DraftOracle:
 
     def attend_windowed(self, q, heads=None):
         Kw, Vw = self.store.stacked()
-        return attention(q, Kw, Vw, sm_scale=self.sm_scale, heads=heads)
+        return attention(q, Kw, Vw, sm_scale=self.sm_scale, heads=heads, k_scale=self.k_scale, v_scale=self.v_scale)
 
     def attend_full(self, q, heads=None):
-        return attention(q, self.Kfull[:, : self.S], self.Vfull[:, : self.S], sm_scale=self.sm_scale, heads=heads)
+        return attention(q, self.Kfull[:, : self.S], self.Vfull[:, : self.S], sm_scale=self.sm_scale, heads=heads,
+                         k_scale=self.k_scale, v_scale=self.v_scale)
 
     def step(self, q, k_row, v_row, full: bool = True, windowed: bool = True):
         """Append this step's K/V, then attend with q.  Returns {'win': (out, lse), 'full': (out, lse)}."""

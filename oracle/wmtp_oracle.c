@@ -90,3 +90,70 @@ int wmtp_oracle_attention(const uint16_t* q, const uint16_t* K, const uint16_t* 
     }
     return fail ? -1 : 0;
 }
+
+/*
+ * fp8 KV variant (Section 6, "Robustness to KV-cache quantization": the KV dtype only sets the bytes
+ * per entry; the key set and the attention are unchanged).  K and V hold e4m3 codes -- 1 sign, 4
+ * exponent (bias 7), 3 mantissa bits; exponent 0 is subnormal (m/8 * 2^-6); exponent 15 with
+ * mantissa 7 is NaN, there are no infinities, the largest finite value is 448 -- and the value of
+ * an entry of KV head g is code_value * k_scale[g] (resp. v_scale[g]).
+ */
+static double e4m3_to_f64(uint8_t b) {
+    const int s = b >> 7, e = (b >> 3) & 15, m = b & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m / 8.0, -6);
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return s ? -v : v;
+}
+
+/* Same contract as wmtp_oracle_attention, with K, V : [Hkv][rows][D] e4m3 codes (head_stride in
+ * elements) and per-KV-head dequantisation scales k_scale, v_scale : [Hkv] fp32. */
+int wmtp_oracle_attention_f8(const uint16_t* q, const uint8_t* K, const uint8_t* V,
+                             int64_t head_stride, const int64_t* keys, int64_t n,
+                             int Hq, int Hkv, int D, double sm_scale,
+                             const float* k_scale, const float* v_scale,
+                             double* out, double* lse, int head_lo, int head_hi) {
+    if (!q || !out || !lse || !k_scale || !v_scale || Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0 || n < 0) return -1;
+    if (n > 0 && (!K || !V)) return -1;
+    if (head_lo < 0) head_lo = 0;
+    if (head_hi > Hq) head_hi = Hq;
+    const int G = Hq / Hkv;
+    int fail = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int h = head_lo; h < head_hi; ++h) {
+        const int g = h / G;
+        const uint8_t* Kg = K + (int64_t)g * head_stride;
+        const uint8_t* Vg = V + (int64_t)g * head_stride;
+        const double ks = (double)k_scale[g], vs = (double)v_scale[g];
+        double* o = out + (int64_t)h * D;
+        for (int d = 0; d < D; ++d) o[d] = 0.0;
+        if (n == 0) { lse[h] = -INFINITY; continue; }
+        double* z = (double*)malloc((size_t)n * sizeof(double));
+        double* qd = (double*)malloc((size_t)D * sizeof(double));
+        if (!z || !qd) { free(z); free(qd); fail = 1; continue; }
+        for (int d = 0; d < D; ++d) qd[d] = bf16_to_f64(q[(int64_t)h * D + d]);
+        double m = -INFINITY;
+        for (int64_t j = 0; j < n; ++j) {
+            const int64_t row = keys ? keys[j] : j;
+            const uint8_t* k = Kg + row * D;
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d) acc += qd[d] * (e4m3_to_f64(k[d]) * ks);
+            z[j] = sm_scale * acc;
+            if (z[j] > m) m = z[j];
+        }
+        double Z = 0.0;
+        for (int64_t j = 0; j < n; ++j) {
+            const int64_t row = keys ? keys[j] : j;
+            const uint8_t* v = Vg + row * D;
+            const double p = exp(z[j] - m);
+            Z += p;
+            for (int d = 0; d < D; ++d) o[d] += p * (e4m3_to_f64(v[d]) * vs);
+        }
+        for (int d = 0; d < D; ++d) o[d] /= Z;
+        lse[h] = m + log(Z);
+        free(z);
+        free(qd);
+    }
+    return fail ? -1 : 0;
+}

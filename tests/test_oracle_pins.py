@@ -327,3 +327,110 @@ def test_tail_out_frac_matches_far_key_contribution():
     # dropping nothing changes nothing
     np.testing.assert_allclose(R.tail_out_frac(of, of, lf, lf), 0.0, atol=1e-15)
     np.testing.assert_allclose(R.win_perturb(of, of), 0.0, atol=1e-15)
+
+
+# ---------------------------------------------------------------- fp8 (e4m3) KV entries
+def test_e4m3_decode_matches_the_format_definition_and_torch():
+    import torch
+    codes = np.arange(256, dtype=np.uint8)
+    val = R.e4m3_decode(codes)
+    # hand-worked codes: zero, smallest subnormal, largest subnormal, smallest normal, one, 1.5, largest finite, NaN
+    hand = {0x00: 0.0, 0x01: 2.0 ** -9, 0x07: 7 * 2.0 ** -9, 0x08: 2.0 ** -6, 0x38: 1.0, 0x3C: 1.5, 0x40: 2.0,
+            0x7E: 448.0, 0x77: 240.0, 0xB8: -1.0, 0xFE: -448.0, 0x81: -(2.0 ** -9)}
+    for c, v in hand.items():
+        assert val[c] == v, hex(c)
+    assert np.isnan(val[0x7F]) and np.isnan(val[0xFF]) and np.isfinite(np.delete(val, [0x7F, 0xFF])).all()
+    assert np.signbit(val[0x80]) and val[0x80] == 0.0
+    pos = val[:0x7F]
+    assert (np.diff(pos) > 0).all()                                        # codes are ordered like their values
+    assert (np.diff(pos)[:8] == 2.0 ** -9).all()                           # subnormal spacing continues into the first binade
+    assert (val[0x80:0xFF] == -pos).all()
+    lib_val = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    assert np.array_equal(np.isnan(val), np.isnan(lib_val)) and (val[~np.isnan(val)] == lib_val[~np.isnan(val)]).all()
+
+
+def test_e4m3_encode_is_nearest_ties_to_even_and_saturates():
+    import torch
+    table = R.e4m3_decode(np.arange(0x7F, dtype=np.uint8))                 # the 127 non-negative finite values, ascending
+    rs = np.random.RandomState(11)
+    x = (rs.standard_normal(60000) * np.exp(rs.uniform(-14, 7, 60000))).astype(np.float32)
+    mid = ((table[:-1] + table[1:]) / 2).astype(np.float32)                # exact ties (representable in fp32)
+    x = np.concatenate([x, mid, -mid, table.astype(np.float32), np.float32([0.0, -0.0, 448, 449, 463.9, 464, 480, 1e9, -1e9,
+                                                                              2.0 ** -10, 3 * 2.0 ** -10, 2.0 ** -11])])
+    got = R.e4m3_encode(x)
+    # brute force: nearest table entry, ties to the even code, beyond the table the last entry
+    a = np.abs(x.astype(np.float64))
+    dist = np.abs(a[:, None] - table[None, :])
+    best = dist.min(axis=1)
+    cand = dist == best[:, None]
+    first = cand.argmax(axis=1)
+    last = cand.shape[1] - 1 - cand[:, ::-1].argmax(axis=1)
+    want = np.where(first == last, first, np.where(first % 2 == 0, first, last))
+    want = want | (np.signbit(x).astype(np.int64) << 7)
+    assert (got == want).all()
+    assert (got[np.abs(x) >= 448] & 0x7F == 0x7E).all()                    # saturation, never NaN
+    assert R.e4m3_encode(np.float32([np.nan]))[0] & 0x7F == 0x7F
+    fin = np.array([c for c in range(256) if c & 0x7F != 0x7F], dtype=np.uint8)
+    assert (R.e4m3_encode(R.e4m3_decode(fin).astype(np.float32)) == fin).all()      # every code is a fixed point
+    m = np.abs(x) <= 448
+    lib_codes = torch.from_numpy(x[m]).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert (got[m] == lib_codes).all()
+
+
+def test_quantize_rows_divides_in_fp32():
+    rs = np.random.RandomState(3)
+    rows = wi.normal_bf16(9, 1, (3, 64))
+    scale = np.float32([0.013, 0.7, 3.1])
+    got = R.quantize_rows(rows, scale)
+    x = (rows.astype(np.uint32) << 16).view(np.float32)
+    for g in range(3):
+        for d in range(64):
+            t = np.float32(x[g, d]) / np.float32(scale[g])
+            assert got[g, d] == R.e4m3_encode(np.float32([t]))[0]
+    # dequantised value within half a code spacing (relative 2^-4) of the input, for inputs inside the range
+    back = R.e4m3_decode(got) * scale[:, None].astype(np.float64)
+    inside = np.abs(x) < 448 * scale[:, None]
+    rel = np.abs(back - x)[inside] / np.maximum(np.abs(x[inside]), 2.0 ** -6 * np.repeat(scale, 64).reshape(3, 64)[inside])
+    assert rel.max() <= 2.0 ** -4 + 1e-7
+
+
+def test_fp8_attention_equals_bf16_attention_on_exactly_representable_values():
+    """With power-of-two scales every dequantised entry is a bf16 value, so the fp8 read-out must equal the bf16
+    read-out of those values; a single key returns code value * v_scale exactly for any scale."""
+    rs = np.random.RandomState(5)
+    Hq, Hkv, D, n = 8, 2, 32, 50
+    q = wi.normal_bf16(21, 1, (Hq, D))
+    codes_k = rs.randint(0, 256, (Hkv, n, D)).astype(np.uint8)
+    codes_v = rs.randint(0, 256, (Hkv, n, D)).astype(np.uint8)
+    codes_k[(codes_k & 0x7F) == 0x7F] = 0x30
+    codes_v[(codes_v & 0x7F) == 0x7F] = 0x30
+    codes_k = (codes_k & 0x80) | np.minimum(codes_k & 0x7F, 0x47)             # keep the logits moderate
+    ks, vs = np.float32([2.0 ** -5, 2.0 ** -3]), np.float32([2.0 ** -7, 2.0 ** 1])
+    Kf = (R.e4m3_decode(codes_k) * ks[:, None, None]).astype(np.float32)
+    Vf = (R.e4m3_decode(codes_v) * vs[:, None, None]).astype(np.float32)
+    Kb, Vb = (Kf.view(np.uint32) >> 16).astype(np.uint16), (Vf.view(np.uint32) >> 16).astype(np.uint16)
+    assert ((Kb.astype(np.uint32) << 16).view(np.float32) == Kf).all()        # exactly representable
+    keys = np.array([3, 17, 4, 44, 45, 9])
+    o8, l8 = R.attention(q, codes_k, codes_v, keys=keys, k_scale=ks, v_scale=vs)
+    ob, lb = R.attention(q, Kb, Vb, keys=keys)
+    assert np.abs(o8 - ob).max() < 1e-12 and np.abs(l8 - lb).max() < 1e-12
+    vs2 = np.float32([0.0371, 1.9])
+    o1, _ = R.attention(q, codes_k, codes_v, keys=np.array([7]), k_scale=ks, v_scale=vs2)
+    for h in range(Hq):
+        assert (o1[h] == R.e4m3_decode(codes_v[h // 4, 7]) * np.float64(vs2[h // 4])).all()
+
+
+def test_fp8_draft_oracle_quantises_on_append():
+    cfg = wi.DraftConfig("f8pin", 1, 20, 8, 2, 32, 16, 4, 3, seed=77, kv_dtype="fp8", key_scale=(0.5, 2.0))
+    wl = wi.make_workload(cfg)
+    assert wl.K[0].dtype == np.uint8 and not (wl.K[0] & 0x7F == 0x7F).any()
+    orc = R.DraftOracle(wl.K[0], wl.V[0], cfg.Hq, cfg.n_sink, cfg.W, k_scale=wl.k_scale, v_scale=wl.v_scale)
+    r = orc.step(wl.q[0, 0], wl.k_new[0, 0], wl.v_new[0, 0])
+    assert (orc.Kfull[:, 20] == R.quantize_rows(wl.k_new[0, 0], wl.k_scale)).all()
+    assert (orc.ring.K[:, orc.ring.slot_pos.tolist().index(20)] == orc.Kfull[:, 20]).all()
+    # S = 21 > n_sink + W = 20: windowed drops exactly position 4
+    keep = R.keep_set(21, 4, 16)
+    assert keep == [0, 1, 2, 3] + list(range(5, 21))
+    ow, lw = R.attention(wl.q[0, 0], orc.Kfull[:, :21], orc.Vfull[:, :21], keys=np.array(keep), k_scale=wl.k_scale, v_scale=wl.v_scale)
+    assert np.abs(ow - r["win"][0]).max() < 1e-12 and np.abs(lw - r["win"][1]).max() < 1e-12
+    assert (r["full"][1] > r["win"][1]).all()

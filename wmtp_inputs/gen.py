@@ -82,3 +82,21 @@ def normal_bf16(seed: int, tensor_id, shape, scale: float = 1.0, mean: float = 0
 def rng(seed: int, tensor_id) -> np.random.Generator:
     """A generator for small integer/structural draws (sequence lengths, page permutations)."""
     return np.random.Generator(np.random.Philox(np.random.SeedSequence([int(seed), *_key(tensor_id)])))
+
+
+def e4m3_codes_trunc(bits: np.ndarray, unit: float) -> np.ndarray:
+    """Synthetic fp8 store contents from bf16 draws: the draw, in units of ``unit``, cut toward zero onto
+    the e4m3 code grid (3 mantissa bits, exponents 2^-6 .. 2^8, magnitudes capped at 448, anything below
+    2^-6 cut to a multiple of 2^-9).  Pure field extraction from the fp32 bit pattern; this defines what
+    the synthetic store contains and is not the store's quantiser."""
+    t = (bf16_bits_to_f32(bits) / np.float32(unit)).astype(np.float32)
+    u = t.view(np.uint32)
+    sign = ((u >> 31) & 1).astype(np.uint8) << 7
+    a = np.minimum(np.abs(t), np.float32(448.0))
+    ua = a.view(np.uint32)
+    expo = ((ua >> 23) & 0xFF).astype(np.int32) - 120          # e4m3 exponent field of a normal code
+    mant = ((ua >> 20) & 7).astype(np.int32)
+    normal = (expo << 3) | mant
+    sub = np.floor(a * np.float32(512.0)).astype(np.int32)      # below 2^-6: multiples of 2^-9
+    code = np.where(expo >= 1, normal, np.minimum(sub, 7))
+    return (code.astype(np.uint8) | sign).reshape(bits.shape)

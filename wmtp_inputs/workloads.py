@@ -1,6 +1,6 @@
 """The synthetic draft-attention workloads (shapes, lengths, layouts) and their tensors.
 
-Every workload is a batch of sequences with a bf16 KV cache for one draft layer
+Every workload is a batch of sequences with a bf16 (or fp8 e4m3) KV cache for one draft layer
 (Hkv KV heads of head_dim D, Hq = G*Hkv query heads), an attention sink of n_sink
 tokens, a window of W tokens and gamma sequential draft steps; each step brings one
 new (q, k, v) per sequence.  Tensors are generated in *logical* form
@@ -18,6 +18,8 @@ from . import gen
 
 T_K, T_V, T_Q, T_KNEW, T_VNEW, T_LENS, T_PAGES = 1, 2, 3, 4, 5, 6, 7
 BF16_NAN = np.uint16(0x7FC0)
+E4M3_NAN = np.uint8(0x7F)
+E4M3_RANGE_SIGMAS = 4.5          # an fp8 store maps +-4.5 standard deviations of its head onto +-448
 
 
 @dataclass(frozen=True)
@@ -37,6 +39,7 @@ class DraftConfig:
     page_size: int = 64
     key_scale: tuple | None = None   # (lo, hi): per-KV-head multiplier on K, log-spaced
     cap_slack: int = 0               # ring capacity = W + cap_slack window slots
+    kv_dtype: str = "bf16"           # "bf16", or "fp8": e4m3 codes with one fp32 scale per KV head for K and for V
 
     @property
     def G(self) -> int:
@@ -44,7 +47,7 @@ class DraftConfig:
 
     @property
     def kv_bytes_per_token(self) -> int:
-        return self.Hkv * self.D * 2 * 2
+        return self.Hkv * self.D * 2 * (1 if self.kv_dtype == "fp8" else 2)
 
 
 # The five workloads named by the benchmark description; index = position in that list.
@@ -84,6 +87,8 @@ class Workload:
     page_table: np.ndarray = None        # int32 [B][max_pages] (paged only)
     num_pages: int = 0
     max_pages: int = 0
+    k_scale: np.ndarray = None           # fp8 stores: float32 [Hkv], value = code * scale (None for bf16)
+    v_scale: np.ndarray = None
 
 
 def head_scales(cfg: DraftConfig) -> np.ndarray:
@@ -110,12 +115,24 @@ def make_workload(cfg: DraftConfig, poison_unused: bool = True, extra_cap: int =
     Rows of the device-layout KV that hold no token yet (positions >= the sequence's
     length) are filled with a bf16 NaN pattern when ``poison_unused`` is set, so a
     kernel that lets a stale row leak into its result fails loudly.
+
+    With ``kv_dtype == "fp8"`` the store holds e4m3 codes: the same N(0, head scale) draws, expressed in
+    units of ``k_scale[g] = 4.5 * head scale / 448`` (``v_scale = 4.5 / 448``) and cut to the code grid by
+    ``gen.e4m3_codes_trunc``; the per-step q / k_new / v_new stay bf16.
     """
     B, Hkv, Hq, D, gam = cfg.batch, cfg.Hkv, cfg.Hq, cfg.D, cfg.gamma
     lens = seq_lens(cfg)
     sc = head_scales(cfg)
     wl = Workload(cfg=cfg, seq_lens=lens)
-    fill = BF16_NAN if poison_unused else np.uint16(0)
+    f8 = cfg.kv_dtype == "fp8"
+    assert cfg.kv_dtype in ("bf16", "fp8")
+    dt = np.uint8 if f8 else np.uint16
+    if f8:
+        wl.k_scale = (E4M3_RANGE_SIGMAS * sc / 448.0).astype(np.float32)
+        wl.v_scale = np.full(Hkv, E4M3_RANGE_SIGMAS / 448.0, dtype=np.float32)
+        fill = E4M3_NAN if poison_unused else np.uint8(0)
+    else:
+        fill = BF16_NAN if poison_unused else np.uint16(0)
 
     if cfg.paged:
         ps = cfg.page_size
@@ -128,19 +145,19 @@ def make_workload(cfg: DraftConfig, poison_unused: bool = True, extra_cap: int =
         for b in range(B):
             wl.page_table[b, : need[b]] = perm[off: off + need[b]]
             off += int(need[b])
-        wl.K_dev = np.full((wl.num_pages, Hkv, ps, D), fill, dtype=np.uint16)
-        wl.V_dev = np.full((wl.num_pages, Hkv, ps, D), fill, dtype=np.uint16)
+        wl.K_dev = np.full((wl.num_pages, Hkv, ps, D), fill, dtype=dt)
+        wl.V_dev = np.full((wl.num_pages, Hkv, ps, D), fill, dtype=dt)
         wl.S_cap = wl.max_pages * ps
     else:
         wl.S_cap = int(lens.max()) + gam + extra_cap
-        wl.K_dev = np.empty((B, Hkv, wl.S_cap, D), dtype=np.uint16)
-        wl.V_dev = np.empty((B, Hkv, wl.S_cap, D), dtype=np.uint16)
+        wl.K_dev = np.empty((B, Hkv, wl.S_cap, D), dtype=dt)
+        wl.V_dev = np.empty((B, Hkv, wl.S_cap, D), dtype=dt)
 
     for b in range(B):
         S = int(lens[b])
         if cfg.paged:
-            Kb = np.empty((Hkv, S, D), dtype=np.uint16)
-            Vb = np.empty((Hkv, S, D), dtype=np.uint16)
+            Kb = np.empty((Hkv, S, D), dtype=dt)
+            Vb = np.empty((Hkv, S, D), dtype=dt)
         else:
             # logical tensors are views of the device-layout buffer (no second copy in host memory)
             Kb = wl.K_dev[b, :, :S, :]
@@ -148,8 +165,13 @@ def make_workload(cfg: DraftConfig, poison_unused: bool = True, extra_cap: int =
             wl.K_dev[b, :, S:, :] = fill
             wl.V_dev[b, :, S:, :] = fill
         for g in range(Hkv):
-            Kb[g] = gen.normal_bf16(cfg.seed, (T_K, b, g), (S, D), scale=float(sc[g]), threads=threads)
-            Vb[g] = gen.normal_bf16(cfg.seed, (T_V, b, g), (S, D), threads=threads)
+            kb = gen.normal_bf16(cfg.seed, (T_K, b, g), (S, D), scale=float(sc[g]), threads=threads)
+            vb = gen.normal_bf16(cfg.seed, (T_V, b, g), (S, D), threads=threads)
+            if f8:
+                kb = gen.e4m3_codes_trunc(kb, float(wl.k_scale[g]))
+                vb = gen.e4m3_codes_trunc(vb, float(wl.v_scale[g]))
+            Kb[g] = kb
+            Vb[g] = vb
         wl.K.append(Kb)
         wl.V.append(Vb)
         if cfg.paged:
