@@ -45,6 +45,21 @@ typedef enum {
 } wmtp_status;
 
 /*
+ * Entry type of a KV store (ring or full-context). WMTP_KV_BF16: bf16 values. WMTP_KV_FP8_E4M3: the fp8-KV variant
+ * (Section 6, "Robustness to KV-cache quantization": the KV dtype only sets the bytes per entry, the key set and the
+ * attention are unchanged): every entry is one e4m3 code (1 sign, 4 exponent, 3 mantissa bits; no infinities, largest
+ * finite value 448) and stands for code_value * k_scale[g] (resp. v_scale[g]) with g its KV head. Layouts, shapes and
+ * alignment rules are the same with 1-byte entries. q, k_new, v_new and out stay bf16: the append calls (and the
+ * appends fused into the draft loops) quantise a new row as code = e4m3(x / scale[g]) -- fp32 division, round to
+ * nearest even, magnitudes beyond 448 saturate -- and the attention kernels widen the codes exactly and apply the
+ * scales to the scores and to the read-out. NaN codes are not valid store contents.
+ */
+typedef enum { WMTP_KV_BF16 = 0, WMTP_KV_FP8_E4M3 = 1 } wmtp_kv_dtype;
+
+/* Bytes per entry of a store of that type (2 or 1); 0 for an unknown type. */
+size_t wmtp_kv_elem_bytes(int kv_dtype);
+
+/*
  * Ring-buffer draft KV store (Section 4 "Memory": the draft KV is kept in a compact
  * n_sink + W + d ring; Appendix A: slot = ring_base(r) + logical position under a modulus).
  * Per sequence r the store has n_sink fixed sink slots followed by `cap` window slots used
@@ -58,6 +73,9 @@ typedef struct wmtp_ring {
     int32_t* slot_pos;  /* device [batch][n_sink + cap]: logical position held by each slot, -1 = never written */
     int64_t* len;       /* device [batch]: logical sequence length S (tokens appended so far) */
     int32_t  batch, Hkv, D, n_sink, W, cap;
+    int32_t  kv_dtype;        /* wmtp_kv_dtype; 0 (bf16) keeps the fields below unused */
+    const float* k_scale;     /* device fp32 [Hkv], WMTP_KV_FP8_E4M3 only: positive, finite */
+    const float* v_scale;     /* device fp32 [Hkv] */
 } wmtp_ring;
 
 /*
@@ -73,12 +91,16 @@ typedef struct wmtp_kv {
     int64_t*       len;        /* device [batch] */
     int64_t        S_cap;      /* host-known capacity in tokens per sequence (contiguous: row count; paged: max_pages * page_size) */
     int32_t        batch, Hkv, D, page_size, max_pages, num_pages;
+    int32_t        kv_dtype;   /* wmtp_kv_dtype */
+    const float*   k_scale;    /* device fp32 [Hkv], WMTP_KV_FP8_E4M3 only */
+    const float*   v_scale;
 } wmtp_kv;
 
 const char* wmtp_status_string(wmtp_status s); /* static storage */
 const char* wmtp_last_error(void);             /* thread-local, valid until the thread's next failing call */
 
-/* Bytes of the ring's K (== V) tensor and of slot_pos, for the caller's allocation. Returns k_bytes. */
+/* Bytes of the ring's K (== V) tensor (bf16 entries; an fp8 ring needs half) and of slot_pos, for the caller's
+ * allocation. Returns k_bytes. */
 size_t wmtp_ring_bytes(int batch, int Hkv, int D, int n_sink, int cap, size_t* pos_bytes);
 
 /*
@@ -104,6 +126,7 @@ wmtp_status wmtp_ring_reset(const wmtp_ring* ring, void* stream);
  * [0, min(S, n_sink)) and [max(n_sink, S - cap), S) into their slots, sets slot_pos and len = S.
  * The result is bit-identical to S sequential wmtp_ring_append calls (Section 6, "Prefill
  * sparsification": only O(W + n_sink) of the context is needed by the windowed draft).
+ * Rows are copied as stored: ring and kv must have the same kv_dtype and, for fp8, equal scales.
  */
 wmtp_status wmtp_ring_init_from_kv(const wmtp_ring* ring, const wmtp_kv* kv, void* stream);
 

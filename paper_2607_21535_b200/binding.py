@@ -24,13 +24,17 @@ STATUS_NAMES = {
 class wmtp_ring(ctypes.Structure):
     _fields_ = [("k", c_void_p), ("v", c_void_p), ("slot_pos", c_void_p), ("len", c_void_p),
                 ("batch", c_int32), ("Hkv", c_int32), ("D", c_int32), ("n_sink", c_int32), ("W", c_int32),
-                ("cap", c_int32)]
+                ("cap", c_int32), ("kv_dtype", c_int32), ("k_scale", c_void_p), ("v_scale", c_void_p)]
 
 
 class wmtp_kv(ctypes.Structure):
     _fields_ = [("k", c_void_p), ("v", c_void_p), ("page_table", c_void_p), ("len", c_void_p),
                 ("S_cap", c_int64), ("batch", c_int32), ("Hkv", c_int32), ("D", c_int32), ("page_size", c_int32),
-                ("max_pages", c_int32), ("num_pages", c_int32)]
+                ("max_pages", c_int32), ("num_pages", c_int32), ("kv_dtype", c_int32), ("k_scale", c_void_p),
+                ("v_scale", c_void_p)]
+
+
+WMTP_KV_BF16, WMTP_KV_FP8_E4M3 = 0, 1
 
 
 class WmtpError(RuntimeError):
@@ -43,6 +47,7 @@ class WmtpError(RuntimeError):
 _SIGNATURES = {
     "wmtp_status_string": (c_char_p, [c_int]),
     "wmtp_last_error": (c_char_p, []),
+    "wmtp_kv_elem_bytes": (c_size_t, [c_int]),
     "wmtp_ring_bytes": (c_size_t, [c_int, c_int, c_int, c_int, c_int, POINTER(c_size_t)]),
     "wmtp_workspace_bytes": (c_size_t, [c_int, c_int, c_int, c_int]),
     "wmtp_workspace_init": (c_int, [c_void_p, c_size_t, c_void_p]),
@@ -126,29 +131,40 @@ def _stream(stream) -> int:
 # Device-memory holders (torch allocations + the C descriptor)
 # ------------------------------------------------------------------------------------------------
 class Ring:
-    """Device ring-buffer KV store for ``batch`` sequences: n_sink sink slots + ``cap`` window slots."""
+    """Device ring-buffer KV store for ``batch`` sequences: n_sink sink slots + ``cap`` window slots.
 
-    def __init__(self, batch, Hkv, D, n_sink, W, cap=None, device="cuda", guard: int = 0):
+    ``k_scale`` / ``v_scale`` (device fp32 [Hkv]) select an fp8 (e4m3) store: uint8 codes, value = code * scale."""
+
+    def __init__(self, batch, Hkv, D, n_sink, W, cap=None, device="cuda", guard: int = 0, k_scale=None, v_scale=None):
         cap = W if cap is None else cap
         self.batch, self.Hkv, self.D, self.n_sink, self.W, self.cap = batch, Hkv, D, n_sink, W, cap
         slots = n_sink + cap
-        self.k = torch.zeros((batch, Hkv, slots, D), dtype=torch.bfloat16, device=device)
-        self.v = torch.zeros((batch, Hkv, slots, D), dtype=torch.bfloat16, device=device)
+        assert (k_scale is None) == (v_scale is None)
+        f8 = k_scale is not None
+        dt = torch.uint8 if f8 else torch.bfloat16
+        self.k_scale, self.v_scale = k_scale, v_scale
+        self.k = torch.zeros((batch, Hkv, slots, D), dtype=dt, device=device)
+        self.v = torch.zeros((batch, Hkv, slots, D), dtype=dt, device=device)
         self.slot_pos = torch.full((batch, slots), -1, dtype=torch.int32, device=device)
         self.len = torch.zeros((batch,), dtype=torch.int64, device=device)
         self.desc = wmtp_ring(self.k.data_ptr(), self.v.data_ptr(), self.slot_pos.data_ptr(), self.len.data_ptr(),
-                              batch, Hkv, D, n_sink, W, cap)
+                              batch, Hkv, D, n_sink, W, cap, WMTP_KV_FP8_E4M3 if f8 else WMTP_KV_BF16, _ptr(k_scale),
+                              _ptr(v_scale))
 
 
 class KV:
     """Full-context KV descriptor over caller-provided device tensors.
 
     Contiguous: k, v bf16 [batch][Hkv][S_cap][D]. Paged: k, v bf16 [num_pages][Hkv][page_size][D]
-    with ``page_table`` int32 [batch][max_pages].
+    with ``page_table`` int32 [batch][max_pages]. uint8 tensors are an fp8 (e4m3) store and need
+    ``k_scale`` / ``v_scale`` (device fp32 [Hkv]).
     """
 
-    def __init__(self, k, v, lens, page_table=None, S_cap=None):
+    def __init__(self, k, v, lens, page_table=None, S_cap=None, k_scale=None, v_scale=None):
         self.k, self.v, self.len, self.page_table = k, v, lens, page_table
+        f8 = k.dtype == torch.uint8
+        assert v.dtype == k.dtype and f8 == (k_scale is not None) == (v_scale is not None)
+        self.k_scale, self.v_scale = k_scale, v_scale
         if page_table is None:
             batch, Hkv, rows, D = k.shape
             self.S_cap = rows if S_cap is None else S_cap
@@ -159,7 +175,8 @@ class KV:
             self.S_cap = max_pages * page_size if S_cap is None else S_cap
         self.batch, self.Hkv, self.D = batch, Hkv, D
         self.desc = wmtp_kv(k.data_ptr(), v.data_ptr(), _ptr(page_table), lens.data_ptr(), self.S_cap, batch, Hkv, D,
-                            page_size, max_pages, num_pages)
+                            page_size, max_pages, num_pages, WMTP_KV_FP8_E4M3 if f8 else WMTP_KV_BF16, _ptr(k_scale),
+                            _ptr(v_scale))
 
 
 class Workspace:
@@ -184,6 +201,10 @@ def wmtp_status_string(status: int) -> str:
 
 def wmtp_last_error() -> str:
     return lib().wmtp_last_error().decode()
+
+
+def wmtp_kv_elem_bytes(kv_dtype: int) -> int:
+    return int(lib().wmtp_kv_elem_bytes(kv_dtype))
 
 
 def wmtp_ring_bytes(batch, Hkv, D, n_sink, cap):

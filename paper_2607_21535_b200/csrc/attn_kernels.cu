@@ -31,6 +31,7 @@
 #include <cuda_bf16.h>
 
 #include "attn_plan.cuh"
+#include "fp8_util.cuh"
 
 namespace wmtp {
 
@@ -56,14 +57,18 @@ constexpr int kStealMinTiles = 16;  // ranges shorter than this are streamed sta
 // contrib[kMaxContrib][4] = {seg, b, g, slot}, reg_k[kMaxContrib] (slot of the group's i-th contribution, producer -> group)
 constexpr int kGroupInts = 4 + 5 * kMaxContrib;
 
-template <int D>
+// D: head_dim; F8: the store holds e4m3 codes (one byte per entry) instead of bf16.
+template <int D, bool F8>
 struct Cfg {
-    static constexpr int kChunks = D / 64;                    // 128-byte column chunks per row
+    static constexpr int kElemBytes = F8 ? 1 : 2;
+    static constexpr int kChunks = D * kElemBytes / 128;      // 128-byte column chunks per row
     static constexpr int kChunkBytes = kTileKeys * 128;       // one TMA box: 64 rows x 128 B
     static constexpr int kTileBytes = kChunks * kChunkBytes;  // K (or V) tile
     static constexpr int kStageBytes = 2 * kTileBytes;
-    static constexpr int kGroups = (D == 256) ? 1 : 2;        // consumer groups
-    static constexpr int kStages = (D == 256) ? 3 : 5;
+    // consumer groups: a tile of fewer bytes brings the same softmax work, so the smaller tiles get two groups
+    static constexpr int kGroups = (kStageBytes >= 65536) ? 1 : 2;
+    static constexpr int kStages = (kStageBytes >= 65536) ? 3 : (kStageBytes >= 32768 ? 5 : 8);
+    static constexpr int kRowVecs = D * kElemBytes / 16;      // 16-byte vectors per stored row
     static constexpr int kConsumerWarps = kGroups * kGroupWarps;
     static constexpr int kThreads = (kConsumerWarps + 1) * 32;
     static constexpr int kKSteps = D / 16;
@@ -175,6 +180,33 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// Two e4m3 codes (low byte first) -> two f16 values, exact.
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
+    uint32_t d;
+    asm("{\n\t.reg .b16 t;\n\tcvt.u16.u32 t, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, t;\n\t}" : "=r"(d) : "r"(x));
+    return d;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__device__ __forceinline__ float f16lo(uint32_t u) {
+    float f;
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %1;\n\tcvt.f32.f16 %0, l;\n\t}" : "=f"(f) : "r"(u));
+    return f;
+}
+__device__ __forceinline__ float f16hi(uint32_t u) {
+    float f;
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %1;\n\tcvt.f32.f16 %0, h;\n\t}" : "=f"(f) : "r"(u));
+    return f;
 }
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
     uint32_t d;
@@ -403,11 +435,11 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
 // ---------------------------------------------------------------------------------------------
 // The attention kernel (one cooperative launch per draft step)
 // ---------------------------------------------------------------------------------------------
-template <int D>
-__global__ void __launch_bounds__(Cfg<D>::kThreads, 1)
+template <int D, bool F8>
+__global__ void __launch_bounds__(Cfg<D, F8>::kThreads, 1)
 attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                const __grid_constant__ AttnParams p) {
-    using C = Cfg<D>;
+    using C = Cfg<D, F8>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char* stages = smem;                                                         // kStages x (K tile, V tile)
@@ -578,7 +610,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 #else
 #pragma unroll
                                 for (int c = 0; c < C::kChunks; ++c)
-                                    tma_load_2d(dstK + c * C::kChunkBytes, &mapK, c * 64, (int)row, bar_fullK + 8 * s, policy);
+                                    tma_load_2d(dstK + c * C::kChunkBytes, &mapK, c * (128 / C::kElemBytes), (int)row, bar_fullK + 8 * s, policy);
 #endif
                                 mbar_expect_tx(bar_fullV + 8 * s, C::kTileBytes);
 #if WMTP_TMA_3D
@@ -586,7 +618,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 #else
 #pragma unroll
                                 for (int c = 0; c < C::kChunks; ++c)
-                                    tma_load_2d(dstV + c * C::kChunkBytes, &mapV, c * 64, (int)row, bar_fullV + 8 * s, policy);
+                                    tma_load_2d(dstV + c * C::kChunkBytes, &mapV, c * (128 / C::kElemBytes), (int)row, bar_fullV + 8 * s, policy);
 #endif
                             }
                         }
@@ -746,6 +778,10 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     uint32_t qb[C::kKSteps][2];
     float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f}, le[2] = {0.f, 0.f};   // l: rounded weights (normaliser), le: exact (lse)
     float o[C::kKSteps][4];
+    // multiplier of the raw scores of heads 2*t4 and 2*t4+1: the softmax scale in log2 units; for an fp8 store also
+    // the key scale of the KV head and the power of two the head's query was normalised by
+    float smul[2] = {scale, scale};
+    float vscale = 1.f;                                  // fp8: dequantisation scale of V, applied to the normalised partial
 
     // Combine every segment this group has contributed to (waits for their last partial), then forget them.
     auto combine_outstanding = [&]() {
@@ -812,7 +848,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                     Le += sm_le[w * kMaxGroup + h] * e;
                 }
             }
-            f[i] = (L > 0.f && m[i] > -INFINITY) ? exp2f(m[i] - M) / L : 0.f;
+            f[i] = (L > 0.f && m[i] > -INFINITY) ? exp2f(m[i] - M) / L * vscale : 0.f;
             if (warp == 0 && g8 == 0 && h < G) p.part_lse[pidx * G + h] = Le > 0.f ? (M + log2f(Le)) * kLn2 : -INFINITY;
         }
         constexpr int kPasses = D / 128;                       // 128 columns of d per pass through the scratch
@@ -822,10 +858,13 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 #pragma unroll
             for (int mbl = 0; mbl < 8; ++mbl) {
                 const int mb = pass * 8 + mbl;
-                float* row0 = scratch + (warp * kMaxGroup + 2 * t4) * kScratchRow + mbl * 16 + g8;
+                // accumulator rows g8 and g8 + 8 of block mb hold d = 16 mb + g8 and + 8 (bf16 store), or, for an fp8
+                // store whose V fragments come out of the transposed load with d pairs interleaved, d = 16 mb + 2 g8 and + 1
+                float* row0 = scratch + (warp * kMaxGroup + 2 * t4) * kScratchRow + mbl * 16 + (F8 ? 2 * g8 : g8);
                 float* row1 = row0 + kScratchRow;
+                constexpr int kSecond = F8 ? 1 : 8;
                 row0[0] = o[mb][0] * f[0]; row1[0] = o[mb][1] * f[1];
-                row0[8] = o[mb][2] * f[0]; row1[8] = o[mb][3] * f[1];
+                row0[kSecond] = o[mb][2] * f[0]; row1[kSecond] = o[mb][3] * f[1];
             }
             group_barrier(grp);
             for (int idx = tid; idx < G * 128; idx += kGroupThreads) {
@@ -873,10 +912,39 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         // Q^T fragments (B operand: k = d, n = head); heads >= G read as zero
         const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
             reinterpret_cast<const __nv_bfloat16*>(p.q) + ((int64_t)sg.b * p.Hq + sg.g * G + g8) * D);
+        if constexpr (!F8) {
 #pragma unroll
-        for (int ks = 0; ks < C::kKSteps; ++ks) {
-            qb[ks][0] = g8 < G ? __ldg(qrow + ks * 8 + t4) : 0u;
-            qb[ks][1] = g8 < G ? __ldg(qrow + ks * 8 + 4 + t4) : 0u;
+            for (int ks = 0; ks < C::kKSteps; ++ks) {
+                qb[ks][0] = g8 < G ? __ldg(qrow + ks * 8 + t4) : 0u;
+                qb[ks][1] = g8 < G ? __ldg(qrow + ks * 8 + 4 + t4) : 0u;
+            }
+        } else {
+            // The e4m3 codes are widened to f16 (exact), so the query goes through the f16 MMA too. Its range is made
+            // safe by a per-head power of two (exact both ways): q' = q * 2^-e with 2^e <= max|q| < 2^(e+1), and 2^e goes
+            // into the score multiplier together with the key scale. MMA k-slot order within 16 columns of d follows the
+            // byte order ldmatrix delivers: thread t4 holds d = 4 t4 .. 4 t4 + 3 of each 16.
+            float amax = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < C::kKSteps; ++ks) {
+                qb[ks][0] = g8 < G ? __ldg(qrow + ks * 8 + 2 * t4) : 0u;
+                qb[ks][1] = g8 < G ? __ldg(qrow + ks * 8 + 2 * t4 + 1) : 0u;
+                amax = fmaxf(fmaxf(amax, fmaxf(fabsf(bf16lo(qb[ks][0])), fabsf(bf16hi(qb[ks][0])))),
+                             fmaxf(fabsf(bf16lo(qb[ks][1])), fabsf(bf16hi(qb[ks][1]))));
+            }
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+            uint32_t eb = (__float_as_uint(amax) >> 23) & 0xffu;
+            eb = eb < 1u ? 1u : (eb > 253u ? 253u : eb);
+            const float down = __uint_as_float((254u - eb) << 23), up = __uint_as_float(eb << 23);
+#pragma unroll
+            for (int ks = 0; ks < C::kKSteps; ++ks) {
+                qb[ks][0] = pack_f16x2(bf16lo(qb[ks][0]) * down, bf16hi(qb[ks][0]) * down);
+                qb[ks][1] = pack_f16x2(bf16lo(qb[ks][1]) * down, bf16hi(qb[ks][1]) * down);
+            }
+            const float hmul = g8 < G ? scale * up * __ldg(p.k_scale + sg.g) : 0.f;
+            smul[0] = __shfl_sync(0xffffffffu, hmul, 8 * t4);
+            smul[1] = __shfl_sync(0xffffffffu, hmul, 8 * t4 + 4);
+            vscale = __ldg(p.v_scale + sg.g);
         }
         m[0] = m[1] = -INFINITY; l[0] = l[1] = 0.f; le[0] = le[1] = 0.f;
 #pragma unroll
@@ -927,12 +995,15 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 new_off = kv_row_offset(p, sg.b, sg.g, key0 + new_row, &new_ok);
                 if (!new_ok && lane == 0) atomicCAS(p.status, 0, kErrBounds);
             }
-            if (has_new && lane < D / 8) {
-                // the row TMA brought may be stale: take it from k_new, in shared memory and in the store
-                const uint4 x = __ldg(reinterpret_cast<const uint4*>(p.k_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8) + lane);
+            if (has_new && lane < C::kRowVecs) {
+                // the row TMA brought may be stale: take it from k_new (quantised for an fp8 store), in shared memory and in the store
+                const uint4* src = reinterpret_cast<const uint4*>(p.k_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8);
+                uint4 x;
+                if constexpr (F8) x = quant16_e4m3(__ldg(src + 2 * lane), __ldg(src + 2 * lane + 1), __ldg(p.k_scale + sg.g));
+                else x = __ldg(src + lane);
                 const uint32_t addr = sK + (lane >> 3) * C::kChunkBytes + new_row * 128 + (((lane & 7) ^ (new_row & 7)) << 4);
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
-                if (new_ok) reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.k) + new_off)[lane] = x;
+                if (new_ok) reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(p.k) + new_off * C::kElemBytes)[lane] = x;
             }
             if (has_new) {
                 if (p.mode == kRing && sg.g == 0 && lane == 0)
@@ -949,17 +1020,35 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 #endif
                 // ---- S^T = K . Q^T for this warp's 16 keys (two accumulator chains)
                 float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+                if constexpr (!F8) {
 #pragma unroll
-                for (int ks = 0; ks < C::kKSteps; ++ks) {
-                    uint32_t a[4];
-                    const uint32_t c16 = (uint32_t)((ks & 3) * 2 + halfK);
-                    ldmatrix_x4(a, sK + (ks >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
-                    if (ks & 1) mma_bf16(sb, a, qb[ks][0], qb[ks][1]);
-                    else mma_bf16(sa, a, qb[ks][0], qb[ks][1]);
+                    for (int ks = 0; ks < C::kKSteps; ++ks) {
+                        uint32_t a[4];
+                        const uint32_t c16 = (uint32_t)((ks & 3) * 2 + halfK);
+                        ldmatrix_x4(a, sK + (ks >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
+                        if (ks & 1) mma_bf16(sb, a, qb[ks][0], qb[ks][1]);
+                        else mma_bf16(sa, a, qb[ks][0], qb[ks][1]);
+                    }
+                } else {
+                    // one ldmatrix brings 32 columns of d for the warp's 16 keys: matrices {keys 0-7, 8-15} x {16 d, next 16 d};
+                    // a thread's word holds 4 consecutive codes of one key, which become the k-slots (2 t4, 2 t4 + 1) and
+                    // (2 t4 + 8, 2 t4 + 9) of that 16-column step (the query fragments use the same order)
+#pragma unroll
+                    for (int j = 0; j < C::kKSteps / 2; ++j) {
+                        uint32_t r[4], a[4];
+                        const uint32_t c16 = (uint32_t)((j & 3) * 2 + halfK);
+                        ldmatrix_x4(r, sK + (j >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
+                        a[0] = e4m3x2_to_f16x2(r[0]); a[1] = e4m3x2_to_f16x2(r[1]);
+                        a[2] = e4m3x2_to_f16x2(r[0] >> 16); a[3] = e4m3x2_to_f16x2(r[1] >> 16);
+                        mma_f16(sa, a, qb[2 * j][0], qb[2 * j][1]);
+                        a[0] = e4m3x2_to_f16x2(r[2]); a[1] = e4m3x2_to_f16x2(r[3]);
+                        a[2] = e4m3x2_to_f16x2(r[2] >> 16); a[3] = e4m3x2_to_f16x2(r[3] >> 16);
+                        mma_f16(sb, a, qb[2 * j + 1][0], qb[2 * j + 1][1]);
+                    }
                 }
                 float sc[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) sc[i] = (sa[i] + sb[i]) * scale;
+                for (int i = 0; i < 4; ++i) sc[i] = (sa[i] + sb[i]) * smul[i & 1];
                 if (!tile_full) {
                     const int ka = wkey0 + g8, kb = ka + 8;
                     bool va = ka >= vlo && ka < vhi, vb = kb >= vlo && kb < vhi;
@@ -983,12 +1072,17 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 corr1 = exp2f(m[1] - mu1);
                 m[0] = mn0; m[1] = mn1;
                 const float p0 = exp2f(sc[0] - mu0), p1 = exp2f(sc[1] - mu1), p2 = exp2f(sc[2] - mu0), p3 = exp2f(sc[3] - mu1);
-                const uint32_t pa = pack_bf16x2(p0, p1);             // key g8   : heads 2t4, 2t4+1
-                const uint32_t pc = pack_bf16x2(p2, p3);             // key g8+8
+                const uint32_t pa = F8 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1);             // key g8   : heads 2t4, 2t4+1
+                const uint32_t pc = F8 ? pack_f16x2(p2, p3) : pack_bf16x2(p2, p3);             // key g8+8
                 le[0] = le[0] * corr0 + p0 + p2;
                 le[1] = le[1] * corr1 + p1 + p3;
-                l[0] = l[0] * corr0 + bf16lo(pa) + bf16lo(pc);      // sums of the rounded weights the MMA will use
-                l[1] = l[1] * corr1 + bf16hi(pa) + bf16hi(pc);
+                if constexpr (F8) {
+                    l[0] = l[0] * corr0 + f16lo(pa) + f16lo(pc);
+                    l[1] = l[1] * corr1 + f16hi(pa) + f16hi(pc);
+                } else {
+                    l[0] = l[0] * corr0 + bf16lo(pa) + bf16lo(pc);      // sums of the rounded weights the MMA will use
+                    l[1] = l[1] * corr1 + bf16hi(pa) + bf16hi(pc);
+                }
                 pb0 = movmatrix_trans(pa);                           // P^T as B operand: k = key, n = head
                 pb1 = movmatrix_trans(pc);
 #pragma unroll
@@ -998,11 +1092,14 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             }
             mbar_wait(bar_fullV + 8 * s, ph, abort_flag, p.status);
             if (it == 0) WMTP_STAMP(p, 4);
-            if (has_new && lane < D / 8) {
-                const uint4 x = __ldg(reinterpret_cast<const uint4*>(p.v_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8) + lane);
+            if (has_new && lane < C::kRowVecs) {
+                const uint4* src = reinterpret_cast<const uint4*>(p.v_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8);
+                uint4 x;
+                if constexpr (F8) x = quant16_e4m3(__ldg(src + 2 * lane), __ldg(src + 2 * lane + 1), __ldg(p.v_scale + sg.g));
+                else x = __ldg(src + lane);
                 const uint32_t addr = sV + (lane >> 3) * C::kChunkBytes + new_row * 128 + (((lane & 7) ^ (new_row & 7)) << 4);
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
-                if (new_ok) reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.v) + new_off)[lane] = x;
+                if (new_ok) reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(p.v) + new_off * C::kElemBytes)[lane] = x;
             }
 #ifdef WMTP_SKIP_COMPUTE
             if (false) {
@@ -1024,12 +1121,31 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                     __syncwarp();
                 }
                 // ---- O^T += V^T . P^T
+                if constexpr (!F8) {
 #pragma unroll
-                for (int mb = 0; mb < C::kKSteps; ++mb) {
-                    uint32_t a[4];
-                    const uint32_t c16 = (uint32_t)((mb & 3) * 2 + halfV);
-                    ldmatrix_x4_trans(a, sV + (mb >> 2) * C::kChunkBytes + offV + ((c16 ^ (uint32_t)rr) << 4));
-                    mma_bf16(o[mb], a, pb0, pb1);
+                    for (int mb = 0; mb < C::kKSteps; ++mb) {
+                        uint32_t a[4];
+                        const uint32_t c16 = (uint32_t)((mb & 3) * 2 + halfV);
+                        ldmatrix_x4_trans(a, sV + (mb >> 2) * C::kChunkBytes + offV + ((c16 ^ (uint32_t)rr) << 4));
+                        mma_bf16(o[mb], a, pb0, pb1);
+                    }
+                } else {
+                    // the transposed load hands a thread, per matrix, the codes of keys (2 t4, 2 t4 + 1) for d = 2 g8 and
+                    // 2 g8 + 1 of a 16-column unit: accumulator row g8 of the block is d = 2 g8, row g8 + 8 is d = 2 g8 + 1
+#pragma unroll
+                    for (int j = 0; j < C::kKSteps / 2; ++j) {
+                        uint32_t r[4], a[4];
+                        const uint32_t c16 = (uint32_t)((j & 3) * 2 + halfK);
+                        ldmatrix_x4_trans(r, sV + (j >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
+                        uint32_t x = __byte_perm(r[0], 0, 0x3120), y = __byte_perm(r[1], 0, 0x3120);
+                        a[0] = e4m3x2_to_f16x2(x); a[1] = e4m3x2_to_f16x2(x >> 16);
+                        a[2] = e4m3x2_to_f16x2(y); a[3] = e4m3x2_to_f16x2(y >> 16);
+                        mma_f16(o[2 * j], a, pb0, pb1);
+                        x = __byte_perm(r[2], 0, 0x3120); y = __byte_perm(r[3], 0, 0x3120);
+                        a[0] = e4m3x2_to_f16x2(x); a[1] = e4m3x2_to_f16x2(x >> 16);
+                        a[2] = e4m3x2_to_f16x2(y); a[3] = e4m3x2_to_f16x2(y >> 16);
+                        mma_f16(o[2 * j + 1], a, pb0, pb1);
+                    }
                 }
             }
             __syncwarp();
@@ -1080,52 +1196,54 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// View of a K or V tensor [rows][D] for TMA, 128-byte swizzle.
-//   3-D (default): dims {64, rows, D/64} with strides {2 D, 128} bytes, box {64, 64, D/64}: one copy per tile.
-//   2-D: dims {D, rows}, box {64, 64}: D/64 copies per tile.
-bool make_map(CUtensorMap* map, const void* base, int64_t rows, int D) {
+// View of a K or V tensor [rows][D] for TMA, 128-byte swizzle; `esz` bytes per entry (2: bf16, 1: e4m3 codes), so a
+// 128-byte chunk of a row holds 128 / esz entries.
+//   3-D (default): dims {128/esz, rows, D esz/128} with strides {D esz, 128} bytes, box {128/esz, 64, D esz/128}: one copy per tile.
+//   2-D: dims {D, rows}, box {128/esz, 64}: D esz/128 copies per tile.
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int D, int esz) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint32_t estr[3] = {1, 1, 1};
+    const cuuint32_t per_chunk = 128 / esz, chunks = D * esz / 128;
 #if WMTP_TMA_3D
-    const cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(D / 64)};
-    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, 128};
-    const cuuint32_t box[3] = {64, (cuuint32_t)kTileKeys, (cuuint32_t)(D / 64)};
+    const cuuint64_t dims[3] = {per_chunk, (cuuint64_t)rows, chunks};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * esz, 128};
+    const cuuint32_t box[3] = {per_chunk, (cuuint32_t)kTileKeys, chunks};
     const cuuint32_t rank = 3;
 #else
     const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kTileKeys};
+    const cuuint64_t strides[1] = {(cuuint64_t)D * esz};
+    const cuuint32_t box[2] = {per_chunk, (cuuint32_t)kTileKeys};
     const cuuint32_t rank = 2;
 #endif
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
+    return fn(map, esz == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, (CUtensorMapL2promotion)WMTP_L2_PROMO,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D>
+template <int D, bool F8>
 size_t partial_smem_bytes(int B) {
-    using C = Cfg<D>;
+    using C = Cfg<D, F8>;
     return 1024 + (size_t)C::kStages * C::kStageBytes +
            sizeof(float) * C::kGroups * (kScratchFloats + 3 * kGroupWarps * kMaxGroup) +
            sizeof(uint64_t) * C::kBarriers + sizeof(int64_t) * C::kStages + sizeof(int64_t) * C::kGroups * 2 * kMaxContrib +
            (sizeof(int64_t) + sizeof(int)) * (B + 1) + sizeof(int) * (C::kGroups * kGroupInts + 4) + 16;
 }
 
-template <int D>
+template <int D, bool F8>
 cudaError_t launch_fused(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaStream_t st) {
-    const size_t smem = partial_smem_bytes<D>(p.B);
+    const size_t smem = partial_smem_bytes<D, F8>(p.B);
     static bool attr_set[64] = {};          // per device: the opt-in to > 48 KB of dynamic shared memory
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(attn_fused_tma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(attn_fused_tma<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     void* args[] = {&mk, &mv, &p};
     // cooperative: the CTAs wait on one another in the combine, so they must all be resident
-    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(attn_fused_tma<D>), dim3(p.num_ctas), dim3(Cfg<D>::kThreads), args, smem, st);
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(attn_fused_tma<D, F8>), dim3(p.num_ctas), dim3(Cfg<D, F8>::kThreads), args, smem, st);
 }
 
 }  // namespace
@@ -1141,8 +1259,11 @@ cudaError_t launch_attention(const AttnParams& p_in, cudaStream_t st) {
     AttnParams p = p_in;
     const int64_t rows = attention_rows(p);
     CUtensorMap mk, mv;
-    if (!make_map(&mk, p.k, rows, p.D) || !make_map(&mv, p.v, rows, p.D)) return cudaErrorInvalidValue;
-    cudaError_t e = p.D == 128 ? launch_fused<128>(mk, mv, p, st) : launch_fused<256>(mk, mv, p, st);
+    const int esz = p.f8 ? 1 : 2;
+    if (!make_map(&mk, p.k, rows, p.D, esz) || !make_map(&mv, p.v, rows, p.D, esz)) return cudaErrorInvalidValue;
+    cudaError_t e;
+    if (p.f8) e = p.D == 128 ? launch_fused<128, true>(mk, mv, p, st) : launch_fused<256, true>(mk, mv, p, st);
+    else e = p.D == 128 ? launch_fused<128, false>(mk, mv, p, st) : launch_fused<256, false>(mk, mv, p, st);
     count_launch(1);
     return e;
 }

@@ -4,12 +4,21 @@
 // position p lives in slot p when p < n_sink, else in n_sink + ((p - n_sink) mod cap).
 // All of this is integer work and copies: results are bit-exact by construction.
 #include "wmtp_internal.h"
+#include "fp8_util.cuh"
 
 namespace wmtp {
 
 namespace {
 
 constexpr int kErrBounds = WMTP_ERR_DEVICE_BOUNDS;
+
+// 16-byte vectors of one stored row of head_dim D: 8 bf16 or 16 e4m3 codes each.
+__device__ __forceinline__ int store_vecs(int D, int f8) { return f8 ? D / 16 : D / 8; }
+// Vector c of the stored form of a bf16 source row (`src`: its D / 8 vectors): a copy, or its e4m3 codes.
+__device__ __forceinline__ uint4 stored_vec(const uint4* __restrict__ src, int c, int f8, float scale) {
+    if (!f8) return src[c];
+    return quant16_e4m3(src[2 * c], src[2 * c + 1], scale);
+}
 
 __device__ __forceinline__ int ring_slot(int64_t p, int n_sink, int cap) {
     return p < n_sink ? (int)p : n_sink + (int)((p - n_sink) % cap);
@@ -35,22 +44,23 @@ __global__ void ring_reset_kernel(RingParams r) {
         for (int b = threadIdx.x; b < r.B; b += blockDim.x) r.len[b] = 0;
 }
 
-// One block per sequence; thread t moves 16 bytes of the token's [Hkv][D] K row and V row.
+// One block per sequence; thread t writes 16 bytes of the token's [Hkv][D] K row and V row (copied, or quantised to
+// e4m3 codes for an fp8 store).
 __global__ void ring_append_kernel(RingParams r, const uint4* __restrict__ k_new, const uint4* __restrict__ v_new) {
     const int b = blockIdx.x;
     const int64_t p = r.len[b];
     const int slots = r.n_sink + r.cap;
     const int slot = ring_slot(p, r.n_sink, r.cap);
-    const int vec_per_row = r.D / 8;
+    const int vec_per_row = store_vecs(r.D, r.f8), src_vecs = r.D / 8;
     const int n_vec = r.Hkv * vec_per_row;
     uint4* K = reinterpret_cast<uint4*>(r.k);
     uint4* V = reinterpret_cast<uint4*>(r.v);
     for (int i = threadIdx.x; i < n_vec; i += blockDim.x) {
         const int g = i / vec_per_row, c = i % vec_per_row;
         const int64_t dst = (((int64_t)b * r.Hkv + g) * slots + slot) * vec_per_row + c;
-        const int64_t src = (int64_t)b * n_vec + i;
-        K[dst] = k_new[src];
-        V[dst] = v_new[src];
+        const int64_t src = ((int64_t)b * r.Hkv + g) * src_vecs;
+        K[dst] = stored_vec(k_new + src, c, r.f8, r.f8 ? r.k_scale[g] : 1.f);
+        V[dst] = stored_vec(v_new + src, c, r.f8, r.f8 ? r.v_scale[g] : 1.f);
     }
     __syncthreads();   // every thread has read len[b] before it moves
     if (threadIdx.x == 0) {
@@ -69,7 +79,7 @@ __device__ __forceinline__ int64_t kv_row_vec(const KvParams& kv, int b, int g, 
 __global__ void kv_append_kernel(KvParams kv, const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, int* status) {
     const int b = blockIdx.x;
     const int64_t p = kv.len[b];
-    const int vec_per_row = kv.D / 8;
+    const int vec_per_row = store_vecs(kv.D, kv.f8), src_vecs = kv.D / 8;
     const int n_vec = kv.Hkv * vec_per_row;
     __shared__ int bad;
     if (threadIdx.x == 0) bad = 0;
@@ -85,9 +95,9 @@ __global__ void kv_append_kernel(KvParams kv, const uint4* __restrict__ k_new, c
         bool ok = true;
         const int64_t dst = kv_row_vec(kv, b, g, p, vec_per_row, &ok) + c;
         if (!ok) { bad = 1; continue; }
-        const int64_t src = (int64_t)b * n_vec + i;
-        K[dst] = k_new[src];
-        V[dst] = v_new[src];
+        const int64_t src = ((int64_t)b * kv.Hkv + g) * src_vecs;
+        K[dst] = stored_vec(k_new + src, c, kv.f8, kv.f8 ? kv.k_scale[g] : 1.f);
+        V[dst] = stored_vec(v_new + src, c, kv.f8, kv.f8 ? kv.v_scale[g] : 1.f);
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -101,7 +111,7 @@ __global__ void ring_init_kernel(RingParams r, KvParams kv) {
     const int b = blockIdx.y;
     const int slots = r.n_sink + r.cap;
     const int64_t S = kv.len[b];
-    const int vec_per_row = r.D / 8;
+    const int vec_per_row = store_vecs(r.D, r.f8);           // rows are copied as stored (same dtype and scales on both sides)
     const int warps = blockDim.x / 32, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const uint4* Ksrc = reinterpret_cast<const uint4*>(kv.k);
     const uint4* Vsrc = reinterpret_cast<const uint4*>(kv.v);
@@ -132,7 +142,7 @@ __global__ void ring_append_many_kernel(RingParams r, int n_tok, const uint4* __
     const int b = blockIdx.x;
     const int64_t p0 = r.len[b];
     const int slots = r.n_sink + r.cap;
-    const int vec_per_row = r.D / 8;
+    const int vec_per_row = store_vecs(r.D, r.f8), src_vecs = r.D / 8;
     const int n_vec = r.Hkv * vec_per_row;
     uint4* K = reinterpret_cast<uint4*>(r.k);
     uint4* V = reinterpret_cast<uint4*>(r.v);
@@ -141,9 +151,9 @@ __global__ void ring_append_many_kernel(RingParams r, int n_tok, const uint4* __
         const int g = i / vec_per_row, c = i % vec_per_row;
         const int slot = ring_slot(p0 + j, r.n_sink, r.cap);
         const int64_t dst = (((int64_t)b * r.Hkv + g) * slots + slot) * vec_per_row + c;
-        const int64_t src = ((int64_t)b * n_tok + j) * n_vec + i;
-        K[dst] = k_new[src];
-        V[dst] = v_new[src];
+        const int64_t src = (((int64_t)b * n_tok + j) * r.Hkv + g) * src_vecs;
+        K[dst] = stored_vec(k_new + src, c, r.f8, r.f8 ? r.k_scale[g] : 1.f);
+        V[dst] = stored_vec(v_new + src, c, r.f8, r.f8 ? r.v_scale[g] : 1.f);
     }
     __syncthreads();   // every thread has read len[b] before it moves
     for (int j = threadIdx.x; j < n_tok; j += blockDim.x)
@@ -155,7 +165,7 @@ __global__ void kv_append_many_kernel(KvParams kv, int n_tok, const uint4* __res
                                       int* status) {
     const int b = blockIdx.x;
     const int64_t p0 = kv.len[b];
-    const int vec_per_row = kv.D / 8;
+    const int vec_per_row = store_vecs(kv.D, kv.f8), src_vecs = kv.D / 8;
     const int n_vec = kv.Hkv * vec_per_row;
     __shared__ int bad;
     if (threadIdx.x == 0) bad = 0;
@@ -172,9 +182,9 @@ __global__ void kv_append_many_kernel(KvParams kv, int n_tok, const uint4* __res
         bool ok = true;
         const int64_t dst = kv_row_vec(kv, b, g, p0 + j, vec_per_row, &ok) + c;
         if (!ok) { bad = 1; continue; }
-        const int64_t src = ((int64_t)b * n_tok + j) * n_vec + i;
-        K[dst] = k_new[src];
-        V[dst] = v_new[src];
+        const int64_t src = (((int64_t)b * n_tok + j) * kv.Hkv + g) * src_vecs;
+        K[dst] = stored_vec(k_new + src, c, kv.f8, kv.f8 ? kv.k_scale[g] : 1.f);
+        V[dst] = stored_vec(v_new + src, c, kv.f8, kv.f8 ? kv.v_scale[g] : 1.f);
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -246,7 +256,7 @@ cudaError_t launch_ring_reset(const RingParams& r, cudaStream_t st) {
 }
 
 cudaError_t launch_ring_append(const RingParams& r, const void* k_new, const void* v_new, cudaStream_t st) {
-    const int n_vec = r.Hkv * r.D / 8;
+    const int n_vec = r.Hkv * r.D / (r.f8 ? 16 : 8);
     const int threads = n_vec < 32 ? 32 : (n_vec > 256 ? 256 : (n_vec + 31) / 32 * 32);
     ring_append_kernel<<<r.B, threads, 0, st>>>(r, (const uint4*)k_new, (const uint4*)v_new);
     count_launch(1);
@@ -254,7 +264,7 @@ cudaError_t launch_ring_append(const RingParams& r, const void* k_new, const voi
 }
 
 cudaError_t launch_kv_append(const KvParams& kv, const void* k_new, const void* v_new, int* status, cudaStream_t st) {
-    const int n_vec = kv.Hkv * kv.D / 8;
+    const int n_vec = kv.Hkv * kv.D / (kv.f8 ? 16 : 8);
     const int threads = n_vec < 32 ? 32 : (n_vec > 256 ? 256 : (n_vec + 31) / 32 * 32);
     kv_append_kernel<<<kv.B, threads, 0, st>>>(kv, (const uint4*)k_new, (const uint4*)v_new, status);
     count_launch(1);

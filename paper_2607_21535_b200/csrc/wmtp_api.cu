@@ -40,9 +40,17 @@ wmtp_status check_shape(int batch, int Hkv, int D) {
     return WMTP_OK;
 }
 
+wmtp_status check_dtype(int kv_dtype, const float* k_scale, const float* v_scale) {
+    if (kv_dtype != WMTP_KV_BF16 && kv_dtype != WMTP_KV_FP8_E4M3) return fail(WMTP_ERR_UNSUPPORTED, "kv_dtype=%d (supported: bf16, fp8 e4m3)", kv_dtype);
+    if (kv_dtype == WMTP_KV_FP8_E4M3 && (!k_scale || !v_scale || !aligned(k_scale, 4) || !aligned(v_scale, 4)))
+        return fail(WMTP_ERR_INVALID_ARG, "an fp8 store needs k_scale and v_scale (device fp32 [Hkv])");
+    return WMTP_OK;
+}
+
 wmtp_status check_ring(const wmtp_ring* r) {
     if (!r) return fail(WMTP_ERR_INVALID_ARG, "ring descriptor is NULL");
     if (wmtp_status s = check_shape(r->batch, r->Hkv, r->D)) return s;
+    if (wmtp_status s = check_dtype(r->kv_dtype, r->k_scale, r->v_scale)) return s;
     if (r->n_sink < 0 || r->W < 1 || r->cap < r->W)
         return fail(WMTP_ERR_INVALID_ARG, "ring needs n_sink >= 0, W >= 1, cap >= W (n_sink=%d W=%d cap=%d)", r->n_sink, r->W, r->cap);
     if ((int64_t)r->n_sink + r->cap > (1 << 30)) return fail(WMTP_ERR_INVALID_ARG, "ring of %lld slots is too large", (long long)r->n_sink + r->cap);
@@ -57,6 +65,7 @@ wmtp_status check_ring(const wmtp_ring* r) {
 wmtp_status check_kv(const wmtp_kv* kv) {
     if (!kv) return fail(WMTP_ERR_INVALID_ARG, "kv descriptor is NULL");
     if (wmtp_status s = check_shape(kv->batch, kv->Hkv, kv->D)) return s;
+    if (wmtp_status s = check_dtype(kv->kv_dtype, kv->k_scale, kv->v_scale)) return s;
     if (!kv->k || !kv->v || !kv->len) return fail(WMTP_ERR_INVALID_ARG, "kv has a NULL pointer");
     if (!aligned(kv->k, 16) || !aligned(kv->v, 16) || !aligned(kv->len, 8))
         return fail(WMTP_ERR_INVALID_ARG, "kv pointers must be 16-byte (k, v), 8-byte (len) aligned");
@@ -75,11 +84,13 @@ wmtp_status check_kv(const wmtp_kv* kv) {
 }
 
 RingParams ring_params(const wmtp_ring* r) {
-    return RingParams{r->k, r->v, r->slot_pos, r->len, r->batch, r->Hkv, r->D, r->n_sink, r->W, r->cap};
+    return RingParams{r->k, r->v, r->slot_pos, r->len, r->batch, r->Hkv, r->D, r->n_sink, r->W, r->cap,
+                      r->kv_dtype == WMTP_KV_FP8_E4M3 ? 1 : 0, r->k_scale, r->v_scale};
 }
 KvParams kv_params(const wmtp_kv* kv) {
     return KvParams{kv->k, kv->v, kv->page_table, kv->len, kv->S_cap, kv->batch, kv->Hkv, kv->D,
-                    kv->page_table ? kv->page_size : 0, kv->max_pages, kv->num_pages};
+                    kv->page_table ? kv->page_size : 0, kv->max_pages, kv->num_pages,
+                    kv->kv_dtype == WMTP_KV_FP8_E4M3 ? 1 : 0, kv->k_scale, kv->v_scale};
 }
 
 wmtp_status check_attn_common(const void* q, int Hq, int Hkv, int batch, int D, const void* out, const float* lse,
@@ -142,6 +153,7 @@ wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm
     fill_attn(p, q, Hq, ring->Hkv, ring->batch * q_len, ring->D, sm_scale, out, lse, ws);
     p.q_len = q_len;
     p.k = ring->k; p.v = ring->v; p.page_table = nullptr; p.len = ring->len;
+    p.f8 = ring->kv_dtype == WMTP_KV_FP8_E4M3 ? 1 : 0; p.k_scale = ring->k_scale; p.v_scale = ring->v_scale;
     p.k_new = k_new; p.v_new = v_new; p.slot_pos = ring->slot_pos;
     p.mode = kRing;
     p.rows_per_head = (int64_t)ring->n_sink + ring->cap;
@@ -166,6 +178,7 @@ wmtp_status attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, 
     fill_attn(p, q, Hq, kv->Hkv, kv->batch * q_len, kv->D, sm_scale, out, lse, ws);
     p.q_len = q_len;
     p.k = kv->k; p.v = kv->v; p.page_table = kv->page_table; p.len = kv->len;
+    p.f8 = kv->kv_dtype == WMTP_KV_FP8_E4M3 ? 1 : 0; p.k_scale = kv->k_scale; p.v_scale = kv->v_scale;
     p.k_new = k_new; p.v_new = v_new; p.slot_pos = nullptr; p.S_cap = kv->S_cap;
     p.mode = kv->page_table ? kPaged : kContiguous;
     p.rows_per_head = kv->page_table ? kv->page_size : kv->S_cap;
@@ -256,6 +269,8 @@ const char* wmtp_status_string(wmtp_status s) {
 
 const char* wmtp_last_error(void) { return g_err; }
 
+size_t wmtp_kv_elem_bytes(int kv_dtype) { return kv_dtype == WMTP_KV_BF16 ? 2 : (kv_dtype == WMTP_KV_FP8_E4M3 ? 1 : 0); }
+
 size_t wmtp_ring_bytes(int batch, int Hkv, int D, int n_sink, int cap, size_t* pos_bytes) {
     if (batch < 1 || Hkv < 1 || D < 1 || n_sink < 0 || cap < 1) { if (pos_bytes) *pos_bytes = 0; return 0; }
     const size_t slots = (size_t)n_sink + cap;
@@ -304,6 +319,7 @@ wmtp_status wmtp_ring_init_from_kv(const wmtp_ring* ring, const wmtp_kv* kv, voi
     if (wmtp_status s = check_kv(kv)) return s;
     if (ring->batch != kv->batch || ring->Hkv != kv->Hkv || ring->D != kv->D)
         return fail(WMTP_ERR_INVALID_ARG, "ring and kv disagree on batch / Hkv / D");
+    if (ring->kv_dtype != kv->kv_dtype) return fail(WMTP_ERR_INVALID_ARG, "ring and kv disagree on kv_dtype (rows are copied as stored)");
     cudaError_t e = launch_ring_init_from_kv(ring_params(ring), kv_params(kv), (cudaStream_t)stream);
     return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "ring init launch");
 }
@@ -592,6 +608,7 @@ wmtp_status wmtp_draft_attn_windowed_noalloc(const void* q, int Hq, const wmtp_r
     const float sc = sm_scale > 0.f ? sm_scale : 1.0f / std::sqrt((float)ring->D);
     p.scale_log2 = sc * 1.4426950408889634f;
     p.k = ring->k; p.v = ring->v; p.page_table = nullptr; p.len = ring->len;
+    p.f8 = ring->kv_dtype == WMTP_KV_FP8_E4M3 ? 1 : 0; p.k_scale = ring->k_scale; p.v_scale = ring->v_scale;
     p.k_new = nullptr; p.v_new = nullptr; p.slot_pos = ring->slot_pos;
     p.mode = kRing;
     p.rows_per_head = (int64_t)ring->n_sink + ring->cap;

@@ -45,8 +45,11 @@ __host__ __device__ inline size_t pool_slots(int nseg) {
 // Everything the attention kernel needs; passed by value.
 struct AttnParams {
     const void* q;            // bf16 [B][Hq][D]
-    void* k;                  // bf16, layout per mode (written only by a fused append)
+    void* k;                  // bf16 (or e4m3 codes when f8), layout per mode (written only by a fused append)
     void* v;
+    const float* k_scale;     // f8 only: [Hkv] dequantisation scales (value = code value * scale)
+    const float* v_scale;
+    int f8;                   // 1: the store holds e4m3 codes
     const int32_t* page_table;
     int64_t* len;             // [B]; advanced at the end of a launch that appends
     const void* k_new;        // bf16 [B][Hkv][D], or nullptr: attention only, no append
@@ -83,12 +86,14 @@ struct AttnParams {
 struct RingParams {
     void* k; void* v; int32_t* slot_pos; int64_t* len;
     int B, Hkv, D, n_sink, W, cap;
+    int f8; const float* k_scale; const float* v_scale;    // f8: e4m3 codes, per-KV-head scales
 };
 
 struct KvParams {
     void* k; void* v; const int32_t* page_table; int64_t* len;
     int64_t S_cap;
     int B, Hkv, D, page_size, max_pages, num_pages;
+    int f8; const float* k_scale; const float* v_scale;
 };
 
 // Launchers (defined in the .cu files). Each returns the cudaError_t of its launch.

@@ -20,7 +20,16 @@ def to_dev_bf16(a: np.ndarray, dev="cuda"):
 
 
 def bits(t: torch.Tensor) -> np.ndarray:
+    if t.dtype == torch.uint8:                       # fp8 store: the codes themselves
+        return t.contiguous().cpu().numpy()
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def to_dev_store(a: np.ndarray, dev="cuda"):
+    """KV store contents: bf16 bit patterns (uint16) or e4m3 codes (uint8)."""
+    if a.dtype == np.uint8:
+        return torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    return to_dev_bf16(a, dev)
 
 
 class DeviceWorkload:
@@ -29,12 +38,15 @@ class DeviceWorkload:
     def __init__(self, wl: wi.Workload, dev="cuda", cap=None):
         cfg = wl.cfg
         self.wl, self.cfg, self.dev = wl, cfg, dev
-        self.K, self.V = to_dev_bf16(wl.K_dev, dev), to_dev_bf16(wl.V_dev, dev)
+        self.K, self.V = to_dev_store(wl.K_dev, dev), to_dev_store(wl.V_dev, dev)
         self.lens = torch.from_numpy(wl.seq_lens.copy()).to(dev)
         pt = torch.from_numpy(wl.page_table).to(dev) if cfg.paged else None
-        self.kv = wm.KV(self.K, self.V, self.lens, page_table=pt, S_cap=None if cfg.paged else wl.S_cap)
+        self.k_scale = torch.from_numpy(wl.k_scale).to(dev) if wl.k_scale is not None else None
+        self.v_scale = torch.from_numpy(wl.v_scale).to(dev) if wl.v_scale is not None else None
+        self.kv = wm.KV(self.K, self.V, self.lens, page_table=pt, S_cap=None if cfg.paged else wl.S_cap,
+                        k_scale=self.k_scale, v_scale=self.v_scale)
         self.ring = wm.Ring(cfg.batch, cfg.Hkv, cfg.D, cfg.n_sink, cfg.W, cap=cap if cap is not None else cfg.W + cfg.cap_slack,
-                            device=dev)
+                            device=dev, k_scale=self.k_scale, v_scale=self.v_scale)
         self.ws = wm.Workspace(cfg.batch, cfg.Hq, cfg.Hkv, cfg.D, device=dev)
         self.q, self.k_new, self.v_new = to_dev_bf16(wl.q, dev), to_dev_bf16(wl.k_new, dev), to_dev_bf16(wl.v_new, dev)
         self.out_w = torch.full_like(self.q, float("nan"))
@@ -82,4 +94,4 @@ def check_ring_against_sim(ring: wm.Ring, b: int, sim: R.RingSim, what=""):
 def oracle_for(wl: wi.Workload, b: int, cap=None, with_ring=True) -> R.DraftOracle:
     cfg = wl.cfg
     return R.DraftOracle(wl.K[b], wl.V[b], cfg.Hq, cfg.n_sink, cfg.W, cap=cap if cap is not None else cfg.W + cfg.cap_slack,
-                         reserve=4 * cfg.gamma + 4, with_ring=with_ring)
+                         reserve=4 * cfg.gamma + 4, with_ring=with_ring, k_scale=wl.k_scale, v_scale=wl.v_scale)
