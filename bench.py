@@ -173,7 +173,7 @@ def config_dict(cfg, args):
     return {
         "workload": f"{cfg.name}: batch {cfg.batch}, S={'log-uniform ' + str(cfg.S0_range) if cfg.S0_range else cfg.S0}, "
                     f"Hq={cfg.Hq}, Hkv={cfg.Hkv}, head_dim={cfg.D}, W={cfg.W}, sink={cfg.n_sink}, gamma={cfg.gamma}, "
-                    f"{'paged(64)' if cfg.paged else 'contiguous'} bf16 KV",
+                    f"{'paged(64)' if cfg.paged else 'contiguous'} {'fp8 e4m3' if cfg.kv_dtype == 'fp8' else 'bf16'} KV",
         "step": "gamma windowed draft steps (ring append + attention) + gamma full-context draft steps (KV append + attention)",
         "draft_steps_per_pass": 2 * cfg.gamma,
         "l2": "inputs larger than L2: every full-context draft step streams the whole KV "
@@ -189,6 +189,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="million", choices=sorted(WORKLOADS))
+    ap.add_argument("--kv-dtype", default="bf16", choices=["bf16", "fp8"],
+                    help="entry type of the KV stores (fp8: e4m3 codes with per-KV-head scales)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -214,6 +216,8 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     cfg = pick_config(args.workload, 0)
+    if args.kv_dtype == "fp8":
+        cfg = wi.scaled(cfg, kv_dtype="fp8", name=cfg.name + "_fp8")
     gam, B = cfg.gamma, cfg.batch
     total_passes = args.warmup + 3 * args.steps + 8          # timed + breakdown + e2e passes, plus slack
     t0 = time.perf_counter()
@@ -221,11 +225,15 @@ def main():
     log(f"[bench] generated {cfg.name} in {time.perf_counter() - t0:.1f}s")
 
     bf = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(dev).view(torch.bfloat16)
-    K, V = bf(wl.K_dev), bf(wl.V_dev)
+    store = (lambda a: torch.from_numpy(a).to(dev)) if cfg.kv_dtype == "fp8" else bf
+    K, V = store(wl.K_dev), store(wl.V_dev)
     lens = torch.from_numpy(wl.seq_lens.copy()).to(dev)
     pt = torch.from_numpy(wl.page_table).to(dev) if cfg.paged else None
-    kv = wm.KV(K, V, lens, page_table=pt)
-    ring = wm.Ring(B, cfg.Hkv, cfg.D, cfg.n_sink, cfg.W, device=dev)
+    scales = {}
+    if cfg.kv_dtype == "fp8":
+        scales = dict(k_scale=torch.from_numpy(wl.k_scale).to(dev), v_scale=torch.from_numpy(wl.v_scale).to(dev))
+    kv = wm.KV(K, V, lens, page_table=pt, **scales)
+    ring = wm.Ring(B, cfg.Hkv, cfg.D, cfg.n_sink, cfg.W, device=dev, **scales)
     ws = wm.Workspace(B, cfg.Hq, cfg.Hkv, cfg.D, device=dev)
     q, kn, vn = bf(wl.q), bf(wl.k_new), bf(wl.v_new)
     out_w, out_f = torch.empty_like(q), torch.empty_like(q)
@@ -334,7 +342,7 @@ def main():
     ext = None
     ql = 4
     if B * ql <= 1024:
-        ring_x = wm.Ring(B, cfg.Hkv, cfg.D, cfg.n_sink, cfg.W, cap=cfg.W + 8, device=dev)
+        ring_x = wm.Ring(B, cfg.Hkv, cfg.D, cfg.n_sink, cfg.W, cap=cfg.W + 8, device=dev, **scales)
         ws_x = wm.Workspace(B * ql, cfg.Hq, cfg.Hkv, cfg.D, device=dev)
         wm.wmtp_ring_init_from_kv(ring_x, kv)
         per_seq = lambda t: t[:ql].transpose(0, 1).contiguous()
@@ -364,6 +372,40 @@ def main():
                "full_us_per_call": x1.elapsed_time(x2) * 1e3 / reps,
                "note": "windowed: append q_len tokens to a ring with 8 slack slots + one multi-query attention launch + "
                        "rollback (3 launches); full: one multi-query attention launch over the whole KV store"}
+    # ---- the fp8 (e4m3) KV variant of the same workload: half the bytes per key, same launches
+    f8 = None
+    if cfg.kv_dtype == "bf16":
+        cfg8 = wi.scaled(cfg, kv_dtype="fp8")
+        wl8 = wi.make_workload(cfg8, poison_unused=False, extra_cap=gam * (reps + 8) + 64)
+        K8, V8 = torch.from_numpy(wl8.K_dev).to(dev), torch.from_numpy(wl8.V_dev).to(dev)
+        lens8 = torch.from_numpy(wl8.seq_lens.copy()).to(dev)
+        ks8, vs8 = torch.from_numpy(wl8.k_scale).to(dev), torch.from_numpy(wl8.v_scale).to(dev)
+        pt8 = torch.from_numpy(wl8.page_table).to(dev) if cfg.paged else None
+        kv8 = wm.KV(K8, V8, lens8, page_table=pt8, k_scale=ks8, v_scale=vs8)
+        ring8 = wm.Ring(B, cfg.Hkv, cfg.D, cfg.n_sink, cfg.W, device=dev, k_scale=ks8, v_scale=vs8)
+        wm.wmtp_ring_init_from_kv(ring8, kv8)
+        for _ in range(2):
+            wm.wmtp_draft_loop_windowed(ring8, q, kn, vn, out_w, ws)
+            wm.wmtp_draft_loop_full(kv8, q, kn, vn, out_f, ws)
+        y0, y1, y2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        y0.record()
+        for _ in range(reps):
+            wm.wmtp_draft_loop_windowed(ring8, q, kn, vn, out_w, ws)
+        y1.record()
+        for _ in range(reps):
+            wm.wmtp_draft_loop_full(kv8, q, kn, vn, out_f, ws)
+        y2.record()
+        torch.cuda.synchronize()
+        wm.wmtp_device_status(ws)
+        lens8_now = lens8.cpu().numpy()
+        us_w8 = y0.elapsed_time(y1) * 1e3 / reps / gam
+        us_f8 = y1.elapsed_time(y2) * 1e3 / reps / gam
+        bytes8 = float(lens8_now.sum()) * cfg8.kv_bytes_per_token
+        f8 = {"windowed_us_per_step": us_w8, "full_us_per_step": us_f8, "kv_bytes_per_full_step": bytes8,
+              "full_algorithmic_gbs": bytes8 / (us_f8 * 1e-6) / 1e9,
+              "full_pct_of_8tbs": bytes8 / (us_f8 * 1e-6) / 8e12 * 100,
+              "note": "e4m3 codes with one fp32 scale per KV head for K and V; q, k_new, v_new, out stay bf16"}
+        del K8, V8, kv8, ring8, wl8
     full_bytes = float(cur_lens.sum()) * cfg.kv_bytes_per_token
     win_bytes = float(np.minimum(cur_lens, cfg.n_sink + cfg.W).sum()) * cfg.kv_bytes_per_token
     peak, peak_src = measured_peaks()
@@ -402,7 +444,8 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic", "config": config_dict(cfg, args),
+            "dtype": "bf16" if cfg.kv_dtype == "bf16" else "f16 (e4m3 KV widened exactly; fp32 softmax)",
+            "data": "synthetic", "config": config_dict(cfg, args),
             "variants": {
                 "windowed": {"us_per_step": us_win, "kv_bytes_per_step": win_bytes,
                              "algorithmic_gbs": win_bytes / (us_win * 1e-6) / 1e9,
@@ -415,13 +458,14 @@ def main():
                          "pct_of_8tbs": full_bytes / (us_full * 1e-6) / 8e12 * 100,
                          "us_per_attention_call": us_full_call},
                 "draft_extend": ext,
+                "fp8_kv": f8,
             },
             "windowed_flatness": flat,
             "roofline": {"bound": "hbm", "kernel": "attn_fused_tma (full-context draft attention: split-KV partials + in-kernel combine)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": peak_src, "pct_of_8tbs": achieved / 8000 * 100,
                          "traffic": (NCU_TRAFFIC_BYTES_PER_KEY[cfg.D] * float(cur_lens.sum())
-                                     if cfg.D in NCU_TRAFFIC_BYTES_PER_KEY and cfg.Hkv == 2 else None),
+                                     if cfg.D in NCU_TRAFFIC_BYTES_PER_KEY and cfg.Hkv == 2 and cfg.kv_dtype == "bf16" else None),
                          "algorithmic_bytes": full_bytes},
             "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},

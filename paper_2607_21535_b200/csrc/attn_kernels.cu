@@ -66,11 +66,34 @@ struct Cfg {
     static constexpr int kTileBytes = kChunks * kChunkBytes;  // K (or V) tile
     static constexpr int kStageBytes = 2 * kTileBytes;
     // consumer groups: a tile of fewer bytes brings the same softmax work, so the smaller tiles get two groups
-    static constexpr int kGroups = (kStageBytes >= 65536) ? 1 : 2;
+#ifndef WMTP_F8_GROUPS_256
+#define WMTP_F8_GROUPS_256 2
+#endif
+    static constexpr int kGroups = (kStageBytes >= 65536) ? 1 : ((F8 && D == 256) ? WMTP_F8_GROUPS_256 : 2);
     static constexpr int kStages = (kStageBytes >= 65536) ? 3 : (kStageBytes >= 32768 ? 5 : 8);
     static constexpr int kRowVecs = D * kElemBytes / 16;      // 16-byte vectors per stored row
+    // With two groups the CTA has 9 warps and a thread at most 168 registers: the query fragments (the same in all four
+    // warps of a group) then live in shared memory, one copy per group, instead of D / 8 registers per thread.
+    static constexpr bool kQShared = (kGroups == 2);
+    static constexpr int kQBytes = kQShared ? kGroups * (D / 16) * 32 * 8 : 0;
     static constexpr int kConsumerWarps = kGroups * kGroupWarps;
-    static constexpr int kThreads = (kConsumerWarps + 1) * 32;
+    // With two consumer groups the CTA would have 9 warps and every thread at most 168 registers (three warps share
+    // one scheduler's register file); the consumers want more and the producer needs about 56. So after the common
+    // prologue the producer's warpgroup hands registers to the consumers' warpgroups (setmaxnreg). The instruction is
+    // warpgroup-wide: the producer's warpgroup is filled up with three warps that execute it and exit.
+#ifndef WMTP_REBALANCE
+#define WMTP_REBALANCE 1
+#endif
+#ifndef WMTP_REGS_P
+#define WMTP_REGS_P 56
+#define WMTP_REGS_C 224
+#endif
+    static constexpr bool kRebalance = (kGroups == 2) && WMTP_REBALANCE;
+    static constexpr int kPadWarps = kRebalance ? 3 : 0;
+    static constexpr int kRegsProducer = WMTP_REGS_P, kRegsConsumer = WMTP_REGS_C;
+    // the 8 consumer warps and the 4 warps of the producer's warpgroup share what the 12 warps were launched with
+    static_assert(8 * kRegsConsumer + 4 * kRegsProducer <= 12 * 168, "register trade must balance");
+    static constexpr int kThreads = (kConsumerWarps + 1 + kPadWarps) * 32;
     static constexpr int kKSteps = D / 16;
     static constexpr int kBarriers = (1 + 2 * kGroups) * kStages;
     // iterations between two uses of the same stage by the same group: lcm(kStages, kGroups)
@@ -436,7 +459,10 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
 // The attention kernel (one cooperative launch per draft step)
 // ---------------------------------------------------------------------------------------------
 template <int D, bool F8>
-__global__ void __launch_bounds__(Cfg<D, F8>::kThreads, 1)
+#ifndef WMTP_LB
+#define WMTP_LB(x) (x)
+#endif
+__global__ void __launch_bounds__(WMTP_LB((Cfg<D, F8>::kThreads)), 1)
 attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                const __grid_constant__ AttnParams p) {
     using C = Cfg<D, F8>;
@@ -448,7 +474,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     // Barriers: empty[stage] (the producer observes every use of a stage) and, per consumer group, fullK / fullV[stage].
     // A group only sees the uses of a stage that are its own, and a parity wait can only tell consecutive phases
     // apart, so the "full" barriers must not be shared between groups.
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sm_stats + C::kGroups * 3 * kGroupWarps * kMaxGroup);
+    uint2* q_sm_all = reinterpret_cast<uint2*>(sm_stats + C::kGroups * 3 * kGroupWarps * kMaxGroup);   // [kGroups][kKSteps][32] (kQShared)
+    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(q_sm_all) + C::kQBytes);
     int64_t* stage_tile = reinterpret_cast<int64_t*>(bars + C::kBarriers);                // [kStages] global tile index, -1 = end
     int64_t* contrib_base_all = stage_tile + C::kStages;                                  // [kGroups][2][kMaxContrib]
     int64_t* tile_prefix = contrib_base_all + C::kGroups * 2 * kMaxContrib;               // [B + 1]
@@ -526,7 +553,14 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     WMTP_STAMP(p, 2);
     const bool slack = (p.mode == kRing) && (p.cap != p.W);
 
-    if ((threadIdx.x >> 5) == C::kConsumerWarps) {
+    if ((int)(threadIdx.x >> 5) >= C::kConsumerWarps) {
+        if constexpr (C::kRebalance) {
+            asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsProducer));
+            if ((int)(threadIdx.x >> 5) > C::kConsumerWarps) return;          // filler warps of the producer's warpgroup
+        }
+#ifdef WMTP_NO_PRODUCER
+        return;
+#endif
         // =================================== producer warp ===================================
         // CTA c < Cn owns the tile range [c n / Cn, (c+1) n / Cn). It streams the first part of it without any
         // bookkeeping; the rest is handed out in small chunks through the per-CTA cursor cur[c], to the owner
@@ -740,6 +774,10 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         return;
     }
 
+    if constexpr (C::kRebalance) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsConsumer));
+#ifdef WMTP_NO_CONSUMER
+    return;
+#endif
     // ===================================== consumer groups =====================================
     const int grp = threadIdx.x / kGroupThreads, tid = threadIdx.x % kGroupThreads;   // group, thread within the group
     const int warp = tid >> 5;                           // warp within the group: owns keys [16 warp, 16 warp + 16) of a tile
@@ -775,7 +813,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     int new_tile = -1;                                   // tile (within the segment) whose row this warp must patch (fused append)
     int new_row = 0;
     int seg_tiles_done = 0;                              // tiles of the current segment this group has processed
-    uint32_t qb[C::kKSteps][2];
+    uint32_t qb[C::kQShared ? 1 : C::kKSteps][2];      // query fragments (registers), or ...
+    uint2* q_sm = q_sm_all + grp * C::kKSteps * 32 + lane;   // ... this lane's column of the group's shared copy
     float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f}, le[2] = {0.f, 0.f};   // l: rounded weights (normaliser), le: exact (lse)
     float o[C::kKSteps][4];
     // multiplier of the raw scores of heads 2*t4 and 2*t4+1: the softmax scale in log2 units; for an fp8 store also
@@ -912,39 +951,51 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         // Q^T fragments (B operand: k = d, n = head); heads >= G read as zero
         const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
             reinterpret_cast<const __nv_bfloat16*>(p.q) + ((int64_t)sg.b * p.Hq + sg.g * G + g8) * D);
-        if constexpr (!F8) {
-#pragma unroll
-            for (int ks = 0; ks < C::kKSteps; ++ks) {
-                qb[ks][0] = g8 < G ? __ldg(qrow + ks * 8 + t4) : 0u;
-                qb[ks][1] = g8 < G ? __ldg(qrow + ks * 8 + 4 + t4) : 0u;
-            }
-        } else {
+        // Words of the query row that make up this lane's fragment of 16-column step ks: ks * 8 + w0 and ks * 8 + w1.
+        // For an fp8 store the MMA k-slot order within 16 columns of d follows the byte order ldmatrix delivers the
+        // codes in: lane t4 holds d = 4 t4 .. 4 t4 + 3 of each 16.
+        const int w0 = F8 ? 2 * t4 : t4, w1 = F8 ? 2 * t4 + 1 : 4 + t4;
+        float down = 1.f;
+        if constexpr (F8) {
             // The e4m3 codes are widened to f16 (exact), so the query goes through the f16 MMA too. Its range is made
             // safe by a per-head power of two (exact both ways): q' = q * 2^-e with 2^e <= max|q| < 2^(e+1), and 2^e goes
-            // into the score multiplier together with the key scale. MMA k-slot order within 16 columns of d follows the
-            // byte order ldmatrix delivers: thread t4 holds d = 4 t4 .. 4 t4 + 3 of each 16.
+            // into the score multiplier together with the key scale.
             float amax = 0.f;
 #pragma unroll
             for (int ks = 0; ks < C::kKSteps; ++ks) {
-                qb[ks][0] = g8 < G ? __ldg(qrow + ks * 8 + 2 * t4) : 0u;
-                qb[ks][1] = g8 < G ? __ldg(qrow + ks * 8 + 2 * t4 + 1) : 0u;
-                amax = fmaxf(fmaxf(amax, fmaxf(fabsf(bf16lo(qb[ks][0])), fabsf(bf16hi(qb[ks][0])))),
-                             fmaxf(fabsf(bf16lo(qb[ks][1])), fabsf(bf16hi(qb[ks][1]))));
+                const uint32_t a = g8 < G ? __ldg(qrow + ks * 8 + w0) : 0u, b = g8 < G ? __ldg(qrow + ks * 8 + w1) : 0u;
+                amax = fmaxf(fmaxf(amax, fmaxf(fabsf(bf16lo(a)), fabsf(bf16hi(a)))), fmaxf(fabsf(bf16lo(b)), fabsf(bf16hi(b))));
             }
             amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
             amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
             uint32_t eb = (__float_as_uint(amax) >> 23) & 0xffu;
             eb = eb < 1u ? 1u : (eb > 253u ? 253u : eb);
-            const float down = __uint_as_float((254u - eb) << 23), up = __uint_as_float(eb << 23);
-#pragma unroll
-            for (int ks = 0; ks < C::kKSteps; ++ks) {
-                qb[ks][0] = pack_f16x2(bf16lo(qb[ks][0]) * down, bf16hi(qb[ks][0]) * down);
-                qb[ks][1] = pack_f16x2(bf16lo(qb[ks][1]) * down, bf16hi(qb[ks][1]) * down);
-            }
-            const float hmul = g8 < G ? scale * up * __ldg(p.k_scale + sg.g) : 0.f;
+            down = __uint_as_float((254u - eb) << 23);
+            const float hmul = g8 < G ? scale * __uint_as_float(eb << 23) * __ldg(p.k_scale + sg.g) : 0.f;
             smul[0] = __shfl_sync(0xffffffffu, hmul, 8 * t4);
             smul[1] = __shfl_sync(0xffffffffu, hmul, 8 * t4 + 4);
             vscale = __ldg(p.v_scale + sg.g);
+        }
+        auto fragment = [&](int ks) {
+            uint2 f;
+            f.x = g8 < G ? __ldg(qrow + ks * 8 + w0) : 0u;
+            f.y = g8 < G ? __ldg(qrow + ks * 8 + w1) : 0u;
+            if constexpr (F8) {
+                f.x = pack_f16x2(bf16lo(f.x) * down, bf16hi(f.x) * down);
+                f.y = pack_f16x2(bf16lo(f.y) * down, bf16hi(f.y) * down);
+            }
+            return f;
+        };
+        if constexpr (C::kQShared) {
+            group_barrier(grp);                          // no warp of the group still reads the previous segment's fragments
+            for (int ks = warp; ks < C::kKSteps; ks += kGroupWarps) q_sm[ks * 32] = fragment(ks);
+            group_barrier(grp);
+        } else {
+#pragma unroll
+            for (int ks = 0; ks < C::kKSteps; ++ks) {
+                const uint2 f = fragment(ks);
+                qb[ks][0] = f.x; qb[ks][1] = f.y;
+            }
         }
         m[0] = m[1] = -INFINITY; l[0] = l[1] = 0.f; le[0] = le[1] = 0.f;
 #pragma unroll
@@ -1026,8 +1077,11 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         uint32_t a[4];
                         const uint32_t c16 = (uint32_t)((ks & 3) * 2 + halfK);
                         ldmatrix_x4(a, sK + (ks >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
-                        if (ks & 1) mma_bf16(sb, a, qb[ks][0], qb[ks][1]);
-                        else mma_bf16(sa, a, qb[ks][0], qb[ks][1]);
+                        uint32_t q0, q1;
+                        if constexpr (C::kQShared) { const uint2 f = q_sm[ks * 32]; q0 = f.x; q1 = f.y; }
+                        else { q0 = qb[ks][0]; q1 = qb[ks][1]; }
+                        if (ks & 1) mma_bf16(sb, a, q0, q1);
+                        else mma_bf16(sa, a, q0, q1);
                     }
                 } else {
                     // one ldmatrix brings 32 columns of d for the warp's 16 keys: matrices {keys 0-7, 8-15} x {16 d, next 16 d};
@@ -1040,10 +1094,13 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         ldmatrix_x4(r, sK + (j >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
                         a[0] = e4m3x2_to_f16x2(r[0]); a[1] = e4m3x2_to_f16x2(r[1]);
                         a[2] = e4m3x2_to_f16x2(r[0] >> 16); a[3] = e4m3x2_to_f16x2(r[1] >> 16);
-                        mma_f16(sa, a, qb[2 * j][0], qb[2 * j][1]);
+                        uint2 qa, qc;
+                        if constexpr (C::kQShared) { qa = q_sm[(2 * j) * 32]; qc = q_sm[(2 * j + 1) * 32]; }
+                        else { qa = make_uint2(qb[2 * j][0], qb[2 * j][1]); qc = make_uint2(qb[2 * j + 1][0], qb[2 * j + 1][1]); }
+                        mma_f16(sa, a, qa.x, qa.y);
                         a[0] = e4m3x2_to_f16x2(r[2]); a[1] = e4m3x2_to_f16x2(r[3]);
                         a[2] = e4m3x2_to_f16x2(r[2] >> 16); a[3] = e4m3x2_to_f16x2(r[3] >> 16);
-                        mma_f16(sb, a, qb[2 * j + 1][0], qb[2 * j + 1][1]);
+                        mma_f16(sb, a, qc.x, qc.y);
                     }
                 }
                 float sc[4];
@@ -1225,7 +1282,7 @@ template <int D, bool F8>
 size_t partial_smem_bytes(int B) {
     using C = Cfg<D, F8>;
     return 1024 + (size_t)C::kStages * C::kStageBytes +
-           sizeof(float) * C::kGroups * (kScratchFloats + 3 * kGroupWarps * kMaxGroup) +
+           sizeof(float) * C::kGroups * (kScratchFloats + 3 * kGroupWarps * kMaxGroup) + C::kQBytes +
            sizeof(uint64_t) * C::kBarriers + sizeof(int64_t) * C::kStages + sizeof(int64_t) * C::kGroups * 2 * kMaxContrib +
            (sizeof(int64_t) + sizeof(int)) * (B + 1) + sizeof(int) * (C::kGroups * kGroupInts + 4) + 16;
 }
