@@ -45,14 +45,18 @@ constexpr int kGroupThreads = kGroupWarps * 32;
 constexpr int kMaxGroups = 2;
 constexpr int kMaxParts = kMaxGroups * kMaxCtas; // partials one segment can receive
 constexpr uint32_t kSpinLimit = 1u << 22;       // bounded waits
-constexpr int kScratchRow = 132;                // floats per (warp, head) row of the merge scratch (128 + pad)
-// per-group scratch: either the warp merge ([4][8][kScratchRow]) or the combine's weights, inverses, ranks and reduction buffer
-constexpr int kCombineFloats = kMaxGroup * kMaxParts + 8 + 4 * kGroupThreads + kMaxParts;
-constexpr int kMergeFloats = kGroupWarps * kMaxGroup * kScratchRow;
-constexpr int kScratchFloats = kMergeFloats > kCombineFloats ? kMergeFloats : kCombineFloats;
+// Per-group scratch, used for two things in turn:
+//   the warp merge of a flush: [4 warps][8 heads][pass columns + 4] floats, `pass columns` of d at a time;
+//   the combine: weights [heads of this contributor's slice][np], inverses [8], a reduction buffer [128] float4 and the
+//   visiting order [np]. A contributor's slice of the (head, d) columns spans at most two heads once there are at least
+//   G contributors, and fewer than G * G (head, partial) pairs otherwise: 2 * kMaxParts weights always suffice.
+constexpr int kCombineWeights = 2 * kMaxParts;
+constexpr int kCombineFloats = kCombineWeights + 8 + 4 * kGroupThreads + kMaxParts;
+static_assert(kMaxGroup * kMaxGroup <= kCombineWeights, "weights of a slice must fit");
 constexpr int kMaxContrib = 32;     // segments a group may have outstanding before it combines them
-constexpr int kStealChunk = 2;      // tiles handed out per cursor step
-constexpr int kStealMinTiles = 16;  // ranges shorter than this are streamed statically
+#ifndef WMTP_CHUNK_BYTES
+#define WMTP_CHUNK_BYTES 262144
+#endif
 // per-group bookkeeping in shared memory (ints): [0] launch-last flag, [1] broadcast word, then
 // contrib[kMaxContrib][4] = {seg, b, g, slot}, reg_k[kMaxContrib] (slot of the group's i-th contribution, producer -> group)
 constexpr int kGroupInts = 4 + 5 * kMaxContrib;
@@ -70,8 +74,20 @@ struct Cfg {
 #define WMTP_F8_GROUPS_256 2
 #endif
     static constexpr int kGroups = (kStageBytes >= 65536) ? 1 : ((F8 && D == 256) ? WMTP_F8_GROUPS_256 : 2);
-    static constexpr int kStages = (kStageBytes >= 65536) ? 3 : (kStageBytes >= 32768 ? 5 : 8);
+    // Stages of the shared-memory ring. What counts for the streaming rate is the bytes a CTA keeps in flight (about
+    // 190 KB per SM saturate HBM at the loaded latency of ~4 us): the host takes as many stages as fit beside the
+    // batch-dependent tables, up to kMaxStages, in multiples of the group count (a stage then always serves one group).
+    static constexpr int kMaxStages = (kStageBytes >= 65536) ? 3 : (kStageBytes >= 32768 ? 6 : 12);
     static constexpr int kRowVecs = D * kElemBytes / 16;      // 16-byte vectors per stored row
+    // Tiles handed out per cursor step. A step costs a global atomic (about 1.5 us) that is fetched one chunk ahead: the
+    // chunk must take longer than that to stream, so it is sized in bytes (256 KB), not in tiles.
+    static constexpr int kStealChunk = WMTP_CHUNK_BYTES / kStageBytes;
+    static constexpr int kStealMinTiles = 8 * kStealChunk;   // ranges shorter than this are streamed statically
+    // columns of d merged per pass of a flush: the two-group configurations trade a second pass for shared memory
+    static constexpr int kPassCols = (kGroups == 2) ? 64 : 128;
+    static constexpr int kScratchRow = kPassCols + 4;
+    static constexpr int kMergeFloats = kGroupWarps * kMaxGroup * kScratchRow;
+    static constexpr int kScratchFloats = kMergeFloats > kCombineFloats ? kMergeFloats : kCombineFloats;
     // With two groups the CTA has 9 warps and a thread at most 168 registers: the query fragments (the same in all four
     // warps of a group) then live in shared memory, one copy per group, instead of D / 8 registers per thread.
     static constexpr bool kQShared = (kGroups == 2);
@@ -95,10 +111,8 @@ struct Cfg {
     static_assert(8 * kRegsConsumer + 4 * kRegsProducer <= 12 * 168, "register trade must balance");
     static constexpr int kThreads = (kConsumerWarps + 1 + kPadWarps) * 32;
     static constexpr int kKSteps = D / 16;
-    static constexpr int kBarriers = (1 + 2 * kGroups) * kStages;
-    // iterations between two uses of the same stage by the same group: lcm(kStages, kGroups)
-    static constexpr int kUsePeriod = (kStages % kGroups == 0) ? kStages : kStages * kGroups;
-    static_assert(kGroups == 1 || kGroups == 2, "kUsePeriod assumes one or two groups");
+    static constexpr int kBarriers = (1 + 2 * kGroups) * kMaxStages;
+    static_assert(kMaxStages % kGroups == 0, "a stage must always serve the same group");
 };
 
 // Development aid (compiled out unless WMTP_TRACE is defined): CTA 0 records %globaltimer at phase boundaries
@@ -325,8 +339,8 @@ __device__ __forceinline__ int64_t kv_row_offset(const AttnParams& p, int b, int
 __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, int64_t pbase, int np, int j, float* scratch,
                                              int tid, int grp) {
     const int G = p.G, D = p.D;
-    float* w_sm = scratch;                                                  // [G][np], np <= kMaxParts
-    float* inv_sm = scratch + kMaxGroup * kMaxParts;                        // [8]
+    float* w_sm = scratch;                                                  // [heads of the slice][np]
+    float* inv_sm = scratch + kCombineWeights;                              // [8], indexed by head - first head of the slice
     float4* red = reinterpret_cast<float4*>(inv_sm + 8);                    // [128]
     int* perm = reinterpret_cast<int*>(inv_sm + 8 + 4 * kGroupThreads);     // [np] visiting order
     WMTP_STAMP(p, 7);
@@ -352,6 +366,8 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
     const int vec = D / 4, cols = G * vec;
     const int cpc = (cols + np - 1) / np;
     const int col_lo = j * cpc, col_hi = col_lo + cpc < cols ? col_lo + cpc : cols;
+    const int h_lo = col_lo < cols ? col_lo / vec : 0;                      // heads the slice touches: [h_lo, h_lo + nh)
+    const int nh = col_lo < col_hi ? (col_hi - 1) / vec - h_lo + 1 : 0;
     const float4* rows = reinterpret_cast<const float4*>(p.part_o);
     float4 pre[kPre];
     {
@@ -365,16 +381,18 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
             }
         }
     }
-    // ---- weights, all heads at once: 16 threads per head, one pass over the partial lse values
+    // ---- weights of the slice's heads, all at once: 16 threads per head, one pass over the partial lse values.
+    //      The contributor whose slice holds a head's first column also writes the head's lse.
     {
-        const int h = tid >> 4, li = tid & 15;
+        const int hh = tid >> 4, h = h_lo + hh, li = tid & 15;
+        const bool act = hh < nh;
         constexpr int kPer = (kMaxParts + 15) / 16;
         float x[kPer];
         float M = -INFINITY;
 #pragma unroll
         for (int u = 0; u < kPer; ++u) {
             const int i = li + 16 * u;
-            x[u] = (h < G && i < np) ? __ldcg(p.part_lse + (pbase + perm[i]) * G + h) : -INFINITY;
+            x[u] = (act && i < np) ? __ldcg(p.part_lse + (pbase + perm[i]) * G + h) : -INFINITY;
             M = fmaxf(M, x[u]);
         }
 #pragma unroll
@@ -383,17 +401,17 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
 #pragma unroll
         for (int u = 0; u < kPer; ++u) {
             const int i = li + 16 * u;
-            if (h < G && i < np) {
+            if (act && i < np) {
                 const float w = (M > -INFINITY) ? __expf(x[u] - M) : 0.f;
-                w_sm[h * np + i] = w;
+                w_sm[hh * np + i] = w;
                 sum += w;
             }
         }
 #pragma unroll
         for (int off = 8; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-        if (li == 0 && h < G) {
-            inv_sm[h] = sum > 0.f ? 1.f / sum : 0.f;
-            if (j == 0 && p.lse) p.lse[(int64_t)b * p.Hq + g * G + h] = sum > 0.f ? M + __logf(sum) : -INFINITY;
+        if (li == 0 && act) {
+            inv_sm[hh] = sum > 0.f ? 1.f / sum : 0.f;
+            if (p.lse && col_lo <= h * vec) p.lse[(int64_t)b * p.Hq + g * G + h] = sum > 0.f ? M + __logf(sum) : -INFINITY;
         }
     }
     group_barrier(grp);
@@ -404,7 +422,7 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
         const int R = kGroupThreads / cb, cl = tid % cb, rg = tid / cb;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (rg < R) {
-            const int col = c0 + cl, h = col / vec;
+            const int col = c0 + cl, h = col / vec - h_lo;
             int i = rg;
             if (c0 == col_lo) {
 #pragma unroll
@@ -432,7 +450,7 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
                 o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
             }
             const int col = c0 + tid;
-            const float inv = inv_sm[col / vec];
+            const float inv = inv_sm[col / vec - h_lo];
             uint2 packed;
             packed.x = pack_bf16x2(o.x * inv, o.y * inv);
             packed.y = pack_bf16x2(o.z * inv, o.w * inv);
@@ -468,16 +486,17 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     using C = Cfg<D, F8>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    unsigned char* stages = smem;                                                         // kStages x (K tile, V tile)
-    float* scratch_all = reinterpret_cast<float*>(stages + C::kStages * C::kStageBytes);  // [kGroups][kScratchFloats]
-    float* sm_stats = scratch_all + C::kGroups * kScratchFloats;                          // [kGroups][3][4][8]: m, l, le per warp and head
+    const uint32_t nst = (uint32_t)p.stages;                                              // stages in use (<= kMaxStages)
+    unsigned char* stages = smem;                                                         // nst x (K tile, V tile)
+    float* scratch_all = reinterpret_cast<float*>(stages + nst * C::kStageBytes);         // [kGroups][kScratchFloats]
+    float* sm_stats = scratch_all + C::kGroups * C::kScratchFloats;                          // [kGroups][3][4][8]: m, l, le per warp and head
     // Barriers: empty[stage] (the producer observes every use of a stage) and, per consumer group, fullK / fullV[stage].
     // A group only sees the uses of a stage that are its own, and a parity wait can only tell consecutive phases
     // apart, so the "full" barriers must not be shared between groups.
     uint2* q_sm_all = reinterpret_cast<uint2*>(sm_stats + C::kGroups * 3 * kGroupWarps * kMaxGroup);   // [kGroups][kKSteps][32] (kQShared)
     uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(q_sm_all) + C::kQBytes);
-    int64_t* stage_tile = reinterpret_cast<int64_t*>(bars + C::kBarriers);                // [kStages] global tile index, -1 = end
-    int64_t* contrib_base_all = stage_tile + C::kStages;                                  // [kGroups][2][kMaxContrib]
+    int64_t* stage_tile = reinterpret_cast<int64_t*>(bars + C::kBarriers);                // [kMaxStages] global tile index, -1 = end
+    int64_t* contrib_base_all = stage_tile + C::kMaxStages;                               // [kGroups][2][kMaxContrib]
     int64_t* tile_prefix = contrib_base_all + C::kGroups * 2 * kMaxContrib;               // [B + 1]
     int* cap_prefix = reinterpret_cast<int*>(tile_prefix + (p.B + 1));                    // [B + 1]
     int* group_ints = cap_prefix + (p.B + 1);                                             // [kGroups][kGroupInts]
@@ -491,13 +510,13 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         asm volatile("prefetch.tensormap [%0];" ::"l"(&mapV) : "memory");
     }
     const int lane = threadIdx.x & 31;
-    const uint32_t bar_empty = smem_u32(bars), bar_fullK0 = smem_u32(bars + C::kStages), bar_fullV0 = smem_u32(bars + (1 + C::kGroups) * C::kStages);
+    const uint32_t bar_empty = smem_u32(bars), bar_fullK0 = smem_u32(bars + C::kMaxStages), bar_fullV0 = smem_u32(bars + (1 + C::kGroups) * C::kMaxStages);
     if (threadIdx.x == 0) {                                  // under the shadow of the len[] round trip
-        for (int s = 0; s < C::kStages; ++s) {
+        for (int s = 0; s < C::kMaxStages; ++s) {
             mbar_init(bar_empty + 8 * s, kGroupWarps);
             for (int q = 0; q < C::kGroups; ++q) {
-                mbar_init(bar_fullK0 + 8 * (q * C::kStages + s), 1);
-                mbar_init(bar_fullV0 + 8 * (q * C::kStages + s), 1);
+                mbar_init(bar_fullK0 + 8 * (q * C::kMaxStages + s), 1);
+                mbar_init(bar_fullV0 + 8 * (q * C::kMaxStages + s), 1);
             }
         }
         cta_flags[0] = 0;
@@ -567,7 +586,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         // and, once they run dry, to other CTAs: SMs do not all stream at the same rate, and the slowest one
         // would otherwise set the launch time. A thief prefers a victim inside the segment it is already in
         // (no new partial); moving into another segment is admitted steal_slots times per segment.
-        // Tile number `it` of this CTA goes to stage it % kStages and to consumer group it % kGroups.
+        // Tile number `it` of this CTA goes to stage it % nst (kept incrementally: ps, with the parity pph of the
+        // stage's use count) and to consumer group it % kGroups.
         const uint32_t stage0 = smem_u32(stages);
         uint64_t policy = 0;
 #if WMTP_TMA_HINT == 1
@@ -576,7 +596,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
 #endif
         (void)policy;
-        uint32_t it = 0;
+        uint32_t it = 0, ps = 0, pph = 0;
         int cur_seg = -1;                    // segment of the last issued tile
         int64_t cur_lo = 0, cur_hi = 0;      // its tile range
         int grp_seg[kMaxGroups], grp_ord[kMaxGroups], pend_k[kMaxGroups];
@@ -613,7 +633,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         }
                     }
                     const int cnt = ntiles - base < 32 ? ntiles - base : 32;
-                    for (int j = 0; j < cnt; ++j, ++it) {
+                    for (int j = 0; j < cnt; ++j, ++it, ps = (ps + 1 == nst ? 0 : ps + 1), pph ^= (ps == 0)) {
                         const int pg = __shfl_sync(0xffffffffu, page, j);
                         const int gq = (int)(it % C::kGroups);
                         settle(gq);
@@ -625,8 +645,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                             ++grp_ord[gq];
                         }
                         if (lane == 0) {
-                            const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
-                            const uint32_t bar_fullK = bar_fullK0 + 8 * (gq * C::kStages), bar_fullV = bar_fullV0 + 8 * (gq * C::kStages);
+                            const uint32_t s = ps, ph = pph;
+                            const uint32_t bar_fullK = bar_fullK0 + 8 * (gq * C::kMaxStages), bar_fullV = bar_fullV0 + 8 * (gq * C::kMaxStages);
                             mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status);
                             if (!*abort_flag) {
                                 int64_t row;
@@ -665,12 +685,12 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         auto range_of = [&](int c, int64_t* lo, int64_t* len, int64_t* first) {
             *lo = cta_range_start(c, n, Cn);
             *len = cta_range_start(c + 1, n, Cn) - *lo;
-            *first = (!p.steal_slots_enabled || *len < kStealMinTiles) ? *len : *len - *len / 4;
+            *first = (!p.steal_slots_enabled || *len < C::kStealMinTiles) ? *len : *len - *len / 4;
         };
 
         // One loop, three sources of work in turn: the static part of the own range, the rest of the own range chunk
         // by chunk through the cursor (thieves may be taking from it too), then other CTAs' cursors.
-        const bool may_steal = p.steal_slots_enabled && n >= (int64_t)kStealMinTiles * Cn;
+        const bool may_steal = p.steal_slots_enabled && n >= (int64_t)C::kStealMinTiles * Cn;
         int phase = is_owner ? 0 : 2;
         int64_t own_lo = 0, own_len = 0, own_first = 0;
         int k_own = 0;                       // own cursor value for the next chunk (phase 1), fetched one chunk ahead
@@ -682,16 +702,16 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 a = own_lo; e = own_lo + own_first;
                 phase = 1;
                 if (own_len > own_first) {
-                    if (lane == 0) k_own = atomicAdd(p.cur + blockIdx.x, kStealChunk);
+                    if (lane == 0) k_own = atomicAdd(p.cur + blockIdx.x, C::kStealChunk);
                 } else {
                     k_own = 0x7fffffff;
                 }
             } else if (phase == 1) {
                 const int k = __shfl_sync(0xffffffffu, k_own, 0);
                 if (k >= own_len - own_first) { phase = 2; continue; }
-                if (lane == 0) k_own = atomicAdd(p.cur + blockIdx.x, kStealChunk);     // overlaps the issue below
+                if (lane == 0) k_own = atomicAdd(p.cur + blockIdx.x, C::kStealChunk);     // overlaps the issue below
                 a = own_lo + own_first + k;
-                e = a + kStealChunk < own_lo + own_len ? a + kStealChunk : own_lo + own_len;
+                e = a + C::kStealChunk < own_lo + own_len ? a + C::kStealChunk : own_lo + own_len;
             } else {
                 if (!may_steal || *abort_flag) break;
                 // ---- steal: look at every cursor, take from the range with the most left
@@ -740,8 +760,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                             }
                         }
                         int64_t take = rem / 8;            // larger bites while much is left: a steal costs two round trips
-                        if (take < kStealChunk) take = kStealChunk;
-                        if (take > 8) take = 8;
+                        if (take < C::kStealChunk) take = C::kStealChunk;
+                        if (take > 4 * C::kStealChunk) take = 4 * C::kStealChunk;
                         if (take > rem) take = rem;
                         if (tv + take > ahi) take = ahi - tv;
                         const int prev = atomicCAS(p.cur + best_v, used, used + (int)take);
@@ -761,13 +781,13 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         for (int q = 0; q < C::kGroups; ++q) settle(q);
         if (lane == 0) {
             // one end marker per consumer group, then: this CTA takes no more tiles
-            for (int q = 0; q < C::kGroups; ++q, ++it) {
-                const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+            for (int q = 0; q < C::kGroups; ++q, ++it, ps = (ps + 1 == nst ? 0 : ps + 1), pph ^= (ps == 0)) {
+                const uint32_t s = ps, ph = pph;
                 const uint32_t gq = it % C::kGroups;
                 mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status);
                 stage_tile[s] = -1;
-                mbar_arrive(bar_fullK0 + 8 * (gq * C::kStages + s));
-                mbar_arrive(bar_fullV0 + 8 * (gq * C::kStages + s));
+                mbar_arrive(bar_fullK0 + 8 * (gq * C::kMaxStages + s));
+                mbar_arrive(bar_fullV0 + 8 * (gq * C::kMaxStages + s));
             }
             atomicAdd(p.grab_done, 1);
         }
@@ -781,7 +801,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     // ===================================== consumer groups =====================================
     const int grp = threadIdx.x / kGroupThreads, tid = threadIdx.x % kGroupThreads;   // group, thread within the group
     const int warp = tid >> 5;                           // warp within the group: owns keys [16 warp, 16 warp + 16) of a tile
-    float* scratch = scratch_all + grp * kScratchFloats;
+    float* scratch = scratch_all + grp * C::kScratchFloats;
     float* sm_m = sm_stats + grp * 3 * kGroupWarps * kMaxGroup;
     float* sm_l = sm_m + kGroupWarps * kMaxGroup;
     float* sm_le = sm_l + kGroupWarps * kMaxGroup;
@@ -798,7 +818,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     const int rowV = warp * 16 + (mi >> 1) * 8 + rr, halfV = mi & 1;       // V as A operand (transposed load)
     const uint32_t offK = rowK * 128, offV = rowV * 128;
     const uint32_t stage0 = smem_u32(stages);
-    const uint32_t bar_fullK = bar_fullK0 + 8 * (grp * C::kStages), bar_fullV = bar_fullV0 + 8 * (grp * C::kStages);
+    const uint32_t bar_fullK = bar_fullK0 + 8 * (grp * C::kMaxStages), bar_fullV = bar_fullV0 + 8 * (grp * C::kMaxStages);
 
     int nonempty_segs = 0;                               // group thread 0 only
     if (tid == 0)
@@ -890,13 +910,14 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             f[i] = (L > 0.f && m[i] > -INFINITY) ? exp2f(m[i] - M) / L * vscale : 0.f;
             if (warp == 0 && g8 == 0 && h < G) p.part_lse[pidx * G + h] = Le > 0.f ? (M + log2f(Le)) * kLn2 : -INFINITY;
         }
-        constexpr int kPasses = D / 128;                       // 128 columns of d per pass through the scratch
+        constexpr int kPasses = D / C::kPassCols;               // kPassCols columns of d per pass through the scratch
+        constexpr int kScratchRow = C::kScratchRow;
 #pragma unroll
         for (int pass = 0; pass < kPasses; ++pass) {
             if (pass > 0) group_barrier(grp);
 #pragma unroll
-            for (int mbl = 0; mbl < 8; ++mbl) {
-                const int mb = pass * 8 + mbl;
+            for (int mbl = 0; mbl < C::kPassCols / 16; ++mbl) {
+                const int mb = pass * (C::kPassCols / 16) + mbl;
                 // accumulator rows g8 and g8 + 8 of block mb hold d = 16 mb + g8 and + 8 (bf16 store), or, for an fp8
                 // store whose V fragments come out of the transposed load with d pairs interleaved, d = 16 mb + 2 g8 and + 1
                 float* row0 = scratch + (warp * kMaxGroup + 2 * t4) * kScratchRow + mbl * 16 + (F8 ? 2 * g8 : g8);
@@ -906,12 +927,12 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 row0[kSecond] = o[mb][2] * f[0]; row1[kSecond] = o[mb][3] * f[1];
             }
             group_barrier(grp);
-            for (int idx = tid; idx < G * 128; idx += kGroupThreads) {
-                const int h = idx >> 7, dd = idx & 127;
+            for (int idx = tid; idx < G * C::kPassCols; idx += kGroupThreads) {
+                const int h = idx / C::kPassCols, dd = idx % C::kPassCols;
                 float acc = 0.f;
 #pragma unroll
                 for (int w = 0; w < kGroupWarps; ++w) acc += scratch[(w * kMaxGroup + h) * kScratchRow + dd];
-                p.part_o[(pidx * G + h) * D + pass * 128 + dd] = acc;
+                p.part_o[(pidx * G + h) * D + pass * C::kPassCols + dd] = acc;
             }
         }
         group_barrier(grp);
@@ -1010,10 +1031,10 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         const int64_t first = cta_range_start(blockIdx.x, n, Cn) + grp;
         if (first < cta_range_start(blockIdx.x + 1, n, Cn)) { tt = first; need_enter = true; }
     }
-    uint32_t it = grp;
+    uint32_t it = grp, cs = grp, cph = 0;
     for (;;) {
         if (need_enter) { enter_segment(tt); need_enter = false; }
-        const uint32_t s = it % C::kStages, ph = (it / C::kUsePeriod) & 1u;   // this group's uses of stage s are kUsePeriod iterations apart
+        const uint32_t s = cs, ph = cph;             // stage of tile `it` and the parity of this group's use count of it
         if (!have_tile) {
             mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
             if (it == 0) { WMTP_STAMP(p, 3); WMTP_CTA_STAMP(p, 1); }
@@ -1209,6 +1230,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             if (lane == 0) mbar_arrive(bar_empty + 8 * s);
         }
         it += C::kGroups;
+        cs += C::kGroups;                            // nst is a multiple of kGroups: the stage stays with this group
+        if (cs >= nst) { cs -= nst; cph ^= 1u; }
     }
     WMTP_STAMP(p, 9);
 
@@ -1279,17 +1302,21 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int D, int esz) 
 }
 
 template <int D, bool F8>
-size_t partial_smem_bytes(int B) {
+size_t partial_smem_bytes(int B, int stages) {
     using C = Cfg<D, F8>;
-    return 1024 + (size_t)C::kStages * C::kStageBytes +
-           sizeof(float) * C::kGroups * (kScratchFloats + 3 * kGroupWarps * kMaxGroup) + C::kQBytes +
-           sizeof(uint64_t) * C::kBarriers + sizeof(int64_t) * C::kStages + sizeof(int64_t) * C::kGroups * 2 * kMaxContrib +
+    return 1024 + (size_t)stages * C::kStageBytes +
+           sizeof(float) * C::kGroups * (C::kScratchFloats + 3 * kGroupWarps * kMaxGroup) + C::kQBytes +
+           sizeof(uint64_t) * C::kBarriers + sizeof(int64_t) * C::kMaxStages + sizeof(int64_t) * C::kGroups * 2 * kMaxContrib +
            (sizeof(int64_t) + sizeof(int)) * (B + 1) + sizeof(int) * (C::kGroups * kGroupInts + 4) + 16;
 }
 
 template <int D, bool F8>
 cudaError_t launch_fused(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaStream_t st) {
-    const size_t smem = partial_smem_bytes<D, F8>(p.B);
+    using C = Cfg<D, F8>;
+    int stages = C::kMaxStages;                                  // as many as fit beside the batch-dependent tables
+    while (stages > C::kGroups && partial_smem_bytes<D, F8>(p.B, stages) > 227 * 1024) stages -= C::kGroups;
+    p.stages = stages;
+    const size_t smem = partial_smem_bytes<D, F8>(p.B, stages);
     static bool attr_set[64] = {};          // per device: the opt-in to > 48 KB of dynamic shared memory
     int dev = 0;
     cudaGetDevice(&dev);

@@ -81,6 +81,7 @@ struct AttnParams {
     int window_view;          // contiguous / paged only: attend over the first n_sink and the last W positions of the KV store
     float scale_log2;         // sm_scale * log2(e)
     int num_ctas;
+    int stages;               // stages of the kernel's shared-memory ring (set by the launcher)
 };
 
 struct RingParams {
