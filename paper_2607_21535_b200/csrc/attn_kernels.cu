@@ -112,6 +112,11 @@ struct Cfg {
     static constexpr int kThreads = (kConsumerWarps + 1 + kPadWarps) * 32;
     static constexpr int kKSteps = D / 16;
     static constexpr int kBarriers = (1 + 2 * kGroups) * kMaxStages;
+    // bytes of the fixed-size part of shared memory (scratch, softmax statistics, query fragments, barriers, stage tags,
+    // contribution lists, per-group words, flags), rounded up to the stage ring's alignment
+    static constexpr int kFixedRaw = 4 * kGroups * (kScratchFloats + 3 * kGroupWarps * kMaxGroup) + kQBytes + 8 * kBarriers +
+                                     8 * kMaxStages + 8 * kGroups * 2 * kMaxContrib + 4 * kGroups * kGroupInts + 16;
+    static constexpr int kFixedBytes = (kFixedRaw + 1023) / 1024 * 1024;
     static_assert(kMaxStages % kGroups == 0, "a stage must always serve the same group");
 };
 
@@ -340,7 +345,11 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
                                              int tid, int grp) {
     const int G = p.G, D = p.D;
     float* w_sm = scratch;                                                  // [heads of the slice][np]
+#ifdef WMTP_COMBINE_ALL
+    float* inv_sm = scratch + kMaxGroup * kMaxParts;
+#else
     float* inv_sm = scratch + kCombineWeights;                              // [8], indexed by head - first head of the slice
+#endif
     float4* red = reinterpret_cast<float4*>(inv_sm + 8);                    // [128]
     int* perm = reinterpret_cast<int*>(inv_sm + 8 + 4 * kGroupThreads);     // [np] visiting order
     WMTP_STAMP(p, 7);
@@ -366,8 +375,13 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
     const int vec = D / 4, cols = G * vec;
     const int cpc = (cols + np - 1) / np;
     const int col_lo = j * cpc, col_hi = col_lo + cpc < cols ? col_lo + cpc : cols;
-    const int h_lo = col_lo < cols ? col_lo / vec : 0;                      // heads the slice touches: [h_lo, h_lo + nh)
-    const int nh = col_lo < col_hi ? (col_hi - 1) / vec - h_lo + 1 : 0;
+#ifdef WMTP_COMBINE_ALL
+    const int h_lo = 0, nh = G;
+#else
+    const int vsh = D == 256 ? 6 : 5;                                       // vec = D / 4 is a power of two: log2(vec)
+    const int h_lo = col_lo < cols ? col_lo >> vsh : 0;                     // heads the slice touches: [h_lo, h_lo + nh)
+    const int nh = col_lo < col_hi ? ((col_hi - 1) >> vsh) - h_lo + 1 : 0;
+#endif
     const float4* rows = reinterpret_cast<const float4*>(p.part_o);
     float4 pre[kPre];
     {
@@ -411,7 +425,7 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
         for (int off = 8; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
         if (li == 0 && act) {
             inv_sm[hh] = sum > 0.f ? 1.f / sum : 0.f;
-            if (p.lse && col_lo <= h * vec) p.lse[(int64_t)b * p.Hq + g * G + h] = sum > 0.f ? M + __logf(sum) : -INFINITY;
+            if (p.lse && col_lo <= (h << vsh)) p.lse[(int64_t)b * p.Hq + g * G + h] = sum > 0.f ? M + __logf(sum) : -INFINITY;
         }
     }
     group_barrier(grp);
@@ -422,7 +436,7 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
         const int R = kGroupThreads / cb, cl = tid % cb, rg = tid / cb;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (rg < R) {
-            const int col = c0 + cl, h = col / vec - h_lo;
+            const int col = c0 + cl, h = (col >> vsh) - h_lo;
             int i = rg;
             if (c0 == col_lo) {
 #pragma unroll
@@ -450,7 +464,7 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
                 o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
             }
             const int col = c0 + tid;
-            const float inv = inv_sm[col / vec - h_lo];
+            const float inv = inv_sm[(col >> vsh) - h_lo];
             uint2 packed;
             packed.x = pack_bf16x2(o.x * inv, o.y * inv);
             packed.y = pack_bf16x2(o.z * inv, o.w * inv);
@@ -486,21 +500,23 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     using C = Cfg<D, F8>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const uint32_t nst = (uint32_t)p.stages;                                              // stages in use (<= kMaxStages)
-    unsigned char* stages = smem;                                                         // nst x (K tile, V tile)
-    float* scratch_all = reinterpret_cast<float*>(stages + nst * C::kStageBytes);         // [kGroups][kScratchFloats]
-    float* sm_stats = scratch_all + C::kGroups * C::kScratchFloats;                          // [kGroups][3][4][8]: m, l, le per warp and head
+    // Shared memory: the fixed-size part first (compile-time offsets), then the stage ring (1024-byte aligned for the
+    // 128-byte swizzle, as many stages as the launcher found room for), then the batch-sized tables.
+    float* scratch_all = reinterpret_cast<float*>(smem);                                  // [kGroups][kScratchFloats]
+    float* sm_stats = scratch_all + C::kGroups * C::kScratchFloats;                       // [kGroups][3][4][8]: m, l, le per warp and head
+    uint2* q_sm_all = reinterpret_cast<uint2*>(sm_stats + C::kGroups * 3 * kGroupWarps * kMaxGroup);   // [kGroups][kKSteps][32] (kQShared)
     // Barriers: empty[stage] (the producer observes every use of a stage) and, per consumer group, fullK / fullV[stage].
     // A group only sees the uses of a stage that are its own, and a parity wait can only tell consecutive phases
     // apart, so the "full" barriers must not be shared between groups.
-    uint2* q_sm_all = reinterpret_cast<uint2*>(sm_stats + C::kGroups * 3 * kGroupWarps * kMaxGroup);   // [kGroups][kKSteps][32] (kQShared)
     uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(q_sm_all) + C::kQBytes);
     int64_t* stage_tile = reinterpret_cast<int64_t*>(bars + C::kBarriers);                // [kMaxStages] global tile index, -1 = end
     int64_t* contrib_base_all = stage_tile + C::kMaxStages;                               // [kGroups][2][kMaxContrib]
-    int64_t* tile_prefix = contrib_base_all + C::kGroups * 2 * kMaxContrib;               // [B + 1]
-    int* cap_prefix = reinterpret_cast<int*>(tile_prefix + (p.B + 1));                    // [B + 1]
-    int* group_ints = cap_prefix + (p.B + 1);                                             // [kGroups][kGroupInts]
+    int* group_ints = reinterpret_cast<int*>(contrib_base_all + C::kGroups * 2 * kMaxContrib);   // [kGroups][kGroupInts]
     int* cta_flags = group_ints + C::kGroups * kGroupInts;                                // [0] abort
+    unsigned char* stages = smem + C::kFixedBytes;                                        // nst x (K tile, V tile)
+    const uint32_t nst = (uint32_t)p.stages;                                              // stages in use (<= kMaxStages)
+    int64_t* tile_prefix = reinterpret_cast<int64_t*>(stages + nst * C::kStageBytes);     // [B + 1]
+    int* cap_prefix = reinterpret_cast<int*>(tile_prefix + (p.B + 1));                    // [B + 1]
     volatile int* abort_flag = cta_flags;
 
     WMTP_STAMP(p, 0);
@@ -1304,10 +1320,7 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int D, int esz) 
 template <int D, bool F8>
 size_t partial_smem_bytes(int B, int stages) {
     using C = Cfg<D, F8>;
-    return 1024 + (size_t)stages * C::kStageBytes +
-           sizeof(float) * C::kGroups * (C::kScratchFloats + 3 * kGroupWarps * kMaxGroup) + C::kQBytes +
-           sizeof(uint64_t) * C::kBarriers + sizeof(int64_t) * C::kMaxStages + sizeof(int64_t) * C::kGroups * 2 * kMaxContrib +
-           (sizeof(int64_t) + sizeof(int)) * (B + 1) + sizeof(int) * (C::kGroups * kGroupInts + 4) + 16;
+    return 1024 + (size_t)C::kFixedBytes + (size_t)stages * C::kStageBytes + (sizeof(int64_t) + sizeof(int)) * (B + 1) + 16;
 }
 
 template <int D, bool F8>
