@@ -229,11 +229,10 @@ __device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], u
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-// Two e4m3 codes (low byte first) -> two f16 values, exact.
-__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
-    uint32_t d;
-    asm("{\n\t.reg .b16 t;\n\tcvt.u16.u32 t, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, t;\n\t}" : "=r"(d) : "r"(x));
-    return d;
+// Four e4m3 codes -> f16 pairs (codes 0,1) and (codes 2,3).
+__device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t x, uint32_t& lo, uint32_t& hi) {
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.rn.f16x2.e4m3x2 %0, l;\n\tcvt.rn.f16x2.e4m3x2 %1, h;\n\t}"
+        : "=r"(lo), "=r"(hi) : "r"(x));
 }
 __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
     uint32_t d;
@@ -1129,14 +1128,14 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         uint32_t r[4], a[4];
                         const uint32_t c16 = (uint32_t)((j & 3) * 2 + halfK);
                         ldmatrix_x4(r, sK + (j >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
-                        a[0] = e4m3x2_to_f16x2(r[0]); a[1] = e4m3x2_to_f16x2(r[1]);
-                        a[2] = e4m3x2_to_f16x2(r[0] >> 16); a[3] = e4m3x2_to_f16x2(r[1] >> 16);
+                        e4m3x4_to_f16x2x2(r[0], a[0], a[2]);
+                        e4m3x4_to_f16x2x2(r[1], a[1], a[3]);
                         uint2 qa, qc;
                         if constexpr (C::kQShared) { qa = q_sm[(2 * j) * 32]; qc = q_sm[(2 * j + 1) * 32]; }
                         else { qa = make_uint2(qb[2 * j][0], qb[2 * j][1]); qc = make_uint2(qb[2 * j + 1][0], qb[2 * j + 1][1]); }
                         mma_f16(sa, a, qa.x, qa.y);
-                        a[0] = e4m3x2_to_f16x2(r[2]); a[1] = e4m3x2_to_f16x2(r[3]);
-                        a[2] = e4m3x2_to_f16x2(r[2] >> 16); a[3] = e4m3x2_to_f16x2(r[3] >> 16);
+                        e4m3x4_to_f16x2x2(r[2], a[0], a[2]);
+                        e4m3x4_to_f16x2x2(r[3], a[1], a[3]);
                         mma_f16(sb, a, qc.x, qc.y);
                     }
                 }
@@ -1179,9 +1178,12 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 }
                 pb0 = movmatrix_trans(pa);                           // P^T as B operand: k = key, n = head
                 pb1 = movmatrix_trans(pc);
+                // the running maxima rarely move after the first tiles of a segment: rescale only when some lane's did
+                if (__any_sync(0xffffffffu, corr0 != 1.f || corr1 != 1.f)) {
 #pragma unroll
-                for (int mb = 0; mb < C::kKSteps; ++mb) {
-                    o[mb][0] *= corr0; o[mb][1] *= corr1; o[mb][2] *= corr0; o[mb][3] *= corr1;
+                    for (int mb = 0; mb < C::kKSteps; ++mb) {
+                        o[mb][0] *= corr0; o[mb][1] *= corr1; o[mb][2] *= corr0; o[mb][3] *= corr1;
+                    }
                 }
             }
             mbar_wait(bar_fullV + 8 * s, ph, abort_flag, p.status);
@@ -1231,13 +1233,11 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         uint32_t r[4], a[4];
                         const uint32_t c16 = (uint32_t)((j & 3) * 2 + halfK);
                         ldmatrix_x4_trans(r, sV + (j >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
-                        uint32_t x = __byte_perm(r[0], 0, 0x3120), y = __byte_perm(r[1], 0, 0x3120);
-                        a[0] = e4m3x2_to_f16x2(x); a[1] = e4m3x2_to_f16x2(x >> 16);
-                        a[2] = e4m3x2_to_f16x2(y); a[3] = e4m3x2_to_f16x2(y >> 16);
+                        e4m3x4_to_f16x2x2(__byte_perm(r[0], 0, 0x3120), a[0], a[1]);
+                        e4m3x4_to_f16x2x2(__byte_perm(r[1], 0, 0x3120), a[2], a[3]);
                         mma_f16(o[2 * j], a, pb0, pb1);
-                        x = __byte_perm(r[2], 0, 0x3120); y = __byte_perm(r[3], 0, 0x3120);
-                        a[0] = e4m3x2_to_f16x2(x); a[1] = e4m3x2_to_f16x2(x >> 16);
-                        a[2] = e4m3x2_to_f16x2(y); a[3] = e4m3x2_to_f16x2(y >> 16);
+                        e4m3x4_to_f16x2x2(__byte_perm(r[2], 0, 0x3120), a[0], a[1]);
+                        e4m3x4_to_f16x2x2(__byte_perm(r[3], 0, 0x3120), a[2], a[3]);
                         mma_f16(o[2 * j + 1], a, pb0, pb1);
                     }
                 }
