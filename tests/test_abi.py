@@ -121,3 +121,18 @@ def test_extend_and_rollback_arguments_rejected_on_host():
     assert L.wmtp_kv_append_many(kb, 2, 4096, None, None, None) == 1
     assert L.wmtp_ring_rewind(rb, None, None, None) == 1
     assert L.wmtp_ring_rewind(ctypes.byref(_ring_desc(W=0)), 4096, None, None) == 1
+
+
+def test_kv_dtype_rejected_on_host():
+    L = wm.lib()
+    assert wm.wmtp_kv_elem_bytes(0) == 2 and wm.wmtp_kv_elem_bytes(1) == 1 and wm.wmtp_kv_elem_bytes(5) == 0
+    # an fp8 store without scales, or with misaligned ones
+    assert L.wmtp_ring_reset(ctypes.byref(_ring_desc(kv_dtype=1)), None) == 1
+    assert L.wmtp_ring_reset(ctypes.byref(_ring_desc(kv_dtype=1, k_scale=4096, v_scale=4098)), None) == 1
+    assert L.wmtp_kv_append(ctypes.byref(_kv_desc(kv_dtype=1, k_scale=4096)), 4096, 4096, None, None) == 1
+    # an unknown entry type
+    assert L.wmtp_ring_reset(ctypes.byref(_ring_desc(kv_dtype=2, k_scale=4096, v_scale=4096)), None) == 2
+    assert L.wmtp_draft_attn_full(4096, 16, ctypes.byref(_kv_desc(kv_dtype=9)), 0.0, 4096, None, 4096, 1 << 30, None) == 2
+    # rows are copied as stored: ring and KV store must agree
+    r8 = _ring_desc(kv_dtype=1, k_scale=4096, v_scale=4096)
+    assert L.wmtp_ring_init_from_kv(ctypes.byref(r8), ctypes.byref(_kv_desc()), None) == 1
