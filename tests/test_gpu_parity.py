@@ -266,6 +266,33 @@ def test_attention_mass_diagnostics_match_oracle():
     assert ((m > 0) & (m <= 1 + 1e-6)).all()
 
 
+@pytest.mark.parametrize("target", [0.78, 0.16])
+def test_attention_mass_on_structured_logit_profiles(target):
+    """Recency-peaked logits calibrated to the in-window mass of a locally peaked (RoPE-like, ~0.75-0.80) and of a
+    diffuse (NoPE-like, 0.16) head of the attention-mass table (Appendix D): the device diagnostics reproduce the
+    oracle's figures, and both land on the calibration target."""
+    S0, W, n_sink, tau = 200000, 4096, 4, 2048.0
+    delta = wi.calibrate_delta(S0 + 1, n_sink, W, tau, target)
+    cfg = _cfg(S0=S0, D=256, W=W, n_sink=n_sink, gamma=1, seed=61, logit_profile=(delta, tau), name=f"profile{target}")
+    wl = wi.make_workload(cfg)
+    dw = DeviceWorkload(wl)
+    dw.run_loops()
+    mass, perturb, tail = (torch.full((cfg.Hq,), float("nan"), device="cuda") for _ in range(3))
+    wm.wmtp_attn_mass_diagnostics(dw.out_w[0], dw.lse_w[0], dw.out_f[0], dw.lse_f[0], mass=mass, perturb=perturb, tail=tail)
+    orc = oracle_for(wl, 0, with_ring=False)
+    r = orc.step(wl.q[0, 0], wl.k_new[0, 0], wl.v_new[0, 0])
+    (ow, lw), (of, lf) = r["win"], r["full"]
+    compare(dw.out_w[0, 0], dw.lse_w[0, 0], ow, lw, what="profile windowed")
+    compare(dw.out_f[0, 0], dw.lse_f[0, 0], of, lf, what="profile full")
+    ref_mass = R.in_window_mass(lw, lf)
+    np.testing.assert_allclose(mass.cpu().numpy(), ref_mass, rtol=2e-3, atol=1e-6)
+    np.testing.assert_allclose(perturb.cpu().numpy(), R.win_perturb(of, ow), atol=2e-2, rtol=2e-2)
+    np.testing.assert_allclose(tail.cpu().numpy(), R.tail_out_frac(of, ow, lw, lf), atol=2e-2, rtol=2e-2)
+    assert abs(float(ref_mass.mean()) - target) < 0.06          # the noise of the other 255 dimensions averages out
+    # far keys carry (1 - mass) of the weight: dropping them moves the read-out more for the diffuse profile
+    assert (float(perturb.mean()) > 0.5) == (target < 0.5)
+
+
 def test_explicit_softmax_scale():
     cfg = _cfg(S0=700, D=128, gamma=1)
     wl = wi.make_workload(cfg)

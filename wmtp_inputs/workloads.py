@@ -40,6 +40,7 @@ class DraftConfig:
     key_scale: tuple | None = None   # (lo, hi): per-KV-head multiplier on K, log-spaced
     cap_slack: int = 0               # ring capacity = W + cap_slack window slots
     kv_dtype: str = "bf16"           # "bf16", or "fp8": e4m3 codes with one fp32 scale per KV head for K and for V
+    logit_profile: tuple | None = None   # (delta, tau): recency-peaked logits, see recency_column (bf16 stores only)
 
     @property
     def G(self) -> int:
@@ -98,6 +99,40 @@ def head_scales(cfg: DraftConfig) -> np.ndarray:
     if cfg.Hkv == 1:
         return np.array([lo])
     return lo * (hi / lo) ** (np.arange(cfg.Hkv) / (cfg.Hkv - 1))
+
+
+Q_ALONG = 4.0     # component of every query along the profile direction (dimension 0)
+
+
+def recency_column(S: int, D: int, delta: float, tau: float, S_ref: int | None = None) -> np.ndarray:
+    """Dimension-0 entries of the keys at positions [0, S) for a recency-peaked logit profile: with every query's
+    dimension 0 set to Q_ALONG, the key at distance dist = S_ref - 1 - pos from the newest token gets
+    delta * exp(-dist / tau) added to its scaled logit (softmax scale 1/sqrt(D)), on top of the i.i.d. noise of the
+    other dimensions.  Large delta with a short tau imitates a locally peaked (RoPE-like) head, small delta a diffuse
+    (NoPE-like) one."""
+    S_ref = S if S_ref is None else S_ref
+    dist = (S_ref - 1 - np.arange(S, dtype=np.float64))
+    return (delta * np.sqrt(D) / Q_ALONG * np.exp(-np.maximum(dist, 0.0) / tau)).astype(np.float32)
+
+
+def profile_window_mass(S: int, n_sink: int, W: int, delta: float, tau: float) -> float:
+    """Share of the softmax mass that the profile alone (noise averaged out) puts on sink + last W at length S."""
+    dist = S - 1 - np.arange(S, dtype=np.float64)
+    w = np.exp(delta * np.exp(-dist / tau))
+    inside = (np.arange(S) < n_sink) | (np.arange(S) >= S - W)
+    return float(w[inside].sum() / w.sum())
+
+
+def calibrate_delta(S: int, n_sink: int, W: int, tau: float, target_mass: float) -> float:
+    """delta for which profile_window_mass equals target_mass (bisection; the mass grows with delta)."""
+    lo, hi = 0.0, 40.0
+    for _ in range(60):
+        mid = (lo + hi) / 2
+        if profile_window_mass(S, n_sink, W, mid, tau) < target_mass:
+            lo = mid
+        else:
+            hi = mid
+    return (lo + hi) / 2
 
 
 def seq_lens(cfg: DraftConfig) -> np.ndarray:
@@ -172,6 +207,12 @@ def make_workload(cfg: DraftConfig, poison_unused: bool = True, extra_cap: int =
                 vb = gen.e4m3_codes_trunc(vb, float(wl.v_scale[g]))
             Kb[g] = kb
             Vb[g] = vb
+        if cfg.logit_profile is not None:
+            assert not f8, "logit profiles are defined for bf16 stores"
+            delta, tau = cfg.logit_profile
+            col = gen.f32_to_bf16_bits(recency_column(S, D, delta, tau))
+            for g in range(Hkv):
+                Kb[g][:, 0] = col
         wl.K.append(Kb)
         wl.V.append(Vb)
         if cfg.paged:
@@ -192,6 +233,10 @@ def make_workload(cfg: DraftConfig, poison_unused: bool = True, extra_cap: int =
     if cfg.key_scale is not None:
         kf = gen.bf16_bits_to_f32(kn) * sc.astype(np.float32)[None, None, :, None]
         kn = gen.f32_to_bf16_bits(kf)
+    if cfg.logit_profile is not None:
+        delta, tau = cfg.logit_profile
+        wl.q[..., 0] = gen.f32_to_bf16_bits(np.float32([Q_ALONG]))[0]
+        kn[..., 0] = gen.f32_to_bf16_bits(np.float32([delta * np.sqrt(D) / Q_ALONG]))[0]       # the newest token: distance 0
     wl.k_new = kn
     wl.v_new = gen.normal_bf16(cfg.seed, T_VNEW, (gam, B, Hkv, D), threads=threads)
     return wl
