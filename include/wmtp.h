@@ -207,6 +207,22 @@ wmtp_status wmtp_draft_loop_windowed_kv(const wmtp_kv* kv, int n_sink, int W, in
                                         const void* k_new, const void* v_new, float sm_scale, void* out, float* lse,
                                         void* workspace, size_t ws_bytes, void* stream);
 
+/*
+ * The reduced block table itself, for callers that run another paged attention backend through it (the paper's
+ * deployment, Section 4 "Mechanism": table = [sink blocks] || [recent-W blocks]). Paged stores only. Per sequence r with
+ * S = len[r]: table[r][0 .. n_s) = pages of the sink positions [0, min(S, n_sink)), table[r][n_s .. n_s + n_w) = pages of
+ * the window positions [max(min(S, n_sink), S - W), S), remaining entries -1; a page holding both kinds appears in both
+ * parts. meta[r][0..5) = { n_s, n_w, rows used in the last sink page, first row used in the first window page, rows
+ * used in the last window page }: the ends stay token-granular. table: device int32 [batch][table_stride],
+ * table_stride >= wmtp_reduced_block_table_width(n_sink, W, page_size) = ceil(n_sink/ps) + ceil(W/ps) + 1;
+ * meta: device int32 [batch][5]. O((n_sink + W) / page_size) work per sequence, no host arithmetic on S (the O(S)
+ * per-step index construction the paper removes has no counterpart in this library: the attention kernels index the
+ * stores arithmetically). A page id outside [0, num_pages) is written as -1 and flagged in `workspace` (may be NULL).
+ */
+int         wmtp_reduced_block_table_width(int n_sink, int W, int page_size);
+wmtp_status wmtp_reduced_block_table(const wmtp_kv* kv, int n_sink, int W, int32_t* table, int table_stride, int32_t* meta,
+                                     void* workspace, void* stream);
+
 /* ---- after verification: rollback and draft-extend -------------------------------------------- */
 
 /*

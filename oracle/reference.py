@@ -7,6 +7,8 @@ What is here, and the passage each part restates:
 
 * ``keep_set``      -- the two-branch key-set rule of the windowing pseudocode (Appendix A):
                        sink positions plus the last W positions when S > n_sink + W, else all.
+* ``reduced_block_table`` -- the block table the windowed draft attends through (Section 4,
+                       "Mechanism": [sink blocks] || [recent-W blocks]), with token-granular ends.
 * ``WindowStore``   -- an explicit list-based sink + window store (Section 4, "Mechanism":
                        the first n_sink tokens plus the most recent W tokens).
 * ``RingSim``       -- a slot-level simulation of the compact ring buffer (Section 4,
@@ -173,6 +175,28 @@ def keep_set(S: int, n_sink: int, W: int) -> list:
     if S > n_sink + W:
         return list(range(0, n_sink)) + list(range(S - W, S))
     return list(range(0, S))
+
+
+def reduced_block_table(S: int, n_sink: int, W: int, page_row, page_size: int):
+    """The windowed draft's block table (Section 4 "Mechanism": the per-request table reduced to
+    [sink blocks] || [recent-W blocks]) for one sequence of length S whose full table is ``page_row``.
+
+    Returns (pages, meta): ``pages`` lists the pages holding the sink positions, then the pages holding the last-W
+    positions (a page that holds both kinds appears in both parts); ``meta`` = [sink pages, window pages, sink rows
+    used in the last sink page, first row used in the first window page, rows used in the last window page] -- what
+    a reader needs to keep the ends token-granular.  Built in O((n_sink + W) / page_size) from S alone."""
+    keep = keep_set(S, n_sink, W)
+    ns = min(S, n_sink)
+    sink_pos = [p for p in keep if p < ns]
+    win_pos = [p for p in keep if p >= ns]
+    sink_pages = sorted({p // page_size for p in sink_pos})
+    win_pages = sorted({p // page_size for p in win_pos})
+    pages = [int(page_row[i]) for i in sink_pages] + [int(page_row[i]) for i in win_pages]
+    meta = [len(sink_pages), len(win_pages),
+            (sink_pos[-1] % page_size + 1) if sink_pos else 0,
+            (win_pos[0] % page_size) if win_pos else 0,
+            (win_pos[-1] % page_size + 1) if win_pos else 0]
+    return pages, meta
 
 
 class WindowStore:

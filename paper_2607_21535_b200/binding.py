@@ -74,6 +74,8 @@ _SIGNATURES = {
                                             c_void_p, c_size_t, c_void_p]),
     "wmtp_draft_loop_windowed_kv": (c_int, [POINTER(wmtp_kv), c_int, c_int, c_int, c_void_p, c_int, c_void_p, c_void_p,
                                             c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "wmtp_reduced_block_table_width": (c_int, [c_int, c_int, c_int]),
+    "wmtp_reduced_block_table": (c_int, [POINTER(wmtp_kv), c_int, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
     "wmtp_ring_rewind": (c_int, [POINTER(wmtp_ring), c_void_p, c_void_p, c_void_p]),
     "wmtp_ring_append_many": (c_int, [POINTER(wmtp_ring), c_int, c_void_p, c_void_p, c_void_p]),
     "wmtp_kv_append_many": (c_int, [POINTER(wmtp_kv), c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -344,6 +346,16 @@ def wmtp_attn_mass_diagnostics(out_win, lse_win, out_full, lse_full, mass=None, 
     rows = out_win.numel() // D
     _check(lib().wmtp_attn_mass_diagnostics(_ptr(out_win), _ptr(lse_win), _ptr(out_full), _ptr(lse_full), rows, D, _ptr(mass),
                                             _ptr(perturb), _ptr(tail), _stream(stream)))
+
+
+def wmtp_reduced_block_table_width(n_sink: int, W: int, page_size: int) -> int:
+    return int(lib().wmtp_reduced_block_table_width(n_sink, W, page_size))
+
+
+def wmtp_reduced_block_table(kv: KV, n_sink: int, W: int, table, meta, ws: Workspace | None = None, stream=None) -> None:
+    """table: device int32 [batch][stride]; meta: device int32 [batch][5]."""
+    _check(lib().wmtp_reduced_block_table(byref(kv.desc), n_sink, W, _ptr(table), table.shape[1], _ptr(meta),
+                                          ws.ptr if ws is not None else None, _stream(stream)))
 
 
 def wmtp_set_max_ctas(n: int) -> None:

@@ -212,6 +212,39 @@ __global__ void ring_rewind_kernel(RingParams r, const int32_t* __restrict__ n_d
     if (threadIdx.x == 0) r.len[b] = S - n;
 }
 
+// The windowed draft's block table over a paged store (Section 4 "Mechanism": the per-request table reduced to
+// [sink blocks] || [recent-W blocks]): O((n_sink + W) / page_size) entries per sequence from the device-resident length,
+// plus the row bounds that keep the ends token-granular. One block per sequence.
+__global__ void reduced_block_table_kernel(KvParams kv, int n_sink, int W, int32_t* __restrict__ table, int stride,
+                                           int32_t* __restrict__ meta, int* status) {
+    const int b = blockIdx.x, ps = kv.page_size;
+    const int64_t S = kv.len[b];
+    const int64_t ns = S < n_sink ? S : n_sink;                 // sink positions [0, ns)
+    const int64_t lo = S - W > ns ? S - W : ns;                 // window positions [lo, S)
+    const int n_s = (int)((ns + ps - 1) / ps);
+    const int first_w = (int)(lo / ps);
+    const int n_w = S > ns ? (int)((S - 1) / ps) - first_w + 1 : 0;
+    const bool fits = n_s + n_w <= stride && (n_w == 0 || first_w + n_w <= kv.max_pages) && n_s <= kv.max_pages;
+    if (!fits && threadIdx.x == 0 && status) atomicCAS(status, 0, kErrBounds);
+    const int n = fits ? n_s + n_w : 0;
+    for (int i = threadIdx.x; i < stride; i += blockDim.x) {
+        int page = -1;
+        if (i < n) {
+            page = kv.page_table[(int64_t)b * kv.max_pages + (i < n_s ? i : first_w + i - n_s)];
+            if (page < 0 || page >= kv.num_pages) { if (status) atomicCAS(status, 0, kErrBounds); page = -1; }
+        }
+        table[(int64_t)b * stride + i] = page;
+    }
+    if (threadIdx.x == 0) {
+        int32_t* m = meta + (int64_t)b * 5;
+        m[0] = fits ? n_s : 0;
+        m[1] = fits ? n_w : 0;
+        m[2] = (fits && ns > 0) ? (int)((ns - 1) % ps) + 1 : 0;         // rows used in the last sink page
+        m[3] = (fits && n_w > 0) ? (int)(lo % ps) : 0;                  // first row used in the first window page
+        m[4] = (fits && n_w > 0) ? (int)((S - 1) % ps) + 1 : 0;         // rows used in the last window page
+    }
+}
+
 __device__ __forceinline__ float bf16_bits_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_bits_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
@@ -299,6 +332,13 @@ cudaError_t launch_ring_append_many(const RingParams& r, int n_tok, const void* 
 
 cudaError_t launch_kv_append_many(const KvParams& kv, int n_tok, const void* k_new, const void* v_new, int* status, cudaStream_t st) {
     kv_append_many_kernel<<<kv.B, 256, 0, st>>>(kv, n_tok, (const uint4*)k_new, (const uint4*)v_new, status);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_reduced_block_table(const KvParams& kv, int n_sink, int W, int32_t* table, int stride, int32_t* meta, int* status,
+                                       cudaStream_t st) {
+    reduced_block_table_kernel<<<kv.B, 128, 0, st>>>(kv, n_sink, W, table, stride, meta, status);
     count_launch(1);
     return cudaGetLastError();
 }

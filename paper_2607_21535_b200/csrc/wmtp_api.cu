@@ -444,6 +444,25 @@ wmtp_status wmtp_draft_attn_windowed_kv(const void* q, int Hq, const wmtp_kv* kv
     return attn_full(q, Hq, kv, sm_scale, out, lse, workspace, ws_bytes, (cudaStream_t)stream, true, nullptr, nullptr, n_sink, W);
 }
 
+int wmtp_reduced_block_table_width(int n_sink, int W, int page_size) {
+    if (n_sink < 0 || W < 1 || page_size < 1) return 0;
+    return (n_sink + page_size - 1) / page_size + (W + page_size - 1) / page_size + 1;
+}
+
+wmtp_status wmtp_reduced_block_table(const wmtp_kv* kv, int n_sink, int W, int32_t* table, int table_stride, int32_t* meta,
+                                     void* workspace, void* stream) {
+    if (wmtp_status s = check_window(n_sink, W)) return s;
+    if (wmtp_status s = check_kv(kv)) return s;
+    if (!kv->page_table) return fail(WMTP_ERR_INVALID_ARG, "a reduced block table needs a paged store");
+    if (!table || !meta || !aligned(table, 4) || !aligned(meta, 4)) return fail(WMTP_ERR_INVALID_ARG, "table or meta is NULL or misaligned");
+    if (table_stride < wmtp_reduced_block_table_width(n_sink, W, kv->page_size))
+        return fail(WMTP_ERR_CAPACITY, "table_stride=%d, %d entries per sequence needed", table_stride,
+                    wmtp_reduced_block_table_width(n_sink, W, kv->page_size));
+    cudaError_t e = launch_reduced_block_table(kv_params(kv), n_sink, W, table, table_stride, meta, static_cast<int*>(workspace),
+                                               (cudaStream_t)stream);
+    return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "reduced block table launch");
+}
+
 wmtp_status wmtp_draft_loop_windowed_kv(const wmtp_kv* kv, int n_sink, int W, int gamma, const void* q, int Hq,
                                         const void* k_new, const void* v_new, float sm_scale, void* out, float* lse,
                                         void* workspace, size_t ws_bytes, void* stream) {

@@ -136,3 +136,14 @@ def test_kv_dtype_rejected_on_host():
     # rows are copied as stored: ring and KV store must agree
     r8 = _ring_desc(kv_dtype=1, k_scale=4096, v_scale=4096)
     assert L.wmtp_ring_init_from_kv(ctypes.byref(r8), ctypes.byref(_kv_desc()), None) == 1
+
+
+def test_reduced_block_table_arguments_rejected_on_host():
+    L = wm.lib()
+    paged = _kv_desc(page_table=4096, page_size=64, max_pages=4, num_pages=8, S_cap=256)
+    assert wm.wmtp_reduced_block_table_width(4, 64, 64) == 3 and wm.wmtp_reduced_block_table_width(64, 4032, 64) == 65
+    assert wm.wmtp_reduced_block_table_width(-1, 64, 64) == 0
+    assert L.wmtp_reduced_block_table(ctypes.byref(paged), 4, 64, 4096, 2, 4096, None, None) == 3      # needs 3 entries
+    assert L.wmtp_reduced_block_table(ctypes.byref(paged), 4, 0, 4096, 8, 4096, None, None) == 1
+    assert L.wmtp_reduced_block_table(ctypes.byref(paged), 4, 64, None, 8, 4096, None, None) == 1
+    assert L.wmtp_reduced_block_table(ctypes.byref(_kv_desc()), 4, 64, 4096, 8, 4096, None, None) == 1  # contiguous store

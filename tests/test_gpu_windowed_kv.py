@@ -6,6 +6,7 @@ import torch
 
 import paper_2607_21535_b200 as wm
 import wmtp_inputs as wi
+from oracle import reference as R
 
 from harness import DeviceWorkload, bits, compare, oracle_for
 
@@ -98,4 +99,41 @@ def test_window_view_rejects_bad_window():
     out = torch.empty_like(dw.q[0])
     with pytest.raises(wm.WmtpError) as ei:
         wm.wmtp_draft_attn_windowed_kv(dw.q[0], dw.kv, 4, 0, out, dw.ws)
+    assert ei.value.status == 1
+
+
+# ------------------------------------------------------------------------------------------ the reduced block table itself
+@pytest.mark.parametrize("n_sink,W", [(4, 64), (0, 100), (64, 252), (70, 130), (4, 2048)])
+def test_reduced_block_table_bit_exact(n_sink, W):
+    cfg = wi.DraftConfig("rbt", 9, 0, 16, 2, 128, W, n_sink, 1, seed=1000 + W, S0_range=(n_sink + W + 2, 9000), paged=True)
+    wl = wi.make_workload(cfg)
+    dw = DeviceWorkload(wl)
+    lens = wl.seq_lens.copy()
+    # shorter than generated (the pages exist): empty, sink only, partly filled window, exactly full, first slide
+    lens[0], lens[1], lens[2], lens[3], lens[4] = 0, max(n_sink - 1, 1), n_sink + W // 2, n_sink + W, n_sink + W + 1
+    dw.lens.copy_(torch.from_numpy(lens))
+    width = wm.wmtp_reduced_block_table_width(n_sink, W, 64)
+    assert width == (n_sink + 63) // 64 + (W + 63) // 64 + 1
+    table = torch.full((cfg.batch, width + 2), -7, dtype=torch.int32, device="cuda")
+    meta = torch.full((cfg.batch, 5), -7, dtype=torch.int32, device="cuda")
+    wm.wmtp_reduced_block_table(dw.kv, n_sink, W, table, meta, dw.ws)
+    wm.wmtp_device_status(dw.ws)
+    tb, mt = table.cpu().numpy(), meta.cpu().numpy()
+    for b in range(cfg.batch):
+        S = int(lens[b])
+        pages, m = R.reduced_block_table(S, n_sink, W, wl.page_table[b], 64)
+        assert mt[b].tolist() == m, (b, S)
+        assert tb[b, :len(pages)].tolist() == pages and (tb[b, len(pages):] == -1).all()
+
+
+def test_reduced_block_table_needs_a_wide_enough_table_and_a_paged_store():
+    cfg = wi.DraftConfig("rbt2", 2, 500, 16, 2, 128, 256, 4, 1, seed=7, paged=True)
+    dw = DeviceWorkload(wi.make_workload(cfg))
+    meta = torch.zeros((2, 5), dtype=torch.int32, device="cuda")
+    with pytest.raises(wm.WmtpError) as ei:
+        wm.wmtp_reduced_block_table(dw.kv, 4, 256, torch.zeros((2, 5), dtype=torch.int32, device="cuda"), meta)
+    assert ei.value.status == 3
+    dc = DeviceWorkload(wi.make_workload(wi.scaled(cfg, paged=False)))
+    with pytest.raises(wm.WmtpError) as ei:
+        wm.wmtp_reduced_block_table(dc.kv, 4, 256, torch.zeros((2, 8), dtype=torch.int32, device="cuda"), meta)
     assert ei.value.status == 1

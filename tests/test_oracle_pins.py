@@ -434,3 +434,26 @@ def test_fp8_draft_oracle_quantises_on_append():
     ow, lw = R.attention(wl.q[0, 0], orc.Kfull[:, :21], orc.Vfull[:, :21], keys=np.array(keep), k_scale=wl.k_scale, v_scale=wl.v_scale)
     assert np.abs(ow - r["win"][0]).max() < 1e-12 and np.abs(lw - r["win"][1]).max() < 1e-12
     assert (r["full"][1] > r["win"][1]).all()
+
+
+# ---------------------------------------------------------------- reduced block table
+@pytest.mark.parametrize("n_sink,W,ps", [(4, 64, 64), (0, 100, 64), (64, 4032 // 16, 64), (70, 130, 64), (3, 5, 4), (4, 8, 16)])
+def test_reduced_block_table_expands_to_the_keep_set(n_sink, W, ps):
+    """Walking the reduced table with its row bounds must visit exactly the rows of the kept positions, in order."""
+    rs = np.random.RandomState(n_sink + W)
+    for S in list(range(0, 3 * ps + 3)) + [n_sink + W, n_sink + W + 1, 10 * ps - 1, 10 * ps, 10 * ps + 1, 977]:
+        n_pages = (S + ps - 1) // ps + 2
+        page_row = rs.permutation(n_pages + 50)[:n_pages]
+        pages, meta = R.reduced_block_table(S, n_sink, W, page_row, ps)
+        n_s, n_w, sink_last, win_first, win_last = meta
+        assert len(pages) == n_s + n_w and n_s <= (n_sink + ps - 1) // ps and n_w <= (W + ps - 1) // ps + 1
+        rows = []                                              # (page, row) pairs a reader would touch
+        for i in range(n_s):
+            hi = sink_last if i == n_s - 1 else ps
+            rows += [(pages[i], r) for r in range(hi)]
+        for i in range(n_w):
+            lo = win_first if i == 0 else 0
+            hi = win_last if i == n_w - 1 else ps
+            rows += [(pages[n_s + i], r) for r in range(lo, hi)]
+        want = [(int(page_row[p // ps]), p % ps) for p in R.keep_set(S, n_sink, W)]        # brute force, token by token
+        assert rows == want, (S, meta)
