@@ -12,9 +12,9 @@
 //   * a producer warp streams K and V tiles into a ring of shared-memory stages with TMA
 //     (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers) and tells the consumers
 //     which tile each stage holds;
-//   * consumer groups of four warps take whole tiles in turn (one group for head_dim 256, two for
-//     head_dim 128, where a tile carries half the bytes for the same softmax work); each warp of a
-//     group takes 16 keys of the tile. Scores are computed as S^T[key, head] = K[key, :] . Q^T (keys
+//   * consumer groups of four warps take whole tiles in turn (one group when a stage holds 64 KB, two
+//     when it holds less -- head_dim 128 or an fp8 store -- where a tile carries fewer bytes for the same
+//     softmax work); each warp of a group takes 16 keys of the tile. Scores are computed as S^T[key, head] = K[key, :] . Q^T (keys
 //     on the MMA M dimension, the G <= 8 query heads of the GQA group exactly on N = 8), the online
 //     softmax runs in fp32, and O^T[d, head] += V^T[d, key] . P^T[key, head] accumulates in
 //     registers. The 8-row problem is far too small for tcgen05 (M >= 64); mma.sync.m16n8k16 needs a
@@ -70,10 +70,7 @@ struct Cfg {
     static constexpr int kTileBytes = kChunks * kChunkBytes;  // K (or V) tile
     static constexpr int kStageBytes = 2 * kTileBytes;
     // consumer groups: a tile of fewer bytes brings the same softmax work, so the smaller tiles get two groups
-#ifndef WMTP_F8_GROUPS_256
-#define WMTP_F8_GROUPS_256 2
-#endif
-    static constexpr int kGroups = (kStageBytes >= 65536) ? 1 : ((F8 && D == 256) ? WMTP_F8_GROUPS_256 : 2);
+    static constexpr int kGroups = (kStageBytes >= 65536) ? 1 : 2;
     // Stages of the shared-memory ring. What counts for the streaming rate is the bytes a CTA keeps in flight (about
     // 190 KB per SM saturate HBM at the loaded latency of ~4 us): the host takes as many stages as fit beside the
     // batch-dependent tables, up to kMaxStages, in multiples of the group count (a stage then always serves one group).
@@ -97,16 +94,9 @@ struct Cfg {
     // one scheduler's register file); the consumers want more and the producer needs about 56. So after the common
     // prologue the producer's warpgroup hands registers to the consumers' warpgroups (setmaxnreg). The instruction is
     // warpgroup-wide: the producer's warpgroup is filled up with three warps that execute it and exit.
-#ifndef WMTP_REBALANCE
-#define WMTP_REBALANCE 1
-#endif
-#ifndef WMTP_REGS_P
-#define WMTP_REGS_P 56
-#define WMTP_REGS_C 224
-#endif
-    static constexpr bool kRebalance = (kGroups == 2) && WMTP_REBALANCE;
+    static constexpr bool kRebalance = (kGroups == 2);
     static constexpr int kPadWarps = kRebalance ? 3 : 0;
-    static constexpr int kRegsProducer = WMTP_REGS_P, kRegsConsumer = WMTP_REGS_C;
+    static constexpr int kRegsProducer = 56, kRegsConsumer = 224;
     // the 8 consumer warps and the 4 warps of the producer's warpgroup share what the 12 warps were launched with
     static_assert(8 * kRegsConsumer + 4 * kRegsProducer <= 12 * 168, "register trade must balance");
     static constexpr int kThreads = (kConsumerWarps + 1 + kPadWarps) * 32;
@@ -344,11 +334,7 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
                                              int tid, int grp) {
     const int G = p.G, D = p.D;
     float* w_sm = scratch;                                                  // [heads of the slice][np]
-#ifdef WMTP_COMBINE_ALL
-    float* inv_sm = scratch + kMaxGroup * kMaxParts;
-#else
     float* inv_sm = scratch + kCombineWeights;                              // [8], indexed by head - first head of the slice
-#endif
     float4* red = reinterpret_cast<float4*>(inv_sm + 8);                    // [128]
     int* perm = reinterpret_cast<int*>(inv_sm + 8 + 4 * kGroupThreads);     // [np] visiting order
     WMTP_STAMP(p, 7);
@@ -374,13 +360,9 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
     const int vec = D / 4, cols = G * vec;
     const int cpc = (cols + np - 1) / np;
     const int col_lo = j * cpc, col_hi = col_lo + cpc < cols ? col_lo + cpc : cols;
-#ifdef WMTP_COMBINE_ALL
-    const int h_lo = 0, nh = G;
-#else
     const int vsh = D == 256 ? 6 : 5;                                       // vec = D / 4 is a power of two: log2(vec)
     const int h_lo = col_lo < cols ? col_lo >> vsh : 0;                     // heads the slice touches: [h_lo, h_lo + nh)
     const int nh = col_lo < col_hi ? ((col_hi - 1) >> vsh) - h_lo + 1 : 0;
-#endif
     const float4* rows = reinterpret_cast<const float4*>(p.part_o);
     float4 pre[kPre];
     {
@@ -490,10 +472,7 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
 // The attention kernel (one cooperative launch per draft step)
 // ---------------------------------------------------------------------------------------------
 template <int D, bool F8>
-#ifndef WMTP_LB
-#define WMTP_LB(x) (x)
-#endif
-__global__ void __launch_bounds__(WMTP_LB((Cfg<D, F8>::kThreads)), 1)
+__global__ void __launch_bounds__(Cfg<D, F8>::kThreads, 1)
 attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                const __grid_constant__ AttnParams p) {
     using C = Cfg<D, F8>;
@@ -592,9 +571,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsProducer));
             if ((int)(threadIdx.x >> 5) > C::kConsumerWarps) return;          // filler warps of the producer's warpgroup
         }
-#ifdef WMTP_NO_PRODUCER
-        return;
-#endif
         // =================================== producer warp ===================================
         // CTA c < Cn owns the tile range [c n / Cn, (c+1) n / Cn). It streams the first part of it without any
         // bookkeeping; the rest is handed out in small chunks through the per-CTA cursor cur[c], to the owner
@@ -810,9 +786,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     }
 
     if constexpr (C::kRebalance) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsConsumer));
-#ifdef WMTP_NO_CONSUMER
-    return;
-#endif
     // ===================================== consumer groups =====================================
     const int grp = threadIdx.x / kGroupThreads, tid = threadIdx.x % kGroupThreads;   // group, thread within the group
     const int warp = tid >> 5;                           // warp within the group: owns keys [16 warp, 16 warp + 16) of a tile

@@ -2,7 +2,8 @@
 //
 // Slot rule (Section 4 "Memory"; Appendix A, RING comment, read with the sink kept fixed):
 // position p lives in slot p when p < n_sink, else in n_sink + ((p - n_sink) mod cap).
-// All of this is integer work and copies: results are bit-exact by construction.
+// All of this is integer work and copies -- bit-exact by construction -- except the quantisation of new rows for an
+// fp8 store, which is defined to the bit (fp32 division, round to nearest even, saturation; fp8_util.cuh).
 #include "wmtp_internal.h"
 #include "fp8_util.cuh"
 
