@@ -226,7 +226,7 @@ def test_config_sweep_shape_fp8():
     _run_and_check(wi.scaled(wi.CONFIGS[4], S0=262144, W=4096, gamma=3, kv_dtype="fp8", name="sweep_fp8"))
 
 
-@pytest.mark.parametrize("kv_dtype,D", [("fp8", 256), ("fp8", 128), ("bf16", 128)])
+@pytest.mark.parametrize("kv_dtype,D", [("fp8", 256), ("fp8", 128), ("bf16", 128), ("bf16", 256)])
 def test_very_large_batch_leaves_room_for_fewer_stages(kv_dtype, D):
     """1000 sequences: the batch-sized tables take shared memory from the stage ring, the kernel runs with fewer stages."""
     cfg = _cfg(batch=1000, S0=0, S0_range=(1, 200), D=D, W=32, n_sink=2, gamma=1, seed=4711, paged=True, kv_dtype=kv_dtype,
