@@ -339,11 +339,10 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
     int* perm = reinterpret_cast<int*>(inv_sm + 8 + 4 * kGroupThreads);     // [np] visiting order
     WMTP_STAMP(p, 7);
 
-    // ---- visiting order
-    if (p.steal_slots_enabled) {
-        for (int i = tid; i < np; i += kGroupThreads) perm[i] = i;
-    } else {
-        int* keys = reinterpret_cast<int*>(red);                            // borrowed until the first barrier below
+    // ---- visiting order: the fixed partition ranks the partials by their keys; with stealing on they are taken as stored
+    const bool ranked = !p.steal_slots_enabled;
+    if (ranked) {
+        int* keys = reinterpret_cast<int*>(red);                            // borrowed until the barrier below
         for (int i = tid; i < np; i += kGroupThreads) keys[i] = __ldcg(p.part_key + pbase + i);
         group_barrier(grp);
         for (int i = tid; i < np; i += kGroupThreads) {
@@ -352,58 +351,73 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
             for (int q = 0; q < np; ++q) r += keys[q] < ki;
             perm[r] = i;
         }
+        group_barrier(grp);
     }
-    group_barrier(grp);
+    auto part = [&](int i) { return ranked ? perm[i] : i; };
 
     // ---- this group's slice of the (head, d) columns; the first rows are requested before the weights exist
     constexpr int kPre = 6;
     const int vec = D / 4, cols = G * vec;
-    const int cpc = (cols + np - 1) / np;
+    // columns per contributor: the smallest power of two that covers all columns (this runs once per launch on the
+    // critical path of the tail: shifts and masks instead of integer divisions)
+    int csh = 0;
+    while ((np << csh) < cols) ++csh;
+    const int cpc = 1 << csh;
+    const int bsh = csh < 7 ? csh : 7, cb = 1 << bsh;                       // columns handled per pass: min(cpc, 128)
+    const int R = kGroupThreads >> bsh, cl = tid & (cb - 1), rg = tid >> bsh;   // R rows of partials in flight per column
     const int col_lo = j * cpc, col_hi = col_lo + cpc < cols ? col_lo + cpc : cols;
     const int vsh = D == 256 ? 6 : 5;                                       // vec = D / 4 is a power of two: log2(vec)
     const int h_lo = col_lo < cols ? col_lo >> vsh : 0;                     // heads the slice touches: [h_lo, h_lo + nh)
     const int nh = col_lo < col_hi ? ((col_hi - 1) >> vsh) - h_lo + 1 : 0;
     const float4* rows = reinterpret_cast<const float4*>(p.part_o);
     float4 pre[kPre];
-    {
-        const int cb = col_hi - col_lo < kGroupThreads ? col_hi - col_lo : kGroupThreads;
-        if (cb > 0) {
-            const int R = kGroupThreads / cb, cl = tid % cb, rg = tid / cb;
 #pragma unroll
-            for (int u = 0; u < kPre; ++u) {
-                const int i = rg + u * R;
-                pre[u] = (rg < R && i < np) ? __ldcg(rows + (pbase + perm[i]) * cols + col_lo + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-        }
+    for (int u = 0; u < kPre; ++u) {
+        const int i = rg + u * R;
+        pre[u] = (col_lo + cl < col_hi && i < np) ? __ldcg(rows + (pbase + part(i)) * cols + col_lo + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    // ---- weights of the slice's heads, all at once: 16 threads per head, one pass over the partial lse values.
+    WMTP_STAMP(p, 11);
+    // ---- weights of the slice's heads, all at once: 16 threads per head, the partial lse values taken 128 at a time
+    //      with a running maximum (weights already stored are rescaled when it moves; one chunk is the common case).
     //      The contributor whose slice holds a head's first column also writes the head's lse.
     {
         const int hh = tid >> 4, h = h_lo + hh, li = tid & 15;
         const bool act = hh < nh;
-        constexpr int kPer = (kMaxParts + 15) / 16;
-        float x[kPer];
-        float M = -INFINITY;
+        constexpr int kPer = 8;
+        float M = -INFINITY, sum = 0.f;
+        for (int c0 = 0; c0 < np; c0 += 16 * kPer) {
+            float x[kPer];
+            float mc = -INFINITY;
 #pragma unroll
-        for (int u = 0; u < kPer; ++u) {
-            const int i = li + 16 * u;
-            x[u] = (act && i < np) ? __ldcg(p.part_lse + (pbase + perm[i]) * G + h) : -INFINITY;
-            M = fmaxf(M, x[u]);
-        }
+            for (int u = 0; u < kPer; ++u) {
+                const int i = c0 + li + 16 * u;
+                x[u] = (act && i < np) ? __ldcg(p.part_lse + (pbase + part(i)) * G + h) : -INFINITY;
+                mc = fmaxf(mc, x[u]);
+            }
 #pragma unroll
-        for (int off = 8; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
-        float sum = 0.f;
+            for (int off = 8; off > 0; off >>= 1) mc = fmaxf(mc, __shfl_xor_sync(0xffffffffu, mc, off));
+            WMTP_STAMP(p, 12);
+            if (mc > M) {
+                if (c0 > 0 && act) {
+                    const float r = __expf(M - mc);                    // 0 when nothing finite was seen before
+                    for (int i = li; i < c0; i += 16) w_sm[hh * np + i] *= r;
+                    sum *= r;
+                }
+                M = mc;
+            }
 #pragma unroll
-        for (int u = 0; u < kPer; ++u) {
-            const int i = li + 16 * u;
-            if (act && i < np) {
-                const float w = (M > -INFINITY) ? __expf(x[u] - M) : 0.f;
-                w_sm[hh * np + i] = w;
-                sum += w;
+            for (int u = 0; u < kPer; ++u) {
+                const int i = c0 + li + 16 * u;
+                if (act && i < np) {
+                    const float w = (M > -INFINITY) ? __expf(x[u] - M) : 0.f;
+                    w_sm[hh * np + i] = w;
+                    sum += w;
+                }
             }
         }
 #pragma unroll
         for (int off = 8; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+        WMTP_STAMP(p, 13);
         if (li == 0 && act) {
             inv_sm[hh] = sum > 0.f ? 1.f / sum : 0.f;
             if (p.lse && col_lo <= (h << vsh)) p.lse[(int64_t)b * p.Hq + g * G + h] = sum > 0.f ? M + __logf(sum) : -INFINITY;
@@ -413,10 +427,8 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
     WMTP_STAMP(p, 8);
     __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + g * G) * D;
     for (int c0 = col_lo; c0 < col_hi; c0 += kGroupThreads) {
-        const int cb = col_hi - c0 < kGroupThreads ? col_hi - c0 : kGroupThreads;
-        const int R = kGroupThreads / cb, cl = tid % cb, rg = tid / cb;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (rg < R) {
+        if (c0 + cl < col_hi) {
             const int col = c0 + cl, h = (col >> vsh) - h_lo;
             int i = rg;
             if (c0 == col_lo) {
@@ -432,13 +444,13 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
 #pragma unroll 4
             for (; i < np; i += R) {
                 const float w = w_sm[h * np + i];
-                const float4 x = __ldcg(rows + (pbase + perm[i]) * cols + col);
+                const float4 x = __ldcg(rows + (pbase + part(i)) * cols + col);
                 acc.x = fmaf(w, x.x, acc.x); acc.y = fmaf(w, x.y, acc.y); acc.z = fmaf(w, x.z, acc.z); acc.w = fmaf(w, x.w, acc.w);
             }
         }
         red[tid] = acc;
         group_barrier(grp);
-        if (tid < cb) {
+        if (tid < cb && c0 + tid < col_hi) {
             float4 o = red[tid];
             for (int r = 1; r < R; ++r) {
                 const float4 x = red[r * cb + tid];
