@@ -376,7 +376,6 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
         const int i = rg + u * R;
         pre[u] = (col_lo + cl < col_hi && i < np) ? __ldcg(rows + (pbase + part(i)) * cols + col_lo + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    WMTP_STAMP(p, 11);
     // ---- weights of the slice's heads, all at once: 16 threads per head, the partial lse values taken 128 at a time
     //      with a running maximum (weights already stored are rescaled when it moves; one chunk is the common case).
     //      The contributor whose slice holds a head's first column also writes the head's lse.
@@ -396,8 +395,7 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
             }
 #pragma unroll
             for (int off = 8; off > 0; off >>= 1) mc = fmaxf(mc, __shfl_xor_sync(0xffffffffu, mc, off));
-            WMTP_STAMP(p, 12);
-            if (mc > M) {
+                    if (mc > M) {
                 if (c0 > 0 && act) {
                     const float r = __expf(M - mc);                    // 0 when nothing finite was seen before
                     for (int i = li; i < c0; i += 16) w_sm[hh * np + i] *= r;
@@ -417,8 +415,7 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
         }
 #pragma unroll
         for (int off = 8; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-        WMTP_STAMP(p, 13);
-        if (li == 0 && act) {
+            if (li == 0 && act) {
             inv_sm[hh] = sum > 0.f ? 1.f / sum : 0.f;
             if (p.lse && col_lo <= (h << vsh)) p.lse[(int64_t)b * p.Hq + g * G + h] = sum > 0.f ? M + __logf(sum) : -INFINITY;
         }
