@@ -319,6 +319,28 @@ def main():
         a.record(); wm.wmtp_draft_attn_windowed(q[0], ring, o1, ws); b.record()
     torch.cuda.synchronize()
     wm.wmtp_device_status(ws)
+    # the windowed loop replayed from a CUDA graph (what a serving stack that captures its decode step sees)
+    us_win_graph = None
+    try:
+        gs = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(gs):
+            wm.wmtp_draft_loop_windowed(ring, q, kn, vn, out_w, ws)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(graph, stream=gs):
+                wm.wmtp_draft_loop_windowed(ring, q, kn, vn, out_w, ws)
+        torch.cuda.synchronize()
+        for _ in range(3):
+            graph.replay()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(reps):
+            graph.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        us_win_graph = g0.elapsed_time(g1) * 1e3 / reps / gam
+    except Exception as exc:                                 # graph capture unavailable: report nothing
+        log(f"[bench] graph replay skipped: {exc}")
     us_full_call = k0.elapsed_time(k1) * 1e3 / reps
     us_win_kv_call = v0.elapsed_time(v1) * 1e3 / reps
     us_win_call_cold = statistics.mean(a.elapsed_time(b) for a, b in wev) * 1e3
@@ -494,7 +516,8 @@ def main():
                              "algorithmic_gbs": win_bytes / (us_win * 1e-6) / 1e9,
                              "pct_of_8tbs": win_bytes / (us_win * 1e-6) / 8e12 * 100,
                              "us_per_call_cold_l2": us_win_call_cold,
-                             "launch_floor_us": us_launch_floor},
+                             "launch_floor_us": us_launch_floor,
+                             "us_per_step_graph_replay": us_win_graph},
                 "windowed_kv_view": {"us_per_attention_call": us_win_kv_call,
                                      "note": "sink + last-W tiles read from the KV store through its page table / rows"},
                 "full": {"us_per_step": us_full, "kv_bytes_per_step": full_bytes,
