@@ -96,7 +96,11 @@ struct Cfg {
     // warpgroup-wide: the producer's warpgroup is filled up with three warps that execute it and exit.
     static constexpr bool kRebalance = (kGroups == 2);
     static constexpr int kPadWarps = kRebalance ? 3 : 0;
-    static constexpr int kRegsProducer = 56, kRegsConsumer = 224;
+#ifndef WMTP_REGS_P
+#define WMTP_REGS_P 56
+#define WMTP_REGS_C 224
+#endif
+    static constexpr int kRegsProducer = WMTP_REGS_P, kRegsConsumer = WMTP_REGS_C;
     // the 8 consumer warps and the 4 warps of the producer's warpgroup share what the 12 warps were launched with
     static_assert(8 * kRegsConsumer + 4 * kRegsProducer <= 12 * 168, "register trade must balance");
     static constexpr int kThreads = (kConsumerWarps + 1 + kPadWarps) * 32;
