@@ -382,10 +382,12 @@ def main():
         drop = torch.full((B,), ql, dtype=torch.int32, device=dev)
 
         def extend_windowed():
-            wm.wmtp_ring_append_many(ring_x, kx, vx)
+            # the draft's update after a verify step: drop the rejected tokens and append the verified ones in one
+            # launch, then attend over them in one launch (dropping as many as are appended keeps the length fixed)
+            wm.wmtp_ring_replace_tail(ring_x, drop, kx, vx, ws_x)
             wm.wmtp_draft_extend_windowed(qx, ring_x, ox, ws_x)
-            wm.wmtp_ring_rewind(ring_x, drop, ws_x)          # keeps the ring at the same length for the next repeat
 
+        wm.wmtp_ring_append_many(ring_x, kx, vx)
         extend_windowed()
         wm.wmtp_draft_extend_full(qx, kv, ox, ws_x)
         x0, x1, x2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
@@ -401,8 +403,8 @@ def main():
         ext = {"q_len": ql,
                "windowed_us_per_iteration": x0.elapsed_time(x1) * 1e3 / reps,
                "full_us_per_call": x1.elapsed_time(x2) * 1e3 / reps,
-               "note": "windowed: append q_len tokens to a ring with 8 slack slots + one multi-query attention launch + "
-                       "rollback (3 launches); full: one multi-query attention launch over the whole KV store"}
+               "note": "windowed: rollback of q_len tokens + append of q_len tokens on a ring with 8 slack slots (one launch) + "
+                       "one multi-query attention launch; full: one multi-query attention launch over the whole KV store"}
     # ---- the fp8 (e4m3) KV variant of the same workload: half the bytes per key, same launches
     f8 = None
     if cfg.kv_dtype == "bf16":

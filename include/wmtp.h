@@ -240,6 +240,9 @@ wmtp_status wmtp_reduced_block_table(const wmtp_kv* kv, int n_sink, int W, int32
  *   sum within cap - W.
  * wmtp_ring_append_many / wmtp_kv_append_many: n_tok tokens per sequence in one launch; k_new, v_new are device bf16
  *   [batch][n_tok][Hkv][D]; token j goes to position len + j; len += n_tok (all or nothing for the KV store).
+ * wmtp_ring_replace_tail: both in one launch, the draft's state update after a verify step: drops the last n_drop[r]
+ *   tokens (n_drop may be NULL: none), then appends n_tok tokens at the positions that follow; slots of dropped
+ *   positions that are not rewritten get slot_pos = -1. Same conditions and error behaviour as wmtp_ring_rewind.
  * wmtp_draft_extend_windowed / _full: q is device bf16 [batch][q_len][Hq][D]; the q_len tokens must already be in the
  *   store. Query i of a sequence attends as a decode step would have at length len - (q_len - 1 - i): over sink + last W
  *   of that length (windowed; needs cap >= W + q_len - 1) or over all positions below it (full). out: device bf16
@@ -249,6 +252,8 @@ wmtp_status wmtp_reduced_block_table(const wmtp_kv* kv, int n_sink, int W, int32
  */
 wmtp_status wmtp_ring_rewind(const wmtp_ring* ring, const int32_t* n_drop, void* workspace, void* stream);
 wmtp_status wmtp_ring_append_many(const wmtp_ring* ring, int n_tok, const void* k_new, const void* v_new, void* stream);
+wmtp_status wmtp_ring_replace_tail(const wmtp_ring* ring, const int32_t* n_drop, int n_tok, const void* k_new, const void* v_new,
+                                   void* workspace, void* stream);
 wmtp_status wmtp_kv_append_many(const wmtp_kv* kv, int n_tok, const void* k_new, const void* v_new, void* workspace,
                                 void* stream);
 wmtp_status wmtp_draft_extend_windowed(const void* q, int q_len, int Hq, const wmtp_ring* ring, float sm_scale, void* out,

@@ -78,6 +78,7 @@ _SIGNATURES = {
     "wmtp_reduced_block_table": (c_int, [POINTER(wmtp_kv), c_int, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
     "wmtp_ring_rewind": (c_int, [POINTER(wmtp_ring), c_void_p, c_void_p, c_void_p]),
     "wmtp_ring_append_many": (c_int, [POINTER(wmtp_ring), c_int, c_void_p, c_void_p, c_void_p]),
+    "wmtp_ring_replace_tail": (c_int, [POINTER(wmtp_ring), c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
     "wmtp_kv_append_many": (c_int, [POINTER(wmtp_kv), c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
     "wmtp_draft_extend_windowed": (c_int, [c_void_p, c_int, c_int, POINTER(wmtp_ring), c_float, c_void_p, c_void_p, c_void_p,
                                            c_size_t, c_void_p]),
@@ -321,6 +322,12 @@ def wmtp_ring_rewind(ring: Ring, n_drop, ws: Workspace | None = None, stream=Non
 def wmtp_ring_append_many(ring: Ring, k_new, v_new, stream=None) -> None:
     """k_new, v_new: [batch][n_tok][Hkv][D]."""
     _check(lib().wmtp_ring_append_many(byref(ring.desc), k_new.shape[1], _ptr(k_new), _ptr(v_new), _stream(stream)))
+
+
+def wmtp_ring_replace_tail(ring: Ring, n_drop, k_new, v_new, ws: Workspace | None = None, stream=None) -> None:
+    """Drop the last n_drop[r] tokens (device int32 [batch] or None), then append k_new / v_new [batch][n_tok][Hkv][D]."""
+    _check(lib().wmtp_ring_replace_tail(byref(ring.desc), _ptr(n_drop), k_new.shape[1], _ptr(k_new), _ptr(v_new),
+                                        ws.ptr if ws is not None else None, _stream(stream)))
 
 
 def wmtp_kv_append_many(kv: KV, k_new, v_new, ws: Workspace | None = None, stream=None) -> None:

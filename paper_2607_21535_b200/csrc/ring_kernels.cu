@@ -246,6 +246,40 @@ __global__ void reduced_block_table_kernel(KvParams kv, int n_sink, int W, int32
     }
 }
 
+// Rollback and append in one launch (the draft's state update after a verify step): drop the last n_drop[b] tokens, then
+// append n_tok new ones at the positions that follow. Slots of dropped positions that are not rewritten are marked
+// empty. Same conditions as ring_rewind_kernel; a violation leaves the sequence unchanged and is flagged.
+__global__ void ring_replace_tail_kernel(RingParams r, const int32_t* __restrict__ n_drop, int n_tok, const uint4* __restrict__ k_new,
+                                         const uint4* __restrict__ v_new, int* status) {
+    const int b = blockIdx.x;
+    const int64_t S = r.len[b];
+    const int slots = r.n_sink + r.cap;
+    const int n = n_drop ? n_drop[b] : 0;
+    if (n < 0 || n > S || n > r.cap - r.W) {
+        if (threadIdx.x == 0 && status) atomicCAS(status, 0, kErrBounds);
+        return;
+    }
+    const int64_t p0 = S - n;
+    const int vec_per_row = store_vecs(r.D, r.f8), src_vecs = r.D / 8;
+    const int n_vec = r.Hkv * vec_per_row;
+    uint4* K = reinterpret_cast<uint4*>(r.k);
+    uint4* V = reinterpret_cast<uint4*>(r.v);
+    for (int idx = threadIdx.x; idx < n_tok * n_vec; idx += blockDim.x) {
+        const int j = idx / n_vec, i = idx % n_vec;
+        const int g = i / vec_per_row, c = i % vec_per_row;
+        const int slot = ring_slot(p0 + j, r.n_sink, r.cap);
+        const int64_t dst = (((int64_t)b * r.Hkv + g) * slots + slot) * vec_per_row + c;
+        const int64_t src = (((int64_t)b * n_tok + j) * r.Hkv + g) * src_vecs;
+        K[dst] = stored_vec(k_new + src, c, r.f8, r.f8 ? r.k_scale[g] : 1.f);
+        V[dst] = stored_vec(v_new + src, c, r.f8, r.f8 ? r.v_scale[g] : 1.f);
+    }
+    __syncthreads();   // every thread has read len[b] before it moves
+    const int m = n > n_tok ? n : n_tok;
+    for (int j = threadIdx.x; j < m; j += blockDim.x)
+        r.slot_pos[(int64_t)b * slots + ring_slot(p0 + j, r.n_sink, r.cap)] = j < n_tok ? (int32_t)(p0 + j) : -1;
+    if (threadIdx.x == 0) r.len[b] = p0 + n_tok;
+}
+
 __device__ __forceinline__ float bf16_bits_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_bits_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
@@ -340,6 +374,13 @@ cudaError_t launch_kv_append_many(const KvParams& kv, int n_tok, const void* k_n
 cudaError_t launch_reduced_block_table(const KvParams& kv, int n_sink, int W, int32_t* table, int stride, int32_t* meta, int* status,
                                        cudaStream_t st) {
     reduced_block_table_kernel<<<kv.B, 128, 0, st>>>(kv, n_sink, W, table, stride, meta, status);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ring_replace_tail(const RingParams& r, const int32_t* n_drop, int n_tok, const void* k_new, const void* v_new,
+                                     int* status, cudaStream_t st) {
+    ring_replace_tail_kernel<<<r.B, 256, 0, st>>>(r, n_drop, n_tok, (const uint4*)k_new, (const uint4*)v_new, status);
     count_launch(1);
     return cudaGetLastError();
 }

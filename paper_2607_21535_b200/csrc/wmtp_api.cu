@@ -416,6 +416,18 @@ wmtp_status wmtp_ring_rewind(const wmtp_ring* ring, const int32_t* n_drop, void*
     return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "ring rewind launch");
 }
 
+wmtp_status wmtp_ring_replace_tail(const wmtp_ring* ring, const int32_t* n_drop, int n_tok, const void* k_new, const void* v_new,
+                                   void* workspace, void* stream) {
+    if (wmtp_status s = check_ring(ring)) return s;
+    if (n_drop && !aligned(n_drop, 4)) return fail(WMTP_ERR_INVALID_ARG, "n_drop is misaligned");
+    if (wmtp_status s = check_loop(n_tok, k_new, v_new)) return s;
+    if (n_tok > ring->cap) return fail(WMTP_ERR_CAPACITY, "n_tok=%d exceeds the ring's %d window slots", n_tok, ring->cap);
+    if (workspace && !aligned(workspace, 256)) return fail(WMTP_ERR_WORKSPACE, "workspace is not 256-byte aligned");
+    cudaError_t e = launch_ring_replace_tail(ring_params(ring), n_drop, n_tok, k_new, v_new, static_cast<int*>(workspace),
+                                             (cudaStream_t)stream);
+    return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "ring replace-tail launch");
+}
+
 wmtp_status wmtp_draft_extend_windowed(const void* q, int q_len, int Hq, const wmtp_ring* ring, float sm_scale, void* out,
                                        float* lse, void* workspace, size_t ws_bytes, void* stream) {
     if (wmtp_status s = check_ring(ring)) return s;

@@ -105,6 +105,8 @@ cudaError_t launch_kv_append(const KvParams& kv, const void* k_new, const void* 
 cudaError_t launch_ring_append_many(const RingParams& r, int n_tok, const void* k_new, const void* v_new, cudaStream_t st);
 cudaError_t launch_kv_append_many(const KvParams& kv, int n_tok, const void* k_new, const void* v_new, int* status, cudaStream_t st);
 cudaError_t launch_ring_rewind(const RingParams& r, const int32_t* n_drop, int* status, cudaStream_t st);
+cudaError_t launch_ring_replace_tail(const RingParams& r, const int32_t* n_drop, int n_tok, const void* k_new, const void* v_new,
+                                     int* status, cudaStream_t st);
 cudaError_t launch_reduced_block_table(const KvParams& kv, int n_sink, int W, int32_t* table, int stride, int32_t* meta, int* status,
                                        cudaStream_t st);
 // One cooperative launch: optional append of (k_new, v_new), split-KV partials, distributed LSE combine.

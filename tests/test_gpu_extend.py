@@ -81,6 +81,43 @@ def test_ring_rewind_beyond_slack_is_flagged_and_ignored():
     assert ei.value.status == 7 and int(ring.len[0]) == 20 and torch.equal(ring.slot_pos, before)
 
 
+@pytest.mark.parametrize("kv_dtype", ["bf16", "fp8"])
+def test_ring_replace_tail_equals_rewind_then_append(kv_dtype):
+    """The one-launch state update after a verify step against the slot simulation: every (rejected, accepted) pair
+    that fits the slack, including more rejected than accepted (left-over slots become empty) and none rejected."""
+    B, Hkv, D, n_sink, W, slack = 3, 2, 128, 4, 16, 6
+    cap = W + slack
+    f8 = kv_dtype == "fp8"
+    k_scale, v_scale = np.float32([0.02, 0.011]), np.float32([0.015, 0.03])
+    ks = dict(k_scale=torch.from_numpy(k_scale).cuda(), v_scale=torch.from_numpy(v_scale).cuda()) if f8 else {}
+    ring = wm.Ring(B, Hkv, D, n_sink, W, cap=cap, **ks)
+    ws = wm.Workspace(B, 16, Hkv, D)
+    wm.wmtp_ring_reset(ring)
+    sims = [R.RingSim(n_sink, cap, Hkv, D, dtype=np.uint8 if f8 else np.uint16) for _ in range(B)]
+    stored = (lambda rows, sc: R.quantize_rows(rows, sc)) if f8 else (lambda rows, sc: rows)
+    rng = np.random.RandomState(17)
+    tid = 0
+    for it in range(40):
+        n_tok = int(rng.randint(1, 8))
+        drops = np.array([int(rng.randint(0, slack + 1)) for _ in range(B)], dtype=np.int32)
+        drops = np.minimum(drops, [s.length for s in sims]).astype(np.int32)
+        if it % 7 == 0:
+            drops[:] = 0
+        k = wi.normal_bf16(3, (1, it), (B, n_tok, Hkv, D)); v = wi.normal_bf16(3, (2, it), (B, n_tok, Hkv, D))
+        wm.wmtp_ring_replace_tail(ring, torch.from_numpy(drops).cuda() if it % 7 else None, to_dev_bf16(k), to_dev_bf16(v), ws)
+        for b in range(B):
+            sims[b].rewind(int(drops[b]))
+            for j in range(n_tok):
+                sims[b].append(stored(k[b, j], k_scale), stored(v[b, j], v_scale))
+            check_ring_against_sim(ring, b, sims[b], f"iteration {it} seq {b}")
+    wm.wmtp_device_status(ws)
+    before = ring.slot_pos.clone()
+    wm.wmtp_ring_replace_tail(ring, torch.full((B,), slack + 1, dtype=torch.int32, device="cuda"), to_dev_bf16(k), to_dev_bf16(v), ws)
+    with pytest.raises(wm.WmtpError) as ei:
+        wm.wmtp_device_status(ws)
+    assert ei.value.status == 7 and torch.equal(ring.slot_pos, before)
+
+
 @pytest.mark.parametrize("paged", [False, True])
 def test_append_many_equals_sequential_appends(paged):
     cfg = _cfg(batch=3, S0=0, S0_range=(50, 400), paged=paged, gamma=6, cap_slack=6)
