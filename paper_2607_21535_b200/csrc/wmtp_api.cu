@@ -116,6 +116,18 @@ int pick_ctas(int64_t max_tiles) {
     return c;
 }
 
+// Launches whose segments all have (about) the same number of tiles -- rings and window views in steady state: a CTA
+// count that is a multiple of the segment count puts the CTAs' range boundaries on the segment boundaries, so no CTA
+// works in two segments, which would cost it a second flush and a second merge (about 5 us on these short launches).
+// Worth up to a fifth of the SMs idle (measured at 16 and 32 sequences: 13 % idle SMs, 8-11 % faster).
+int align_ctas_to_segments(int ctas, int nseg, int64_t tiles) {
+    if (nseg > 1 && nseg < ctas && tiles > ctas) {
+        const int aligned_ctas = ctas / nseg * nseg;
+        if ((ctas - aligned_ctas) * 5 <= ctas) return aligned_ctas;
+    }
+    return ctas;
+}
+
 void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, float sm_scale, void* out, float* lse,
                void* ws) {
     const WorkspaceLayout L = workspace_layout(batch, Hq, Hkv, D);
@@ -160,6 +172,7 @@ wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm
     p.n_sink = ring->n_sink; p.W = ring->W; p.cap = ring->cap;
     const int64_t tiles = (p.rows_per_head + kTileKeys - 1) / kTileKeys * ring->batch * q_len * ring->Hkv;
     p.num_ctas = pick_ctas(tiles);
+    p.num_ctas = align_ctas_to_segments(p.num_ctas, ring->batch * q_len * ring->Hkv, tiles);
     if (p.num_ctas <= 0) return fail(WMTP_ERR_CUDA, "no CUDA device available");
     cudaError_t e = launch_attention(p, st);
     if (e != cudaSuccess) return cuda_fail(e, "windowed attention launch");
@@ -190,6 +203,7 @@ wmtp_status attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, 
         if (view_tiles < tiles_per_seg) tiles_per_seg = view_tiles;
     }
     p.num_ctas = pick_ctas(tiles_per_seg * kv->batch * q_len * kv->Hkv);
+    if (W > 0) p.num_ctas = align_ctas_to_segments(p.num_ctas, kv->batch * q_len * kv->Hkv, tiles_per_seg * kv->batch * q_len * kv->Hkv);
     if (p.num_ctas <= 0) return fail(WMTP_ERR_CUDA, "no CUDA device available");
     cudaError_t e = launch_attention(p, st);
     if (e != cudaSuccess) return cuda_fail(e, W > 0 ? "windowed (KV view) attention launch" : "full attention launch");
