@@ -288,6 +288,24 @@ __device__ __forceinline__ int wait_tiles(const unsigned long long* word, uint32
 }
 __device__ __forceinline__ int kMaxSegmentsPadded(const AttnParams& p) { return p.seg_stride; }
 
+// In-place inclusive running sum of a[0 .. n) in shared memory by one warp: every lane sums a contiguous chunk, the
+// lanes' totals are scanned with shuffles, the offsets are added back. n <= kMaxBatch: at most 32 elements per lane.
+template <typename T>
+__device__ __forceinline__ void warp_inclusive_scan(T* a, int n) {
+    const int lane = threadIdx.x & 31;
+    const int per = (n + 31) >> 5, lo = lane * per, hi = lo + per < n ? lo + per : n;
+    T sum = 0;
+    for (int i = lo; i < hi; ++i) { sum += a[i]; a[i] = sum; }
+    T incl = sum;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const T up = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    const T before = incl - sum;
+    for (int i = lo; i < hi; ++i) a[i] += before;
+}
+
 // One (sequence, KV head) segment as seen by a CTA.
 struct Segment {
     int b, g, seg;
@@ -527,33 +545,35 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             }
         }
         cta_flags[0] = 0;
+        cta_flags[1] = 0;                                    // segments that hold at least one tile (counted below)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     const uint32_t epoch = *reinterpret_cast<const volatile uint32_t*>(p.epoch);
     const int par_off = (epoch & 1u) ? kMaxSegmentsPadded(p) : 0;        // which copy of the per-segment words this launch uses
 
-    // ---- plan: tiles per sequence and partial-slot capacity per sequence (all from len[], O(B))
+    // ---- plan: tiles per sequence and partial-slot capacity per sequence (all from len[]; O(B / 32) steps: the
+    //      per-sequence values are computed by all threads, the two running sums by one warp)
     for (int b = threadIdx.x; b < p.B; b += blockDim.x)
         tile_prefix[b + 1] = seq_view(p, b).tiles;
+    if (threadIdx.x == 0) { tile_prefix[0] = 0; cap_prefix[0] = 0; }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        int64_t acc = 0;
-        tile_prefix[0] = 0;
-        for (int b = 0; b < p.B; ++b) { acc += tile_prefix[b + 1]; tile_prefix[b + 1] = acc; }
-        const int64_t n_ = acc * p.Hkv;
+    if (threadIdx.x < 32) warp_inclusive_scan(tile_prefix + 1, p.B);
+    __syncthreads();
+    {
+        const int64_t n_ = tile_prefix[p.B] * p.Hkv;
         const int cn_ = effective_ctas(gridDim.x, n_);
-        int cacc = 0;
-        cap_prefix[0] = 0;
-        for (int b = 0; b < p.B; ++b) {
+        for (int b = threadIdx.x; b < p.B; b += blockDim.x) {
             // contributors of a segment: per CTA whose static range meets it (<= T * Cn / n + 2 of them), per thief
             // admitted from another segment (<= steal_slots) and per chunk straddling into it, one partial per group
             const int64_t tb = tile_prefix[b + 1] - tile_prefix[b];
             int64_t own = tb == 0 ? 0 : (n_ < (1 << 23) ? (int64_t)(((uint32_t)tb * (uint32_t)cn_) / (uint32_t)n_) : tb * cn_ / n_) + 2;
             if (own > tb) own = tb;
-            cacc += tb == 0 ? 0 : kMaxGroups * ((int)own + p.steal_slots + 1);
-            cap_prefix[b + 1] = cacc;
+            cap_prefix[b + 1] = tb == 0 ? 0 : kMaxGroups * ((int)own + p.steal_slots + 1);
+            if (tb != 0) atomicAdd(cta_flags + 1, p.Hkv);
         }
     }
+    __syncthreads();
+    if (threadIdx.x < 32) warp_inclusive_scan(cap_prefix + 1, p.B);
     __syncthreads();
     WMTP_STAMP(p, 1);
     const int G = p.G;
@@ -821,9 +841,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     const uint32_t stage0 = smem_u32(stages);
     const uint32_t bar_fullK = bar_fullK0 + 8 * (grp * C::kMaxStages), bar_fullV = bar_fullV0 + 8 * (grp * C::kMaxStages);
 
-    int nonempty_segs = 0;                               // group thread 0 only
-    if (tid == 0)
-        for (int b = 0; b < p.B; ++b) nonempty_segs += (tile_prefix[b + 1] != tile_prefix[b]) ? p.Hkv : 0;
+    const int nonempty_segs = cta_flags[1];
     bool launch_last = false;                            // group thread 0: did this group complete the launch's last segment?
     int ncontrib = 0;                                    // uniform across the group
     int ord = 0;                                         // segment entries so far (mirrors the producer's count for this group)
