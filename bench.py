@@ -209,11 +209,16 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
-    wm.lib()
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    if local_rank == 0:
+        from paper_2607_21535_b200 import build as _build
+        _build.build()                                       # no-op when libwmtp.so is up to date
+    if world > 1:
+        dist.barrier()
+    wm.lib()
 
     cfg = pick_config(args.workload, 0)
     if args.kv_dtype == "fp8":

@@ -10,6 +10,9 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
+    # the tests exercise the in-tree library: (re)build it when it is missing or older than its sources
+    from paper_2607_21535_b200 import build as _build
+    _build.build()
 
 
 @pytest.fixture(scope="session")
