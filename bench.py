@@ -121,6 +121,16 @@ def pick_config(name: str, steps_total: int):
     return cfg
 
 
+def cpu_model() -> str:
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.lower().startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def oracle_sample(wl, n_threads_hint=None):
     """Times the CPU oracle, as it stands, on one windowed and one full-context draft step (sequence 0)."""
     from oracle import reference as R
@@ -162,7 +172,7 @@ def run_reference(args, rank):
         "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": config_dict(cfg, args),
         "variants": {"windowed": {"us_per_step": statistics.mean(tw) * 1e6}, "full": {"us_per_step": statistics.mean(tf) * 1e6}},
-        "cpu_baseline": {"value": per_step_us, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": per_step_us, "unit": UNIT, "cores": thr, "kind": "oracle", "cpu_model": cpu_model(), "sample": sample},
         "e2e": {"value": per_step_us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -509,7 +519,7 @@ def main():
                 t_win, t_full, thr = oracle_sample(wl)
                 tws.append(t_win); tfs.append(t_full)
             t_win, t_full = statistics.mean(tws), statistics.mean(tfs)
-            cpu = {"value": (t_win + t_full) / 2 * 1e6, "unit": UNIT, "cores": thr, "kind": "oracle",
+            cpu = {"value": (t_win + t_full) / 2 * 1e6, "unit": UNIT, "cores": thr, "kind": "oracle", "cpu_model": cpu_model(),
                    "sample": f"{len(tws)} x [1 windowed ({t_win * 1e3:.1f} ms) + 1 full-context ({t_full * 1e3:.1f} ms) draft-attention "
                              f"step of sequence 0, all {cfg.Hq} query heads], {time.perf_counter() - t_begin:.1f} s of CPU work, "
                              f"host has {os.cpu_count()} logical cores"}
