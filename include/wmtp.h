@@ -40,7 +40,8 @@ typedef enum {
     WMTP_ERR_CAPACITY = 3,       /* a length would exceed the ring / KV capacity */
     WMTP_ERR_WORKSPACE = 4,      /* workspace missing, misaligned or too small */
     WMTP_ERR_CUDA = 5,           /* a CUDA runtime / driver call failed (no device, launch error) */
-    WMTP_ERR_DEVICE_TIMEOUT = 6, /* a bounded device-side wait expired; outputs of that call are invalid */
+    WMTP_ERR_DEVICE_TIMEOUT = 6, /* a bounded device-side wait expired; outputs of that call are invalid and the workspace
+                                    must be initialised again (wmtp_workspace_init) before it is reused */
     WMTP_ERR_DEVICE_BOUNDS = 7   /* a device-side index check failed (page id, append past capacity) */
 } wmtp_status;
 
