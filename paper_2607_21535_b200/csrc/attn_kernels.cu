@@ -6,19 +6,21 @@
 // all S positions for the full-context (native) draft of Section 3. The work is bound by the
 // HBM read of K and V, so the kernel is organised around keeping bytes in flight:
 //
-//   * one persistent CTA per SM; the tile line (attn_plan.cuh) is split into one contiguous range per
-//     CTA, and the tail of every range can be taken over by CTAs that finish early (SMs do not all
-//     stream at the same rate);
+//   * at most one persistent CTA per SM (the launcher takes seven eighths of the SMs for long bf16 streams:
+//     the memory system delivers more to fewer requesters); the tile line (attn_plan.cuh) is split into one
+//     contiguous range per CTA, and the tail of every range can be taken over by CTAs that finish early
+//     (SMs do not all stream at the same rate);
 //   * a producer warp streams K and V tiles into a ring of shared-memory stages with TMA
 //     (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers) and tells the consumers
 //     which tile each stage holds;
 //   * consumer groups of four warps take whole tiles in turn (one group when a stage holds 64 KB, two
 //     when it holds less -- head_dim 128 or an fp8 store -- where a tile carries fewer bytes for the same
-//     softmax work); each warp of a group takes 16 keys of the tile. Scores are computed as S^T[key, head] = K[key, :] . Q^T (keys
-//     on the MMA M dimension, the G <= 8 query heads of the GQA group exactly on N = 8), the online
-//     softmax runs in fp32, and O^T[d, head] += V^T[d, key] . P^T[key, head] accumulates in
-//     registers. The 8-row problem is far too small for tcgen05 (M >= 64); mma.sync.m16n8k16 needs a
-//     few percent of tensor peak here;
+//     softmax work, and the producer's warpgroup then hands registers to the consumers'); each warp of a
+//     group takes 16 keys of the tile. Scores are computed as S^T[key, head] = K[key, :] . Q^T (keys on the
+//     MMA M dimension, the G <= 8 query heads of the GQA group exactly on N = 8), the online softmax runs
+//     in fp32, and O^T[d, head] += V^T[d, key] . P^T[key, head] accumulates in registers. The 8-row problem
+//     is far too small for tcgen05 (M >= 64); mma.sync.m16n8k16 needs a few percent of tensor peak here.
+//     The codes of an fp8 store are widened to f16 after ldmatrix and take the f16 MMA;
 //   * every K/V byte is read once from HBM and once from shared memory, shared by all heads
 //     of the group;
 //   * the launch is cooperative (all CTAs co-resident): after publishing its partial a group waits,
