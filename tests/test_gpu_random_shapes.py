@@ -38,6 +38,11 @@ def test_random_shape(idx):
         wl = wi.make_workload(cfg)
         dw = DeviceWorkload(wl)
         dw.run_loops()
+        # the same windowed steps read straight from a second copy of the KV store (window view), loop form
+        dv = DeviceWorkload(wl)
+        out_v, lse_v = torch.full_like(dv.q, float("nan")), torch.full_like(dv.lse_w, float("nan"))
+        wm.wmtp_draft_loop_windowed_kv(dv.kv, cfg.n_sink, cfg.W, dv.q, dv.k_new, dv.v_new, out_v, dv.ws, lse=lse_v)
+        wm.wmtp_device_status(dv.ws)
         seqs = sorted(set([0, cfg.batch - 1, int(np.argmax(wl.seq_lens)), int(np.argmin(wl.seq_lens))]))
         for b in seqs:
             orc = oracle_for(wl, b)
@@ -46,6 +51,7 @@ def test_random_shape(idx):
                 tag = f"{cfg} ctas={max_ctas} stealing={stealing} seq={b} step={i}"
                 compare(dw.out_w[i, b], dw.lse_w[i, b], *r["win"], what=tag + " windowed")
                 compare(dw.out_f[i, b], dw.lse_f[i, b], *r["full"], what=tag + " full")
+                compare(out_v[i, b], lse_v[i, b], *r["win"], what=tag + " window view")
             check_ring_against_sim(dw.ring, b, orc.ring, f"{cfg} seq={b}")
             assert int(dw.lens[b]) == orc.S
     finally:
