@@ -330,6 +330,22 @@ def test_tail_out_frac_matches_far_key_contribution():
 
 
 # ---------------------------------------------------------------- fp8 (e4m3) KV entries
+def test_e4m3_decode_matches_hand_worked_codes(golden_dir):
+    n = 0
+    for line in _read_golden(os.path.join(golden_dir, "e4m3_codes.txt")):
+        code, rest = line.split(None, 1)
+        got = float(R.e4m3_decode(np.array([int(code, 16)], dtype=np.uint8))[0])
+        if rest.strip() == "nan":
+            assert math.isnan(got), line
+        else:
+            num, shift = rest.split("/")
+            want = float(num) / 2.0 ** int(shift.strip()[2:])
+            assert got == want and math.copysign(1.0, got) == math.copysign(1.0, float(num)), line
+            assert int(code, 16) == int(R.e4m3_encode(np.float32([want]))[0]), line          # and back
+        n += 1
+    assert n >= 25
+
+
 def test_e4m3_decode_matches_the_format_definition_and_torch():
     import torch
     codes = np.arange(256, dtype=np.uint8)
