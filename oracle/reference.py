@@ -24,8 +24,7 @@ What is here, and the passage each part restates:
                        scale per KV head, value = code value * scale; new rows are quantised
                        on append with round-to-nearest-even and saturation at 448.
 
-Readings of points the paper leaves open are listed in the repository's design notes;
-the ones that matter here: the window includes the token appended in the same step; sink
+Readings of points the paper leaves open, as far as they matter here: the window includes the token appended in the same step; sink
 and window never double-count a position; the sink slots are fixed and only the window
 region of the ring is circular; query head h reads KV head h // (Hq // Hkv); the softmax
 scale defaults to 1/sqrt(D).
@@ -35,7 +34,8 @@ pure-Python twin on tiny inputs, torch's scaled_dot_product_attention in fp64, t
 windowed == full identity for S <= n_sink + W, the mass identity, hand-written key sets
 under tests/golden/; for fp8: hand-worked codes of the format, torch's float8_e4m3fn cast,
 brute-force nearest-code search, equality with the bf16 read-out on exactly representable
-values.  No function here is "parity unpinned".
+values; ``win_perturb`` by hand vectors that fix its numerator and denominator separately.
+No function here is "parity unpinned".
 """
 from __future__ import annotations
 

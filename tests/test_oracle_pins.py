@@ -329,6 +329,32 @@ def test_tail_out_frac_matches_far_key_contribution():
     np.testing.assert_allclose(R.win_perturb(of, of), 0.0, atol=1e-15)
 
 
+def test_win_perturb_is_the_difference_norm_over_the_full_norm():
+    """Appendix D, caption of the attention-mass table: win_perturb = ||o_full - o_win|| / ||o_full||.
+    Hand vectors fix numerator and denominator separately: a 3-4-5 triangle whose windowed read-out has
+    another norm than the full one, so dividing by ||o_win|| (4/3) or by nothing (4) cannot pass."""
+    assert R.win_perturb([3.0, 4.0], [3.0, 0.0]) == pytest.approx(4.0 / 5.0, abs=1e-15)
+    assert R.win_perturb([3.0, 0.0], [3.0, 4.0]) == pytest.approx(4.0 / 3.0, abs=1e-15)     # not symmetric in its arguments
+    assert R.win_perturb([0.0, 5.0], [0.0, -5.0]) == pytest.approx(2.0, abs=1e-15)          # a sign flip doubles, not cancels
+    # rows are treated one by one (the last axis is the head dimension)
+    got = R.win_perturb([[3.0, 4.0], [6.0, 8.0]], [[3.0, 0.0], [0.0, 8.0]])
+    np.testing.assert_allclose(got, [0.8, 0.6], atol=1e-15)
+    # on real oracle read-outs with ||o_win|| != ||o_full||: the norms written out as plain sums
+    cfg = _small_cfg(S0=240, W=16, n_sink=2, D=16)
+    wl = wi.make_workload(cfg, threads=1)
+    o = R.DraftOracle(wl.K[0], wl.V[0], cfg.Hq, cfg.n_sink, cfg.W)
+    r = o.step(wl.q[0, 0], wl.k_new[0, 0], wl.v_new[0, 0])
+    (ow, _), (of, _) = r["win"], r["full"]
+    got = R.win_perturb(of, ow)
+    for h in range(cfg.Hq):
+        num = math.sqrt(sum((float(of[h, d]) - float(ow[h, d])) ** 2 for d in range(cfg.D)))
+        den_full = math.sqrt(sum(float(of[h, d]) ** 2 for d in range(cfg.D)))
+        den_win = math.sqrt(sum(float(ow[h, d]) ** 2 for d in range(cfg.D)))
+        assert abs(den_full - den_win) > 0.05 * den_full          # the case separates the two denominators
+        assert got[h] == pytest.approx(num / den_full, rel=1e-12)
+        assert abs(got[h] - num / den_win) > 1e-3
+
+
 # ---------------------------------------------------------------- fp8 (e4m3) KV entries
 def test_e4m3_decode_matches_hand_worked_codes(golden_dir):
     n = 0
