@@ -9,6 +9,9 @@
  * Conventions for every call
  *  - Pointers marked "device" are CUDA device memory owned by the caller; the library
  *    allocates nothing on the device and keeps no reference after the call's work has run.
+ *    Process-wide state: a launch counter, per-device caches of device attributes, and the three
+ *    test knobs at the end of this file (wmtp_set_max_ctas, wmtp_set_work_stealing,
+ *    wmtp_set_wait_limit); nothing else outlives a call.
  *    Descriptors (wmtp_ring, wmtp_kv) are plain host structs, read during the call only.
  *  - bf16 tensors are row-major with head_dim D contiguous; base pointers 16-byte aligned.
  *  - `stream` is a cudaStream_t passed as void*. Calls only enqueue work on it; nothing
@@ -108,8 +111,9 @@ size_t wmtp_ring_bytes(int batch, int Hkv, int D, int n_sink, int cap, size_t* p
  * Workspace for the attention calls: split-KV partial results, their completion counters and
  * the sticky device status word. Size depends only on (batch, Hq, Hkv, D). The workspace must be
  * 256-byte aligned and initialised once with wmtp_workspace_init before its first use; after that
- * the kernels leave it ready for the next call. Calls sharing one workspace must be ordered on
- * one stream.
+ * the kernels leave it ready for the next call, whatever its shape: one workspace sized for the
+ * largest (batch, Hq, Hkv, D) serves decode steps and draft-extend launches in any order. Calls
+ * sharing one workspace must be ordered on one stream.
  */
 size_t      wmtp_workspace_bytes(int batch, int Hq, int Hkv, int D);
 wmtp_status wmtp_workspace_init(void* workspace, size_t ws_bytes, void* stream);
@@ -286,6 +290,12 @@ void    wmtp_set_max_ctas(int max_ctas);
  * shortens long launches by several percent but makes the low bits of the result depend on timing. 0 selects a
  * fixed partition: bit-reproducible results. Process-wide. */
 void    wmtp_set_work_stealing(int enabled);
+/* Polls a CTA of the attention kernels spends waiting for a word another CTA of the same launch writes (a segment's
+ * arrival count, the end-of-launch count) before it gives up, flags WMTP_ERR_DEVICE_TIMEOUT in the workspace and
+ * carries on to the end of the kernel; 0 restores the default (2^22 polls, seconds). Waits on the kernel's own
+ * shared-memory barriers are not affected. Process-wide; meant for tests of the give-up path: with a limit of one
+ * poll a multi-CTA launch reports the timeout, its outputs are invalid and the workspace needs wmtp_workspace_init. */
+void    wmtp_set_wait_limit(int polls);
 /* Number of kernels this library has launched in this process (all threads). */
 int64_t wmtp_launch_count(void);
 
@@ -307,7 +317,9 @@ int64_t wmtp_launch_count(void);
  *     clears the words that must start at zero. Two calls whose GPU work can overlap (different
  *     streams without ordering) race on it: order them on one stream or with events.
  *   - The sticky device status lives in the array too and is cleared at the start of each call; it is
- *     not reported (the windowed path has no page table whose ids could be out of range).
+ *     not reported. The windowed path has no page table whose ids could be out of range; a bounded
+ *     device-side wait that expired goes unnoticed here, so callers that need that report use the
+ *     workspace form and wmtp_device_status.
  * Arguments as wmtp_draft_attn_windowed, without workspace.
  */
 wmtp_status wmtp_draft_attn_windowed_noalloc(const void* q, int Hq, const wmtp_ring* ring, float sm_scale,

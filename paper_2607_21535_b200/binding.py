@@ -88,6 +88,7 @@ _SIGNATURES = {
                                            c_void_p]),
     "wmtp_set_max_ctas": (None, [c_int]),
     "wmtp_set_work_stealing": (None, [c_int]),
+    "wmtp_set_wait_limit": (None, [c_int]),
     "wmtp_launch_count": (c_int64, []),
 }
 
@@ -138,7 +139,7 @@ class Ring:
 
     ``k_scale`` / ``v_scale`` (device fp32 [Hkv]) select an fp8 (e4m3) store: uint8 codes, value = code * scale."""
 
-    def __init__(self, batch, Hkv, D, n_sink, W, cap=None, device="cuda", guard: int = 0, k_scale=None, v_scale=None):
+    def __init__(self, batch, Hkv, D, n_sink, W, cap=None, device="cuda", k_scale=None, v_scale=None):
         cap = W if cap is None else cap
         self.batch, self.Hkv, self.D, self.n_sink, self.W, self.cap = batch, Hkv, D, n_sink, W, cap
         slots = n_sink + cap
@@ -371,6 +372,10 @@ def wmtp_set_max_ctas(n: int) -> None:
 
 def wmtp_set_work_stealing(enabled: bool) -> None:
     lib().wmtp_set_work_stealing(1 if enabled else 0)
+
+
+def wmtp_set_wait_limit(polls: int) -> None:
+    lib().wmtp_set_wait_limit(int(polls))
 
 
 def wmtp_launch_count() -> int:

@@ -32,6 +32,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <mutex>
+
 #include "attn_plan.cuh"
 #include "fp8_util.cuh"
 
@@ -46,7 +48,9 @@ constexpr int kGroupWarps = 4;                  // warps per consumer group: 4 x
 constexpr int kGroupThreads = kGroupWarps * 32;
 constexpr int kMaxGroups = 2;
 constexpr int kMaxParts = kMaxGroups * kMaxCtas; // partials one segment can receive
-constexpr uint32_t kSpinLimit = 1u << 22;       // bounded waits
+constexpr uint32_t kSpinLimit = 1u << 22;       // bounded waits on mbarriers (the waits on other CTAs take AttnParams::spin_limit)
+constexpr uint32_t kDrainLimit = 1u << 12;      // polls per barrier when a CTA that gave up waits for its copies in flight
+constexpr int kAbortWord = 1, kAbortBarrier = 2; // values of a CTA's abort flag: which kind of wait expired first
 // Per-group scratch, used for two things in turn:
 //   the warp merge of a flush: [4 warps][8 heads][pass columns + 4] floats, `pass columns` of d at a time;
 //   the combine: weights [heads of this contributor's slice][np], inverses [8], a reduction buffer [128] float4 and the
@@ -56,9 +60,7 @@ constexpr int kCombineWeights = 2 * kMaxParts;
 constexpr int kCombineFloats = kCombineWeights + 8 + 4 * kGroupThreads + kMaxParts;
 static_assert(kMaxGroup * kMaxGroup <= kCombineWeights, "weights of a slice must fit");
 constexpr int kMaxContrib = 32;     // segments a group may have outstanding before it combines them
-#ifndef WMTP_CHUNK_BYTES
-#define WMTP_CHUNK_BYTES 262144
-#endif
+constexpr int kStealChunkBytes = 262144;        // bytes of K/V handed out per cursor step
 // per-group bookkeeping in shared memory (ints): [0] launch-last flag, [1] broadcast word, then
 // contrib[kMaxContrib][4] = {seg, b, g, slot}, reg_k[kMaxContrib] (slot of the group's i-th contribution, producer -> group)
 constexpr int kGroupInts = 4 + 5 * kMaxContrib;
@@ -80,7 +82,7 @@ struct Cfg {
     static constexpr int kRowVecs = D * kElemBytes / 16;      // 16-byte vectors per stored row
     // Tiles handed out per cursor step. A step costs a global atomic (about 1.5 us) that is fetched one chunk ahead: the
     // chunk must take longer than that to stream, so it is sized in bytes (256 KB), not in tiles.
-    static constexpr int kStealChunk = WMTP_CHUNK_BYTES / kStageBytes;
+    static constexpr int kStealChunk = kStealChunkBytes / kStageBytes;
     static constexpr int kStealMinTiles = 8 * kStealChunk;   // ranges shorter than this are streamed statically
     // columns of d merged per pass of a flush: the two-group configurations trade a second pass for shared memory
     static constexpr int kPassCols = (kGroups == 2) ? 64 : 128;
@@ -98,11 +100,7 @@ struct Cfg {
     // warpgroup-wide: the producer's warpgroup is filled up with three warps that execute it and exit.
     static constexpr bool kRebalance = (kGroups == 2);
     static constexpr int kPadWarps = kRebalance ? 3 : 0;
-#ifndef WMTP_REGS_P
-#define WMTP_REGS_P 56
-#define WMTP_REGS_C 224
-#endif
-    static constexpr int kRegsProducer = WMTP_REGS_P, kRegsConsumer = WMTP_REGS_C;
+    static constexpr int kRegsProducer = 56, kRegsConsumer = 224;
     // the 8 consumer warps and the 4 warps of the producer's warpgroup share what the 12 warps were launched with
     static_assert(8 * kRegsConsumer + 4 * kRegsProducer <= 12 * 168, "register trade must balance");
     static constexpr int kThreads = (kConsumerWarps + 1 + kPadWarps) * 32;
@@ -115,34 +113,6 @@ struct Cfg {
     static constexpr int kFixedBytes = (kFixedRaw + 1023) / 1024 * 1024;
     static_assert(kMaxStages % kGroups == 0, "a stage must always serve the same group");
 };
-
-// Development aid (compiled out unless WMTP_TRACE is defined): CTA 0 records %globaltimer at phase boundaries
-// into the workspace header, bytes [64, 256).
-#ifdef WMTP_TRACE
-#define WMTP_STAMP(p, i)                                                                      \
-    do {                                                                                      \
-        if (blockIdx.x == 0 && (threadIdx.x == 0)) {                                          \
-            unsigned long long t_;                                                            \
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                            \
-            reinterpret_cast<unsigned long long*>(reinterpret_cast<char*>((p).status) + 64)[i] = t_; \
-        }                                                                                     \
-    } while (0)
-// per-CTA record {entry, first tile landed, tiles done, smid} right behind the partial-o area (trace builds enlarge the workspace)
-#define WMTP_CTA_STAMP(p, i)                                                                  \
-    do {                                                                                      \
-        if (threadIdx.x == 0) {                                                               \
-            unsigned long long t_;                                                            \
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                            \
-            unsigned long long* rec_ = reinterpret_cast<unsigned long long*>(                 \
-                (p).part_o + pool_slots((p).B * (p).Hkv) * (p).G * (p).D) + 4 * blockIdx.x; \
-            rec_[i] = t_;                                                                     \
-            if ((i) == 0) { unsigned sm_; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_)); rec_[3] = sm_; } \
-        }                                                                                     \
-    } while (0)
-#else
-#define WMTP_STAMP(p, i) do { } while (0)
-#define WMTP_CTA_STAMP(p, i) do { } while (0)
-#endif
 
 // ---- PTX wrappers -----------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -167,40 +137,30 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: gives up after kSpinLimit polls (or as soon as another thread has given up), raises
 // the CTA's abort flag and the sticky device status; the caller carries on with invalid data so that
-// every thread still follows the same control flow and nobody is left waiting.
+// every thread still follows the same control flow and nobody is left waiting. Before a CTA that gave up
+// on a barrier leaves the kernel it waits, again bounded, for the copies that may still be in flight
+// into its shared memory (drain_stages).
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
     if (mbar_try_wait(bar, parity)) return;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return;
         if ((i & 1023u) == 1023u && *abort_flag) return;
     }
-    *abort_flag = 1;
+    if (*abort_flag == 0) *abort_flag = kAbortBarrier;
     atomicCAS(status, 0, kErrTimeout);
 }
-#ifndef WMTP_TMA_3D
-#define WMTP_TMA_3D 1
-#endif
-#ifndef WMTP_TMA_HINT
-#define WMTP_TMA_HINT 0
-#endif
-#ifndef WMTP_L2_PROMO
-#define WMTP_L2_PROMO 3
-#endif
-[[maybe_unused]] __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t policy) {
-#if WMTP_TMA_HINT
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
-#else
-    (void)policy;
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-#endif
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
 }
 // Whole K (or V) tile in one instruction: box {64 elements, 64 rows, D/64 column chunks} of the 3-D view
 // [chunk][row][64] of the tensor; lands in shared memory as [chunk][row][128 B], 128-byte swizzled.
-[[maybe_unused]] __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int y, uint32_t bar) {
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(map), "r"(0), "r"(y), "r"(0), "r"(bar) : "memory");
@@ -261,30 +221,31 @@ __device__ __forceinline__ void group_barrier(int grp) { asm volatile("bar.sync 
 
 // Bounded spin on a global word written by other CTAs of this (cooperative) launch: waits until
 // (value - base) >= target in wrap-around arithmetic.
-__device__ __forceinline__ uint32_t wait_word(const void* word, uint32_t base, uint32_t target, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ uint32_t wait_word(const void* word, uint32_t base, uint32_t target, uint32_t limit, volatile int* abort_flag,
+                                              int* status) {
     uint32_t v = 0;
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(word) : "memory");
         if (v - base >= target) return v;
         if ((i & 255u) == 255u && *abort_flag) return v;
         __nanosleep(32);
     }
-    *abort_flag = 1;
+    if (*abort_flag == 0) *abort_flag = kAbortWord;
     atomicCAS(status, 0, kErrTimeout);
     return v;
 }
 
 // Bounded spin on a segment's arrival word until its tile count (low half) reaches `tiles`; returns the number of
 // published partials (high half).
-__device__ __forceinline__ int wait_tiles(const unsigned long long* word, uint32_t tiles, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ int wait_tiles(const unsigned long long* word, uint32_t tiles, uint32_t limit, volatile int* abort_flag, int* status) {
     unsigned long long v = 0;
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(word) : "memory");
         if ((uint32_t)v >= tiles) return (int)(v >> 32);
         if ((i & 255u) == 255u && *abort_flag) return 0;
         __nanosleep(32);
     }
-    *abort_flag = 1;
+    if (*abort_flag == 0) *abort_flag = kAbortWord;
     atomicCAS(status, 0, kErrTimeout);
     return 0;
 }
@@ -361,7 +322,6 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
     float* inv_sm = scratch + kCombineWeights;                              // [8], indexed by head - first head of the slice
     float4* red = reinterpret_cast<float4*>(inv_sm + 8);                    // [128]
     int* perm = reinterpret_cast<int*>(inv_sm + 8 + 4 * kGroupThreads);     // [np] visiting order
-    WMTP_STAMP(p, 7);
 
     // ---- visiting order: the fixed partition ranks the partials by their keys; with stealing on they are taken as stored
     const bool ranked = !p.steal_slots_enabled;
@@ -445,7 +405,6 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
         }
     }
     group_barrier(grp);
-    WMTP_STAMP(p, 8);
     __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + g * G) * D;
     for (int c0 = col_lo; c0 < col_hi; c0 += kGroupThreads) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -499,7 +458,10 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
 //                half is the number of partials to combine. One hop, no "ready" flag;
 //   segs_done    completed segments; the group that completes the last one advances the epoch and, after every
 //                CTA has stopped taking tiles (grab_done, which also means it has read len[] for the last
-//                time), resets the cursors, clears the other copy and advances the lengths of a fused append.
+//                time), resets the cursors, clears the other copy and advances the lengths of a fused append;
+//   dirty[2]     (header) segments whose words each copy may hold non-zero: launches on one workspace may differ in
+//                their segment count (a draft-extend between decode steps), so the other copy is cleared over the
+//                count of the launch that used it last, not over this launch's.
 
 // ---------------------------------------------------------------------------------------------
 // The attention kernel (one cooperative launch per draft step)
@@ -530,8 +492,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     int* cap_prefix = reinterpret_cast<int*>(tile_prefix + (p.B + 1));                    // [B + 1]
     volatile int* abort_flag = cta_flags;
 
-    WMTP_STAMP(p, 0);
-    WMTP_CTA_STAMP(p, 0);
     if (threadIdx.x == C::kConsumerWarps * 32) {            // descriptor fetch overlaps the len[] round trip
         asm volatile("prefetch.tensormap [%0];" ::"l"(&mapK) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&mapV) : "memory");
@@ -577,7 +537,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     __syncthreads();
     if (threadIdx.x < 32) warp_inclusive_scan(cap_prefix + 1, p.B);
     __syncthreads();
-    WMTP_STAMP(p, 1);
     const int G = p.G;
     const int nseg = p.B * p.Hkv;
     const int64_t n = (int64_t)p.Hkv * tile_prefix[p.B];
@@ -598,7 +557,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         }
         return;
     }
-    WMTP_STAMP(p, 2);
     const bool slack = (p.mode == kRing) && (p.cap != p.W);
 
     if ((int)(threadIdx.x >> 5) >= C::kConsumerWarps) {
@@ -615,13 +573,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         // Tile number `it` of this CTA goes to stage it % nst (kept incrementally: ps, with the parity pph of the
         // stage's use count) and to consumer group it % kGroups.
         const uint32_t stage0 = smem_u32(stages);
-        uint64_t policy = 0;
-#if WMTP_TMA_HINT == 1
-        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-#elif WMTP_TMA_HINT == 2
-        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
-#endif
-        (void)policy;
         uint32_t it = 0, ps = 0, pph = 0;
         int cur_seg = -1;                    // segment of the last issued tile
         int64_t cur_lo = 0, cur_hi = 0;      // its tile range
@@ -685,21 +636,9 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                                 const uint32_t dstK = stage0 + s * C::kStageBytes, dstV = dstK + C::kTileBytes;
                                 stage_tile[s] = t + base + j;          // ordered before the consumers' wait by the arrive below
                                 mbar_expect_tx(bar_fullK + 8 * s, C::kTileBytes);
-#if WMTP_TMA_3D
                                 tma_load_3d(dstK, &mapK, (int)row, bar_fullK + 8 * s);
-#else
-#pragma unroll
-                                for (int c = 0; c < C::kChunks; ++c)
-                                    tma_load_2d(dstK + c * C::kChunkBytes, &mapK, c * (128 / C::kElemBytes), (int)row, bar_fullK + 8 * s, policy);
-#endif
                                 mbar_expect_tx(bar_fullV + 8 * s, C::kTileBytes);
-#if WMTP_TMA_3D
                                 tma_load_3d(dstV, &mapV, (int)row, bar_fullV + 8 * s);
-#else
-#pragma unroll
-                                for (int c = 0; c < C::kChunks; ++c)
-                                    tma_load_2d(dstV + c * C::kChunkBytes, &mapV, c * (128 / C::kElemBytes), (int)row, bar_fullV + 8 * s, policy);
-#endif
                             }
                         }
                     }
@@ -868,7 +807,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         for (int i = 0; i < ncontrib; ++i) {
             const int seg = contrib[4 * i], b = contrib[4 * i + 1], g = contrib[4 * i + 2], k = contrib[4 * i + 3];
             if (tid == 0) {
-                gints[1] = wait_tiles(p.arrive + par_off + seg, (uint32_t)contrib_tiles[i], abort_flag, p.status);
+                gints[1] = wait_tiles(p.arrive + par_off + seg, (uint32_t)contrib_tiles[i], p.spin_limit, abort_flag, p.status);
             }
             group_barrier(grp);
             const int np = gints[1];
@@ -880,8 +819,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 
     // Merge the four warps' states, publish the partial of (this group, current segment), note the contribution.
     auto flush_segment = [&]() {
-        WMTP_STAMP(p, 5);
-        WMTP_CTA_STAMP(p, 2);
 #pragma unroll
         for (int off = 4; off <= 16; off <<= 1) {
             l[0] += __shfl_xor_sync(0xffffffffu, l[0], off);
@@ -968,7 +905,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 }
             }
         }
-        WMTP_STAMP(p, 6);
         ++ncontrib;
     };
 
@@ -1058,7 +994,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         const uint32_t s = cs, ph = cph;             // stage of tile `it` and the parity of this group's use count of it
         if (!have_tile) {
             mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
-            if (it == 0) { WMTP_STAMP(p, 3); WMTP_CTA_STAMP(p, 1); }
             tt = *reinterpret_cast<volatile int64_t*>(stage_tile + s);
             const bool end = tt < 0 || *abort_flag;
             const bool outside = sg.seg < 0 || tt < sg.seg_start || tt >= sg.seg_start + sg.tiles;
@@ -1106,11 +1041,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             }
             uint32_t pb0 = 0, pb1 = 0;
             float corr0 = 1.f, corr1 = 1.f;
-#ifdef WMTP_SKIP_COMPUTE
-            if (false) {
-#else
             if (any_valid) {
-#endif
                 // ---- S^T = K . Q^T for this warp's 16 keys (two accumulator chains)
                 float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
                 if constexpr (!F8) {
@@ -1193,7 +1124,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 }
             }
             mbar_wait(bar_fullV + 8 * s, ph, abort_flag, p.status);
-            if (it == 0) WMTP_STAMP(p, 4);
             if (has_new && lane < C::kRowVecs) {
                 const uint4* src = reinterpret_cast<const uint4*>(p.v_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8);
                 uint4 x;
@@ -1203,11 +1133,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
                 if (new_ok) reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(p.v) + new_off * C::kElemBytes)[lane] = x;
             }
-#ifdef WMTP_SKIP_COMPUTE
-            if (false) {
-#else
             if (any_valid) {
-#endif
                 if (wkey0 + 16 > vhi) {
                     // rows past the end were never written (or, in a sink tile of a window view, may be): they can hold
                     // NaN/Inf bit patterns, and 0 * NaN would poison the accumulators. Zero them in shared memory.
@@ -1255,22 +1181,36 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         cs += C::kGroups;                            // nst is a multiple of kGroups: the stage stays with this group
         if (cs >= nst) { cs -= nst; cph ^= 1u; }
     }
-    WMTP_STAMP(p, 9);
 
+    // ---- a CTA that gave up on a barrier must not leave while copies into its shared memory may still land:
+    //      wait (bounded) for this group's next use of each of its stages; a stage nothing was issued for just runs
+    //      the short limit out. If even that expires the copy is lost with the CTA: the launch's results were
+    //      already invalid, the memory written is still this kernel's own.
+    if (*abort_flag == kAbortBarrier && tid == 0) {
+        for (uint32_t s2 = grp; s2 < nst; s2 += C::kGroups) {
+            const uint32_t par = s2 >= cs ? cph : cph ^ 1u;
+            for (uint32_t i = 0; i < kDrainLimit && !mbar_test_wait(bar_fullK + 8 * s2, par); ++i) { }
+            for (uint32_t i = 0; i < kDrainLimit && !mbar_test_wait(bar_fullV + 8 * s2, par); ++i) { }
+        }
+    }
     // ---- the group that completed the launch's last segment closes the launch
     if (tid == 0) gints[0] = launch_last ? 1 : 0;
     group_barrier(grp);
     if (gints[0]) {
         if (tid == 0) {
-            wait_word(p.grab_done, 0u, (uint32_t)Cg, abort_flag, p.status);   // nobody takes tiles or reads len[] any more
+            wait_word(p.grab_done, 0u, (uint32_t)Cg, p.spin_limit, abort_flag, p.status);   // nobody takes tiles or reads len[] any more
             *p.grab_done = 0;
         }
         group_barrier(grp);
         for (int c = tid; c < Cg; c += kGroupThreads) p.cur[c] = 0;
         const int other = (epoch & 1u) ? 0 : kMaxSegmentsPadded(p);
-        for (int sgi = tid; sgi < nseg; sgi += kGroupThreads) {               // the next launch's copy
+        int* dirty = p.status + 4;                                             // header ints [4], [5]
+        const int nclear = dirty[(epoch & 1u) ^ 1u];                           // segments the other copy's last user touched
+        group_barrier(grp);
+        for (int sgi = tid; sgi < nclear; sgi += kGroupThreads) {              // the next launch's copy
             p.arrive[other + sgi] = 0ull; p.nparts[other + sgi] = 0; p.nthief[other + sgi] = 0;
         }
+        if (tid == 0) { dirty[(epoch & 1u) ^ 1u] = 0; dirty[epoch & 1u] = nseg; }
         if (p.k_new) {
             for (int b = tid; b < p.B; b += kGroupThreads) {
                 if (appends_to(p, b)) p.len[b] += 1;
@@ -1278,7 +1218,6 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             }
         }
     }
-    WMTP_STAMP(p, 10);
 }
 
 // ---- host side: tensor maps and launch --------------------------------------------------------
@@ -1300,26 +1239,18 @@ EncodeTiledFn encode_fn() {
 
 // View of a K or V tensor [rows][D] for TMA, 128-byte swizzle; `esz` bytes per entry (2: bf16, 1: e4m3 codes), so a
 // 128-byte chunk of a row holds 128 / esz entries.
-//   3-D (default): dims {128/esz, rows, D esz/128} with strides {D esz, 128} bytes, box {128/esz, 64, D esz/128}: one copy per tile.
-//   2-D: dims {D, rows}, box {128/esz, 64}: D esz/128 copies per tile.
+// 3-D view: dims {128/esz, rows, D esz/128} with strides {D esz, 128} bytes, box {128/esz, 64, D esz/128}: one copy per tile.
 bool make_map(CUtensorMap* map, const void* base, int64_t rows, int D, int esz) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint32_t estr[3] = {1, 1, 1};
     const cuuint32_t per_chunk = 128 / esz, chunks = D * esz / 128;
-#if WMTP_TMA_3D
     const cuuint64_t dims[3] = {per_chunk, (cuuint64_t)rows, chunks};
     const cuuint64_t strides[2] = {(cuuint64_t)D * esz, 128};
     const cuuint32_t box[3] = {per_chunk, (cuuint32_t)kTileKeys, chunks};
     const cuuint32_t rank = 3;
-#else
-    const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)D * esz};
-    const cuuint32_t box[2] = {per_chunk, (cuuint32_t)kTileKeys};
-    const cuuint32_t rank = 2;
-#endif
     return fn(map, esz == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, (CUtensorMapL2promotion)WMTP_L2_PROMO,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -1336,13 +1267,17 @@ cudaError_t launch_fused(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaSt
     while (stages > C::kGroups && partial_smem_bytes<D, F8>(p.B, stages) > 227 * 1024) stages -= C::kGroups;
     p.stages = stages;
     const size_t smem = partial_smem_bytes<D, F8>(p.B, stages);
-    static bool attr_set[64] = {};          // per device: the opt-in to > 48 KB of dynamic shared memory
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(attn_fused_tma<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    {
+        static std::mutex mu;
+        static bool attr_set[64] = {};      // per device: the opt-in to > 48 KB of dynamic shared memory
+        int dev = 0;
+        cudaGetDevice(&dev);
+        std::lock_guard<std::mutex> lock(mu);
+        if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+            cudaError_t e = cudaFuncSetAttribute(attn_fused_tma<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+            if (e != cudaSuccess) return e;
+            if (dev >= 0 && dev < 64) attr_set[dev] = true;
+        }
     }
     void* args[] = {&mk, &mv, &p};
     // cooperative: the CTAs wait on one another in the combine, so they must all be resident

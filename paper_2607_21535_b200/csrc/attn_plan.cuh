@@ -2,10 +2,10 @@
 //
 // Every (sequence b, KV head g) pair is a *segment* of tiles_b = ceil(keys_b / kTileKeys) tiles;
 // segments are laid end to end on one line of n tiles in (b, g) order. CTA c of C owns the tile
-// range [c*n/C, (c+1)*n/C). A CTA emits one partial result per segment it touches; the partial of
-// (CTA c, segment s) is stored at index c + s, which is injective and makes the partials of one
-// segment contiguous. Everything is computed from the device-resident lengths in O(B) per CTA;
-// nothing is O(S) and nothing comes from the host.
+// range [c*n/C, (c+1)*n/C). A consumer group emits one partial result per segment it enters; a
+// segment's partials live in its own run of slots (handed out by an atomic counter in the order of
+// entry). Everything is computed from the device-resident lengths in O(B) per CTA; nothing is O(S)
+// and nothing comes from the host.
 #pragma once
 
 #include "wmtp_internal.h"
@@ -89,37 +89,16 @@ __device__ __forceinline__ bool ring_slot_live(int s, int64_t S, int n_sink, int
     return age < W;
 }
 
-// Fills tile_prefix[0..B] (exclusive prefix of per-sequence tile counts) in shared memory.
-// Must be called by all threads of the block; ends with a __syncthreads().
-__device__ __forceinline__ void build_tile_prefix(const AttnParams& p, int64_t* tile_prefix) {
-    for (int b = threadIdx.x; b < p.B; b += blockDim.x)
-        tile_prefix[b + 1] = (scan_keys(p, b) + kTileKeys - 1) / kTileKeys;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int64_t acc = 0;
-        tile_prefix[0] = 0;
-        for (int b = 0; b < p.B; ++b) { acc += tile_prefix[b + 1]; tile_prefix[b + 1] = acc; }
-    }
-    __syncthreads();
-}
-
-// CTAs that take part: never more than there are tiles, so every participating CTA owns >= 1 tile
-// and the CTAs touching a segment are exactly tile_owner(first tile) .. tile_owner(last tile).
+// CTAs that take part: never more than there are tiles, so every participating CTA owns >= 1 tile.
 __device__ __forceinline__ int effective_ctas(int launched, int64_t n) {
     return n < (int64_t)launched ? (int)n : launched;
 }
 
-// (Tile counts below 2^23 keep c * n and (t + 1) * C inside 32 bits for C <= kMaxCtas = 256; 64-bit division
+// (Tile counts below 2^23 keep c * n and (t + 1) * C inside 32 bits for C <= kMaxCtas; 64-bit division
 // costs hundreds of dependent cycles on one thread, which the short windowed launches would feel.)
 __device__ __forceinline__ int64_t cta_range_start(int c, int64_t n, int C) {
     if (n < (1 << 23)) return (int64_t)(((uint32_t)c * (uint32_t)n) / (uint32_t)C);
     return ((int64_t)c * n) / C;   // c <= kMaxCtas and n < 2^40: no overflow
-}
-
-// CTA owning tile t: the largest c with cta_range_start(c) <= t.
-__device__ __forceinline__ int tile_owner(int64_t t, int64_t n, int C) {
-    if (n < (1 << 23)) return (int)((((uint32_t)t + 1u) * (uint32_t)C - 1u) / (uint32_t)n);
-    return (int)(((t + 1) * (int64_t)C - 1) / n);
 }
 
 // Sequence whose segment group contains global tile t (Hkv segments per sequence).

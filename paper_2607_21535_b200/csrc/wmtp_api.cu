@@ -16,6 +16,8 @@ thread_local char g_err[512] = "";
 std::atomic<int64_t> g_launches{0};
 std::atomic<int> g_max_ctas{0};
 std::atomic<int> g_stealing{1};
+std::atomic<uint32_t> g_wait_limit{0};          // 0: the default below
+constexpr uint32_t kDefaultWaitLimit = 1u << 22;
 
 wmtp_status fail(wmtp_status s, const char* fmt, ...) {
     va_list ap;
@@ -132,10 +134,19 @@ int align_ctas_to_segments(int ctas, int nseg, int64_t tiles) {
     return ctas;
 }
 
+// Where the kernel's scratch lives: the header at `base`, the cursors behind it, two copies of the per-segment words
+// `seg_stride` elements apart, then the partial results. Both the caller's workspace and the library's built-in
+// scratch array are described this way.
+struct ScratchLayout {
+    size_t counters_off;
+    int seg_stride;
+    size_t part_key_off, part_lse_off, part_o_off;
+};
+
+// Everything of AttnParams that does not depend on the kind of store.
 void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, float sm_scale, void* out, float* lse,
-               void* ws) {
-    const WorkspaceLayout L = workspace_layout(batch, Hq, Hkv, D);
-    char* base = static_cast<char*>(ws);
+               void* scratch, const ScratchLayout& L, bool stealing) {
+    char* base = static_cast<char*>(scratch);
     p.q = q; p.out = out; p.lse = lse;
     p.status = reinterpret_cast<int*>(base);
     p.epoch = reinterpret_cast<uint32_t*>(base + 4);
@@ -143,11 +154,11 @@ void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, 
     p.grab_done = reinterpret_cast<int*>(base + 12);
     p.cur = reinterpret_cast<int*>(base + 256);
     p.arrive = reinterpret_cast<unsigned long long*>(base + L.counters_off);
-    p.nparts = reinterpret_cast<int*>(p.arrive + 2 * kMaxSegments);
-    p.nthief = p.nparts + 2 * kMaxSegments;
-    p.seg_stride = kMaxSegments;
-    p.steal_slots_enabled = g_stealing.load() ? 1 : 0;
-    p.steal_slots = p.steal_slots_enabled ? steal_slots_for(batch * Hkv) : 0;
+    p.nparts = reinterpret_cast<int*>(p.arrive + 2 * L.seg_stride);
+    p.nthief = p.nparts + 2 * L.seg_stride;
+    p.seg_stride = L.seg_stride;
+    p.steal_slots_enabled = stealing ? 1 : 0;
+    p.steal_slots = stealing ? steal_slots_for(batch * Hkv) : 0;
     p.part_key = reinterpret_cast<int*>(base + L.part_key_off);
     p.part_lse = reinterpret_cast<float*>(base + L.part_lse_off);
     p.part_o = reinterpret_cast<float*>(base + L.part_o_off);
@@ -155,6 +166,25 @@ void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, 
     p.q_len = 1;
     const float s = sm_scale > 0.f ? sm_scale : 1.0f / std::sqrt((float)D);
     p.scale_log2 = s * 1.4426950408889634f;
+    const uint32_t wl = g_wait_limit.load();
+    p.spin_limit = wl ? wl : kDefaultWaitLimit;
+}
+
+void fill_attn(AttnParams& p, const void* q, int Hq, int Hkv, int batch, int D, float sm_scale, void* out, float* lse,
+               void* ws) {
+    const WorkspaceLayout W = workspace_layout(batch, Hq, Hkv, D);
+    fill_attn(p, q, Hq, Hkv, batch, D, sm_scale, out, lse, ws,
+              ScratchLayout{W.counters_off, kMaxSegments, W.part_key_off, W.part_lse_off, W.part_o_off}, g_stealing.load() != 0);
+}
+
+// The ring as the attention kernel sees it.
+void bind_ring(AttnParams& p, const wmtp_ring* ring, const void* k_new, const void* v_new) {
+    p.k = ring->k; p.v = ring->v; p.page_table = nullptr; p.len = ring->len;
+    p.f8 = ring->kv_dtype == WMTP_KV_FP8_E4M3 ? 1 : 0; p.k_scale = ring->k_scale; p.v_scale = ring->v_scale;
+    p.k_new = k_new; p.v_new = v_new; p.slot_pos = ring->slot_pos;
+    p.mode = kRing;
+    p.rows_per_head = (int64_t)ring->n_sink + ring->cap;
+    p.n_sink = ring->n_sink; p.W = ring->W; p.cap = ring->cap;
 }
 
 // k_new / v_new non-NULL: a fused draft step (append, then attend) in one launch.
@@ -168,12 +198,7 @@ wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm
     AttnParams p{};
     fill_attn(p, q, Hq, ring->Hkv, ring->batch * q_len, ring->D, sm_scale, out, lse, ws);
     p.q_len = q_len;
-    p.k = ring->k; p.v = ring->v; p.page_table = nullptr; p.len = ring->len;
-    p.f8 = ring->kv_dtype == WMTP_KV_FP8_E4M3 ? 1 : 0; p.k_scale = ring->k_scale; p.v_scale = ring->v_scale;
-    p.k_new = k_new; p.v_new = v_new; p.slot_pos = ring->slot_pos;
-    p.mode = kRing;
-    p.rows_per_head = (int64_t)ring->n_sink + ring->cap;
-    p.n_sink = ring->n_sink; p.W = ring->W; p.cap = ring->cap;
+    bind_ring(p, ring, k_new, v_new);
     const int64_t tiles = (p.rows_per_head + kTileKeys - 1) / kTileKeys * ring->batch * q_len * ring->Hkv;
     p.num_ctas = pick_ctas(tiles);
     p.num_ctas = align_ctas_to_segments(p.num_ctas, ring->batch * q_len * ring->Hkv, tiles);
@@ -243,14 +268,17 @@ void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 
 int sm_count() {
-    static std::atomic<int> cached{0};
-    int c = cached.load();
-    if (c > 0) return c;
+    static std::atomic<int> cached[64];     // per device ordinal; zero-initialised
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    const bool slot = dev >= 0 && dev < 64;
+    if (slot) {
+        const int c = cached[dev].load();
+        if (c > 0) return c;
+    }
     int n = 0;
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    cached.store(n);
+    if (slot) cached[dev].store(n);
     return n;
 }
 
@@ -262,9 +290,6 @@ WorkspaceLayout workspace_layout(int batch, int Hq, int Hkv, int D) {
     L.part_lse_off = L.part_key_off + round_up(np * sizeof(int), 256);
     L.part_o_off = L.part_lse_off + round_up(np * G * sizeof(float), 256);
     L.total = L.part_o_off + round_up(np * G * D * sizeof(float), 256);
-#ifdef WMTP_TRACE
-    L.total += 32 * kMaxCtas;     // per-CTA trace records
-#endif
     return L;
 }
 
@@ -577,6 +602,8 @@ void wmtp_set_max_ctas(int max_ctas) { g_max_ctas.store(max_ctas < 0 ? 0 : max_c
 
 void wmtp_set_work_stealing(int enabled) { g_stealing.store(enabled ? 1 : 0); }
 
+void wmtp_set_wait_limit(int polls) { g_wait_limit.store(polls > 0 ? (uint32_t)polls : 0u); }
+
 int64_t wmtp_launch_count(void) { return g_launches.load(); }
 
 // ---- allocation-free windowed attention ---------------------------------------------------------
@@ -586,16 +613,23 @@ int64_t wmtp_launch_count(void) { return g_launches.load(); }
 // the split-KV scratch of the windowed attention lives in this file-scope device array instead of a
 // caller buffer. Every GPU that loads the library holds it until the process exits.
 namespace {
-constexpr int kStaticMaxCtas = 160;        // CTAs (KV splits) the static scratch has room for
+constexpr int kStaticMaxCtas = kMaxCtas;   // CTAs (KV splits) the static scratch has room for
 constexpr int kStaticMaxSegments = 32;     // batch * Hkv
 constexpr size_t kStaticCountersOff = 256 + kCursorBytes;
-constexpr size_t kStaticPartLseOff = kStaticCountersOff + 2 * (8 + 4 + 4) * kStaticMaxSegments;       // two copies of the per-segment words
+constexpr size_t kStaticZeroBytes = kStaticCountersOff + 2 * (8 + 4 + 4) * kStaticMaxSegments;   // header, cursors, two copies of the per-segment words
+// Partial slots: with the fixed partition a segment receives at most one partial per consumer group of every CTA whose
+// range meets it; the kernel reserves kMaxGroups * (own + 1) slots per segment with own <= CTAs * tiles_b / tiles + 2,
+// which sums to at most kMaxGroups * (CTAs + 3 * segments) over a launch.
 constexpr size_t kStaticSlots = (size_t)kMaxGroups * (kStaticMaxCtas + 3 * kStaticMaxSegments);
-constexpr size_t kStaticPartKeyOff = kStaticPartLseOff;                      // int [kStaticSlots]
-constexpr size_t kStaticPartLse2Off = kStaticPartKeyOff + kStaticSlots * sizeof(int);
-constexpr size_t kStaticPartOOff = kStaticPartLse2Off + kStaticSlots * kMaxGroup * sizeof(float);
+constexpr size_t kStaticPartKeyOff = kStaticZeroBytes;                        // int [kStaticSlots]
+constexpr size_t kStaticPartLseOff = kStaticPartKeyOff + kStaticSlots * sizeof(int);
+constexpr size_t kStaticPartOOff = kStaticPartLseOff + kStaticSlots * kMaxGroup * sizeof(float);
 constexpr size_t kStaticBytes = kStaticPartOOff + kStaticSlots * kMaxGroup * 256 * sizeof(float);
-static_assert(kStaticPartLseOff % 256 == 0 && kStaticPartOOff % 256 == 0, "static scratch regions must stay 256-byte aligned");
+static_assert(kStaticMaxCtas >= kMaxCtas, "the launcher may use up to kMaxCtas CTAs");
+static_assert(kStaticSlots >= (size_t)kMaxGroups * (kMaxCtas + 3 * kStaticMaxSegments), "partial slots of the largest accepted launch");
+static_assert(kStaticPartKeyOff % 256 == 0 && kStaticPartLseOff % 256 == 0 && kStaticPartOOff % 256 == 0,
+              "static scratch regions must stay 256-byte aligned");
+static_assert(kStaticMaxSegments <= kMaxSegments, "per-segment words");
 
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];   // ~4 MiB
 
@@ -637,34 +671,14 @@ wmtp_status wmtp_draft_attn_windowed_noalloc(const void* q, int Hq, const wmtp_r
     char* base = static_cast<char*>(base_v);
     cudaStream_t st = (cudaStream_t)stream;
     // status word and this call's counters must start at zero; the array keeps the previous call's contents
-    cudaError_t e = cudaMemsetAsync(base, 0, kStaticPartLseOff, st);
+    cudaError_t e = cudaMemsetAsync(base, 0, kStaticZeroBytes, st);
     if (e != cudaSuccess) return cuda_fail(e, "clearing the static scratch header");
 
     AttnParams p{};
-    p.q = q; p.out = out; p.lse = lse;
-    p.status = reinterpret_cast<int*>(base);
-    p.epoch = reinterpret_cast<uint32_t*>(base + 4);
-    p.segs_done = reinterpret_cast<int*>(base + 8);
-    p.grab_done = reinterpret_cast<int*>(base + 12);
-    p.cur = reinterpret_cast<int*>(base + 256);
-    p.arrive = reinterpret_cast<unsigned long long*>(base + kStaticCountersOff);
-    p.nparts = reinterpret_cast<int*>(p.arrive + 2 * kStaticMaxSegments);
-    p.nthief = p.nparts + 2 * kStaticMaxSegments;
-    p.seg_stride = kStaticMaxSegments;
-    p.steal_slots_enabled = 0;                 // static partition: deterministic and the smallest partial pool
-    p.steal_slots = 0;
-    p.part_key = reinterpret_cast<int*>(base + kStaticPartKeyOff);
-    p.part_lse = reinterpret_cast<float*>(base + kStaticPartLse2Off);
-    p.part_o = reinterpret_cast<float*>(base + kStaticPartOOff);
-    p.B = ring->batch; p.Hq = Hq; p.Hkv = ring->Hkv; p.D = ring->D; p.G = Hq / ring->Hkv;
-    const float sc = sm_scale > 0.f ? sm_scale : 1.0f / std::sqrt((float)ring->D);
-    p.scale_log2 = sc * 1.4426950408889634f;
-    p.k = ring->k; p.v = ring->v; p.page_table = nullptr; p.len = ring->len;
-    p.f8 = ring->kv_dtype == WMTP_KV_FP8_E4M3 ? 1 : 0; p.k_scale = ring->k_scale; p.v_scale = ring->v_scale;
-    p.k_new = nullptr; p.v_new = nullptr; p.slot_pos = ring->slot_pos;
-    p.mode = kRing;
-    p.rows_per_head = (int64_t)ring->n_sink + ring->cap;
-    p.n_sink = ring->n_sink; p.W = ring->W; p.cap = ring->cap;
+    // static partition: deterministic and the smallest partial pool
+    fill_attn(p, q, Hq, ring->Hkv, ring->batch, ring->D, sm_scale, out, lse, base,
+              ScratchLayout{kStaticCountersOff, kStaticMaxSegments, kStaticPartKeyOff, kStaticPartLseOff, kStaticPartOOff}, false);
+    bind_ring(p, ring, nullptr, nullptr);
     const int64_t tiles = (p.rows_per_head + kTileKeys - 1) / kTileKeys * ring->batch * ring->Hkv;
     p.num_ctas = pick_ctas(tiles);
     if (p.num_ctas <= 0) return fail(WMTP_ERR_CUDA, "no CUDA device available");

@@ -21,7 +21,8 @@ constexpr size_t kWorkspaceZeroBytes = 256 + kCursorBytes + 2 * (8 + 4 + 4) * kM
 enum KvMode : int { kContiguous = 0, kPaged = 1, kRing = 2 };
 
 // Workspace layout (all offsets from a 256-byte aligned base):
-//   [0, 256)            header: int status @0, uint epoch @4, int segs_done @8, int grab_done @12
+//   [0, 256)            header: int status @0, uint epoch @4, int segs_done @8, int grab_done @12, int dirty[2] @16
+//                       (segments whose per-segment words each copy may hold non-zero), diagnostic record @32
 //   [256, 1280)         int cur[kMaxCtas]: per-CTA cursors of the work-stealing scheme
 //   counters            u64 arrive[2][kMaxSegments], int nparts[2][..], int nthief[2][..]
 //                       (fixed size: initialisation needs no shape)
@@ -82,6 +83,7 @@ struct AttnParams {
     float scale_log2;         // sm_scale * log2(e)
     int num_ctas;
     int stages;               // stages of the kernel's shared-memory ring (set by the launcher)
+    uint32_t spin_limit;      // polls a CTA spends waiting for another CTA's global word before it gives up
 };
 
 struct RingParams {
@@ -116,6 +118,6 @@ cudaError_t launch_mass_diagnostics(const void* o_win, const float* lse_win, con
                                     int D, float* mass, float* perturb, float* tail, cudaStream_t st);
 
 void count_launch(int n);
-int  sm_count();   // multiprocessors of the current device (cached), 0 on failure
+int  sm_count();   // multiprocessors of the current device (cached per device), 0 on failure
 
 }  // namespace wmtp

@@ -227,3 +227,88 @@ def test_speculative_cycle_draft_rewind_extend():
             assert pos[s] == p and (Kb[:, s] == orc.ring.K[:, s]).all()
             seen += 1
     assert seen == len(keep) and (pos < orc.S).all()
+
+
+# ------------------------------------------------------------------------------------------ one workspace, changing shapes
+@pytest.mark.parametrize("D", [128, 256])
+def test_one_workspace_serves_extend_and_decode_launches_in_turn(D):
+    """The normal speculative cycle on ONE workspace: a draft-extend launch (q_len times the (sequence, KV head) pairs
+    of a decode step), some decode steps, the next extend, ... The kernels keep two copies of their per-segment words
+    and each launch prepares the other copy for the next one, whose segment count may be larger than its own: with an
+    odd number of decode launches between two extends the second extend lands on the copy the first one used. Every
+    output is compared with the oracle's sequential steps."""
+    q_len = 4
+    cycles = [(3, False), (1, True), (2, False), (3, True)]      # (decode steps, also run the full-context loop)
+    total = sum(q_len + d for d, _ in cycles)
+    cfg = _cfg(batch=2, S0=0, S0_range=(40, 900), D=D, gamma=total, cap_slack=q_len, W=96, seed=4242 + D)
+    wl = wi.make_workload(cfg)
+    dw = DeviceWorkload(wl)
+    ws = wm.Workspace(cfg.batch * q_len, cfg.Hq, cfg.Hkv, cfg.D)
+    wm.wmtp_ring_init_from_kv(dw.ring, dw.kv)
+    orcs = [oracle_for(wl, b, with_ring=False) for b in range(cfg.batch)]
+    i = 0
+    for cyc, (d, with_full) in enumerate(cycles):
+        # ---- extend: q_len tokens appended, then attended in one launch per variant
+        sl = slice(i, i + q_len)
+        km, vm, qm = (to_dev_bf16(_per_seq(a[sl])) for a in (wl.k_new, wl.v_new, wl.q))
+        wm.wmtp_ring_append_many(dw.ring, km, vm)
+        wm.wmtp_kv_append_many(dw.kv, km, vm, ws)
+        out_w, out_f = torch.full_like(qm, float("nan")), torch.full_like(qm, float("nan"))
+        lse_w = torch.full(qm.shape[:-1], float("nan"), dtype=torch.float32, device="cuda")
+        lse_f = torch.full_like(lse_w, float("nan"))
+        wm.wmtp_draft_extend_windowed(qm, dw.ring, out_w, ws, lse=lse_w)
+        wm.wmtp_draft_extend_full(qm, dw.kv, out_f, ws, lse=lse_f)
+        wm.wmtp_device_status(ws)
+        for b in range(cfg.batch):
+            for j in range(q_len):
+                r = orcs[b].step(wl.q[i + j, b], wl.k_new[i + j, b], wl.v_new[i + j, b])
+                compare(out_w[b, j], lse_w[b, j], *r["win"], what=f"cycle {cyc} extend windowed seq {b} token {j}")
+                compare(out_f[b, j], lse_f[b, j], *r["full"], what=f"cycle {cyc} extend full seq {b} token {j}")
+        i += q_len
+        # ---- d decode steps on the same workspace
+        sl = slice(i, i + d)
+        q, kn, vn = dw.q[sl], dw.k_new[sl], dw.v_new[sl]
+        ow, of = torch.full_like(q, float("nan")), torch.full_like(q, float("nan"))
+        lw = torch.full(q.shape[:-1], float("nan"), dtype=torch.float32, device="cuda")
+        lf = torch.full_like(lw, float("nan"))
+        wm.wmtp_draft_loop_windowed(dw.ring, q, kn, vn, ow, ws, lse=lw)
+        if with_full:
+            wm.wmtp_draft_loop_full(dw.kv, q, kn, vn, of, ws, lse=lf)
+        else:
+            wm.wmtp_kv_append_many(dw.kv, to_dev_bf16(_per_seq(wl.k_new[sl])), to_dev_bf16(_per_seq(wl.v_new[sl])), ws)
+        wm.wmtp_device_status(ws)
+        for b in range(cfg.batch):
+            for j in range(d):
+                r = orcs[b].step(wl.q[i + j, b], wl.k_new[i + j, b], wl.v_new[i + j, b], full=with_full)
+                compare(ow[j, b], lw[j, b], *r["win"], what=f"cycle {cyc} decode windowed seq {b} step {j}")
+                if with_full:
+                    compare(of[j, b], lf[j, b], *r["full"], what=f"cycle {cyc} decode full seq {b} step {j}")
+        i += d
+    assert all(int(dw.ring.len[b]) == orcs[b].S and int(dw.lens[b]) == orcs[b].S for b in range(cfg.batch))
+
+
+def test_one_workspace_serves_two_batch_sizes_in_turn():
+    """Two stores of different batch size share one workspace (sized for the larger); runs of odd and even length
+    alternate, so a large launch meets per-segment words that only smaller launches have prepared since."""
+    big = _cfg(name="big", batch=4, S0=0, S0_range=(30, 1200), D=128, gamma=8, W=64, seed=515)
+    small = _cfg(name="small", batch=1, S0=700, D=128, gamma=8, W=64, seed=516)
+    wls = {c.name: wi.make_workload(c) for c in (big, small)}
+    dws = {n: DeviceWorkload(w) for n, w in wls.items()}
+    ws = wm.Workspace(big.batch, big.Hq, big.Hkv, big.D)
+    orcs = {n: [oracle_for(w, b, with_ring=False) for b in range(w.cfg.batch)] for n, w in wls.items()}
+    done = {"big": 0, "small": 0}
+    for dw in dws.values():
+        wm.wmtp_ring_init_from_kv(dw.ring, dw.kv)
+    for name, steps in (("big", 3), ("small", 3), ("big", 3), ("small", 1), ("big", 2), ("small", 2)):
+        dw, wl, i = dws[name], wls[name], done[name]
+        sl = slice(i, i + steps)
+        q = dw.q[sl]
+        ow = torch.full_like(q, float("nan"))
+        lw = torch.full(q.shape[:-1], float("nan"), dtype=torch.float32, device="cuda")
+        wm.wmtp_draft_loop_windowed(dw.ring, q, dw.k_new[sl], dw.v_new[sl], ow, ws, lse=lw)
+        wm.wmtp_device_status(ws)
+        for b in range(wl.cfg.batch):
+            for j in range(steps):
+                r = orcs[name][b].step(wl.q[i + j, b], wl.k_new[i + j, b], wl.v_new[i + j, b], full=False)
+                compare(ow[j, b], lw[j, b], *r["win"], what=f"{name} step {i + j} seq {b}")
+        done[name] += steps

@@ -396,3 +396,9 @@ def test_config_batched_paged_full_size_sampled_sequences():
 @pytest.mark.parametrize("S0,W", [(65536, 1024), (262144, 4096)])
 def test_config_sweep_shapes(S0, W):
     _run_and_check(wi.scaled(wi.CONFIGS[4], S0=S0, W=W, gamma=3, name=f"sweep_{S0}_{W}"))
+
+
+def test_config_sweep_shape_at_full_size():
+    # Hq=32, Hkv=4, D=128 at S=1,048,576 (the two-consumer-group kernel at the size the benchmark times), default CTAs;
+    # first and last draft step
+    _run_and_check(wi.scaled(wi.CONFIGS[4], name="sweep_full_size"), steps={0, 6})
