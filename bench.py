@@ -360,11 +360,11 @@ def main():
         us_win_graph = g0.elapsed_time(g1) * 1e3 / reps / gam
     except Exception as exc:                                 # graph capture unavailable: report nothing
         log(f"[bench] graph replay skipped: {exc}")
-    us_full_call = k0.elapsed_time(k1) * 1e3 / reps
     us_win_kv_call = v0.elapsed_time(v1) * 1e3 / reps
     us_win_call_cold = statistics.mean(a.elapsed_time(b) for a, b in wev) * 1e3
     us_launch_floor = l0.elapsed_time(l1) * 1e3 / reps
     cur_lens = lens.cpu().numpy()
+    us_full_call = k0.elapsed_time(k1) * 1e3 / reps
 
     # ---- windowed step time against context length: same ring shape, ring re-seeded at other lengths
     flat = None
@@ -419,9 +419,15 @@ def main():
         x2.record()
         torch.cuda.synchronize()
         wm.wmtp_device_status(ws_x)
+        ext_full_us = x1.elapsed_time(x2) * 1e3 / reps
+        ext_bytes = float(lens.cpu().numpy().sum()) * cfg.kv_bytes_per_token      # one pass over the K/V serves all q_len queries
         ext = {"q_len": ql,
                "windowed_us_per_iteration": x0.elapsed_time(x1) * 1e3 / reps,
-               "full_us_per_call": x1.elapsed_time(x2) * 1e3 / reps,
+               "full_us_per_call": ext_full_us,
+               "full_kv_bytes_per_call": ext_bytes,
+               "full_algorithmic_gbs": ext_bytes / (ext_full_us * 1e-6) / 1e9,
+               "full_pct_of_8tbs": ext_bytes / (ext_full_us * 1e-6) / 8e12 * 100,
+               "full_vs_one_decode_call": ext_full_us / us_full_call,
                "note": "windowed: rollback of q_len tokens + append of q_len tokens on a ring with 8 slack slots (one launch) + "
                        "one multi-query attention launch; full: one multi-query attention launch over the whole KV store"}
     # ---- the fp8 (e4m3) KV variant of the same workload: half the bytes per key, same launches

@@ -101,6 +101,24 @@ __device__ __forceinline__ int64_t cta_range_start(int c, int64_t n, int C) {
     return ((int64_t)c * n) / C;   // c <= kMaxCtas and n < 2^40: no overflow
 }
 
+// In-place inclusive running sum of a[0 .. n) in shared memory by one warp: every lane sums a contiguous chunk, the
+// lanes' totals are scanned with shuffles, the offsets are added back. n <= kMaxBatch: at most 32 elements per lane.
+template <typename T>
+__device__ __forceinline__ void warp_inclusive_scan(T* a, int n) {
+    const int lane = threadIdx.x & 31;
+    const int per = (n + 31) >> 5, lo = lane * per, hi = lo + per < n ? lo + per : n;
+    T sum = 0;
+    for (int i = lo; i < hi; ++i) { sum += a[i]; a[i] = sum; }
+    T incl = sum;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const T up = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    const T before = incl - sum;
+    for (int i = lo; i < hi; ++i) a[i] += before;
+}
+
 // Sequence whose segment group contains global tile t (Hkv segments per sequence).
 __device__ __forceinline__ int find_seq(const int64_t* tile_prefix, int B, int Hkv, int64_t t) {
     int lo = 0, hi = B - 1;

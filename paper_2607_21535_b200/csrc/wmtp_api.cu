@@ -484,10 +484,41 @@ wmtp_status wmtp_draft_extend_windowed(const void* q, int q_len, int Hq, const w
     return attn_windowed(q, Hq, ring, sm_scale, out, lse, workspace, ws_bytes, (cudaStream_t)stream, true, nullptr, nullptr, q_len);
 }
 
+// The shared-tile multi-query kernel (extend_kernels.cu): every K/V tile is read once for up to kExtendChunk queries of
+// a sequence. Returns false when the launch does not fit it (the per-query path then serves the call).
+static bool extend_full_shared_tiles(const void* q, int q_len, int Hq, const wmtp_kv* kv, float sm_scale, void* out, float* lse,
+                                     void* ws, cudaStream_t st, wmtp_status* result) {
+    if (q_len < 2 || kv->kv_dtype != WMTP_KV_BF16 || !extend_mq_fits(kv->batch, kv->D)) return false;
+    const int nch = (q_len + kExtendChunk - 1) / kExtendChunk, nstreams = kv->batch * kv->Hkv * nch;
+    const int slot_rows = q_len < kExtendChunk ? q_len : kExtendChunk;
+    // the partial pool of a workspace sized for batch * q_len sequences holds pool_slots rows of G x (D + 1) floats
+    const int64_t max_ctas = (int64_t)pool_slots(kv->batch * q_len * kv->Hkv) / slot_rows - nstreams;
+    if (max_ctas < 1) return false;
+    AttnParams p{};
+    fill_attn(p, q, Hq, kv->Hkv, kv->batch * q_len, kv->D, sm_scale, out, lse, ws);
+    p.B = kv->batch;                        // this kernel counts sequences, not queries
+    p.q_len = q_len;
+    p.k = kv->k; p.v = kv->v; p.page_table = kv->page_table; p.len = kv->len;
+    p.S_cap = kv->S_cap;
+    p.mode = kv->page_table ? kPaged : kContiguous;
+    p.rows_per_head = kv->page_table ? kv->page_size : kv->S_cap;
+    p.page_size = kv->page_size; p.max_pages = kv->max_pages; p.num_pages = kv->num_pages;
+    const int64_t tiles = (kv->S_cap + kTileKeys - 1) / kTileKeys * nstreams;
+    p.num_ctas = pick_ctas(tiles);
+    if (p.num_ctas <= 0) { *result = fail(WMTP_ERR_CUDA, "no CUDA device available"); return true; }
+    if (p.num_ctas > max_ctas) p.num_ctas = (int)max_ctas;
+    const cudaError_t e = launch_extend_mq(p, st);
+    *result = e == cudaSuccess ? WMTP_OK : cuda_fail(e, "multi-query draft-extend launch");
+    return true;
+}
+
 wmtp_status wmtp_draft_extend_full(const void* q, int q_len, int Hq, const wmtp_kv* kv, float sm_scale, void* out, float* lse,
                                    void* workspace, size_t ws_bytes, void* stream) {
     if (wmtp_status s = check_kv(kv)) return s;
     if (wmtp_status s = check_extend(q_len, kv->batch)) return s;
+    if (wmtp_status s = check_attn_common(q, Hq, kv->Hkv, kv->batch * q_len, kv->D, out, lse, workspace, ws_bytes)) return s;
+    wmtp_status r = WMTP_OK;
+    if (extend_full_shared_tiles(q, q_len, Hq, kv, sm_scale, out, lse, workspace, (cudaStream_t)stream, &r)) return r;
     return attn_full(q, Hq, kv, sm_scale, out, lse, workspace, ws_bytes, (cudaStream_t)stream, true, nullptr, nullptr, 0, 0, q_len);
 }
 

@@ -15,6 +15,7 @@ constexpr int kMaxGroups = 2;        // consumer groups per CTA (each contribute
 constexpr int kMaxBatch = 1024;     // sequences per call (prefix table lives in shared memory)
 constexpr int kMaxGroup = 8;        // query heads per KV head
 constexpr int kMaxSegments = 16384; // batch * Hkv per call
+constexpr int kExtendChunk = 4;     // new tokens of a sequence whose queries share one pass over its K/V (draft-extend)
 constexpr size_t kCursorBytes = 1024;                                          // int cur[kMaxCtas], padded
 constexpr size_t kWorkspaceZeroBytes = 256 + kCursorBytes + 2 * (8 + 4 + 4) * kMaxSegments;   // header + cursors + two copies of the per-segment words
 
@@ -113,6 +114,11 @@ cudaError_t launch_reduced_block_table(const KvParams& kv, int n_sink, int W, in
                                        cudaStream_t st);
 // One cooperative launch: optional append of (k_new, v_new), split-KV partials, distributed LSE combine.
 cudaError_t launch_attention(const AttnParams& p, cudaStream_t st);
+
+// Full-context draft-extend with shared K/V tiles (bf16 stores): p.B counts sequences, p.q_len their new tokens;
+// partial results go to p.part_lse / p.part_o, (p.num_ctas + streams) * min(q_len, kExtendChunk) rows of G (x D) floats.
+cudaError_t launch_extend_mq(const AttnParams& p, cudaStream_t st);
+bool extend_mq_fits(int B, int D);     // does the kernel's shared memory hold the tables of B sequences?
 
 cudaError_t launch_mass_diagnostics(const void* o_win, const float* lse_win, const void* o_full, const float* lse_full, int rows,
                                     int D, float* mass, float* perturb, float* tail, cudaStream_t st);

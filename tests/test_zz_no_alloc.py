@@ -110,7 +110,7 @@ def test_noalloc_calls_of_differing_shape_share_the_scratch():
     """A run of calls whose (batch * Hkv) goes up and down: the array keeps the previous call's words, a larger call
     must not trip over what a smaller or larger one left behind."""
     small = _Case(_cfg(name="noalloc_b1", batch=1, gamma=4, seed=21))
-    wide = _Case(_cfg(name="noalloc_b12", batch=12, Hq=32, Hkv=4, D=128, W=256, S0_range=(20, 1500), gamma=4, seed=22))
+    wide = _Case(_cfg(name="noalloc_b8", batch=8, Hq=32, Hkv=4, D=128, W=256, S0_range=(20, 1500), gamma=4, seed=22))
     mid = _Case(_cfg(name="noalloc_b5", batch=5, gamma=4, seed=23))
     for case in (wide, small, small, small, wide, mid, wide, small, mid, mid, wide):
         if case is wide and case.i == 3:
