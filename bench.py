@@ -36,8 +36,8 @@ UNIT = "us"
 WORKLOADS = {"tiny": 0, "s128k": 1, "million": 2, "batched": 3, "sweep": 4}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (attn_fused_tma on the full
-# context). Captured with ncu on the s128k workload (profiles/attn_fused_tma_D256_s128k_ncu_full.md: 272.8 MB
-# for 131,075 keys = 2081.3 B per key, against 2048 algorithmic) and scaled by the keys one launch scans.
+# context), from an ncu capture of that kernel on the s128k workload (272.8 MB for 131,075 keys = 2081.3 B per key,
+# against 2048 algorithmic), scaled by the keys one launch scans: DRAM traffic grows in proportion to the keys.
 NCU_TRAFFIC_BYTES_PER_KEY = {256: 2081.3}
 
 
@@ -53,7 +53,7 @@ def measured_peaks():
             return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, STREAM-style copy)"
         except Exception:
             pass
-    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+    return 6650.0, "fallback (6.65 TB/s; no MEASURED_PEAKS.json beside bench.py)"
 
 
 class ClockSampler:
@@ -119,10 +119,9 @@ def replica_value(ms_per_step_max: float, gamma: int, world: int) -> float:
     return ms_per_step_max * 1e3 / (2 * gamma) / world
 
 
-def pick_config(name: str, steps_total: int):
+def pick_config(name: str):
     import wmtp_inputs as wi
-    cfg = wi.CONFIGS[WORKLOADS[name]]
-    return cfg
+    return wi.CONFIGS[WORKLOADS[name]]
 
 
 def cpu_model() -> str:
@@ -159,7 +158,7 @@ def run_reference(args, rank):
     import wmtp_inputs as wi
     from oracle import reference as R
     R.build()
-    cfg = pick_config(args.workload, 0)
+    cfg = pick_config(args.workload)
     wl = wi.make_workload(cfg, poison_unused=False)
     for _ in range(max(0, min(args.warmup, 1))):
         oracle_sample(wl)
@@ -206,6 +205,8 @@ def main():
     ap.add_argument("--kv-dtype", default="bf16", choices=["bf16", "fp8"],
                     help="entry type of the KV stores (fp8: e4m3 codes with per-KV-head scales)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--grid", action="store_true",
+                    help="with --workload sweep: also time the context / depth / window grid (S x gamma x W, 24 points)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -234,7 +235,7 @@ def main():
         dist.barrier()
     wm.lib()
 
-    cfg = pick_config(args.workload, 0)
+    cfg = pick_config(args.workload)
     if args.kv_dtype == "fp8":
         cfg = wi.scaled(cfg, kv_dtype="fp8", name=cfg.name + "_fp8")
     gam, B = cfg.gamma, cfg.batch
@@ -303,8 +304,9 @@ def main():
         wm.wmtp_draft_loop_full(kv, q, kn, vn, out_f, ws)
         ev[k][2].record()
     torch.cuda.synchronize()
-    us_win = statistics.mean(ev[k][0].elapsed_time(ev[k][1]) for k in range(args.steps)) * 1e3 / gam
-    us_full = statistics.mean(ev[k][1].elapsed_time(ev[k][2]) for k in range(args.steps)) * 1e3 / gam
+    win_samples = [ev[k][0].elapsed_time(ev[k][1]) * 1e3 / gam for k in range(args.steps)]
+    full_samples = [ev[k][1].elapsed_time(ev[k][2]) * 1e3 / gam for k in range(args.steps)]
+    us_win, us_full = statistics.mean(win_samples), statistics.mean(full_samples)
 
     # ---- the dominant kernel alone: `reps` launches of the full-context attention kernel back to back between one
     #      pair of events on the launching stream (average launch duration, inter-launch gap included)
@@ -464,6 +466,48 @@ def main():
               "full_pct_of_8tbs": bytes8 / (us_f8 * 1e-6) / 8e12 * 100,
               "note": "e4m3 codes with one fp32 scale per KV head for K and V; q, k_new, v_new, out stay bf16"}
         del K8, V8, kv8, ring8, wl8
+    # ---- the context / depth / window grid of the sweep workload: S x gamma x W on the same store (a sequence of
+    #      length S is the first S positions), windowed and full-context loops timed separately per point
+    grid = None
+    if args.grid and B == 1 and not cfg.paged:
+        grid = []
+        S_full = int(cur_lens[0])
+        gmax = max(c.gamma for c in wi.sweep_configs())
+        qg = torch.randn((gmax, B, cfg.Hq, cfg.D), device=dev).to(torch.bfloat16)
+        kg = torch.randn((gmax, B, cfg.Hkv, cfg.D), device=dev).to(torch.bfloat16)
+        og = torch.empty_like(qg)
+        rings = {}
+        for pt in wi.sweep_configs():
+            S_pt = min(pt.S0, S_full - gmax * (reps + 4))
+            if pt.W not in rings:
+                rings[pt.W] = wm.Ring(B, cfg.Hkv, cfg.D, cfg.n_sink, pt.W, device=dev, **scales)
+            rg = rings[pt.W]
+            res = {}
+            for name, fn in (("windowed", lambda: wm.wmtp_draft_loop_windowed(rg, qg[:pt.gamma], kg[:pt.gamma], kg[:pt.gamma], og[:pt.gamma], ws)),
+                             ("full", lambda: wm.wmtp_draft_loop_full(kv, qg[:pt.gamma], kg[:pt.gamma], kg[:pt.gamma], og[:pt.gamma], ws))):
+                lens.fill_(S_pt)
+                wm.wmtp_ring_init_from_kv(rg, kv)
+                for _ in range(2):
+                    fn()
+                lens.fill_(S_pt)
+                wm.wmtp_ring_init_from_kv(rg, kv)
+                n_rep = max(3, min(reps, 10))
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record()
+                for _ in range(n_rep):
+                    fn()
+                g1.record()
+                torch.cuda.synchronize()
+                res[name] = g0.elapsed_time(g1) * 1e3 / n_rep / pt.gamma
+            kvb = cfg.kv_bytes_per_token
+            grid.append({"S": pt.S0, "gamma": pt.gamma, "W": pt.W,
+                         "windowed_us_per_step": res["windowed"], "full_us_per_step": res["full"],
+                         "windowed_pct_of_8tbs": min(S_pt, cfg.n_sink + pt.W) * kvb / (res["windowed"] * 1e-6) / 8e12 * 100,
+                         "full_pct_of_8tbs": S_pt * kvb / (res["full"] * 1e-6) / 8e12 * 100})
+        wm.wmtp_device_status(ws)
+        lens.copy_(torch.from_numpy(cur_lens).to(dev))
+        wm.wmtp_ring_init_from_kv(ring, kv)
+        torch.cuda.synchronize()
     full_bytes = float(cur_lens.sum()) * cfg.kv_bytes_per_token
     win_bytes = float(np.minimum(cur_lens, cfg.n_sink + cfg.W).sum()) * cfg.kv_bytes_per_token
     peak, peak_src = measured_peaks()
@@ -531,7 +575,10 @@ def main():
         mass_rep = {}
         S_now = int(lens[0].item())
         tau = cfg.W / 2
-        qx1 = q[0].clone()
+        # the profile carries the logits; the other query components are scaled down (by a power of two: exact) so that
+        # the i.i.d. part of the logits stays small against it and the figures land on the calibration target whatever
+        # the head's key scale and however many tokens the timed loops have appended
+        qx1 = (q[0].float() * 0.125).to(torch.bfloat16)
         qx1[..., 0] = wi.Q_ALONG
         lw = torch.empty((B, cfg.Hq), dtype=torch.float32, device=dev)
         lf, mm, pp, tt = (torch.empty_like(lw) for _ in range(4))
@@ -571,7 +618,8 @@ def main():
             "dtype": "bf16" if cfg.kv_dtype == "bf16" else "f16 (e4m3 KV widened exactly; fp32 softmax)",
             "data": "synthetic", "config": config_dict(cfg, args),
             "variants": {
-                "windowed": {"us_per_step": us_win, "kv_bytes_per_step": win_bytes,
+                "windowed": {"us_per_step": us_win, "us_per_step_median": statistics.median(win_samples),
+                             "us_per_step_min": min(win_samples), "kv_bytes_per_step": win_bytes,
                              "algorithmic_gbs": win_bytes / (us_win * 1e-6) / 1e9,
                              "pct_of_8tbs": win_bytes / (us_win * 1e-6) / 8e12 * 100,
                              "us_per_call_cold_l2": us_win_call_cold,
@@ -579,7 +627,8 @@ def main():
                              "us_per_step_graph_replay": us_win_graph},
                 "windowed_kv_view": {"us_per_attention_call": us_win_kv_call,
                                      "note": "sink + last-W tiles read from the KV store through its page table / rows"},
-                "full": {"us_per_step": us_full, "kv_bytes_per_step": full_bytes,
+                "full": {"us_per_step": us_full, "us_per_step_median": statistics.median(full_samples),
+                         "us_per_step_min": min(full_samples), "kv_bytes_per_step": full_bytes,
                          "algorithmic_gbs": full_bytes / (us_full * 1e-6) / 1e9,
                          "pct_of_8tbs": full_bytes / (us_full * 1e-6) / 8e12 * 100,
                          "us_per_attention_call": us_full_call},
@@ -587,6 +636,7 @@ def main():
                 "fp8_kv": f8,
             },
             "windowed_flatness": flat,
+            "grid": grid,
             "attention_mass": mass_rep,
             "windowed_batch_scaling": batch_scaling,
             "roofline": {"bound": "hbm", "kernel": "attn_fused_tma (full-context draft attention: split-KV partials + in-kernel combine)",

@@ -497,8 +497,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         if (lane == 0) {
                             const uint32_t s = ps, ph = pph;
                             const uint32_t bar_fullK = bar_fullK0 + 8 * (gq * C::kMaxStages), bar_fullV = bar_fullV0 + 8 * (gq * C::kMaxStages);
-                            mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status);
-                            if (!*abort_flag) {
+                            if (mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status)) {
                                 int64_t row;
                                 if (p.mode == kPaged) row = ((int64_t)pg * p.Hkv + sg.g) * kTileKeys;
                                 else {
@@ -866,9 +865,9 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         if (need_enter) { enter_segment(tt); need_enter = false; }
         const uint32_t s = cs, ph = cph;             // stage of tile `it` and the parity of this group's use count of it
         if (!have_tile) {
-            mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
+            const bool landed = mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
             tt = *reinterpret_cast<volatile int64_t*>(stage_tile + s);
-            const bool end = tt < 0 || *abort_flag;
+            const bool end = tt < 0 || !landed;
             const bool outside = sg.seg < 0 || tt < sg.seg_start || tt >= sg.seg_start + sg.tiles;
             if ((end || outside) && sg.seg >= 0 && seg_tiles_done > 0) flush_segment();
             if (end || ncontrib == kMaxContrib) {
@@ -971,10 +970,10 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 }
                 const float mn0 = fmaxf(m[0], mx0), mn1 = fmaxf(m[1], mx1);
                 const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
-                corr0 = exp2f(m[0] - mu0);
-                corr1 = exp2f(m[1] - mu1);
+                corr0 = ex2(m[0] - mu0);
+                corr1 = ex2(m[1] - mu1);
                 m[0] = mn0; m[1] = mn1;
-                const float p0 = exp2f(sc[0] - mu0), p1 = exp2f(sc[1] - mu1), p2 = exp2f(sc[2] - mu0), p3 = exp2f(sc[3] - mu1);
+                const float p0 = ex2(sc[0] - mu0), p1 = ex2(sc[1] - mu1), p2 = ex2(sc[2] - mu0), p3 = ex2(sc[3] - mu1);
                 const uint32_t pa = F8 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1);             // key g8   : heads 2t4, 2t4+1
                 const uint32_t pc = F8 ? pack_f16x2(p2, p3) : pack_bf16x2(p2, p3);             // key g8+8
                 le[0] = le[0] * corr0 + p0 + p2;

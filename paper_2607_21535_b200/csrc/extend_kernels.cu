@@ -204,14 +204,12 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         if (p.mode == kPaged) row = ((int64_t)pg * p.Hkv + sg.g) * kTileKeys;
                         else row = ((int64_t)sg.b * p.Hkv + sg.g) * p.rows_per_head + (first_tile + base + j) * kTileKeys;
                         const uint32_t dstK = stage0 + s * C::kStageBytes, dstV = dstK + C::kTileBytes;
-                        mbar_wait(bar_emptyK + 8 * s, ph ^ 1u, abort_flag, p.status);
-                        if (!*abort_flag) {
+                        if (mbar_wait(bar_emptyK + 8 * s, ph ^ 1u, abort_flag, p.status)) {
                             stage_tile[s] = t + base + j;          // ordered before the consumers' wait by the arrive below
                             mbar_expect_tx(bar_fullK + 8 * s, C::kTileBytes);
                             tma_load_3d(dstK, &mapK, (int)row, bar_fullK + 8 * s);
                         }
-                        mbar_wait(bar_emptyV + 8 * s, ph ^ 1u, abort_flag, p.status);
-                        if (!*abort_flag) {
+                        if (mbar_wait(bar_emptyV + 8 * s, ph ^ 1u, abort_flag, p.status)) {
                             mbar_expect_tx(bar_fullV + 8 * s, C::kTileBytes);
                             tma_load_3d(dstV, &mapV, (int)row, bar_fullV + 8 * s);
                         }
@@ -484,9 +482,9 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     uint32_t pb[kQW][2], pbn[kQW][2];
 #pragma unroll
     for (int j = 0; j < kQW; ++j) { pb[j][0] = pb[j][1] = 0u; pbn[j][0] = pbn[j][1] = 0u; }
-    mbar_wait(bar_fullK, 0u, abort_flag, p.status);
+    const bool first_landed = mbar_wait(bar_fullK, 0u, abort_flag, p.status);
     int64_t tt = *reinterpret_cast<volatile int64_t*>(stage_tile);
-    if (tt >= 0 && !*abort_flag) {
+    if (tt >= 0 && first_landed) {
         enter(tt);
         bool valid_c = slab_valid(tt);
         if (valid_c) {
@@ -500,9 +498,9 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             const int key0 = (int)(tt - sg.start) * kTileKeys;           // first row of the tile in hand within the sequence
             // ---- the next tile's K slot: same stream?
             const uint32_t ns = cs + 1 == (uint32_t)C::kStages ? 0u : cs + 1, nph = ns == 0 ? cph ^ 1u : cph;
-            mbar_wait(bar_fullK + 8 * ns, nph, abort_flag, p.status);
+            const bool landed = mbar_wait(bar_fullK + 8 * ns, nph, abort_flag, p.status);
             const int64_t tn = *reinterpret_cast<volatile int64_t*>(stage_tile + ns);
-            const bool end = tn < 0 || *abort_flag;
+            const bool end = tn < 0 || !landed;
             const bool same = !end && tn >= sg.start && tn < sg.start + sg.tiles;
             bool valid_n = same && slab_valid(tn);
             const int key0n = (int)(tn - sg.start) * kTileKeys;

@@ -36,19 +36,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after kSpinLimit polls (or as soon as another thread has given up), raises
-// the CTA's abort flag and the sticky device status; the caller carries on with invalid data so that
-// every thread still follows the same control flow and nobody is left waiting. Before a CTA that gave up
-// on a barrier leaves the kernel it waits, again bounded, for the copies that may still be in flight
-// into its shared memory (drain_stages).
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    if (mbar_try_wait(bar, parity)) return;
+// Bounded wait; true when the phase completed. It gives up after kSpinLimit polls (or, while it is waiting, as soon as
+// another thread of the CTA has given up), raises the CTA's abort flag and the sticky device status and returns false;
+// the caller carries on to the end of the kernel without using the data, so that every thread still follows the same
+// control flow and nobody is left waiting. The abort flag is read only inside the wait loop: a wait that succeeds at
+// once -- the steady state -- costs no shared-memory round trip beyond the barrier's own. Before a CTA that gave up on
+// a barrier leaves the kernel it waits, again bounded, for the copies that may still be in flight into its shared memory.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    if (mbar_try_wait(bar, parity)) return true;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return;
-        if ((i & 1023u) == 1023u && *abort_flag) return;
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 1023u) == 1023u && *abort_flag) return false;
     }
     if (*abort_flag == 0) *abort_flag = kAbortBarrier;
     atomicCAS(status, 0, kErrTimeout);
+    return false;
 }
 __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
