@@ -170,6 +170,23 @@ __device__ __forceinline__ Segment locate_segment(const AttnParams& p, const int
     return s;
 }
 
+// The segment (b, g) by itself, tiles numbered from 0 (cluster launches: one cluster per segment, no tile line).
+__device__ __forceinline__ Segment make_segment(const AttnParams& p, int b, int g) {
+    Segment s;
+    s.b = b; s.g = g; s.seg = b * p.Hkv + g;
+    const SeqView v = seq_view(p, b);
+    s.seg_start = 0; s.tiles = (int)v.tiles;
+    s.S = v.S; s.nk = (int)v.nk; s.ns = (int)v.ns; s.lo = (int)v.lo; s.sink_tiles = (int)v.sink_tiles; s.win_first = (int)v.win_first;
+    s.hi = (int)(v.S < 0x7fffffffLL ? v.S : 0x7fffffffLL);
+    s.cap = 0; s.slot_base = 0;
+    return s;
+}
+// Barrier over all threads of the cluster that have not exited: what was written to shared memory before it is visible
+// to the other CTAs' distributed-shared-memory reads after it.
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // Element offset of row `key` of (b, g) in the K / V tensor; *ok = false on a bad page id.
 __device__ __forceinline__ int64_t kv_row_offset(const AttnParams& p, int b, int g, int64_t key, bool* ok) {
     if (p.mode == kPaged) {
@@ -337,9 +354,19 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
 //                count of the launch that used it last, not over this launch's.
 
 // ---------------------------------------------------------------------------------------------
-// The attention kernel (one cooperative launch per draft step)
+// The attention kernel (one launch per draft step), in two forms.
+//   CL = false: the cooperative launch described above -- one tile line over all segments, work stealing, partials in the
+//     workspace, distributed combine. Made for long streams, where its fixed cost (about 13 us of plan, flush, arrival
+//     and combine round trips through L2) does not matter.
+//   CL = true: a thread-block cluster per segment, for launches whose segments are short (the windowed draft: a ring
+//     or a window view of a few thousand keys per sequence). CTA r of the cluster's n takes tiles [r T / n, (r + 1) T / n)
+//     of its segment; every consumer group leaves its partial in its own shared memory, and after one cluster barrier
+//     CTA r reduces the r-th slice of the output columns over all partials of the cluster through distributed shared
+//     memory (log-sum-exp weights from the partials' lse values). No workspace traffic, no atomics, no polling; the
+//     launch is an ordinary one (no CTA waits for another cluster), and the cluster that finishes last -- a ticket in
+//     the workspace header -- advances the lengths of a fused append. Tile processing is the same code in both forms.
 // ---------------------------------------------------------------------------------------------
-template <int D, bool F8>
+template <int D, bool F8, bool CL>
 __global__ void __launch_bounds__(Cfg<D, F8>::kThreads, 1)
 attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                const __grid_constant__ AttnParams p) {
@@ -361,8 +388,9 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     int* cta_flags = group_ints + C::kGroups * kGroupInts;                                // [0] abort
     unsigned char* stages = smem + C::kFixedBytes;                                        // nst x (K tile, V tile)
     const uint32_t nst = (uint32_t)p.stages;                                              // stages in use (<= kMaxStages)
-    int64_t* tile_prefix = reinterpret_cast<int64_t*>(stages + nst * C::kStageBytes);     // [B + 1]
+    int64_t* tile_prefix = reinterpret_cast<int64_t*>(stages + nst * C::kStageBytes);     // [B + 1]       (CL = false)
     int* cap_prefix = reinterpret_cast<int*>(tile_prefix + (p.B + 1));                    // [B + 1]
+    float* part_sm = reinterpret_cast<float*>(stages + nst * C::kStageBytes);             // [kGroups][8 D + 8] (CL = true): o, lse
     volatile int* abort_flag = cta_flags;
 
     if (threadIdx.x == C::kConsumerWarps * 32) {            // descriptor fetch overlaps the len[] round trip
@@ -383,9 +411,37 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         cta_flags[1] = 0;                                    // segments that hold at least one tile (counted below)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    const uint32_t epoch = *reinterpret_cast<const volatile uint32_t*>(p.epoch);
+    if constexpr (CL) {
+        // Programmatic dependent launch: the cluster form is launched so that it may start while the kernel before it on
+        // the stream (normally the previous draft step) is still finishing on other SMs. Everything above touches only
+        // shared memory and the kernel's parameters; from here on global memory is read and written, which has to wait
+        // until that kernel has completed and its writes (lengths, the appended row, the ticket word) are visible. The
+        // next kernel on the stream may be set up from now on.
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
+    // ---- cluster form: this cluster's segment and this CTA's share of its tiles (one length to read, no tables)
+    Segment csg;
+    csg.seg = -1; csg.seg_start = 0; csg.tiles = 0; csg.b = 0; csg.g = 0; csg.nk = 0; csg.S = 0; csg.slot_base = 0; csg.cap = 0;
+    csg.ns = 0; csg.lo = 0; csg.hi = 0; csg.sink_tiles = 0; csg.win_first = 0;
+    int c_lo = 0, c_hi = 0;
+    uint32_t crank = 0, csize = 1;
+    if constexpr (CL) {
+        asm("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
+        asm("mov.u32 %0, %%cluster_nctarank;" : "=r"(csize));
+        const int cseg = (int)(blockIdx.x / csize);
+        csg = make_segment(p, cseg / p.Hkv, cseg % p.Hkv);
+        c_lo = (int)(crank * (uint32_t)csg.tiles / csize);
+        c_hi = (int)((crank + 1) * (uint32_t)csg.tiles / csize);
+        // a group that gets no tile contributes an empty partial
+        if (threadIdx.x < C::kGroups * kMaxGroup)
+            part_sm[(threadIdx.x / kMaxGroup) * (kMaxGroup * D + kMaxGroup) + kMaxGroup * D + threadIdx.x % kMaxGroup] = -INFINITY;
+        __syncthreads();
+    }
+    const uint32_t epoch = CL ? 0u : *reinterpret_cast<const volatile uint32_t*>(p.epoch);
     const int par_off = (epoch & 1u) ? kMaxSegmentsPadded(p) : 0;        // which copy of the per-segment words this launch uses
 
+    if constexpr (!CL) {
     // ---- plan: tiles per sequence and partial-slot capacity per sequence (all from len[]; O(B / 32) steps: the
     //      per-sequence values are computed by all threads, the two running sums by one warp)
     for (int b = threadIdx.x; b < p.B; b += blockDim.x)
@@ -410,20 +466,21 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     __syncthreads();
     if (threadIdx.x < 32) warp_inclusive_scan(cap_prefix + 1, p.B);
     __syncthreads();
+    }
     const int G = p.G;
     const int nseg = p.B * p.Hkv;
-    const int64_t n = (int64_t)p.Hkv * tile_prefix[p.B];
+    const int64_t n = CL ? (int64_t)csg.tiles : (int64_t)p.Hkv * tile_prefix[p.B];
     const int Cg = gridDim.x;
-    const int Cn = effective_ctas(Cg, n);
+    const int Cn = CL ? Cg : effective_ctas(Cg, n);
     // ---- sequences that hold no token: out = 0, lse = -inf (no CTA owns a tile of theirs)
-    for (int seg = blockIdx.x; seg < nseg; seg += gridDim.x) {
+    for (int seg = blockIdx.x; !CL && seg < nseg; seg += gridDim.x) {
         const int b = seg / p.Hkv, g = seg % p.Hkv;
         if (tile_prefix[b + 1] != tile_prefix[b]) continue;
         __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + g * G) * D;
         for (int idx = threadIdx.x; idx < G * D; idx += blockDim.x) o[idx] = __float2bfloat16(0.f);
         if (p.lse && threadIdx.x < G) p.lse[(int64_t)b * p.Hq + g * G + threadIdx.x] = -INFINITY;
     }
-    if (n == 0) {                                            // nothing to attend over at all
+    if (!CL && n == 0) {                                     // nothing to attend over at all
         if (threadIdx.x == 0 && atomicAdd(p.grab_done, 1) + 1 == Cg) {
             *p.grab_done = 0;
             if (p.k_new) atomicCAS(p.status, 0, kErrBounds);
@@ -435,7 +492,10 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     if ((int)(threadIdx.x >> 5) >= C::kConsumerWarps) {
         if constexpr (C::kRebalance) {
             asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsProducer));
-            if ((int)(threadIdx.x >> 5) > C::kConsumerWarps) return;          // filler warps of the producer's warpgroup
+            if ((int)(threadIdx.x >> 5) > C::kConsumerWarps) {                // filler warps of the producer's warpgroup
+                if constexpr (CL) { cluster_sync_all(); cluster_sync_all(); }   // every thread of the cluster joins its two barriers
+                return;
+            }
         }
         // =================================== producer warp ===================================
         // CTA c < Cn owns the tile range [c n / Cn, (c+1) n / Cn). It streams the first part of it without any
@@ -447,6 +507,59 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         // stage's use count) and to consumer group it % kGroups.
         const uint32_t stage0 = smem_u32(stages);
         uint32_t it = 0, ps = 0, pph = 0;
+        if constexpr (CL) {
+            // ---- cluster form: tiles [c_lo, c_hi) of the cluster's segment, in order; page ids fetched 32 at a time
+            const int ntiles = c_hi - c_lo;
+            for (int base = 0; base < ntiles; base += 32) {
+                int page = 0;
+                if (p.mode == kPaged) {
+                    const int64_t tj = c_lo + base + lane;
+                    const int64_t ti = tj < csg.sink_tiles ? tj : csg.win_first + tj - csg.sink_tiles;   // source tile = page index
+                    if (base + lane < ntiles) {
+                        page = p.page_table[(int64_t)kv_seq(p, csg.b) * p.max_pages + ti];
+                        if (page < 0 || page >= p.num_pages) { atomicCAS(p.status, 0, kErrBounds); page = 0; }
+                    }
+                }
+                const int cnt = ntiles - base < 32 ? ntiles - base : 32;
+                for (int j = 0; j < cnt; ++j, ++it, ps = (ps + 1 == nst ? 0 : ps + 1), pph ^= (ps == 0)) {
+                    const int pg = __shfl_sync(0xffffffffu, page, j);
+                    if (lane == 0) {
+                        const uint32_t s = ps, ph = pph, gq = it % C::kGroups;
+                        const uint32_t bar_fullK = bar_fullK0 + 8 * (gq * C::kMaxStages), bar_fullV = bar_fullV0 + 8 * (gq * C::kMaxStages);
+                        if (mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status)) {
+                            int64_t row;
+                            if (p.mode == kPaged) row = ((int64_t)pg * p.Hkv + csg.g) * kTileKeys;
+                            else {
+                                const int64_t tj = c_lo + base + j;
+                                const int64_t src = tj < csg.sink_tiles ? tj : csg.win_first + tj - csg.sink_tiles;
+                                row = ((int64_t)kv_seq(p, csg.b) * p.Hkv + csg.g) * p.rows_per_head + src * kTileKeys;
+                            }
+                            const uint32_t dstK = stage0 + s * C::kStageBytes, dstV = dstK + C::kTileBytes;
+                            stage_tile[s] = c_lo + base + j;       // ordered before the consumers' wait by the arrive below
+                            mbar_expect_tx(bar_fullK + 8 * s, C::kTileBytes);
+                            tma_load_3d(dstK, &mapK, (int)row, bar_fullK + 8 * s);
+                            mbar_expect_tx(bar_fullV + 8 * s, C::kTileBytes);
+                            tma_load_3d(dstV, &mapV, (int)row, bar_fullV + 8 * s);
+                        }
+                    }
+                }
+            }
+            if (lane == 0) {
+                // one end marker per consumer group
+                for (int q = 0; q < C::kGroups; ++q, ++it, ps = (ps + 1 == nst ? 0 : ps + 1), pph ^= (ps == 0)) {
+                    const uint32_t s = ps, ph = pph;
+                    const uint32_t gq = it % C::kGroups;
+                    mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status);
+                    stage_tile[s] = -1;
+                    mbar_arrive(bar_fullK0 + 8 * (gq * C::kMaxStages + s));
+                    mbar_arrive(bar_fullV0 + 8 * (gq * C::kMaxStages + s));
+                }
+            }
+            __syncwarp();
+            cluster_sync_all();                  // the two barriers of the cluster's merge (the consumers' work lies between them)
+            cluster_sync_all();
+            return;
+        }
         int cur_seg = -1;                    // segment of the last issued tile
         int64_t cur_lo = 0, cur_hi = 0;      // its tile range
         int grp_seg[kMaxGroups], grp_ord[kMaxGroups], pend_k[kMaxGroups];
@@ -676,7 +789,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 
     // Combine every segment this group has contributed to (waits for their last partial), then forget them.
     auto combine_outstanding = [&]() {
-        for (int i = 0; i < ncontrib; ++i) {
+        for (int i = 0; !CL && i < ncontrib; ++i) {
             const int seg = contrib[4 * i], b = contrib[4 * i + 1], g = contrib[4 * i + 2], k = contrib[4 * i + 3];
             if (tid == 0) {
                 gints[1] = wait_tiles(p.arrive + par_off + seg, (uint32_t)contrib_tiles[i], p.spin_limit, abort_flag, p.status);
@@ -705,8 +818,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             sm_le[warp * kMaxGroup + 2 * t4] = le[0]; sm_le[warp * kMaxGroup + 2 * t4 + 1] = le[1];
         }
         group_barrier(grp);
-        int k = reg_k[ord % kMaxContrib];                     // slot the producer took when this group entered the segment
-        if (k < 0 || k >= sg.cap) {
+        int k = CL ? 0 : reg_k[ord % kMaxContrib];            // slot the producer took when this group entered the segment
+        if (!CL && (k < 0 || k >= sg.cap)) {
             // cannot happen while the admission rules hold; never write outside the segment's slots
             if (tid == 0) {
                 atomicCAS(p.status, 0, kErrBounds);
@@ -715,12 +828,15 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             }
             k = sg.cap - 1;
         }
-        if (tid == 0) {
+        if (!CL && tid == 0) {
             contrib[4 * ncontrib + 3] = k;
             p.part_key[sg.slot_base + k] = (int)blockIdx.x * kMaxGroups + grp;
         }
         ++ord;
         const int64_t pidx = (int64_t)sg.slot_base + k;
+        // where the partial goes: the workspace, or (cluster form) this group's buffer in shared memory, rows of D floats
+        float* const dst_o = CL ? part_sm + grp * (kMaxGroup * D + kMaxGroup) : p.part_o + pidx * G * D;
+        float* const dst_lse = CL ? part_sm + grp * (kMaxGroup * D + kMaxGroup) + kMaxGroup * D : p.part_lse + pidx * G;
         float f[2];
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
@@ -738,7 +854,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 }
             }
             f[i] = (L > 0.f && m[i] > -INFINITY) ? exp2f(m[i] - M) / L * vscale : 0.f;
-            if (warp == 0 && g8 == 0 && h < G) p.part_lse[pidx * G + h] = Le > 0.f ? (M + log2f(Le)) * kLn2 : -INFINITY;
+            if (warp == 0 && g8 == 0 && h < G) dst_lse[h] = Le > 0.f ? (M + log2f(Le)) * kLn2 : -INFINITY;
         }
         constexpr int kPasses = D / C::kPassCols;               // kPassCols columns of d per pass through the scratch
         constexpr int kScratchRow = C::kScratchRow;
@@ -762,11 +878,11 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 float acc = 0.f;
 #pragma unroll
                 for (int w = 0; w < kGroupWarps; ++w) acc += scratch[(w * kMaxGroup + h) * kScratchRow + dd];
-                p.part_o[(pidx * G + h) * D + pass * C::kPassCols + dd] = acc;
+                dst_o[h * D + pass * C::kPassCols + dd] = acc;
             }
         }
         group_barrier(grp);
-        if (tid == 0) {
+        if (!CL && tid == 0) {
             __threadfence();                                   // the group's partial is visible device-wide before the arrival
             const unsigned long long old = atomicAdd(p.arrive + par_off + sg.seg, (1ull << 32) | (unsigned long long)seg_tiles_done);
             if ((int)(uint32_t)old + seg_tiles_done == sg.tiles) {        // this contribution completes the segment
@@ -782,8 +898,9 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 
     // Start work on the segment that holds tile tt: partial bookkeeping, append target, query fragments, fresh state.
     auto enter_segment = [&](int64_t tt) {
-        sg = locate_segment(p, tile_prefix, cap_prefix, tt);
-        if (tid == 0) {
+        if constexpr (CL) sg = csg;
+        else sg = locate_segment(p, tile_prefix, cap_prefix, tt);
+        if (!CL && tid == 0) {
             contrib[4 * ncontrib] = sg.seg; contrib[4 * ncontrib + 1] = sg.b; contrib[4 * ncontrib + 2] = sg.g;
             contrib_base[ncontrib] = sg.slot_base;
             contrib_tiles[ncontrib] = sg.tiles;
@@ -855,7 +972,9 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     // tail runs once per launch, from a cold instruction cache: code size is latency there).
     int64_t tt = -1;                                     // tile in hand
     bool have_tile = false, need_enter = false;
-    if ((int)blockIdx.x < Cn) {
+    if constexpr (CL) {
+        if (c_lo + grp < c_hi) { tt = c_lo + grp; need_enter = true; }
+    } else if ((int)blockIdx.x < Cn) {
         // an owner knows its first tiles: fetch the query while they are still in flight
         const int64_t first = cta_range_start(blockIdx.x, n, Cn) + grp;
         if (first < cta_range_start(blockIdx.x + 1, n, Cn)) { tt = first; need_enter = true; }
@@ -1065,6 +1184,108 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             for (uint32_t i = 0; i < kDrainLimit && !mbar_test_wait(bar_fullV + 8 * s2, par); ++i) { }
         }
     }
+    if constexpr (CL) {
+        // ---- cluster form: merge the cluster's partials through distributed shared memory. CTA r reduces the r-th slice
+        //      of the (head, d) columns: weights exp(lse_s - lse) from all partials' lse values, then the weighted sum.
+        cluster_sync_all();                                   // every group of every CTA has left its partial (or none)
+        if (grp == 0) {
+            constexpr int kVec = D / 4;                       // float4 columns per head
+            constexpr int kPart = kMaxGroup * D + kMaxGroup;  // floats per partial: o [8][D], lse [8]
+            const int cols = G * kVec, np = (int)csize * C::kGroups;
+            const int per = (cols + (int)csize - 1) / (int)csize;
+            const int col_lo = (int)crank * per, col_hi = col_lo + per < cols ? col_lo + per : cols;
+            const uint32_t part_local = smem_u32(part_sm);
+            float4* red = reinterpret_cast<float4*>(scratch);  // [4 warps][32]
+            __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)csg.b * p.Hq + csg.g * G) * D;
+            auto remote = [&](int s_, int off_floats) {       // shared::cluster address of float `off` of partial s_
+                uint32_t a;
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
+                             : "=r"(a) : "r"(part_local + 4u * (uint32_t)((s_ % C::kGroups) * kPart + off_floats)), "r"((uint32_t)(s_ / C::kGroups)));
+                return a;
+            };
+            constexpr int kMaxNp = 16 * kMaxGroups;           // partials of the largest cluster
+            constexpr int kMaxOwn = kMaxNp / kGroupWarps;     // ... of which a warp sums every fourth
+            for (int c0 = col_lo; c0 < col_hi; c0 += 32) {
+                const int col = c0 + lane;
+                const bool act = col < col_hi;
+                const int h = act ? col / kVec : 0;
+                // one round trip through the cluster: all partials' lse values of head h (every thread computes the
+                // weights of its own column) and, with them, the rows of the partials this warp sums
+                float x[kMaxNp];
+                float4 v[kMaxOwn];
+#pragma unroll
+                for (int s_ = 0; s_ < kMaxNp; ++s_) {
+                    x[s_] = -INFINITY;
+                    if (s_ < np) asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(x[s_]) : "r"(remote(s_, kMaxGroup * D + h)));
+                }
+#pragma unroll
+                for (int u = 0; u < kMaxOwn; ++u) {
+                    const int s_ = warp + kGroupWarps * u;
+                    v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (s_ < np && act)
+                        asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
+                                     : "=f"(v[u].x), "=f"(v[u].y), "=f"(v[u].z), "=f"(v[u].w) : "r"(remote(s_, col * 4)));
+                }
+                float M = -INFINITY;
+#pragma unroll
+                for (int s_ = 0; s_ < kMaxNp; ++s_) M = fmaxf(M, x[s_]);
+                float sum = 0.f;
+#pragma unroll
+                for (int s_ = 0; s_ < kMaxNp; ++s_) {
+                    x[s_] = (s_ < np && M > -INFINITY) ? __expf(x[s_] - M) : 0.f;
+                    sum += x[s_];
+                }
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int u = 0; u < kMaxOwn; ++u) {
+                    // x[warp + 4 u], by a select chain (a register array cannot be indexed by a run-time value)
+                    float w = 0.f;
+#pragma unroll
+                    for (int q = 0; q < kGroupWarps; ++q) w = (warp == q) ? x[q + kGroupWarps * u] : w;
+                    if (w > 0.f) {                           // an empty partial's rows were never written
+                        acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
+                        acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);
+                    }
+                }
+                red[warp * 32 + lane] = acc;
+                group_barrier(grp);
+                if (warp == 0 && act) {
+                    float4 o4 = red[lane];
+#pragma unroll
+                    for (int w2 = 1; w2 < kGroupWarps; ++w2) {
+                        const float4 y = red[w2 * 32 + lane];
+                        o4.x += y.x; o4.y += y.y; o4.z += y.z; o4.w += y.w;
+                    }
+                    const float inv = sum > 0.f ? 1.f / sum : 0.f;
+                    uint2 packed;
+                    packed.x = pack_bf16x2(o4.x * inv, o4.y * inv);
+                    packed.y = pack_bf16x2(o4.z * inv, o4.w * inv);
+                    *reinterpret_cast<uint2*>(out + (int64_t)col * 4) = packed;
+                    if (p.lse && col % kVec == 0) p.lse[(int64_t)csg.b * p.Hq + csg.g * G + h] = sum > 0.f ? M + __logf(sum) : -INFINITY;
+                }
+                group_barrier(grp);
+            }
+        }
+        cluster_sync_all();                                   // nobody's shared memory goes away while it is being read
+        // ---- the cluster that finishes last closes the launch (all others have read len[] for the last time)
+        if (grp == 0) {
+            if (tid == 0) {
+                gints[0] = 0;
+                if (crank == 0 && atomicAdd(p.segs_done, 1) + 1 == (int)(gridDim.x / csize)) {
+                    *p.segs_done = 0;
+                    gints[0] = 1;
+                }
+            }
+            group_barrier(grp);
+            if (gints[0] && p.k_new) {
+                for (int b = tid; b < p.B; b += kGroupThreads) {
+                    if (appends_to(p, b)) p.len[b] += 1;
+                    else atomicCAS(p.status, 0, kErrBounds);      // append past S_cap: skipped and flagged
+                }
+            }
+        }
+        return;
+    }
     // ---- the group that completed the launch's last segment closes the launch
     if (tid == 0) gints[0] = launch_last ? 1 : 0;
     group_barrier(grp);
@@ -1113,14 +1334,84 @@ cudaError_t launch_fused(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaSt
         cudaGetDevice(&dev);
         std::lock_guard<std::mutex> lock(mu);
         if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-            cudaError_t e = cudaFuncSetAttribute(attn_fused_tma<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+            cudaError_t e = cudaFuncSetAttribute(attn_fused_tma<D, F8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
             if (e != cudaSuccess) return e;
             if (dev >= 0 && dev < 64) attr_set[dev] = true;
         }
     }
     void* args[] = {&mk, &mv, &p};
     // cooperative: the CTAs wait on one another in the combine, so they must all be resident
-    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(attn_fused_tma<D, F8>), dim3(p.num_ctas), dim3(Cfg<D, F8>::kThreads), args, smem, st);
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(attn_fused_tma<D, F8, false>), dim3(p.num_ctas), dim3(Cfg<D, F8>::kThreads), args, smem, st);
+}
+
+// ---- cluster form ----
+// Stages of the cluster form: as many as fit beside the groups' partial buffers (the data comes from L2: depth matters less
+// than in the streaming form).
+template <int D, bool F8>
+constexpr int cluster_stages() {
+    using C = Cfg<D, F8>;
+    int stages = C::kMaxStages;
+    while (stages > C::kGroups &&
+           1024 + C::kFixedBytes + stages * C::kStageBytes + (int)sizeof(float) * C::kGroups * (kMaxGroup * D + kMaxGroup) + 16 > 227 * 1024)
+        stages -= C::kGroups;
+    return stages;
+}
+template <int D, bool F8>
+size_t cluster_smem_bytes() {
+    using C = Cfg<D, F8>;
+    return 1024 + (size_t)C::kFixedBytes + (size_t)cluster_stages<D, F8>() * C::kStageBytes +
+           sizeof(float) * C::kGroups * (kMaxGroup * D + kMaxGroup) + 16;
+}
+static_assert(cluster_stages<256, false>() == 3 && cluster_stages<256, true>() >= 4 && cluster_stages<128, false>() >= 4 &&
+              cluster_stages<128, true>() >= 4, "cluster form: stages that fit shared memory");
+
+// One-time set-up per device: shared-memory opt-in, non-portable cluster sizes, and how many clusters of each size the
+// device holds at once (index: log2 of the cluster size).
+struct ClusterInfo { bool ready; int active[5]; };
+template <int D, bool F8>
+cudaError_t cluster_info(const ClusterInfo** out) {
+    static std::mutex mu;
+    static ClusterInfo info[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!info[dev].ready) {
+        auto* fn = attn_fused_tma<D, F8, true>;
+        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) return e;
+        for (int l2 = 0; l2 < 5; ++l2) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(1 << l2); cfg.blockDim = dim3(Cfg<D, F8>::kThreads); cfg.dynamicSmemBytes = cluster_smem_bytes<D, F8>();
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = 1u << l2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            cfg.attrs = at; cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, fn, &cfg) != cudaSuccess) { n = 0; (void)cudaGetLastError(); }
+            info[dev].active[l2] = n;
+        }
+        info[dev].ready = true;
+    }
+    *out = &info[dev];
+    return cudaSuccess;
+}
+
+template <int D, bool F8>
+cudaError_t launch_cluster(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaStream_t st) {
+    using C = Cfg<D, F8>;
+    p.stages = cluster_stages<D, F8>();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.num_ctas); cfg.blockDim = dim3(C::kThreads); cfg.dynamicSmemBytes = cluster_smem_bytes<D, F8>(); cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)p.cluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    // may be set up while the previous kernel on the stream drains (the kernel waits before it touches global memory)
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, attn_fused_tma<D, F8, true>, mk, mv, p);
 }
 
 }  // namespace
@@ -1132,17 +1423,52 @@ int64_t attention_rows(const AttnParams& p) {
     return (int64_t)(p.B / (p.q_len > 1 ? p.q_len : 1)) * p.Hkv * p.rows_per_head;
 }
 
-cudaError_t launch_attention(const AttnParams& p_in, cudaStream_t st) {
-    AttnParams p = p_in;
+cudaError_t make_attention_maps(const AttnParams& p, AttnMaps* maps) {
     const int64_t rows = attention_rows(p);
-    CUtensorMap mk, mv;
     const int esz = p.f8 ? 1 : 2;
-    if (!make_map(&mk, p.k, rows, p.D, esz) || !make_map(&mv, p.v, rows, p.D, esz)) return cudaErrorInvalidValue;
+    if (!make_map(&maps->k, p.k, rows, p.D, esz) || !make_map(&maps->v, p.v, rows, p.D, esz)) return cudaErrorInvalidValue;
+    return cudaSuccess;
+}
+
+cudaError_t launch_attention(const AttnParams& p_in, const AttnMaps& maps, cudaStream_t st) {
+    AttnParams p = p_in;
+    CUtensorMap mk = maps.k, mv = maps.v;
     cudaError_t e;
-    if (p.f8) e = p.D == 128 ? launch_fused<128, true>(mk, mv, p, st) : launch_fused<256, true>(mk, mv, p, st);
-    else e = p.D == 128 ? launch_fused<128, false>(mk, mv, p, st) : launch_fused<256, false>(mk, mv, p, st);
+    if (p.cluster > 0) {
+        if (p.f8) e = p.D == 128 ? launch_cluster<128, true>(mk, mv, p, st) : launch_cluster<256, true>(mk, mv, p, st);
+        else e = p.D == 128 ? launch_cluster<128, false>(mk, mv, p, st) : launch_cluster<256, false>(mk, mv, p, st);
+    } else {
+        if (p.f8) e = p.D == 128 ? launch_fused<128, true>(mk, mv, p, st) : launch_fused<256, true>(mk, mv, p, st);
+        else e = p.D == 128 ? launch_fused<128, false>(mk, mv, p, st) : launch_fused<256, false>(mk, mv, p, st);
+    }
     count_launch(1);
     return e;
+}
+
+// CTAs per cluster for a launch of `nseg` segments of at most `tiles` tiles each through the cluster form of the kernel,
+// or 0 when the cooperative form should serve it: the largest power of two (at most 16, at most `max_ctas` CTAs in all
+// when that is positive) whose clusters are all resident at once, as long as that leaves a CTA a handful of tiles.
+int pick_cluster(int D, int f8, int nseg, int64_t tiles, int max_ctas) {
+    const ClusterInfo* info = nullptr;
+    cudaError_t e;
+    if (f8) e = D == 128 ? cluster_info<128, true>(&info) : cluster_info<256, true>(&info);
+    else e = D == 128 ? cluster_info<128, false>(&info) : cluster_info<256, false>(&info);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    int best = 0;
+    for (int l2 = 0; l2 < 5; ++l2) {
+        const int cl = 1 << l2;
+        if (info->active[l2] <= 0) continue;
+        if (cl > 1 && cl > tiles) break;
+        if (max_ctas > 0 && (int64_t)nseg * cl > max_ctas && cl > 1) break;
+        if (l2 > 0 && nseg > info->active[l2]) break;               // a second wave of clusters would double the time
+        best = cl;
+    }
+    if (best == 0) return 0;
+    // long segments: the cooperative form spreads them over all SMs (a CTA with one consumer group takes about 1 us per
+    // 64 KB tile out of L2, one with two groups half of that)
+    const bool one_group = 2 * kTileKeys * D * (f8 ? 1 : 2) >= 65536;
+    if ((tiles + best - 1) / best > (one_group ? kClusterMaxTiles1 : kClusterMaxTiles2)) return 0;
+    return best;
 }
 
 }  // namespace wmtp

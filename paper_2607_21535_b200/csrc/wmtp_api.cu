@@ -188,9 +188,22 @@ void bind_ring(AttnParams& p, const wmtp_ring* ring, const void* k_new, const vo
 }
 
 // k_new / v_new non-NULL: a fused draft step (append, then attend) in one launch.
+// A chain of launches on one store encodes the store's TMA descriptors once.
+struct MapCache { AttnMaps maps; bool ready = false; };
+cudaError_t launch_with(const AttnParams& p, MapCache* cache, cudaStream_t st) {
+    MapCache local;
+    if (!cache) cache = &local;
+    if (!cache->ready) {
+        cudaError_t e = make_attention_maps(p, &cache->maps);
+        if (e != cudaSuccess) return e;
+        cache->ready = true;
+    }
+    return launch_attention(p, cache->maps, st);
+}
+
 wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm_scale, void* out, float* lse,
                           void* ws, size_t ws_bytes, cudaStream_t st, bool validate, const void* k_new = nullptr,
-                          const void* v_new = nullptr, int q_len = 1) {
+                          const void* v_new = nullptr, int q_len = 1, MapCache* cache = nullptr) {
     if (validate) {
         if (wmtp_status s = check_ring(ring)) return s;
         if (wmtp_status s = check_attn_common(q, Hq, ring->Hkv, ring->batch * q_len, ring->D, out, lse, ws, ws_bytes)) return s;
@@ -199,11 +212,17 @@ wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm
     fill_attn(p, q, Hq, ring->Hkv, ring->batch * q_len, ring->D, sm_scale, out, lse, ws);
     p.q_len = q_len;
     bind_ring(p, ring, k_new, v_new);
-    const int64_t tiles = (p.rows_per_head + kTileKeys - 1) / kTileKeys * ring->batch * q_len * ring->Hkv;
-    p.num_ctas = pick_ctas(tiles);
-    p.num_ctas = align_ctas_to_segments(p.num_ctas, ring->batch * q_len * ring->Hkv, tiles);
+    const int nseg = ring->batch * q_len * ring->Hkv;
+    const int64_t tiles_per_seg = (p.rows_per_head + kTileKeys - 1) / kTileKeys, tiles = tiles_per_seg * nseg;
+    p.cluster = pick_cluster(p.D, p.f8, nseg, tiles_per_seg, g_max_ctas.load());
+    if (p.cluster > 0) {
+        p.num_ctas = nseg * p.cluster;
+    } else {
+        p.num_ctas = pick_ctas(tiles);
+        p.num_ctas = align_ctas_to_segments(p.num_ctas, nseg, tiles);
+    }
     if (p.num_ctas <= 0) return fail(WMTP_ERR_CUDA, "no CUDA device available");
-    cudaError_t e = launch_attention(p, st);
+    cudaError_t e = launch_with(p, cache, st);
     if (e != cudaSuccess) return cuda_fail(e, "windowed attention launch");
     return WMTP_OK;
 }
@@ -211,7 +230,7 @@ wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm
 // W > 0: window view (attend over the first n_sink and the last W positions of the KV store); W == 0: all positions.
 wmtp_status attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, void* out, float* lse, void* ws,
                       size_t ws_bytes, cudaStream_t st, bool validate, const void* k_new = nullptr,
-                      const void* v_new = nullptr, int n_sink = 0, int W = 0, int q_len = 1) {
+                      const void* v_new = nullptr, int n_sink = 0, int W = 0, int q_len = 1, MapCache* cache = nullptr) {
     if (validate) {
         if (wmtp_status s = check_kv(kv)) return s;
         if (wmtp_status s = check_attn_common(q, Hq, kv->Hkv, kv->batch * q_len, kv->D, out, lse, ws, ws_bytes)) return s;
@@ -234,10 +253,16 @@ wmtp_status attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, 
     // few long segments of a bf16 store, one query each: see pick_ctas (a ragged 32-sequence batch and the multi-query
     // extend, which re-reads rows through L2, measured slower on fewer SMs)
     const bool streaming = W == 0 && !p.f8 && q_len == 1 && kv->batch * kv->Hkv <= 8;
-    p.num_ctas = pick_ctas(tiles_per_seg * kv->batch * q_len * kv->Hkv, streaming);
-    if (W > 0) p.num_ctas = align_ctas_to_segments(p.num_ctas, kv->batch * q_len * kv->Hkv, tiles_per_seg * kv->batch * q_len * kv->Hkv);
+    const int nseg = kv->batch * q_len * kv->Hkv;
+    if (W > 0) p.cluster = pick_cluster(p.D, p.f8, nseg, tiles_per_seg, g_max_ctas.load());
+    if (p.cluster > 0) {
+        p.num_ctas = nseg * p.cluster;
+    } else {
+        p.num_ctas = pick_ctas(tiles_per_seg * nseg, streaming);
+        if (W > 0) p.num_ctas = align_ctas_to_segments(p.num_ctas, nseg, tiles_per_seg * nseg);
+    }
     if (p.num_ctas <= 0) return fail(WMTP_ERR_CUDA, "no CUDA device available");
-    cudaError_t e = launch_attention(p, st);
+    cudaError_t e = launch_with(p, cache, st);
     if (e != cudaSuccess) return cuda_fail(e, W > 0 ? "windowed (KV view) attention launch" : "full attention launch");
     return WMTP_OK;
 }
@@ -402,12 +427,13 @@ wmtp_status wmtp_draft_loop_windowed(const wmtp_ring* ring, int gamma, const voi
     if (wmtp_status s = check_loop(gamma, k_new, v_new)) return s;
     if (wmtp_status s = check_attn_common(q, Hq, ring->Hkv, ring->batch, ring->D, out, lse, workspace, ws_bytes)) return s;
     const size_t q_step = (size_t)ring->batch * Hq * ring->D * 2, kv_step = (size_t)ring->batch * ring->Hkv * ring->D * 2;
+    MapCache cache;
     for (int i = 0; i < gamma; ++i) {
         // one launch per draft step: the kernel appends step i's K/V row, then attends
         if (wmtp_status s = attn_windowed((const char*)q + i * q_step, Hq, ring, sm_scale, (char*)out + i * q_step,
                                           lse ? lse + (size_t)i * ring->batch * Hq : nullptr, workspace, ws_bytes,
                                           (cudaStream_t)stream, false, (const char*)k_new + i * kv_step,
-                                          (const char*)v_new + i * kv_step))
+                                          (const char*)v_new + i * kv_step, 1, &cache))
             return s;
     }
     return WMTP_OK;
@@ -420,11 +446,12 @@ wmtp_status wmtp_draft_loop_full(const wmtp_kv* kv, int gamma, const void* q, in
     if (wmtp_status s = check_loop(gamma, k_new, v_new)) return s;
     if (wmtp_status s = check_attn_common(q, Hq, kv->Hkv, kv->batch, kv->D, out, lse, workspace, ws_bytes)) return s;
     const size_t q_step = (size_t)kv->batch * Hq * kv->D * 2, kv_step = (size_t)kv->batch * kv->Hkv * kv->D * 2;
+    MapCache cache;
     for (int i = 0; i < gamma; ++i) {
         if (wmtp_status s = attn_full((const char*)q + i * q_step, Hq, kv, sm_scale, (char*)out + i * q_step,
                                       lse ? lse + (size_t)i * kv->batch * Hq : nullptr, workspace, ws_bytes,
                                       (cudaStream_t)stream, false, (const char*)k_new + i * kv_step,
-                                      (const char*)v_new + i * kv_step))
+                                      (const char*)v_new + i * kv_step, 0, 0, 1, &cache))
             return s;
     }
     return WMTP_OK;
@@ -560,11 +587,12 @@ wmtp_status wmtp_draft_loop_windowed_kv(const wmtp_kv* kv, int n_sink, int W, in
     if (wmtp_status s = check_loop(gamma, k_new, v_new)) return s;
     if (wmtp_status s = check_attn_common(q, Hq, kv->Hkv, kv->batch, kv->D, out, lse, workspace, ws_bytes)) return s;
     const size_t q_step = (size_t)kv->batch * Hq * kv->D * 2, kv_step = (size_t)kv->batch * kv->Hkv * kv->D * 2;
+    MapCache cache;
     for (int i = 0; i < gamma; ++i) {
         if (wmtp_status s = attn_full((const char*)q + i * q_step, Hq, kv, sm_scale, (char*)out + i * q_step,
                                       lse ? lse + (size_t)i * kv->batch * Hq : nullptr, workspace, ws_bytes,
                                       (cudaStream_t)stream, false, (const char*)k_new + i * kv_step,
-                                      (const char*)v_new + i * kv_step, n_sink, W))
+                                      (const char*)v_new + i * kv_step, n_sink, W, 1, &cache))
             return s;
     }
     return WMTP_OK;
@@ -714,7 +742,7 @@ wmtp_status wmtp_draft_attn_windowed_noalloc(const void* q, int Hq, const wmtp_r
     p.num_ctas = pick_ctas(tiles);
     if (p.num_ctas <= 0) return fail(WMTP_ERR_CUDA, "no CUDA device available");
     if (p.num_ctas > kStaticMaxCtas) p.num_ctas = kStaticMaxCtas;
-    e = launch_attention(p, st);
+    e = launch_with(p, nullptr, st);
     if (e != cudaSuccess) return cuda_fail(e, "windowed attention launch (static scratch)");
     return WMTP_OK;
 }

@@ -1,6 +1,7 @@
 // Internal declarations shared by the library's translation units (not part of the C ABI).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -15,6 +16,7 @@ constexpr int kMaxGroups = 2;        // consumer groups per CTA (each contribute
 constexpr int kMaxBatch = 1024;     // sequences per call (prefix table lives in shared memory)
 constexpr int kMaxGroup = 8;        // query heads per KV head
 constexpr int kMaxSegments = 16384; // batch * Hkv per call
+constexpr int kClusterMaxTiles1 = 10, kClusterMaxTiles2 = 20;   // the cluster form serves launches whose CTAs get at most this many tiles (one / two consumer groups)
 constexpr int kExtendChunk = 4;     // new tokens of a sequence whose queries share one pass over its K/V (draft-extend)
 constexpr size_t kCursorBytes = 1024;                                          // int cur[kMaxCtas], padded
 constexpr size_t kWorkspaceZeroBytes = 256 + kCursorBytes + 2 * (8 + 4 + 4) * kMaxSegments;   // header + cursors + two copies of the per-segment words
@@ -85,6 +87,7 @@ struct AttnParams {
     int num_ctas;
     int stages;               // stages of the kernel's shared-memory ring (set by the launcher)
     uint32_t spin_limit;      // polls a CTA spends waiting for another CTA's global word before it gives up
+    int cluster;              // > 0: the cluster form of the kernel, one cluster of this many CTAs per segment (num_ctas = segments * cluster)
 };
 
 struct RingParams {
@@ -112,8 +115,13 @@ cudaError_t launch_ring_replace_tail(const RingParams& r, const int32_t* n_drop,
                                      int* status, cudaStream_t st);
 cudaError_t launch_reduced_block_table(const KvParams& kv, int n_sink, int W, int32_t* table, int stride, int32_t* meta, int* status,
                                        cudaStream_t st);
-// One cooperative launch: optional append of (k_new, v_new), split-KV partials, distributed LSE combine.
-cudaError_t launch_attention(const AttnParams& p, cudaStream_t st);
+// The TMA descriptors of a store's K and V tensors. They depend on the store only (base pointers, rows, head_dim, entry
+// size), so a chain of launches on one store encodes them once.
+struct AttnMaps { CUtensorMap k, v; };
+cudaError_t make_attention_maps(const AttnParams& p, AttnMaps* maps);
+// One launch: optional append of (k_new, v_new), split-KV partials, LSE combine (cooperative or cluster form: p.cluster).
+cudaError_t launch_attention(const AttnParams& p, const AttnMaps& maps, cudaStream_t st);
+int pick_cluster(int D, int f8, int nseg, int64_t tiles_per_segment, int max_ctas);
 
 // Full-context draft-extend with shared K/V tiles (bf16 stores): p.B counts sequences, p.q_len their new tokens;
 // partial results go to p.part_lse / p.part_o, (p.num_ctas + streams) * min(q_len, kExtendChunk) rows of G (x D) floats.
