@@ -143,10 +143,11 @@ def oracle_sample(wl, n_threads_hint=None):
     q = wl.q[0, 0]
     keep = R.keep_set(S, cfg.n_sink, cfg.W)
     t0 = time.perf_counter()
-    R.attention(q, K0, V0, keys=keep)
+    sc = dict(k_scale=wl.k_scale, v_scale=wl.v_scale) if wl.k_scale is not None else {}
+    R.attention(q, K0, V0, keys=keep, **sc)
     t_win = time.perf_counter() - t0
     t0 = time.perf_counter()
-    R.attention(q, K0, V0)
+    R.attention(q, K0, V0, **sc)
     t_full = time.perf_counter() - t0
     return t_win, t_full, R.threads()
 

@@ -283,8 +283,10 @@ wmtp_status wmtp_attn_mass_diagnostics(const void* out_win, const float* lse_win
 
 /* ---- tuning and accounting ---------------------------------------------------------------- */
 
-/* Upper bound on the CTAs (KV splits) of the attention kernels; 0 restores the default
- * (one CTA per SM). Process-wide; meant for tests that exercise the split/merge path. */
+/* Upper bound on the CTAs (KV splits) of the attention kernels; 0 restores the default (up to one CTA per SM).
+ * Windowed launches, which run one thread-block cluster per (sequence, KV head), take the largest cluster size that
+ * keeps the launch within the bound (never less than one CTA per pair). Process-wide; meant for tests that exercise
+ * the split/merge paths. */
 void    wmtp_set_max_ctas(int max_ctas);
 /* Tile-level work stealing between CTAs (default on): SMs that stream faster take tiles from slower ones, which
  * shortens long launches by several percent but makes the low bits of the result depend on timing. 0 selects a

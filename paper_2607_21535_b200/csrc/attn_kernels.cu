@@ -23,9 +23,11 @@
 //     The codes of an fp8 store are widened to f16 after ldmatrix and take the f16 MMA;
 //   * every K/V byte is read once from HBM and once from shared memory, shared by all heads
 //     of the group;
-//   * the launch is cooperative (all CTAs co-resident): after publishing its partial a group waits,
-//     with a bounded spin, for the other contributors of its segment and reduces its slice of the
-//     output, so the merge needs no second launch and no single CTA serialises it;
+//   * long launches (the full-context draft) are cooperative (all CTAs co-resident): after publishing its partial a
+//     group waits, with a bounded spin, for the other contributors of its segment and reduces its slice of the output,
+//     so the merge needs no second launch and no single CTA serialises it; short launches (the windowed draft: a few
+//     thousand keys per sequence, out of L2) run as one thread-block cluster per segment and merge through distributed
+//     shared memory instead (see the kernel's two forms below);
 //   * a draft step's append (Appendix A, RING; the KV write of a draft forward) is fused: the warp
 //     that owns the new token's row patches the tile in shared memory from k_new / v_new and stores
 //     the row to the KV store; the group that completes the launch's last segment advances len[].
@@ -1205,19 +1207,19 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             };
             constexpr int kMaxNp = 16 * kMaxGroups;           // partials of the largest cluster
             constexpr int kMaxOwn = kMaxNp / kGroupWarps;     // ... of which a warp sums every fourth
+            float* lse_all = scratch + 4 * kGroupThreads;     // [np][8], behind the reduction buffer
+            // one round trip through the cluster: the lse values of all partials (staged in shared memory for everybody)
+            // and, for the first pass of columns, the rows of the partials this warp sums
+            for (int i = tid; i < np * kMaxGroup; i += kGroupThreads) {
+                float x;
+                asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(x) : "r"(remote(i / kMaxGroup, kMaxGroup * D + i % kMaxGroup)));
+                lse_all[i] = x;
+            }
             for (int c0 = col_lo; c0 < col_hi; c0 += 32) {
                 const int col = c0 + lane;
                 const bool act = col < col_hi;
                 const int h = act ? col / kVec : 0;
-                // one round trip through the cluster: all partials' lse values of head h (every thread computes the
-                // weights of its own column) and, with them, the rows of the partials this warp sums
-                float x[kMaxNp];
                 float4 v[kMaxOwn];
-#pragma unroll
-                for (int s_ = 0; s_ < kMaxNp; ++s_) {
-                    x[s_] = -INFINITY;
-                    if (s_ < np) asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(x[s_]) : "r"(remote(s_, kMaxGroup * D + h)));
-                }
 #pragma unroll
                 for (int u = 0; u < kMaxOwn; ++u) {
                     const int s_ = warp + kGroupWarps * u;
@@ -1226,22 +1228,16 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
                                      : "=f"(v[u].x), "=f"(v[u].y), "=f"(v[u].z), "=f"(v[u].w) : "r"(remote(s_, col * 4)));
                 }
-                float M = -INFINITY;
-#pragma unroll
-                for (int s_ = 0; s_ < kMaxNp; ++s_) M = fmaxf(M, x[s_]);
-                float sum = 0.f;
-#pragma unroll
-                for (int s_ = 0; s_ < kMaxNp; ++s_) {
-                    x[s_] = (s_ < np && M > -INFINITY) ? __expf(x[s_] - M) : 0.f;
-                    sum += x[s_];
-                }
+                if (c0 == col_lo) group_barrier(grp);       // lse_all is in place
+                // weights of head h: every thread computes them for its own column
+                float M = -INFINITY, sum = 0.f;
+                for (int s_ = 0; s_ < np; ++s_) M = fmaxf(M, lse_all[s_ * kMaxGroup + h]);
+                for (int s_ = 0; s_ < np; ++s_) sum += M > -INFINITY ? __expf(lse_all[s_ * kMaxGroup + h] - M) : 0.f;
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                 for (int u = 0; u < kMaxOwn; ++u) {
-                    // x[warp + 4 u], by a select chain (a register array cannot be indexed by a run-time value)
-                    float w = 0.f;
-#pragma unroll
-                    for (int q = 0; q < kGroupWarps; ++q) w = (warp == q) ? x[q + kGroupWarps * u] : w;
+                    const int s_ = warp + kGroupWarps * u;
+                    const float w = (s_ < np && M > -INFINITY) ? __expf(lse_all[s_ * kMaxGroup + h] - M) : 0.f;
                     if (w > 0.f) {                           // an empty partial's rows were never written
                         acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
                         acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);

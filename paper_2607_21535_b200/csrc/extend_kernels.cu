@@ -165,6 +165,8 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         cta_flags[0] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // the merge kernel that follows on the stream may be set up from now on (it waits for this grid before it reads)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     for (int b = threadIdx.x; b < p.B; b += blockDim.x) tile_prefix[b + 1] = mq_seq_tiles(p, b);
     if (threadIdx.x == 0) tile_prefix[0] = 0;
     __syncthreads();
@@ -568,6 +570,9 @@ extend_mq_combine(const AttnParams p) {
     const int G = p.G, g = hq / G, h = hq % G;
     const int ch = jq / kQC, qi = jq % kQC, nch = mq_chunks(p);
     if (tid < 2) sums[tid] = 0;
+    // launched as a programmatic dependent of the partials kernel: nothing of global memory is read before that grid
+    // has completed and its partials are visible
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();
     {
         long long before = 0, all = 0;
@@ -670,8 +675,13 @@ cudaError_t launch_mq(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaStrea
     attn_extend_mq<D><<<p.num_ctas, MqCfg<D>::kThreads, smem, st>>>(mk, mv, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    extend_mq_combine<D><<<p.B * p.q_len * p.Hq, D / 4 * kCombineRows, 0, st>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.B * p.q_len * p.Hq); cfg.blockDim = dim3(D / 4 * kCombineRows); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, extend_mq_combine<D>, p);
 }
 
 }  // namespace

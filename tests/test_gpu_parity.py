@@ -148,6 +148,14 @@ def test_small_shapes_all_boundaries(D, max_ctas, S0):
     _run_and_check(_cfg(S0=S0, D=D, W=64, n_sink=4, seed=100 + S0), max_ctas=max_ctas)
 
 
+@pytest.mark.parametrize("D", [128, 256])
+@pytest.mark.parametrize("max_ctas", [2, 4, 8, 16, 32])
+def test_windowed_cluster_sizes(D, max_ctas):
+    # windowed launches run one thread-block cluster per (sequence, KV head); with two such pairs the CTA cap selects
+    # clusters of 1, 2, 4, 8 and 16 CTAs. 1100 ring slots are 18 tiles: ranks without a tile, ranks with two, a ragged end.
+    _run_and_check(_cfg(S0=5000, D=D, W=1096, n_sink=4, gamma=3, seed=4100 + max_ctas), max_ctas=max_ctas)
+
+
 @pytest.mark.parametrize("paged", [False, True])
 @pytest.mark.parametrize("max_ctas", [3, 0])
 def test_batched_ragged_lengths(paged, max_ctas):
