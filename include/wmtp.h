@@ -74,7 +74,8 @@ size_t wmtp_kv_elem_bytes(int kv_dtype);
 typedef struct wmtp_ring {
     void*    k;         /* device bf16 [batch][Hkv][n_sink + cap][D] */
     void*    v;         /* device bf16 [batch][Hkv][n_sink + cap][D] */
-    int32_t* slot_pos;  /* device [batch][n_sink + cap]: logical position held by each slot, -1 = never written */
+    int32_t* slot_pos;  /* device [batch][n_sink + cap]: logical position held by each slot, -1 = never written
+                           (32 bits: the bookkeeping is exact for logical lengths up to 2^31 - 1 tokens) */
     int64_t* len;       /* device [batch]: logical sequence length S (tokens appended so far) */
     int32_t  batch, Hkv, D, n_sink, W, cap;
     int32_t  kv_dtype;        /* wmtp_kv_dtype; 0 (bf16) keeps the fields below unused */
@@ -132,6 +133,9 @@ wmtp_status wmtp_ring_reset(const wmtp_ring* ring, void* stream);
  * The result is bit-identical to S sequential wmtp_ring_append calls (Section 6, "Prefill
  * sparsification": only O(W + n_sink) of the context is needed by the windowed draft).
  * Rows are copied as stored: ring and kv must have the same kv_dtype and, for fp8, equal scales.
+ * The call has no workspace to flag device-side findings in: a position whose page id lies outside [0, num_pages)
+ * is not copied and its slot is marked empty (slot_pos = -1) while len is still set to S; callers that cannot vouch for
+ * their page table check it first (wmtp_reduced_block_table and wmtp_kv_append flag bad ids in a workspace).
  */
 wmtp_status wmtp_ring_init_from_kv(const wmtp_ring* ring, const wmtp_kv* kv, void* stream);
 

@@ -339,6 +339,25 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
     }
 }
 
+// Fused append, one tensor (K or V): the row TMA brought for the new token's slot may be stale, so the warp that owns
+// it takes the row from the step's input (quantised for an fp8 store), writes it into the landed tile in shared memory
+// (`tile`: shared-memory address of the K or V tile, 128-byte swizzle) and into the store (`dst_row`, or nullptr when
+// the row has no valid place there). Kept out of line: it runs once per launch and sequence, and inside the tile loop
+// its code (the fp8 quantiser above all) would sit in the middle of every iteration's instruction stream.
+template <int D, bool F8>
+__device__ __noinline__ void patch_new_row(const void* new_rows, int64_t row_index, const float* scale, int g, uint32_t tile,
+                                           int new_row, void* dst_row, int lane) {
+    using C = Cfg<D, F8>;
+    if (lane >= C::kRowVecs) return;
+    const uint4* src = reinterpret_cast<const uint4*>(new_rows) + row_index * (D / 8);
+    uint4 x;
+    if constexpr (F8) x = quant16_e4m3(__ldg(src + 2 * lane), __ldg(src + 2 * lane + 1), __ldg(scale + g));
+    else x = __ldg(src + lane);
+    const uint32_t addr = tile + (lane >> 3) * C::kChunkBytes + new_row * 128 + (((lane & 7) ^ (new_row & 7)) << 4);
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
+    if (dst_row) reinterpret_cast<uint4*>(dst_row)[lane] = x;
+}
+
 // Launch-level bookkeeping (workspace header and per-segment words), with no reset pass and no grid barrier.
 // The per-segment words exist twice; a launch uses the copy selected by the parity of the launch epoch and,
 // at its very end, clears the other copy for the next launch (nobody can be using that one).
@@ -983,20 +1002,20 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     }
     uint32_t it = grp, cs = grp, cph = 0;
     for (;;) {
-        if (need_enter) { enter_segment(tt); need_enter = false; }
+        if (__builtin_expect(need_enter, 0)) { enter_segment(tt); need_enter = false; }
         const uint32_t s = cs, ph = cph;             // stage of tile `it` and the parity of this group's use count of it
         if (!have_tile) {
             const bool landed = mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
             tt = *reinterpret_cast<volatile int64_t*>(stage_tile + s);
             const bool end = tt < 0 || !landed;
             const bool outside = sg.seg < 0 || tt < sg.seg_start || tt >= sg.seg_start + sg.tiles;
-            if ((end || outside) && sg.seg >= 0 && seg_tiles_done > 0) flush_segment();
-            if (end || ncontrib == kMaxContrib) {
+            if (__builtin_expect((end || outside) && sg.seg >= 0 && seg_tiles_done > 0, 0)) flush_segment();
+            if (__builtin_expect(end || ncontrib == kMaxContrib, 0)) {
                 combine_outstanding();           // every segment this group contributed to (normally: once, at the end)
                 if (end) break;
             }
             have_tile = true;
-            if (outside) { need_enter = true; continue; }
+            if (__builtin_expect(outside, 0)) { need_enter = true; continue; }
         }
         have_tile = false;
         ++seg_tiles_done;
@@ -1012,28 +1031,20 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             const uint32_t sK = stage0 + s * C::kStageBytes, sV = sK + C::kTileBytes;
             int64_t new_off = 0;
             bool new_ok = true;
-            if (has_new) {
+            if (__builtin_expect(has_new, 0)) {
                 new_off = kv_row_offset(p, sg.b, sg.g, key0 + new_row, &new_ok);
                 if (!new_ok && lane == 0) atomicCAS(p.status, 0, kErrBounds);
             }
-            if (has_new && lane < C::kRowVecs) {
-                // the row TMA brought may be stale: take it from k_new (quantised for an fp8 store), in shared memory and in the store
-                const uint4* src = reinterpret_cast<const uint4*>(p.k_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8);
-                uint4 x;
-                if constexpr (F8) x = quant16_e4m3(__ldg(src + 2 * lane), __ldg(src + 2 * lane + 1), __ldg(p.k_scale + sg.g));
-                else x = __ldg(src + lane);
-                const uint32_t addr = sK + (lane >> 3) * C::kChunkBytes + new_row * 128 + (((lane & 7) ^ (new_row & 7)) << 4);
-                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
-                if (new_ok) reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(p.k) + new_off * C::kElemBytes)[lane] = x;
-            }
-            if (has_new) {
+            if (__builtin_expect(has_new, 0))
+                patch_new_row<D, F8>(p.k_new, (int64_t)sg.b * p.Hkv + sg.g, p.k_scale, sg.g, sK, new_row,
+                                     new_ok ? reinterpret_cast<unsigned char*>(p.k) + new_off * C::kElemBytes : nullptr, lane);
+            if (__builtin_expect(has_new, 0)) {
                 if (p.mode == kRing && sg.g == 0 && lane == 0)
                     p.slot_pos[(int64_t)sg.b * p.rows_per_head + key0 + new_row] = (int32_t)(sg.S - 1);
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
             }
             uint32_t pb0 = 0, pb1 = 0;
-            float corr0 = 1.f, corr1 = 1.f;
             if (any_valid) {
                 // ---- S^T = K . Q^T for this warp's 16 keys (two accumulator chains)
                 float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
@@ -1069,10 +1080,12 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         mma_f16(sb, a, qc.x, qc.y);
                     }
                 }
+                // raw scores; the multipliers smul (softmax scale in log2 units, for an fp8 store also the key scale and the
+                // query's power of two: all positive) are applied to the maxima and inside the exponentials
                 float sc[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) sc[i] = (sa[i] + sb[i]) * smul[i & 1];
-                if (!tile_full) {
+                for (int i = 0; i < 4; ++i) sc[i] = sa[i] + sb[i];
+                if (__builtin_expect(!tile_full, 0)) {
                     const int ka = wkey0 + g8, kb = ka + 8;
                     bool va = ka >= vlo && ka < vhi, vb = kb >= vlo && kb < vhi;
                     if (slack) {
@@ -1089,45 +1102,41 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                     mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
                     mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
                 }
-                const float mn0 = fmaxf(m[0], mx0), mn1 = fmaxf(m[1], mx1);
-                const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
-                corr0 = ex2(m[0] - mu0);
-                corr1 = ex2(m[1] - mu1);
-                m[0] = mn0; m[1] = mn1;
-                const float p0 = ex2(sc[0] - mu0), p1 = ex2(sc[1] - mu1), p2 = ex2(sc[2] - mu0), p3 = ex2(sc[3] - mu1);
-                const uint32_t pa = F8 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1);             // key g8   : heads 2t4, 2t4+1
-                const uint32_t pc = F8 ? pack_f16x2(p2, p3) : pack_bf16x2(p2, p3);             // key g8+8
-                le[0] = le[0] * corr0 + p0 + p2;
-                le[1] = le[1] * corr1 + p1 + p3;
-                if constexpr (F8) {
-                    l[0] = l[0] * corr0 + f16lo(pa) + f16lo(pc);
-                    l[1] = l[1] * corr1 + f16hi(pa) + f16hi(pc);
-                } else {
-                    l[0] = l[0] * corr0 + bf16lo(pa) + bf16lo(pc);      // sums of the rounded weights the MMA will use
-                    l[1] = l[1] * corr1 + bf16hi(pa) + bf16hi(pc);
-                }
-                pb0 = movmatrix_trans(pa);                           // P^T as B operand: k = key, n = head
-                pb1 = movmatrix_trans(pc);
+                const float mn0 = fmaxf(m[0], mx0 * smul[0]), mn1 = fmaxf(m[1], mx1 * smul[1]);
                 // the running maxima rarely move after the first tiles of a segment: rescale only when some lane's did
-                if (__any_sync(0xffffffffu, corr0 != 1.f || corr1 != 1.f)) {
+                if (__builtin_expect(__any_sync(0xffffffffu, mn0 != m[0] || mn1 != m[1]), 0)) {
+                    const float corr0 = mn0 == -INFINITY ? 1.f : ex2(m[0] - mn0), corr1 = mn1 == -INFINITY ? 1.f : ex2(m[1] - mn1);
+                    le[0] *= corr0; le[1] *= corr1;
+                    l[0] *= corr0; l[1] *= corr1;
 #pragma unroll
                     for (int mb = 0; mb < C::kKSteps; ++mb) {
                         o[mb][0] *= corr0; o[mb][1] *= corr1; o[mb][2] *= corr0; o[mb][3] *= corr1;
                     }
+                    m[0] = mn0; m[1] = mn1;
                 }
+                const float nu0 = mn0 == -INFINITY ? 0.f : -mn0, nu1 = mn1 == -INFINITY ? 0.f : -mn1;
+                const float p0 = ex2(fmaf(sc[0], smul[0], nu0)), p1 = ex2(fmaf(sc[1], smul[1], nu1));
+                const float p2 = ex2(fmaf(sc[2], smul[0], nu0)), p3 = ex2(fmaf(sc[3], smul[1], nu1));
+                const uint32_t pa = F8 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1);             // key g8   : heads 2t4, 2t4+1
+                const uint32_t pc = F8 ? pack_f16x2(p2, p3) : pack_bf16x2(p2, p3);             // key g8+8
+                le[0] += p0 + p2;
+                le[1] += p1 + p3;
+                if constexpr (F8) {
+                    l[0] += f16lo(pa) + f16lo(pc);
+                    l[1] += f16hi(pa) + f16hi(pc);
+                } else {
+                    l[0] += bf16lo(pa) + bf16lo(pc);      // sums of the rounded weights the MMA will use
+                    l[1] += bf16hi(pa) + bf16hi(pc);
+                }
+                pb0 = movmatrix_trans(pa);                           // P^T as B operand: k = key, n = head
+                pb1 = movmatrix_trans(pc);
             }
             mbar_wait(bar_fullV + 8 * s, ph, abort_flag, p.status);
-            if (has_new && lane < C::kRowVecs) {
-                const uint4* src = reinterpret_cast<const uint4*>(p.v_new) + ((int64_t)sg.b * p.Hkv + sg.g) * (D / 8);
-                uint4 x;
-                if constexpr (F8) x = quant16_e4m3(__ldg(src + 2 * lane), __ldg(src + 2 * lane + 1), __ldg(p.v_scale + sg.g));
-                else x = __ldg(src + lane);
-                const uint32_t addr = sV + (lane >> 3) * C::kChunkBytes + new_row * 128 + (((lane & 7) ^ (new_row & 7)) << 4);
-                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
-                if (new_ok) reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(p.v) + new_off * C::kElemBytes)[lane] = x;
-            }
+            if (__builtin_expect(has_new, 0))
+                patch_new_row<D, F8>(p.v_new, (int64_t)sg.b * p.Hkv + sg.g, p.v_scale, sg.g, sV, new_row,
+                                     new_ok ? reinterpret_cast<unsigned char*>(p.v) + new_off * C::kElemBytes : nullptr, lane);
             if (any_valid) {
-                if (wkey0 + 16 > vhi) {
+                if (__builtin_expect(wkey0 + 16 > vhi, 0)) {
                     // rows past the end were never written (or, in a sink tile of a window view, may be): they can hold
                     // NaN/Inf bit patterns, and 0 * NaN would poison the accumulators. Zero them in shared memory.
                     const int first_bad = vhi > wkey0 ? vhi - wkey0 : 0;
@@ -1137,7 +1146,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
                     }
                 }
-                if (has_new || wkey0 + 16 > vhi) {
+                if (__builtin_expect(has_new || wkey0 + 16 > vhi, 0)) {
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                 }

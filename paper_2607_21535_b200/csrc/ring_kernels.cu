@@ -120,8 +120,11 @@ __global__ void ring_init_kernel(RingParams r, KvParams kv) {
     uint4* V = reinterpret_cast<uint4*>(r.v);
     for (int s = blockIdx.x * warps + warp; s < slots; s += gridDim.x * warps) {
         const int64_t p = ring_slot_position(s, S, r.n_sink, r.cap);
-        if (lane == 0) r.slot_pos[(int64_t)b * slots + s] = (int32_t)p;
-        if (p < 0) continue;
+        bool page_ok = true;
+        if (p >= 0) kv_row_vec(kv, b, 0, p, vec_per_row, &page_ok);
+        // a position whose page id is out of range cannot be copied: the slot is marked empty rather than claimed
+        if (lane == 0) r.slot_pos[(int64_t)b * slots + s] = page_ok ? (int32_t)p : -1;
+        if (p < 0 || !page_ok) continue;
         for (int g = 0; g < r.Hkv; ++g) {
             bool ok = true;
             const int64_t src = kv_row_vec(kv, b, g, p, vec_per_row, &ok);
