@@ -869,13 +869,13 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             if (M > -INFINITY) {
 #pragma unroll
                 for (int w = 0; w < kGroupWarps; ++w) {
-                    const float e = exp2f(sm_m[w * kMaxGroup + h] - M);
+                    const float e = ex2(sm_m[w * kMaxGroup + h] - M);
                     L += sm_l[w * kMaxGroup + h] * e;
                     Le += sm_le[w * kMaxGroup + h] * e;
                 }
             }
-            f[i] = (L > 0.f && m[i] > -INFINITY) ? exp2f(m[i] - M) / L * vscale : 0.f;
-            if (warp == 0 && g8 == 0 && h < G) dst_lse[h] = Le > 0.f ? (M + log2f(Le)) * kLn2 : -INFINITY;
+            f[i] = (L > 0.f && m[i] > -INFINITY) ? ex2(m[i] - M) / L * vscale : 0.f;
+            if (warp == 0 && g8 == 0 && h < G) dst_lse[h] = Le > 0.f ? (M + lg2(Le)) * kLn2 : -INFINITY;
         }
         constexpr int kPasses = D / C::kPassCols;               // kPassCols columns of d per pass through the scratch
         constexpr int kScratchRow = C::kScratchRow;

@@ -295,13 +295,13 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 if (M > -INFINITY) {
 #pragma unroll
                     for (int w = 0; w < kMqWarps; ++w) {
-                        const float e = exp2f(sm_m[w * kMaxGroup + h] - M);
+                        const float e = ex2(sm_m[w * kMaxGroup + h] - M);
                         L += sm_l[w * kMaxGroup + h] * e;
                         Le += sm_le[w * kMaxGroup + h] * e;
                     }
                 }
-                f[i] = (L > 0.f && m[j][i] > -INFINITY) ? exp2f(m[j][i] - M) / L : 0.f;
-                if (warp == 0 && g8 == 0 && h < G) p.part_lse[prow * G + h] = Le > 0.f ? (M + log2f(Le)) * kLn2f : -INFINITY;
+                f[i] = (L > 0.f && m[j][i] > -INFINITY) ? ex2(m[j][i] - M) / L : 0.f;
+                if (warp == 0 && g8 == 0 && h < G) p.part_lse[prow * G + h] = Le > 0.f ? (M + lg2(Le)) * kLn2f : -INFINITY;
             }
             constexpr int kPasses = D / C::kPassCols;
 #pragma unroll
@@ -453,7 +453,7 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         bool moved = false;
 #pragma unroll
         for (int j = 0; j < kQW; ++j) moved = moved || mn[j][0] != m[j][0] || mn[j][1] != m[j][1];
-        if (__any_sync(0xffffffffu, moved)) {
+        if (__builtin_expect(__any_sync(0xffffffffu, moved), 0)) {
 #pragma unroll
             for (int j = 0; j < kQW; ++j) {
                 const float corr0 = mn[j][0] == -INFINITY ? 1.f : ex2(m[j][0] - mn[j][0]);
@@ -508,7 +508,7 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             const int key0n = (int)(tn - sg.start) * kTileKeys;
             const uint32_t sKn = stage0 + ns * C::kStageBytes, sV = stage0 + cs * C::kStageBytes + C::kTileBytes;
             mbar_wait(bar_fullV + 8 * cs, cph, abort_flag, p.status);
-            if (valid_c && key0 + warp * 16 + 16 > sg.S_last) {
+            if (__builtin_expect(valid_c && key0 + warp * 16 + 16 > sg.S_last, 0)) {
                 // rows past the end of the sequence were never written: they can hold NaN/Inf bit patterns, and 0 * NaN
                 // would poison the accumulators. Zero them in shared memory (the other group's warp on the same keys
                 // writes the same zeros).
@@ -522,12 +522,12 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
             }
-            if (valid_c && valid_n) { qk_pv(Yes{}, sKn, scn, Yes{}, sV, pb); weights(scn, key0n, pbn); }
+            if (__builtin_expect(valid_c && valid_n, 1)) { qk_pv(Yes{}, sKn, scn, Yes{}, sV, pb); weights(scn, key0n, pbn); }
             else if (valid_c) qk_pv(No{}, 0u, scn, Yes{}, sV, pb);
             else if (valid_n) { qk_pv(Yes{}, sKn, scn, No{}, 0u, pb); weights(scn, key0n, pbn); }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_emptyV + 8 * cs);
-            if (!same) {
+            if (__builtin_expect(!same, 0)) {
                 flush();
                 if (end) break;
                 enter(tn);
