@@ -1214,7 +1214,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                              : "=r"(a) : "r"(part_local + 4u * (uint32_t)((s_ % C::kGroups) * kPart + off_floats)), "r"((uint32_t)(s_ / C::kGroups)));
                 return a;
             };
-            constexpr int kMaxNp = 16 * kMaxGroups;           // partials of the largest cluster
+            constexpr int kMaxNp = kMaxCluster * kMaxGroups;           // partials of the largest cluster
             constexpr int kMaxOwn = kMaxNp / kGroupWarps;     // ... of which a warp sums every fourth
             float* lse_all = scratch + 4 * kGroupThreads;     // [np][8], behind the reduction buffer
             // one round trip through the cluster: the lse values of all partials (staged in shared memory for everybody)
@@ -1372,7 +1372,7 @@ static_assert(cluster_stages<256, false>() == 3 && cluster_stages<256, true>() >
 
 // One-time set-up per device: shared-memory opt-in, non-portable cluster sizes, and how many clusters of each size the
 // device holds at once (index: log2 of the cluster size).
-struct ClusterInfo { bool ready; int active[5]; };
+struct ClusterInfo { bool ready; int sms; int active[kMaxCluster + 1]; };   // active[c]: resident clusters of c CTAs
 template <int D, bool F8>
 cudaError_t cluster_info(const ClusterInfo** out) {
     static std::mutex mu;
@@ -1386,16 +1386,17 @@ cudaError_t cluster_info(const ClusterInfo** out) {
         cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
-        for (int l2 = 0; l2 < 5; ++l2) {
+        if (cudaDeviceGetAttribute(&info[dev].sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) info[dev].sms = 0;
+        for (int cl = 1; cl <= kMaxCluster; ++cl) {
             cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(1 << l2); cfg.blockDim = dim3(Cfg<D, F8>::kThreads); cfg.dynamicSmemBytes = cluster_smem_bytes<D, F8>();
+            cfg.gridDim = dim3(cl); cfg.blockDim = dim3(Cfg<D, F8>::kThreads); cfg.dynamicSmemBytes = cluster_smem_bytes<D, F8>();
             cudaLaunchAttribute at[1];
             at[0].id = cudaLaunchAttributeClusterDimension;
-            at[0].val.clusterDim.x = 1u << l2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            at[0].val.clusterDim.x = (unsigned)cl; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
             cfg.attrs = at; cfg.numAttrs = 1;
             int n = 0;
             if (cudaOccupancyMaxActiveClusters(&n, fn, &cfg) != cudaSuccess) { n = 0; (void)cudaGetLastError(); }
-            info[dev].active[l2] = n;
+            info[dev].active[cl] = n;
         }
         info[dev].ready = true;
     }
@@ -1459,20 +1460,23 @@ int pick_cluster(int D, int f8, int nseg, int64_t tiles, int max_ctas) {
     if (f8) e = D == 128 ? cluster_info<128, true>(&info) : cluster_info<256, true>(&info);
     else e = D == 128 ? cluster_info<128, false>(&info) : cluster_info<256, false>(&info);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    // the largest cluster all of whose copies are resident at once (a second wave of clusters would double the time)
     int best = 0;
-    for (int l2 = 0; l2 < 5; ++l2) {
-        const int cl = 1 << l2;
-        if (info->active[l2] <= 0) continue;
+    for (int cl = 1; cl <= kMaxCluster; ++cl) {
+        if (info->active[cl] <= 0 || (cl > 1 && nseg > info->active[cl])) continue;
         if (cl > 1 && cl > tiles) break;
         if (max_ctas > 0 && (int64_t)nseg * cl > max_ctas && cl > 1) break;
-        if (l2 > 0 && nseg > info->active[l2]) break;               // a second wave of clusters would double the time
         best = cl;
     }
     if (best == 0) return 0;
-    // long segments: the cooperative form spreads them over all SMs (a CTA with one consumer group takes about 1 us per
-    // 64 KB tile out of L2, one with two groups half of that)
-    const bool one_group = 2 * kTileKeys * D * (f8 ? 1 : 2) >= 65536;
-    if ((tiles + best - 1) / best > (one_group ? kClusterMaxTiles1 : kClusterMaxTiles2)) return 0;
+    // Which form is faster: a cluster CTA streams ceil(tiles / best) tiles of its segment, the cooperative form spreads
+    // all tiles over every SM but pays a longer launch, a grid-wide combine and no overlap with the launch before it.
+    // Measured per-tile times of one CTA reading through L2 and the difference of the fixed costs decide.
+    const int64_t per_cta = (tiles + best - 1) / best;
+    const int coop_ctas = max_ctas > 0 && max_ctas < info->sms ? max_ctas : info->sms;
+    const int64_t per_coop = (tiles * nseg + coop_ctas - 1) / (coop_ctas > 0 ? coop_ctas : 1);
+    const int tile_ns = f8 ? (D == 256 ? kTileNsF8D256 : kTileNsF8D128) : (D == 256 ? kTileNsD256 : kTileNsD128);
+    if ((per_cta - per_coop) * tile_ns > kClusterFixedGainNs) return 0;
     return best;
 }
 

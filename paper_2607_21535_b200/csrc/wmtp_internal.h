@@ -16,7 +16,11 @@ constexpr int kMaxGroups = 2;        // consumer groups per CTA (each contribute
 constexpr int kMaxBatch = 1024;     // sequences per call (prefix table lives in shared memory)
 constexpr int kMaxGroup = 8;        // query heads per KV head
 constexpr int kMaxSegments = 16384; // batch * Hkv per call
-constexpr int kClusterMaxTiles1 = 10, kClusterMaxTiles2 = 20;   // the cluster form serves launches whose CTAs get at most this many tiles (one / two consumer groups)
+constexpr int kMaxCluster = 16;                                  // CTAs in a thread-block cluster (the non-portable limit)
+// Choice between the cluster form and the cooperative form of a windowed launch: time one CTA takes per 64-key tile (ns,
+// measured with the ring in L2) and what the cluster form saves in fixed cost (launch overlap, no grid-wide combine).
+constexpr int kTileNsD256 = 1000, kTileNsD128 = 500, kTileNsF8D256 = 800, kTileNsF8D128 = 450;
+constexpr int kClusterFixedGainNs = 5500;
 constexpr int kExtendChunk = 4;     // new tokens of a sequence whose queries share one pass over its K/V (draft-extend)
 constexpr size_t kCursorBytes = 1024;                                          // int cur[kMaxCtas], padded
 constexpr size_t kWorkspaceZeroBytes = 256 + kCursorBytes + 2 * (8 + 4 + 4) * kMaxSegments;   // header + cursors + two copies of the per-segment words

@@ -149,10 +149,11 @@ def test_small_shapes_all_boundaries(D, max_ctas, S0):
 
 
 @pytest.mark.parametrize("D", [128, 256])
-@pytest.mark.parametrize("max_ctas", [2, 4, 8, 16, 32])
+@pytest.mark.parametrize("max_ctas", [2, 4, 6, 8, 10, 14, 16, 22, 26, 32])
 def test_windowed_cluster_sizes(D, max_ctas):
     # windowed launches run one thread-block cluster per (sequence, KV head); with two such pairs the CTA cap selects
-    # clusters of 1, 2, 4, 8 and 16 CTAs. 1100 ring slots are 18 tiles: ranks without a tile, ranks with two, a ragged end.
+    # clusters of 1, 2, 3, 4, 5, 7, 8, 11, 13 and 16 CTAs (any size up to 16 is used, not only powers of two). 1100 ring
+    # slots are 18 tiles: ranks with one tile and ranks with two or three, output columns that do not divide evenly.
     _run_and_check(_cfg(S0=5000, D=D, W=1096, n_sink=4, gamma=3, seed=4100 + max_ctas), max_ctas=max_ctas)
 
 
