@@ -20,7 +20,9 @@
 //     MMA M dimension, the G <= 8 query heads of the GQA group exactly on N = 8), the online softmax runs
 //     in fp32, and O^T[d, head] += V^T[d, key] . P^T[key, head] accumulates in registers. The 8-row problem
 //     is far too small for tcgen05 (M >= 64); mma.sync.m16n8k16 needs a few percent of tensor peak here.
-//     The codes of an fp8 store are widened to f16 after ldmatrix and take the f16 MMA;
+//     The codes of an fp8 store are widened to f16 after ldmatrix and take the f16 MMA. The smallest tiles (8 KB:
+//     head_dim 128, fp8) are streamed and consumed two at a time -- a stage holds two consecutive tiles of a segment and
+//     a warp works on its 16 keys of both, one softmax update over the 32 keys;
 //   * every K/V byte is read once from HBM and once from shared memory, shared by all heads
 //     of the group;
 //   * long launches (the full-context draft) are cooperative (all CTAs co-resident): after publishing its partial a
@@ -35,6 +37,7 @@
 #include <cuda_bf16.h>
 
 #include <mutex>
+#include <type_traits>
 
 #include "attn_plan.cuh"
 #include "fp8_util.cuh"
@@ -47,15 +50,15 @@ namespace {
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kGroupWarps = 4;                  // warps per consumer group: 4 x 16 keys = one tile
 constexpr int kGroupThreads = kGroupWarps * 32;
-constexpr int kMaxGroups = 2;
 constexpr int kMaxParts = kMaxGroups * kMaxCtas; // partials one segment can receive
 // Per-group scratch, used for two things in turn:
 //   the warp merge of a flush: [4 warps][8 heads][pass columns + 4] floats, `pass columns` of d at a time;
 //   the combine: weights [heads of this contributor's slice][np], inverses [8], a reduction buffer [128] float4 and the
-//   visiting order [np]. A contributor's slice of the (head, d) columns spans at most two heads once there are at least
+//   visiting order [np] (16-bit entries). A contributor's slice of the (head, d) columns spans at most two heads once there are at least
 //   G contributors, and fewer than G * G (head, partial) pairs otherwise: 2 * kMaxParts weights always suffice.
 constexpr int kCombineWeights = 2 * kMaxParts;
-constexpr int kCombineFloats = kCombineWeights + 8 + 4 * kGroupThreads + kMaxParts;
+constexpr int kCombineFloats = kCombineWeights + 8 + 4 * kGroupThreads + kMaxParts / 2;
+static_assert(kMaxParts < 65536 && kMaxParts % 2 == 0, "visiting order held in 16-bit entries");
 static_assert(kMaxGroup * kMaxGroup <= kCombineWeights, "weights of a slice must fit");
 constexpr int kMaxContrib = 32;     // segments a group may have outstanding before it combines them
 constexpr int kStealChunkBytes = 262144;        // bytes of K/V handed out per cursor step
@@ -63,24 +66,28 @@ constexpr int kStealChunkBytes = 262144;        // bytes of K/V handed out per c
 // contrib[kMaxContrib][4] = {seg, b, g, slot}, reg_k[kMaxContrib] (slot of the group's i-th contribution, producer -> group)
 constexpr int kGroupInts = 4 + 5 * kMaxContrib;
 
-// D: head_dim; F8: the store holds e4m3 codes (one byte per entry) instead of bf16.
-template <int D, bool F8>
+// D: head_dim; F8: the store holds e4m3 codes (one byte per entry) instead of bf16; CL: the cluster form of the kernel.
+template <int D, bool F8, bool CL = false>
 struct Cfg {
     static constexpr int kElemBytes = F8 ? 1 : 2;
     static constexpr int kChunks = D * kElemBytes / 128;      // 128-byte column chunks per row
     static constexpr int kChunkBytes = kTileKeys * 128;       // one TMA box: 64 rows x 128 B
     static constexpr int kTileBytes = kChunks * kChunkBytes;  // K (or V) tile
-    static constexpr int kStageBytes = 2 * kTileBytes;
+    // Tiles per stage. The smallest tiles (8 KB: head_dim 128, fp8) travel and are consumed in pairs of consecutive tiles
+    // of a segment in the streaming form: a warp then works on two independent 16-key slabs at once (its dependent
+    // chain per tile, not any unit of the SM, limits the rate), and the producer's per-stage work is halved.
+    static constexpr int kPair = (F8 && D == 128 && !CL) ? 2 : 1;
+    static constexpr int kStageBytes = kPair * 2 * kTileBytes;
     // consumer groups: a tile of fewer bytes brings the same softmax work, so the smaller tiles get two groups
-    static constexpr int kGroups = (kStageBytes >= 65536) ? 1 : 2;
+    static constexpr int kGroups = (D == 256 && !F8) ? 1 : 2;
     // Stages of the shared-memory ring. What counts for the streaming rate is the bytes a CTA keeps in flight (about
     // 190 KB per SM saturate HBM at the loaded latency of ~4 us): the host takes as many stages as fit beside the
     // batch-dependent tables, up to kMaxStages, in multiples of the group count (a stage then always serves one group).
     static constexpr int kMaxStages = (kStageBytes >= 65536) ? 3 : (kStageBytes >= 32768 ? 6 : 12);
-    static constexpr int kRowVecs = D * kElemBytes / 16;      // 16-byte vectors per stored row
     // Tiles handed out per cursor step. A step costs a global atomic (about 1.5 us) that is fetched one chunk ahead: the
     // chunk must take longer than that to stream, so it is sized in bytes (256 KB), not in tiles.
-    static constexpr int kStealChunk = kStealChunkBytes / kStageBytes;
+    static constexpr int kStealChunk = kStealChunkBytes / (2 * kTileBytes);
+    static_assert(kStealChunk % kPair == 0, "a cursor step hands out whole stages");
     static constexpr int kStealMinTiles = 8 * kStealChunk;   // ranges shorter than this are streamed statically
     // columns of d merged per pass of a flush: the two-group configurations trade a second pass for shared memory
     static constexpr int kPassCols = (kGroups == 2) ? 64 : 128;
@@ -89,19 +96,19 @@ struct Cfg {
     static constexpr int kScratchFloats = kMergeFloats > kCombineFloats ? kMergeFloats : kCombineFloats;
     // With two groups the CTA has 9 warps and a thread at most 168 registers: the query fragments (the same in all four
     // warps of a group) then live in shared memory, one copy per group, instead of D / 8 registers per thread.
-    static constexpr bool kQShared = (kGroups == 2);
+    static constexpr bool kQShared = (kGroups >= 2);
     static constexpr int kQBytes = kQShared ? kGroups * (D / 16) * 32 * 8 : 0;
     static constexpr int kConsumerWarps = kGroups * kGroupWarps;
     // With two consumer groups the CTA would have 9 warps and every thread at most 168 registers (three warps share
     // one scheduler's register file); the consumers want more and the producer needs about 56. So after the common
     // prologue the producer's warpgroup hands registers to the consumers' warpgroups (setmaxnreg). The instruction is
     // warpgroup-wide: the producer's warpgroup is filled up with three warps that execute it and exit.
-    static constexpr bool kRebalance = (kGroups == 2);
+    static constexpr bool kRebalance = (kGroups >= 2);
     static constexpr int kPadWarps = kRebalance ? 3 : 0;
+    static constexpr int kThreads = (kConsumerWarps + 1 + kPadWarps) * 32;
     static constexpr int kRegsProducer = 56, kRegsConsumer = 224;
     // the 8 consumer warps and the 4 warps of the producer's warpgroup share what the 12 warps were launched with
-    static_assert(8 * kRegsConsumer + 4 * kRegsProducer <= 12 * 168, "register trade must balance");
-    static constexpr int kThreads = (kConsumerWarps + 1 + kPadWarps) * 32;
+    static_assert(!kRebalance || (kGroups == 2 && 8 * kRegsConsumer + 4 * kRegsProducer <= 12 * 168), "register trade must balance");
     static constexpr int kKSteps = D / 16;
     static constexpr int kBarriers = (1 + 2 * kGroups) * kMaxStages;
     // bytes of the fixed-size part of shared memory (scratch, softmax statistics, query fragments, barriers, stage tags,
@@ -110,6 +117,7 @@ struct Cfg {
                                      8 * kMaxStages + 8 * kGroups * 2 * kMaxContrib + 4 * kGroups * kGroupInts + 16;
     static constexpr int kFixedBytes = (kFixedRaw + 1023) / 1024 * 1024;
     static_assert(kMaxStages % kGroups == 0, "a stage must always serve the same group");
+    static_assert(kGroups <= kMaxGroups, "partial slots are reserved for kMaxGroups groups per CTA");
 };
 
 // Bounded spin on a global word written by other CTAs of this (cooperative) launch: waits until
@@ -213,7 +221,7 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
     float* w_sm = scratch;                                                  // [heads of the slice][np]
     float* inv_sm = scratch + kCombineWeights;                              // [8], indexed by head - first head of the slice
     float4* red = reinterpret_cast<float4*>(inv_sm + 8);                    // [128]
-    int* perm = reinterpret_cast<int*>(inv_sm + 8 + 4 * kGroupThreads);     // [np] visiting order
+    uint16_t* perm = reinterpret_cast<uint16_t*>(inv_sm + 8 + 4 * kGroupThreads);   // [np] visiting order
 
     // ---- visiting order: the fixed partition ranks the partials by their keys; with stealing on they are taken as stored
     const bool ranked = !p.steal_slots_enabled;
@@ -225,11 +233,11 @@ __device__ __noinline__ void combine_segment(const AttnParams& p, int b, int g, 
             const int ki = keys[i];
             int r = 0;
             for (int q = 0; q < np; ++q) r += keys[q] < ki;
-            perm[r] = i;
+            perm[r] = (uint16_t)i;
         }
         group_barrier(grp);
     }
-    auto part = [&](int i) { return ranked ? perm[i] : i; };
+    auto part = [&](int i) { return ranked ? (int)perm[i] : i; };
 
     // ---- this group's slice of the (head, d) columns; the first rows are requested before the weights exist
     constexpr int kPre = 6;
@@ -348,7 +356,8 @@ template <int D, bool F8>
 __device__ __noinline__ void patch_new_row(const void* new_rows, int64_t row_index, const float* scale, int g, uint32_t tile,
                                            int new_row, void* dst_row, int lane) {
     using C = Cfg<D, F8>;
-    if (lane >= C::kRowVecs) return;
+    constexpr int kRowVecs = D * C::kElemBytes / 16;        // 16-byte vectors per stored row
+    if (lane >= kRowVecs) return;
     const uint4* src = reinterpret_cast<const uint4*>(new_rows) + row_index * (D / 8);
     uint4 x;
     if constexpr (F8) x = quant16_e4m3(__ldg(src + 2 * lane), __ldg(src + 2 * lane + 1), __ldg(scale + g));
@@ -388,10 +397,10 @@ __device__ __noinline__ void patch_new_row(const void* new_rows, int64_t row_ind
 //     the workspace header -- advances the lengths of a fused append. Tile processing is the same code in both forms.
 // ---------------------------------------------------------------------------------------------
 template <int D, bool F8, bool CL>
-__global__ void __launch_bounds__(Cfg<D, F8>::kThreads, 1)
+__global__ void __launch_bounds__(Cfg<D, F8, CL>::kThreads, 1)
 attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                const __grid_constant__ AttnParams p) {
-    using C = Cfg<D, F8>;
+    using C = Cfg<D, F8, CL>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     // Shared memory: the fixed-size part first (compile-time offsets), then the stage ring (1024-byte aligned for the
@@ -617,8 +626,12 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         }
                     }
                     const int cnt = ntiles - base < 32 ? ntiles - base : 32;
-                    for (int j = 0; j < cnt; ++j, ++it, ps = (ps + 1 == nst ? 0 : ps + 1), pph ^= (ps == 0)) {
-                        const int pg = __shfl_sync(0xffffffffu, page, j);
+                    // one stage per step: kPair consecutive tiles of the segment (a single one at an odd end)
+                    for (int j = 0; j < cnt; j += C::kPair, ++it, ps = (ps + 1 == nst ? 0 : ps + 1), pph ^= (ps == 0)) {
+                        const int c2 = cnt - j < C::kPair ? cnt - j : C::kPair;       // tiles in this stage
+                        int pg[C::kPair];
+#pragma unroll
+                        for (int h = 0; h < C::kPair; ++h) pg[h] = __shfl_sync(0xffffffffu, page, (j + h) & 31);
                         const int gq = (int)(it % C::kGroups);
                         settle(gq);
                         if (grp_seg[gq] != sg.seg) {
@@ -632,19 +645,27 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                             const uint32_t s = ps, ph = pph;
                             const uint32_t bar_fullK = bar_fullK0 + 8 * (gq * C::kMaxStages), bar_fullV = bar_fullV0 + 8 * (gq * C::kMaxStages);
                             if (mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status)) {
-                                int64_t row;
-                                if (p.mode == kPaged) row = ((int64_t)pg * p.Hkv + sg.g) * kTileKeys;
-                                else {
-                                    const int64_t tj = first_tile + base + j;
-                                    const int64_t src = tj < sg.sink_tiles ? tj : sg.win_first + tj - sg.sink_tiles;
-                                    row = ((int64_t)kv_seq(p, sg.b) * p.Hkv + sg.g) * p.rows_per_head + src * kTileKeys;
+                                const uint32_t dstK = stage0 + s * C::kStageBytes, dstV = dstK + C::kPair * C::kTileBytes;
+                                // ordered before the consumers' wait by the arrive below
+                                stage_tile[s] = C::kPair == 1 ? t + base + j : (((t + base + j) << 1) | (int64_t)(c2 - 1));
+                                int64_t row[C::kPair];
+#pragma unroll
+                                for (int h = 0; h < C::kPair; ++h) {
+                                    if (p.mode == kPaged) row[h] = ((int64_t)pg[h] * p.Hkv + sg.g) * kTileKeys;
+                                    else {
+                                        const int64_t tj = first_tile + base + j + h;
+                                        const int64_t src = tj < sg.sink_tiles ? tj : sg.win_first + tj - sg.sink_tiles;
+                                        row[h] = ((int64_t)kv_seq(p, sg.b) * p.Hkv + sg.g) * p.rows_per_head + src * kTileKeys;
+                                    }
                                 }
-                                const uint32_t dstK = stage0 + s * C::kStageBytes, dstV = dstK + C::kTileBytes;
-                                stage_tile[s] = t + base + j;          // ordered before the consumers' wait by the arrive below
-                                mbar_expect_tx(bar_fullK + 8 * s, C::kTileBytes);
-                                tma_load_3d(dstK, &mapK, (int)row, bar_fullK + 8 * s);
-                                mbar_expect_tx(bar_fullV + 8 * s, C::kTileBytes);
-                                tma_load_3d(dstV, &mapV, (int)row, bar_fullV + 8 * s);
+                                mbar_expect_tx(bar_fullK + 8 * s, c2 * C::kTileBytes);
+#pragma unroll
+                                for (int h = 0; h < C::kPair; ++h)
+                                    if (h < c2) tma_load_3d(dstK + h * C::kTileBytes, &mapK, (int)row[h], bar_fullK + 8 * s);
+                                mbar_expect_tx(bar_fullV + 8 * s, c2 * C::kTileBytes);
+#pragma unroll
+                                for (int h = 0; h < C::kPair; ++h)
+                                    if (h < c2) tma_load_3d(dstV + h * C::kTileBytes, &mapV, (int)row[h], bar_fullV + 8 * s);
                             }
                         }
                     }
@@ -989,134 +1010,139 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 #pragma unroll
         for (int mb = 0; mb < C::kKSteps; ++mb) { o[mb][0] = o[mb][1] = o[mb][2] = o[mb][3] = 0.f; }
     };
-    // The loop is written so that enter / flush / tile processing each appear once in the code (the kernel's
-    // tail runs once per launch, from a cold instruction cache: code size is latency there).
-    int64_t tt = -1;                                     // tile in hand
-    bool have_tile = false, need_enter = false;
-    if constexpr (CL) {
-        if (c_lo + grp < c_hi) { tt = c_lo + grp; need_enter = true; }
-    } else if ((int)blockIdx.x < Cn) {
-        // an owner knows its first tiles: fetch the query while they are still in flight
-        const int64_t first = cta_range_start(blockIdx.x, n, Cn) + grp;
-        if (first < cta_range_start(blockIdx.x + 1, n, Cn)) { tt = first; need_enter = true; }
-    }
-    uint32_t it = grp, cs = grp, cph = 0;
-    for (;;) {
-        if (__builtin_expect(need_enter, 0)) { enter_segment(tt); need_enter = false; }
-        const uint32_t s = cs, ph = cph;             // stage of tile `it` and the parity of this group's use count of it
-        if (!have_tile) {
-            const bool landed = mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
-            tt = *reinterpret_cast<volatile int64_t*>(stage_tile + s);
-            const bool end = tt < 0 || !landed;
-            const bool outside = sg.seg < 0 || tt < sg.seg_start || tt >= sg.seg_start + sg.tiles;
-            if (__builtin_expect((end || outside) && sg.seg >= 0 && seg_tiles_done > 0, 0)) flush_segment();
-            if (__builtin_expect(end || ncontrib == kMaxContrib, 0)) {
-                combine_outstanding();           // every segment this group contributed to (normally: once, at the end)
-                if (end) break;
-            }
-            have_tile = true;
-            if (__builtin_expect(outside, 0)) { need_enter = true; continue; }
-        }
-        have_tile = false;
-        ++seg_tiles_done;
-        {
-            const int tj = (int)tt - sg.seg_start;                     // tile within the segment
+    // One stage: NH consecutive tiles of the current segment (tiles tj0 .. tj0 + NH - 1 of it) in stage s, this warp's 16
+    // keys of each. With NH = 2 the two slabs are independent until the softmax, which takes them as one block of 32 keys.
+    auto process_stage = [&](auto nh_tag, uint32_t s, uint32_t ph, int tj0) {
+        constexpr int NH = decltype(nh_tag)::value;
+        const uint32_t sK = stage0 + s * C::kStageBytes, sV = sK + C::kPair * C::kTileBytes;
+        int key0[NH], vlo[NH], vhi[NH], wkey0[NH];
+        bool has_new[NH];
+        bool any_valid = false, all_full = true, any_new = false, any_tail = false;
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+            const int tj = tj0 + h;                                    // tile within the segment
             const bool sink_part = tj < sg.sink_tiles;
-            const int key0 = (sink_part ? tj : sg.win_first + tj - sg.sink_tiles) * kTileKeys;   // first row of the tile
-            const int vlo = sink_part ? 0 : sg.lo, vhi = sink_part ? sg.ns : sg.hi;             // rows of it that count
-            const int wkey0 = key0 + warp * 16;
-            const bool tile_full = key0 >= vlo && key0 + kTileKeys <= vhi && !slack;
-            const bool any_valid = wkey0 < vhi && wkey0 + 16 > vlo;
-            const bool has_new = tj == new_tile;                       // this warp owns the appended row in this tile
-            const uint32_t sK = stage0 + s * C::kStageBytes, sV = sK + C::kTileBytes;
-            int64_t new_off = 0;
-            bool new_ok = true;
-            if (__builtin_expect(has_new, 0)) {
-                new_off = kv_row_offset(p, sg.b, sg.g, key0 + new_row, &new_ok);
+            key0[h] = (sink_part ? tj : sg.win_first + tj - sg.sink_tiles) * kTileKeys;      // first row of the tile
+            vlo[h] = sink_part ? 0 : sg.lo; vhi[h] = sink_part ? sg.ns : sg.hi;              // rows of it that count
+            wkey0[h] = key0[h] + warp * 16;
+            all_full = all_full && key0[h] >= vlo[h] && key0[h] + kTileKeys <= vhi[h] && !slack;
+            any_valid = any_valid || (wkey0[h] < vhi[h] && wkey0[h] + 16 > vlo[h]);
+            has_new[h] = tj == new_tile;                               // this warp owns the appended row in this tile
+            any_new = any_new || has_new[h];
+            any_tail = any_tail || wkey0[h] + 16 > vhi[h];
+        }
+        int64_t new_off = 0;
+        bool new_ok = true;
+        if (__builtin_expect(any_new, 0)) {
+#pragma unroll
+            for (int h = 0; h < NH; ++h) {
+                if (!has_new[h]) continue;
+                new_off = kv_row_offset(p, sg.b, sg.g, key0[h] + new_row, &new_ok);
                 if (!new_ok && lane == 0) atomicCAS(p.status, 0, kErrBounds);
-            }
-            if (__builtin_expect(has_new, 0))
-                patch_new_row<D, F8>(p.k_new, (int64_t)sg.b * p.Hkv + sg.g, p.k_scale, sg.g, sK, new_row,
+                patch_new_row<D, F8>(p.k_new, (int64_t)sg.b * p.Hkv + sg.g, p.k_scale, sg.g, sK + h * C::kTileBytes, new_row,
                                      new_ok ? reinterpret_cast<unsigned char*>(p.k) + new_off * C::kElemBytes : nullptr, lane);
-            if (__builtin_expect(has_new, 0)) {
                 if (p.mode == kRing && sg.g == 0 && lane == 0)
-                    p.slot_pos[(int64_t)sg.b * p.rows_per_head + key0 + new_row] = (int32_t)(sg.S - 1);
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
+                    p.slot_pos[(int64_t)sg.b * p.rows_per_head + key0[h] + new_row] = (int32_t)(sg.S - 1);
             }
-            uint32_t pb0 = 0, pb1 = 0;
-            if (any_valid) {
-                // ---- S^T = K . Q^T for this warp's 16 keys (two accumulator chains)
-                float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
-                if constexpr (!F8) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+        }
+        uint32_t pb[NH][2];
 #pragma unroll
-                    for (int ks = 0; ks < C::kKSteps; ++ks) {
+        for (int h = 0; h < NH; ++h) pb[h][0] = pb[h][1] = 0;
+        if (any_valid) {
+            // ---- S^T = K . Q^T for this warp's 16 keys of every tile (two accumulator chains per tile)
+            float sa[NH][4], sb[NH][4];
+#pragma unroll
+            for (int h = 0; h < NH; ++h) { sa[h][0] = sa[h][1] = sa[h][2] = sa[h][3] = 0.f; sb[h][0] = sb[h][1] = sb[h][2] = sb[h][3] = 0.f; }
+            if constexpr (!F8) {
+#pragma unroll
+                for (int ks = 0; ks < C::kKSteps; ++ks) {
+                    uint32_t q0, q1;
+                    if constexpr (C::kQShared) { const uint2 f = q_sm[ks * 32]; q0 = f.x; q1 = f.y; }
+                    else { q0 = qb[ks][0]; q1 = qb[ks][1]; }
+                    const uint32_t c16 = (uint32_t)((ks & 3) * 2 + halfK);
+#pragma unroll
+                    for (int h = 0; h < NH; ++h) {
                         uint32_t a[4];
-                        const uint32_t c16 = (uint32_t)((ks & 3) * 2 + halfK);
-                        ldmatrix_x4(a, sK + (ks >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
-                        uint32_t q0, q1;
-                        if constexpr (C::kQShared) { const uint2 f = q_sm[ks * 32]; q0 = f.x; q1 = f.y; }
-                        else { q0 = qb[ks][0]; q1 = qb[ks][1]; }
-                        if (ks & 1) mma_bf16(sb, a, q0, q1);
-                        else mma_bf16(sa, a, q0, q1);
-                    }
-                } else {
-                    // one ldmatrix brings 32 columns of d for the warp's 16 keys: matrices {keys 0-7, 8-15} x {16 d, next 16 d};
-                    // a thread's word holds 4 consecutive codes of one key, which become the k-slots (2 t4, 2 t4 + 1) and
-                    // (2 t4 + 8, 2 t4 + 9) of that 16-column step (the query fragments use the same order)
-#pragma unroll
-                    for (int j = 0; j < C::kKSteps / 2; ++j) {
-                        uint32_t r[4], a[4];
-                        const uint32_t c16 = (uint32_t)((j & 3) * 2 + halfK);
-                        ldmatrix_x4(r, sK + (j >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
-                        e4m3x4_to_f16x2x2(r[0], a[0], a[2]);
-                        e4m3x4_to_f16x2x2(r[1], a[1], a[3]);
-                        uint2 qa, qc;
-                        if constexpr (C::kQShared) { qa = q_sm[(2 * j) * 32]; qc = q_sm[(2 * j + 1) * 32]; }
-                        else { qa = make_uint2(qb[2 * j][0], qb[2 * j][1]); qc = make_uint2(qb[2 * j + 1][0], qb[2 * j + 1][1]); }
-                        mma_f16(sa, a, qa.x, qa.y);
-                        e4m3x4_to_f16x2x2(r[2], a[0], a[2]);
-                        e4m3x4_to_f16x2x2(r[3], a[1], a[3]);
-                        mma_f16(sb, a, qc.x, qc.y);
+                        ldmatrix_x4(a, sK + h * C::kTileBytes + (ks >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
+                        if (ks & 1) mma_bf16(sb[h], a, q0, q1);
+                        else mma_bf16(sa[h], a, q0, q1);
                     }
                 }
-                // raw scores; the multipliers smul (softmax scale in log2 units, for an fp8 store also the key scale and the
-                // query's power of two: all positive) are applied to the maxima and inside the exponentials
-                float sc[4];
+            } else {
+                // one ldmatrix brings 32 columns of d for the warp's 16 keys: matrices {keys 0-7, 8-15} x {16 d, next 16 d};
+                // a thread's word holds 4 consecutive codes of one key, which become the k-slots (2 t4, 2 t4 + 1) and
+                // (2 t4 + 8, 2 t4 + 9) of that 16-column step (the query fragments use the same order)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) sc[i] = sa[i] + sb[i];
-                if (__builtin_expect(!tile_full, 0)) {
-                    const int ka = wkey0 + g8, kb = ka + 8;
-                    bool va = ka >= vlo && ka < vhi, vb = kb >= vlo && kb < vhi;
+                for (int j = 0; j < C::kKSteps / 2; ++j) {
+                    uint2 qa, qc;
+                    if constexpr (C::kQShared) { qa = q_sm[(2 * j) * 32]; qc = q_sm[(2 * j + 1) * 32]; }
+                    else { qa = make_uint2(qb[2 * j][0], qb[2 * j][1]); qc = make_uint2(qb[2 * j + 1][0], qb[2 * j + 1][1]); }
+                    const uint32_t c16 = (uint32_t)((j & 3) * 2 + halfK);
+#pragma unroll
+                    for (int h = 0; h < NH; ++h) {
+                        uint32_t r[4], a[4];
+                        ldmatrix_x4(r, sK + h * C::kTileBytes + (j >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
+                        e4m3x4_to_f16x2x2(r[0], a[0], a[2]);
+                        e4m3x4_to_f16x2x2(r[1], a[1], a[3]);
+                        mma_f16(sa[h], a, qa.x, qa.y);
+                        e4m3x4_to_f16x2x2(r[2], a[0], a[2]);
+                        e4m3x4_to_f16x2x2(r[3], a[1], a[3]);
+                        mma_f16(sb[h], a, qc.x, qc.y);
+                    }
+                }
+            }
+            // raw scores; the multipliers smul (softmax scale in log2 units, for an fp8 store also the key scale and the
+            // query's power of two: all positive) are applied to the maxima and inside the exponentials
+            float sc[NH][4];
+#pragma unroll
+            for (int h = 0; h < NH; ++h) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sc[h][i] = sa[h][i] + sb[h][i];
+            }
+            if (__builtin_expect(!all_full, 0)) {
+#pragma unroll
+                for (int h = 0; h < NH; ++h) {
+                    const int ka = wkey0[h] + g8, kb = ka + 8;
+                    bool va = ka >= vlo[h] && ka < vhi[h], vb = kb >= vlo[h] && kb < vhi[h];
                     if (slack) {
                         va = va && ring_slot_live(ka, sg.S, p.n_sink, p.W, p.cap);
                         vb = vb && ring_slot_live(kb, sg.S, p.n_sink, p.W, p.cap);
                     }
-                    if (!va) { sc[0] = -INFINITY; sc[1] = -INFINITY; }
-                    if (!vb) { sc[2] = -INFINITY; sc[3] = -INFINITY; }
+                    if (!va) { sc[h][0] = -INFINITY; sc[h][1] = -INFINITY; }
+                    if (!vb) { sc[h][2] = -INFINITY; sc[h][3] = -INFINITY; }
                 }
-                // ---- online softmax; this thread holds heads 2*t4, 2*t4+1 for keys g8 and g8+8
-                float mx0 = fmaxf(sc[0], sc[2]), mx1 = fmaxf(sc[1], sc[3]);
+            }
+            // ---- online softmax; this thread holds heads 2*t4, 2*t4+1 for keys g8 and g8+8 of every tile
+            float mx0 = fmaxf(sc[0][0], sc[0][2]), mx1 = fmaxf(sc[0][1], sc[0][3]);
 #pragma unroll
-                for (int off = 4; off <= 16; off <<= 1) {
-                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
-                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
-                }
-                const float mn0 = fmaxf(m[0], mx0 * smul[0]), mn1 = fmaxf(m[1], mx1 * smul[1]);
-                // the running maxima rarely move after the first tiles of a segment: rescale only when some lane's did
-                if (__builtin_expect(__any_sync(0xffffffffu, mn0 != m[0] || mn1 != m[1]), 0)) {
-                    const float corr0 = mn0 == -INFINITY ? 1.f : ex2(m[0] - mn0), corr1 = mn1 == -INFINITY ? 1.f : ex2(m[1] - mn1);
-                    le[0] *= corr0; le[1] *= corr1;
-                    l[0] *= corr0; l[1] *= corr1;
+            for (int h = 1; h < NH; ++h) {
+                mx0 = fmaxf(mx0, fmaxf(sc[h][0], sc[h][2]));
+                mx1 = fmaxf(mx1, fmaxf(sc[h][1], sc[h][3]));
+            }
 #pragma unroll
-                    for (int mb = 0; mb < C::kKSteps; ++mb) {
-                        o[mb][0] *= corr0; o[mb][1] *= corr1; o[mb][2] *= corr0; o[mb][3] *= corr1;
-                    }
-                    m[0] = mn0; m[1] = mn1;
+            for (int off = 4; off <= 16; off <<= 1) {
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+            }
+            const float mn0 = fmaxf(m[0], mx0 * smul[0]), mn1 = fmaxf(m[1], mx1 * smul[1]);
+            // the running maxima rarely move after the first tiles of a segment: rescale only when some lane's did
+            if (__builtin_expect(__any_sync(0xffffffffu, mn0 != m[0] || mn1 != m[1]), 0)) {
+                const float corr0 = mn0 == -INFINITY ? 1.f : ex2(m[0] - mn0), corr1 = mn1 == -INFINITY ? 1.f : ex2(m[1] - mn1);
+                le[0] *= corr0; le[1] *= corr1;
+                l[0] *= corr0; l[1] *= corr1;
+#pragma unroll
+                for (int mb = 0; mb < C::kKSteps; ++mb) {
+                    o[mb][0] *= corr0; o[mb][1] *= corr1; o[mb][2] *= corr0; o[mb][3] *= corr1;
                 }
-                const float nu0 = mn0 == -INFINITY ? 0.f : -mn0, nu1 = mn1 == -INFINITY ? 0.f : -mn1;
-                const float p0 = ex2(fmaf(sc[0], smul[0], nu0)), p1 = ex2(fmaf(sc[1], smul[1], nu1));
-                const float p2 = ex2(fmaf(sc[2], smul[0], nu0)), p3 = ex2(fmaf(sc[3], smul[1], nu1));
+                m[0] = mn0; m[1] = mn1;
+            }
+            const float nu0 = mn0 == -INFINITY ? 0.f : -mn0, nu1 = mn1 == -INFINITY ? 0.f : -mn1;
+#pragma unroll
+            for (int h = 0; h < NH; ++h) {
+                const float p0 = ex2(fmaf(sc[h][0], smul[0], nu0)), p1 = ex2(fmaf(sc[h][1], smul[1], nu1));
+                const float p2 = ex2(fmaf(sc[h][2], smul[0], nu0)), p3 = ex2(fmaf(sc[h][3], smul[1], nu1));
                 const uint32_t pa = F8 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1);             // key g8   : heads 2t4, 2t4+1
                 const uint32_t pc = F8 ? pack_f16x2(p2, p3) : pack_bf16x2(p2, p3);             // key g8+8
                 le[0] += p0 + p2;
@@ -1128,57 +1154,106 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                     l[0] += bf16lo(pa) + bf16lo(pc);      // sums of the rounded weights the MMA will use
                     l[1] += bf16hi(pa) + bf16hi(pc);
                 }
-                pb0 = movmatrix_trans(pa);                           // P^T as B operand: k = key, n = head
-                pb1 = movmatrix_trans(pc);
+                pb[h][0] = movmatrix_trans(pa);                      // P^T as B operand: k = key, n = head
+                pb[h][1] = movmatrix_trans(pc);
             }
-            mbar_wait(bar_fullV + 8 * s, ph, abort_flag, p.status);
-            if (__builtin_expect(has_new, 0))
-                patch_new_row<D, F8>(p.v_new, (int64_t)sg.b * p.Hkv + sg.g, p.v_scale, sg.g, sV, new_row,
-                                     new_ok ? reinterpret_cast<unsigned char*>(p.v) + new_off * C::kElemBytes : nullptr, lane);
-            if (any_valid) {
-                if (__builtin_expect(wkey0 + 16 > vhi, 0)) {
-                    // rows past the end were never written (or, in a sink tile of a window view, may be): they can hold
-                    // NaN/Inf bit patterns, and 0 * NaN would poison the accumulators. Zero them in shared memory.
-                    const int first_bad = vhi > wkey0 ? vhi - wkey0 : 0;
+        }
+        mbar_wait(bar_fullV + 8 * s, ph, abort_flag, p.status);
+        if (__builtin_expect(any_new, 0)) {
+#pragma unroll
+            for (int h = 0; h < NH; ++h)
+                if (has_new[h])
+                    patch_new_row<D, F8>(p.v_new, (int64_t)sg.b * p.Hkv + sg.g, p.v_scale, sg.g, sV + h * C::kTileBytes, new_row,
+                                         new_ok ? reinterpret_cast<unsigned char*>(p.v) + new_off * C::kElemBytes : nullptr, lane);
+        }
+        if (any_valid) {
+            if (__builtin_expect(any_tail, 0)) {
+                // rows past the end were never written (or, in a sink tile of a window view, may be): they can hold
+                // NaN/Inf bit patterns, and 0 * NaN would poison the accumulators. Zero them in shared memory.
+#pragma unroll
+                for (int h = 0; h < NH; ++h) {
+                    if (wkey0[h] + 16 <= vhi[h]) continue;
+                    const int first_bad = vhi[h] > wkey0[h] ? vhi[h] - wkey0[h] : 0;
                     for (int idx = lane; idx < (16 - first_bad) * C::kChunks * 8; idx += 32) {
                         const int r = first_bad + idx / (C::kChunks * 8), rem = idx % (C::kChunks * 8);
-                        const uint32_t addr = sV + (rem >> 3) * C::kChunkBytes + (warp * 16 + r) * 128 + ((rem & 7) << 4);
+                        const uint32_t addr = sV + h * C::kTileBytes + (rem >> 3) * C::kChunkBytes + (warp * 16 + r) * 128 + ((rem & 7) << 4);
                         asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
                     }
                 }
-                if (__builtin_expect(has_new || wkey0 + 16 > vhi, 0)) {
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
-                }
-                // ---- O^T += V^T . P^T
-                if constexpr (!F8) {
+            }
+            if (__builtin_expect(any_new || any_tail, 0)) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+            }
+            // ---- O^T += V^T . P^T
+            if constexpr (!F8) {
 #pragma unroll
-                    for (int mb = 0; mb < C::kKSteps; ++mb) {
+                for (int mb = 0; mb < C::kKSteps; ++mb) {
+                    const uint32_t c16 = (uint32_t)((mb & 3) * 2 + halfV);
+#pragma unroll
+                    for (int h = 0; h < NH; ++h) {
                         uint32_t a[4];
-                        const uint32_t c16 = (uint32_t)((mb & 3) * 2 + halfV);
-                        ldmatrix_x4_trans(a, sV + (mb >> 2) * C::kChunkBytes + offV + ((c16 ^ (uint32_t)rr) << 4));
-                        mma_bf16(o[mb], a, pb0, pb1);
+                        ldmatrix_x4_trans(a, sV + h * C::kTileBytes + (mb >> 2) * C::kChunkBytes + offV + ((c16 ^ (uint32_t)rr) << 4));
+                        mma_bf16(o[mb], a, pb[h][0], pb[h][1]);
                     }
-                } else {
-                    // the transposed load hands a thread, per matrix, the codes of keys (2 t4, 2 t4 + 1) for d = 2 g8 and
-                    // 2 g8 + 1 of a 16-column unit: accumulator row g8 of the block is d = 2 g8, row g8 + 8 is d = 2 g8 + 1
+                }
+            } else {
+                // the transposed load hands a thread, per matrix, the codes of keys (2 t4, 2 t4 + 1) for d = 2 g8 and
+                // 2 g8 + 1 of a 16-column unit: accumulator row g8 of the block is d = 2 g8, row g8 + 8 is d = 2 g8 + 1
 #pragma unroll
-                    for (int j = 0; j < C::kKSteps / 2; ++j) {
+                for (int j = 0; j < C::kKSteps / 2; ++j) {
+                    const uint32_t c16 = (uint32_t)((j & 3) * 2 + halfK);
+#pragma unroll
+                    for (int h = 0; h < NH; ++h) {
                         uint32_t r[4], a[4];
-                        const uint32_t c16 = (uint32_t)((j & 3) * 2 + halfK);
-                        ldmatrix_x4_trans(r, sV + (j >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
+                        ldmatrix_x4_trans(r, sV + h * C::kTileBytes + (j >> 2) * C::kChunkBytes + offK + ((c16 ^ (uint32_t)rr) << 4));
                         e4m3x4_to_f16x2x2(__byte_perm(r[0], 0, 0x3120), a[0], a[1]);
                         e4m3x4_to_f16x2x2(__byte_perm(r[1], 0, 0x3120), a[2], a[3]);
-                        mma_f16(o[2 * j], a, pb0, pb1);
+                        mma_f16(o[2 * j], a, pb[h][0], pb[h][1]);
                         e4m3x4_to_f16x2x2(__byte_perm(r[2], 0, 0x3120), a[0], a[1]);
                         e4m3x4_to_f16x2x2(__byte_perm(r[3], 0, 0x3120), a[2], a[3]);
-                        mma_f16(o[2 * j + 1], a, pb0, pb1);
+                        mma_f16(o[2 * j + 1], a, pb[h][0], pb[h][1]);
                     }
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_empty + 8 * s);
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+    };
+    // The loop is written so that enter / flush / tile processing each appear once in the code (the kernel's
+    // tail runs once per launch, from a cold instruction cache: code size is latency there).
+    int64_t tt = -1;                                     // (first) tile in hand
+    int tcnt = 1;                                        // tiles in the stage in hand
+    bool have_tile = false, need_enter = false;
+    if constexpr (CL) {
+        if (c_lo + grp < c_hi) { tt = c_lo + grp; need_enter = true; }
+    } else if ((int)blockIdx.x < Cn) {
+        // an owner knows its first tiles: fetch the query while they are still in flight
+        const int64_t first = cta_range_start(blockIdx.x, n, Cn) + grp * C::kPair;
+        if (first < cta_range_start(blockIdx.x + 1, n, Cn)) { tt = first; need_enter = true; }
+    }
+    uint32_t it = grp, cs = grp, cph = 0;
+    for (;;) {
+        if (__builtin_expect(need_enter, 0)) { enter_segment(tt); need_enter = false; }
+        const uint32_t s = cs, ph = cph;             // stage of tile `it` and the parity of this group's use count of it
+        if (!have_tile) {
+            const bool landed = mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
+            tt = *reinterpret_cast<volatile int64_t*>(stage_tile + s);
+            if (C::kPair == 2 && tt >= 0) { tcnt = (int)(tt & 1) + 1; tt >>= 1; }          // (first tile << 1) | (tiles - 1)
+            const bool end = tt < 0 || !landed;
+            const bool outside = sg.seg < 0 || tt < sg.seg_start || tt >= sg.seg_start + sg.tiles;
+            if (__builtin_expect((end || outside) && sg.seg >= 0 && seg_tiles_done > 0, 0)) flush_segment();
+            if (__builtin_expect(end || ncontrib == kMaxContrib, 0)) {
+                combine_outstanding();           // every segment this group contributed to (normally: once, at the end)
+                if (end) break;
+            }
+            have_tile = true;
+            if (__builtin_expect(outside, 0)) { need_enter = true; continue; }
+        }
+        have_tile = false;
+        seg_tiles_done += tcnt;
+        if (C::kPair == 2 && tcnt == 2) process_stage(std::integral_constant<int, C::kPair>{}, s, ph, (int)tt - sg.seg_start);
+        else process_stage(std::integral_constant<int, 1>{}, s, ph, (int)tt - sg.seg_start);
         it += C::kGroups;
         cs += C::kGroups;                            // nst is a multiple of kGroups: the stage stays with this group
         if (cs >= nst) { cs -= nst; cph ^= 1u; }
@@ -1214,7 +1289,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                              : "=r"(a) : "r"(part_local + 4u * (uint32_t)((s_ % C::kGroups) * kPart + off_floats)), "r"((uint32_t)(s_ / C::kGroups)));
                 return a;
             };
-            constexpr int kMaxNp = kMaxCluster * kMaxGroups;           // partials of the largest cluster
+            constexpr int kMaxNp = kMaxCluster * C::kGroups;           // partials of the largest cluster
             constexpr int kMaxOwn = kMaxNp / kGroupWarps;     // ... of which a warp sums every fourth
             float* lse_all = scratch + 4 * kGroupThreads;     // [np][8], behind the reduction buffer
             // one round trip through the cluster: the lse values of all partials (staged in shared memory for everybody)
@@ -1354,7 +1429,7 @@ cudaError_t launch_fused(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaSt
 // than in the streaming form).
 template <int D, bool F8>
 constexpr int cluster_stages() {
-    using C = Cfg<D, F8>;
+    using C = Cfg<D, F8, true>;
     int stages = C::kMaxStages;
     while (stages > C::kGroups &&
            1024 + C::kFixedBytes + stages * C::kStageBytes + (int)sizeof(float) * C::kGroups * (kMaxGroup * D + kMaxGroup) + 16 > 227 * 1024)
@@ -1363,7 +1438,7 @@ constexpr int cluster_stages() {
 }
 template <int D, bool F8>
 size_t cluster_smem_bytes() {
-    using C = Cfg<D, F8>;
+    using C = Cfg<D, F8, true>;
     return 1024 + (size_t)C::kFixedBytes + (size_t)cluster_stages<D, F8>() * C::kStageBytes +
            sizeof(float) * C::kGroups * (kMaxGroup * D + kMaxGroup) + 16;
 }
@@ -1389,7 +1464,7 @@ cudaError_t cluster_info(const ClusterInfo** out) {
         if (cudaDeviceGetAttribute(&info[dev].sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) info[dev].sms = 0;
         for (int cl = 1; cl <= kMaxCluster; ++cl) {
             cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(cl); cfg.blockDim = dim3(Cfg<D, F8>::kThreads); cfg.dynamicSmemBytes = cluster_smem_bytes<D, F8>();
+            cfg.gridDim = dim3(cl); cfg.blockDim = dim3(Cfg<D, F8, true>::kThreads); cfg.dynamicSmemBytes = cluster_smem_bytes<D, F8>();
             cudaLaunchAttribute at[1];
             at[0].id = cudaLaunchAttributeClusterDimension;
             at[0].val.clusterDim.x = (unsigned)cl; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
@@ -1406,7 +1481,7 @@ cudaError_t cluster_info(const ClusterInfo** out) {
 
 template <int D, bool F8>
 cudaError_t launch_cluster(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaStream_t st) {
-    using C = Cfg<D, F8>;
+    using C = Cfg<D, F8, true>;
     p.stages = cluster_stages<D, F8>();
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.num_ctas); cfg.blockDim = dim3(C::kThreads); cfg.dynamicSmemBytes = cluster_smem_bytes<D, F8>(); cfg.stream = st;
