@@ -36,9 +36,9 @@ UNIT = "us"
 WORKLOADS = {"tiny": 0, "s128k": 1, "million": 2, "batched": 3, "sweep": 4}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (attn_fused_tma on the full
-# context), from an ncu capture of that kernel on the s128k workload (272.8 MB for 131,075 keys = 2081.3 B per key,
-# against 2048 algorithmic), scaled by the keys one launch scans: DRAM traffic grows in proportion to the keys.
-NCU_TRAFFIC_BYTES_PER_KEY = {256: 2081.3}
+# context), from an ncu capture of that kernel on this benchmark's own default workload (2152.0 MB for 1,048,590 keys
+# = 2052.3 B per key, against 2048 algorithmic), times the keys one launch scans.
+NCU_TRAFFIC_BYTES_PER_KEY = {256: 2052.3}
 
 
 def log(*a):
