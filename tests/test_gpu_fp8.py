@@ -138,6 +138,24 @@ def test_batched_ragged_lengths(paged, D):
     _run_and_check(_cfg(batch=5, S0=0, S0_range=(1, 3000), paged=paged, D=D, W=128, gamma=2, seed=77))
 
 
+@pytest.mark.parametrize("max_ctas", [1, 3, 0])
+@pytest.mark.parametrize("S0", [62, 63, 64, 126, 127, 128, 190, 191, 192, 320])
+def test_paired_tiles_odd_and_even_tile_counts(S0, max_ctas):
+    """head_dim 128 fp8 stores travel two tiles to a stage: lengths around tile boundaries give stages of one and of
+    two tiles, and put the appended row into the first and into the second tile of a pair (gamma = 3 appends)."""
+    _run_and_check(_cfg(S0=S0, D=128, seed=500 + S0), max_ctas=max_ctas)
+
+
+@pytest.mark.parametrize("paged", [False, True])
+@pytest.mark.parametrize("stealing", [True, False])
+def test_paired_tiles_long_ragged_batch(paged, stealing):
+    """Ranges long enough for the cursor-driven tail (and thieves) on a ragged batch (37 CTAs over some 9000 tiles):
+    chunks and stolen runs end at segment ends, where a stage may hold a single tile."""
+    wm.wmtp_set_work_stealing(stealing)
+    _run_and_check(_cfg(batch=3, S0=0, S0_range=(150001, 260000), paged=paged, D=128, Hq=8, Hkv=1, W=512, gamma=2, seed=91),
+                   max_ctas=37, check_store=False)
+
+
 @pytest.mark.parametrize("Hq,Hkv", [(8, 8), (4, 2), (32, 4), (6, 2)])
 def test_group_sizes(Hq, Hkv):
     _run_and_check(_cfg(Hq=Hq, Hkv=Hkv, S0=900, key_scale=None, seed=Hq * 10 + Hkv), max_ctas=0)
