@@ -240,7 +240,8 @@ def main():
     if args.kv_dtype == "fp8":
         cfg = wi.scaled(cfg, kv_dtype="fp8", name=cfg.name + "_fp8")
     gam, B = cfg.gamma, cfg.batch
-    total_passes = args.warmup + 3 * args.steps + 8          # timed + breakdown + e2e passes, plus slack
+    # timed + breakdown + e2e passes, the graph replays of the full-context loop, plus slack
+    total_passes = args.warmup + 3 * args.steps + max(10, args.steps) + 5 + 8
     t0 = time.perf_counter()
     wl = wi.make_workload(cfg, poison_unused=False, extra_cap=gam * total_passes + 64)
     log(f"[bench] generated {cfg.name} in {time.perf_counter() - t0:.1f}s")
@@ -341,28 +342,32 @@ def main():
         a.record(); wm.wmtp_draft_attn_windowed(q[0], ring, o1, ws); b.record()
     torch.cuda.synchronize()
     wm.wmtp_device_status(ws)
-    # the windowed loop replayed from a CUDA graph (what a serving stack that captures its decode step sees)
-    us_win_graph = None
-    try:
-        gs = torch.cuda.Stream()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(gs):
-            wm.wmtp_draft_loop_windowed(ring, q, kn, vn, out_w, ws)
+    # both loops replayed from CUDA graphs (what a serving stack that captures its decode step sees)
+    def graph_replay_us(loop):
+        try:
+            gs = torch.cuda.Stream()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(gs):
+                loop()
+                torch.cuda.synchronize()
+                with torch.cuda.graph(graph, stream=gs):
+                    loop()
             torch.cuda.synchronize()
-            with torch.cuda.graph(graph, stream=gs):
-                wm.wmtp_draft_loop_windowed(ring, q, kn, vn, out_w, ws)
-        torch.cuda.synchronize()
-        for _ in range(3):
-            graph.replay()
-        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        g0.record()
-        for _ in range(reps):
-            graph.replay()
-        g1.record()
-        torch.cuda.synchronize()
-        us_win_graph = g0.elapsed_time(g1) * 1e3 / reps / gam
-    except Exception as exc:                                 # graph capture unavailable: report nothing
-        log(f"[bench] graph replay skipped: {exc}")
+            for _ in range(3):
+                graph.replay()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record()
+            for _ in range(reps):
+                graph.replay()
+            g1.record()
+            torch.cuda.synchronize()
+            return g0.elapsed_time(g1) * 1e3 / reps / gam
+        except Exception as exc:                             # graph capture unavailable: report nothing
+            log(f"[bench] graph replay skipped: {exc}")
+            return None
+    us_win_graph = graph_replay_us(lambda: wm.wmtp_draft_loop_windowed(ring, q, kn, vn, out_w, ws))
+    us_full_graph = graph_replay_us(lambda: wm.wmtp_draft_loop_full(kv, q, kn, vn, out_f, ws))
+    wm.wmtp_device_status(ws)
     us_win_kv_call = v0.elapsed_time(v1) * 1e3 / reps
     us_win_call_cold = statistics.mean(a.elapsed_time(b) for a, b in wev) * 1e3
     us_launch_floor = l0.elapsed_time(l1) * 1e3 / reps
@@ -632,7 +637,8 @@ def main():
                          "us_per_step_min": min(full_samples), "kv_bytes_per_step": full_bytes,
                          "algorithmic_gbs": full_bytes / (us_full * 1e-6) / 1e9,
                          "pct_of_8tbs": full_bytes / (us_full * 1e-6) / 8e12 * 100,
-                         "us_per_attention_call": us_full_call},
+                         "us_per_attention_call": us_full_call,
+                         "us_per_step_graph_replay": us_full_graph},
                 "draft_extend": ext,
                 "fp8_kv": f8,
             },

@@ -35,6 +35,7 @@
 #include <type_traits>
 
 #include "attn_plan.cuh"
+#include "fp8_util.cuh"
 #include "ptx_util.cuh"
 
 namespace wmtp {
@@ -49,9 +50,11 @@ constexpr int kMqWarps = 4;                // warps per group: 4 x 16 keys = one
 constexpr int kMqGroupThreads = kMqWarps * 32;
 constexpr int kCombineRows = 8;            // partials in flight per output column in the merge kernel
 
-template <int D>
+// D: head_dim; F8: the store holds e4m3 codes (one byte per entry) instead of bf16.
+template <int D, bool F8>
 struct MqCfg {
-    static constexpr int kChunks = D * 2 / 128;                // 128-byte column chunks per row
+    static constexpr int kElemBytes = F8 ? 1 : 2;
+    static constexpr int kChunks = D * kElemBytes / 128;       // 128-byte column chunks per row
     static constexpr int kChunkBytes = kTileKeys * 128;        // one TMA box: 64 rows x 128 B
     static constexpr int kTileBytes = kChunks * kChunkBytes;   // K (or V) tile
     static constexpr int kStageBytes = 2 * kTileBytes;
@@ -131,11 +134,11 @@ __device__ __forceinline__ void mq_group_barrier(int grp) { asm volatile("bar.sy
 // ---------------------------------------------------------------------------------------------
 // Partials: one launch, fixed partition, no inter-CTA wait
 // ---------------------------------------------------------------------------------------------
-template <int D>
-__global__ void __launch_bounds__(MqCfg<D>::kThreads, 1)
+template <int D, bool F8>
+__global__ void __launch_bounds__(MqCfg<D, F8>::kThreads, 1)
 attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                const __grid_constant__ AttnParams p) {
-    using C = MqCfg<D>;
+    using C = MqCfg<D, F8>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     float* scratch_all = reinterpret_cast<float*>(smem);                                   // [groups][kScratchFloats]
@@ -258,8 +261,12 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     // copy per group (head_dim 256: 64 registers of fragments next to 128 of accumulators spill, and keeping only one
     // query's fragments in registers measured no faster).
     uint32_t qreg[C::kQRegs > 0 ? C::kQRegs : 1][C::kKSteps][2];
+    // multipliers of the raw scores of heads 2 t4 and 2 t4 + 1 of each query: the softmax scale in log2 units; for an fp8
+    // store also the key scale of the KV head and the power of two the head's query was normalised by (all positive)
+    float smul[kQW][2];
+    float vscale = 1.f;                      // fp8: dequantisation scale of V, applied to the normalised partial
 #pragma unroll
-    for (int j = 0; j < kQW; ++j) Sq[j] = 0;
+    for (int j = 0; j < kQW; ++j) { Sq[j] = 0; smul[j][0] = smul[j][1] = scale; }
 
     // Merge the four warps' states per query, write the partial of (this CTA, current stream, query).
     auto flush = [&]() {
@@ -300,7 +307,7 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                         Le += sm_le[w * kMaxGroup + h] * e;
                     }
                 }
-                f[i] = (L > 0.f && m[j][i] > -INFINITY) ? ex2(m[j][i] - M) / L : 0.f;
+                f[i] = (L > 0.f && m[j][i] > -INFINITY) ? ex2(m[j][i] - M) / L * vscale : 0.f;
                 if (warp == 0 && g8 == 0 && h < G) p.part_lse[prow * G + h] = Le > 0.f ? (M + lg2(Le)) * kLn2f : -INFINITY;
             }
             constexpr int kPasses = D / C::kPassCols;
@@ -310,11 +317,13 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
 #pragma unroll
                 for (int mbl = 0; mbl < C::kPassCols / 16; ++mbl) {
                     const int mb = pass * (C::kPassCols / 16) + mbl;
-                    // accumulator rows g8 and g8 + 8 of block mb hold d = 16 mb + g8 and + 8
-                    float* row0 = scratch + (warp * kMaxGroup + 2 * t4) * C::kScratchRow + mbl * 16 + g8;
+                    // accumulator rows g8 and g8 + 8 of block mb hold d = 16 mb + g8 and + 8 (bf16 store), or, for an fp8
+                    // store whose V fragments come out of the transposed load with d pairs interleaved, d = 16 mb + 2 g8 and + 1
+                    float* row0 = scratch + (warp * kMaxGroup + 2 * t4) * C::kScratchRow + mbl * 16 + (F8 ? 2 * g8 : g8);
                     float* row1 = row0 + C::kScratchRow;
+                    constexpr int kSecond = F8 ? 1 : 8;
                     row0[0] = o[j][mb][0] * f[0]; row1[0] = o[j][mb][1] * f[1];
-                    row0[8] = o[j][mb][2] * f[0]; row1[8] = o[j][mb][3] * f[1];
+                    row0[kSecond] = o[j][mb][2] * f[0]; row1[kSecond] = o[j][mb][3] * f[1];
                 }
                 mq_group_barrier(grp);
                 for (int idx = tid; idx < G * C::kPassCols; idx += kMqGroupThreads) {
@@ -342,19 +351,50 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
                 reinterpret_cast<const __nv_bfloat16*>(p.q) +
                 ((((int64_t)sg.b * p.q_len + sg.ch * kQC + (qi < sg.nq ? qi : 0)) * p.Hq) + sg.g * G + (g8 < G ? g8 : 0)) * D);
+            // Words of the query row that make up this lane's fragment of 16-column step ks: ks * 8 + w0 and ks * 8 + w1.
+            // For an fp8 store the MMA k-slot order within 16 columns of d follows the byte order ldmatrix delivers the
+            // codes in: lane t4 holds d = 4 t4 .. 4 t4 + 3 of each 16.
+            const int w0 = F8 ? 2 * t4 : t4, w1 = F8 ? 2 * t4 + 1 : 4 + t4;
+            float down = 1.f;
+            if constexpr (F8) {
+                // The e4m3 codes are widened to f16 (exact), so the query goes through the f16 MMA too. Its range is made
+                // safe by a per-head power of two (exact both ways): q' = q * 2^-e with 2^e <= max|q| < 2^(e+1), and 2^e
+                // goes into the score multiplier together with the key scale.
+                float amax = 0.f;
+#pragma unroll
+                for (int ks = 0; ks < C::kKSteps; ++ks) {
+                    const uint32_t a = have ? __ldg(qrow + ks * 8 + w0) : 0u, b = have ? __ldg(qrow + ks * 8 + w1) : 0u;
+                    amax = fmaxf(fmaxf(amax, fmaxf(fabsf(bf16lo(a)), fabsf(bf16hi(a)))), fmaxf(fabsf(bf16lo(b)), fabsf(bf16hi(b))));
+                }
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+                uint32_t eb = (__float_as_uint(amax) >> 23) & 0xffu;
+                eb = eb < 1u ? 1u : (eb > 253u ? 253u : eb);
+                down = __uint_as_float((254u - eb) << 23);
+                const float hmul = g8 < G ? scale * __uint_as_float(eb << 23) * __ldg(p.k_scale + sg.g) : 0.f;
+                smul[j][0] = __shfl_sync(0xffffffffu, hmul, 8 * t4);
+                smul[j][1] = __shfl_sync(0xffffffffu, hmul, 8 * t4 + 4);
+                vscale = __ldg(p.v_scale + sg.g);
+            }
+            auto fragment = [&](int ks) {
+                uint2 f;
+                f.x = have ? __ldg(qrow + ks * 8 + w0) : 0u;
+                f.y = have ? __ldg(qrow + ks * 8 + w1) : 0u;
+                if constexpr (F8) {
+                    f.x = pack_f16x2(bf16lo(f.x) * down, bf16hi(f.x) * down);
+                    f.y = pack_f16x2(bf16lo(f.y) * down, bf16hi(f.y) * down);
+                }
+                return f;
+            };
             if (j < C::kQRegs) {
 #pragma unroll
                 for (int ks = 0; ks < C::kKSteps; ++ks) {
-                    qreg[j < C::kQRegs ? j : 0][ks][0] = have ? __ldg(qrow + ks * 8 + t4) : 0u;
-                    qreg[j < C::kQRegs ? j : 0][ks][1] = have ? __ldg(qrow + ks * 8 + 4 + t4) : 0u;
+                    const uint2 f = fragment(ks);
+                    qreg[j < C::kQRegs ? j : 0][ks][0] = f.x;
+                    qreg[j < C::kQRegs ? j : 0][ks][1] = f.y;
                 }
             } else {
-                for (int ks = warp; ks < C::kKSteps; ks += kMqWarps) {
-                    uint2 f;
-                    f.x = have ? __ldg(qrow + ks * 8 + t4) : 0u;
-                    f.y = have ? __ldg(qrow + ks * 8 + 4 + t4) : 0u;
-                    q_sm[(j * C::kKSteps + ks) * 32] = f;
-                }
+                for (int ks = warp; ks < C::kKSteps; ks += kMqWarps) q_sm[(j * C::kKSteps + ks) * 32] = fragment(ks);
             }
             m[j][0] = m[j][1] = -INFINITY; le[j][0] = le[j][1] = 0.f;
             lacc[j][0] = lacc[j][1] = lacc[j][2] = lacc[j][3] = 0.f;
@@ -377,32 +417,81 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 sd[j][0] = sd[j][1] = sd[j][2] = sd[j][3] = 0.f;
             }
         }
+        auto qfrag = [&](int j, int ks, uint32_t& q0, uint32_t& q1) {
+            if (j < C::kQRegs) { q0 = qreg[j < C::kQRegs ? j : 0][ks][0]; q1 = qreg[j < C::kQRegs ? j : 0][ks][1]; }
+            else { const uint2 f = q_sm[(j * C::kKSteps + ks) * 32]; q0 = f.x; q1 = f.y; }
+        };
+        if constexpr (!F8) {
 #pragma unroll
-        for (int ks = 0; ks < C::kKSteps; ++ks) {
-            if constexpr (kQK) {
-                uint32_t a[4];
-                ldmatrix_x4(a, sK + (ks >> 2) * C::kChunkBytes + koff[ks & 3]);
+            for (int ks = 0; ks < C::kKSteps; ++ks) {
+                if constexpr (kQK) {
+                    uint32_t a[4];
+                    ldmatrix_x4(a, sK + (ks >> 2) * C::kChunkBytes + koff[ks & 3]);
 #pragma unroll
-                for (int j = 0; j < kQW; ++j) {
-                    uint32_t q0, q1;
-                    if (j < C::kQRegs) { q0 = qreg[j < C::kQRegs ? j : 0][ks][0]; q1 = qreg[j < C::kQRegs ? j : 0][ks][1]; }
-                    else { const uint2 f = q_sm[(j * C::kKSteps + ks) * 32]; q0 = f.x; q1 = f.y; }
-                    if (ks & 1) mma_bf16(sd[j], a, q0, q1);
-                    else mma_bf16(scn[j], a, q0, q1);
+                    for (int j = 0; j < kQW; ++j) {
+                        uint32_t q0, q1;
+                        qfrag(j, ks, q0, q1);
+                        if (ks & 1) mma_bf16(sd[j], a, q0, q1);
+                        else mma_bf16(scn[j], a, q0, q1);
+                    }
+                }
+                if constexpr (kPV) {
+                    uint32_t a[4];
+                    ldmatrix_x4_trans(a, sV + (ks >> 2) * C::kChunkBytes + voff[ks & 3]);
+#pragma unroll
+                    for (int j = 0; j < kQW; ++j) mma_bf16(o[j][ks], a, pb[j][0], pb[j][1]);
                 }
             }
-            if constexpr (kPV) {
-                uint32_t a[4];
-                ldmatrix_x4_trans(a, sV + (ks >> 2) * C::kChunkBytes + voff[ks & 3]);
+        } else {
+            // e4m3 codes: one ldmatrix brings 32 columns of d for the warp's 16 keys; a thread's word holds 4 consecutive
+            // codes of one key (K) or, from the transposed load, the codes of two keys for two consecutive d (V, after one
+            // byte permute). They are widened to f16 (exact) four at a time and take the f16 MMA; the query fragments are
+            // stored in the matching k-slot order, the accumulator rows of the read-out come out with d pairs interleaved.
 #pragma unroll
-                for (int j = 0; j < kQW; ++j) mma_bf16(o[j][ks], a, pb[j][0], pb[j][1]);
+            for (int jj = 0; jj < C::kKSteps / 2; ++jj) {
+                if constexpr (kQK) {
+                    uint32_t r[4], a[4];
+                    ldmatrix_x4(r, sK + (jj >> 2) * C::kChunkBytes + koff[jj & 3]);
+                    e4m3x4_to_f16x2x2(r[0], a[0], a[2]);
+                    e4m3x4_to_f16x2x2(r[1], a[1], a[3]);
+#pragma unroll
+                    for (int j = 0; j < kQW; ++j) {
+                        uint32_t q0, q1;
+                        qfrag(j, 2 * jj, q0, q1);
+                        mma_f16(scn[j], a, q0, q1);
+                    }
+                    e4m3x4_to_f16x2x2(r[2], a[0], a[2]);
+                    e4m3x4_to_f16x2x2(r[3], a[1], a[3]);
+#pragma unroll
+                    for (int j = 0; j < kQW; ++j) {
+                        uint32_t q0, q1;
+                        qfrag(j, 2 * jj + 1, q0, q1);
+                        mma_f16(sd[j], a, q0, q1);
+                    }
+                }
+                if constexpr (kPV) {
+                    uint32_t r[4], a[4];
+                    ldmatrix_x4_trans(r, sV + (jj >> 2) * C::kChunkBytes + koff[jj & 3]);
+                    e4m3x4_to_f16x2x2(__byte_perm(r[0], 0, 0x3120), a[0], a[1]);
+                    e4m3x4_to_f16x2x2(__byte_perm(r[1], 0, 0x3120), a[2], a[3]);
+#pragma unroll
+                    for (int j = 0; j < kQW; ++j) mma_f16(o[j][2 * jj], a, pb[j][0], pb[j][1]);
+                    e4m3x4_to_f16x2x2(__byte_perm(r[2], 0, 0x3120), a[0], a[1]);
+                    e4m3x4_to_f16x2x2(__byte_perm(r[3], 0, 0x3120), a[2], a[3]);
+#pragma unroll
+                    for (int j = 0; j < kQW; ++j) mma_f16(o[j][2 * jj + 1], a, pb[j][0], pb[j][1]);
+                }
             }
         }
         if constexpr (kPV) {
             // the normaliser: sums of the rounded weights, as one more row block of the product (V^T = all ones)
-            const uint32_t ones[4] = {0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u};
+            constexpr uint32_t kOne = F8 ? 0x3c003c00u : 0x3f803f80u;      // 1.0 twice, in the weights' format
+            const uint32_t ones[4] = {kOne, kOne, kOne, kOne};
 #pragma unroll
-            for (int j = 0; j < kQW; ++j) mma_bf16(lacc[j], ones, pb[j][0], pb[j][1]);
+            for (int j = 0; j < kQW; ++j) {
+                if constexpr (F8) mma_f16(lacc[j], ones, pb[j][0], pb[j][1]);
+                else mma_bf16(lacc[j], ones, pb[j][0], pb[j][1]);
+            }
         }
         if constexpr (kQK) {
 #pragma unroll
@@ -437,12 +526,12 @@ attn_extend_mq(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
                 mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
             }
-            mn[j][0] = fmaxf(m[j][0], mx0 * scale); mn[j][1] = fmaxf(m[j][1], mx1 * scale);
+            mn[j][0] = fmaxf(m[j][0], mx0 * smul[j][0]); mn[j][1] = fmaxf(m[j][1], mx1 * smul[j][1]);
             const float nu0 = mn[j][0] == -INFINITY ? 0.f : -mn[j][0], nu1 = mn[j][1] == -INFINITY ? 0.f : -mn[j][1];
-            const float p0 = ex2(fmaf(sc[j][0], scale, nu0)), p1 = ex2(fmaf(sc[j][1], scale, nu1));
-            const float p2 = ex2(fmaf(sc[j][2], scale, nu0)), p3 = ex2(fmaf(sc[j][3], scale, nu1));
-            const uint32_t pa = pack_bf16x2(p0, p1);             // key g8   : heads 2t4, 2t4+1
-            const uint32_t pc = pack_bf16x2(p2, p3);             // key g8+8
+            const float p0 = ex2(fmaf(sc[j][0], smul[j][0], nu0)), p1 = ex2(fmaf(sc[j][1], smul[j][1], nu1));
+            const float p2 = ex2(fmaf(sc[j][2], smul[j][0], nu0)), p3 = ex2(fmaf(sc[j][3], smul[j][1], nu1));
+            const uint32_t pa = F8 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1);             // key g8   : heads 2t4, 2t4+1
+            const uint32_t pc = F8 ? pack_f16x2(p2, p3) : pack_bf16x2(p2, p3);             // key g8+8
             psum[j][0] = p0 + p2;                                  // exact weights: the lse
             psum[j][1] = p1 + p3;
             pbn[j][0] = movmatrix_trans(pa);                       // P^T as B operand: k = key, n = head
@@ -651,15 +740,15 @@ extend_mq_combine(const AttnParams p) {
     }
 }
 
-template <int D>
+template <int D, bool F8>
 size_t mq_smem_bytes(int B) {
-    using C = MqCfg<D>;
+    using C = MqCfg<D, F8>;
     return 1024 + (size_t)C::kFixedBytes + (size_t)C::kStages * C::kStageBytes + sizeof(int64_t) * (B + 1) + 16;
 }
 
-template <int D>
+template <int D, bool F8>
 cudaError_t launch_mq(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaStream_t st) {
-    const size_t smem = mq_smem_bytes<D>(p.B);
+    const size_t smem = mq_smem_bytes<D, F8>(p.B);
     {
         static std::mutex mu;
         static bool attr_set[64] = {};      // per device: the opt-in to > 48 KB of dynamic shared memory
@@ -667,12 +756,12 @@ cudaError_t launch_mq(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaStrea
         cudaGetDevice(&dev);
         std::lock_guard<std::mutex> lock(mu);
         if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-            cudaError_t e = cudaFuncSetAttribute(attn_extend_mq<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+            cudaError_t e = cudaFuncSetAttribute(attn_extend_mq<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
             if (e != cudaSuccess) return e;
             if (dev >= 0 && dev < 64) attr_set[dev] = true;
         }
     }
-    attn_extend_mq<D><<<p.num_ctas, MqCfg<D>::kThreads, smem, st>>>(mk, mv, p);
+    attn_extend_mq<D, F8><<<p.num_ctas, MqCfg<D, F8>::kThreads, smem, st>>>(mk, mv, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
@@ -686,8 +775,9 @@ cudaError_t launch_mq(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaStrea
 
 }  // namespace
 
-bool extend_mq_fits(int B, int D) {
-    const size_t need = D == 128 ? mq_smem_bytes<128>(B) : mq_smem_bytes<256>(B);
+bool extend_mq_fits(int B, int D, int f8) {
+    const size_t need = f8 ? (D == 128 ? mq_smem_bytes<128, true>(B) : mq_smem_bytes<256, true>(B))
+                           : (D == 128 ? mq_smem_bytes<128, false>(B) : mq_smem_bytes<256, false>(B));
     return need <= 227 * 1024;
 }
 
@@ -695,8 +785,11 @@ cudaError_t launch_extend_mq(const AttnParams& p_in, cudaStream_t st) {
     AttnParams p = p_in;
     const int64_t rows = p.mode == kPaged ? (int64_t)p.num_pages * p.Hkv * p.page_size : (int64_t)p.B * p.Hkv * p.rows_per_head;
     CUtensorMap mk, mv;
-    if (!make_map(&mk, p.k, rows, p.D, 2) || !make_map(&mv, p.v, rows, p.D, 2)) return cudaErrorInvalidValue;
-    cudaError_t e = p.D == 128 ? launch_mq<128>(mk, mv, p, st) : launch_mq<256>(mk, mv, p, st);
+    const int esz = p.f8 ? 1 : 2;
+    if (!make_map(&mk, p.k, rows, p.D, esz) || !make_map(&mv, p.v, rows, p.D, esz)) return cudaErrorInvalidValue;
+    cudaError_t e;
+    if (p.f8) e = p.D == 128 ? launch_mq<128, true>(mk, mv, p, st) : launch_mq<256, true>(mk, mv, p, st);
+    else e = p.D == 128 ? launch_mq<128, false>(mk, mv, p, st) : launch_mq<256, false>(mk, mv, p, st);
     count_launch(2);
     return e;
 }

@@ -515,7 +515,7 @@ wmtp_status wmtp_draft_extend_windowed(const void* q, int q_len, int Hq, const w
 // a sequence. Returns false when the launch does not fit it (the per-query path then serves the call).
 static bool extend_full_shared_tiles(const void* q, int q_len, int Hq, const wmtp_kv* kv, float sm_scale, void* out, float* lse,
                                      void* ws, cudaStream_t st, wmtp_status* result) {
-    if (q_len < 2 || kv->kv_dtype != WMTP_KV_BF16 || !extend_mq_fits(kv->batch, kv->D)) return false;
+    if (q_len < 2 || !extend_mq_fits(kv->batch, kv->D, kv->kv_dtype == WMTP_KV_FP8_E4M3)) return false;
     const int nch = (q_len + kExtendChunk - 1) / kExtendChunk, nstreams = kv->batch * kv->Hkv * nch;
     const int slot_rows = q_len < kExtendChunk ? q_len : kExtendChunk;
     // the partial pool of a workspace sized for batch * q_len sequences holds pool_slots rows of G x (D + 1) floats
@@ -526,6 +526,7 @@ static bool extend_full_shared_tiles(const void* q, int q_len, int Hq, const wmt
     p.B = kv->batch;                        // this kernel counts sequences, not queries
     p.q_len = q_len;
     p.k = kv->k; p.v = kv->v; p.page_table = kv->page_table; p.len = kv->len;
+    p.f8 = kv->kv_dtype == WMTP_KV_FP8_E4M3 ? 1 : 0; p.k_scale = kv->k_scale; p.v_scale = kv->v_scale;
     p.S_cap = kv->S_cap;
     p.mode = kv->page_table ? kPaged : kContiguous;
     p.rows_per_head = kv->page_table ? kv->page_size : kv->S_cap;

@@ -127,10 +127,10 @@ cudaError_t make_attention_maps(const AttnParams& p, AttnMaps* maps);
 cudaError_t launch_attention(const AttnParams& p, const AttnMaps& maps, cudaStream_t st);
 int pick_cluster(int D, int f8, int nseg, int64_t tiles_per_segment, int max_ctas);
 
-// Full-context draft-extend with shared K/V tiles (bf16 stores): p.B counts sequences, p.q_len their new tokens;
+// Full-context draft-extend with shared K/V tiles: p.B counts sequences, p.q_len their new tokens;
 // partial results go to p.part_lse / p.part_o, (p.num_ctas + streams) * min(q_len, kExtendChunk) rows of G (x D) floats.
 cudaError_t launch_extend_mq(const AttnParams& p, cudaStream_t st);
-bool extend_mq_fits(int B, int D);     // does the kernel's shared memory hold the tables of B sequences?
+bool extend_mq_fits(int B, int D, int f8);     // does the kernel's shared memory hold the tables of B sequences?
 
 cudaError_t launch_mass_diagnostics(const void* o_win, const float* lse_win, const void* o_full, const float* lse_full, int rows,
                                     int D, float* mass, float* perturb, float* tail, cudaStream_t st);

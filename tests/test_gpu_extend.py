@@ -163,21 +163,32 @@ def _extend_and_check(cfg, max_ctas=0, seqs=None):
             compare(out_f[b, i], lse_f[b, i], *r["full"], what=tag + " extend full")
 
 
+@pytest.mark.parametrize("kv_dtype", ["bf16", "fp8"])
 @pytest.mark.parametrize("D", [128, 256])
 @pytest.mark.parametrize("S0", [0, 2, 60, 66, 70, 300, 2000])
 @pytest.mark.parametrize("max_ctas", [1, 0])
-def test_extend_matches_sequential_steps(D, S0, max_ctas):
+def test_extend_matches_sequential_steps(D, S0, max_ctas, kv_dtype):
     # n_sink + W = 68 and five new tokens: the queries straddle sink-filling, window-filling and sliding states
-    _extend_and_check(_cfg(S0=S0, D=D, cap_slack=4, seed=900 + S0), max_ctas=max_ctas)
+    _extend_and_check(_cfg(S0=S0, D=D, cap_slack=4, seed=900 + S0, kv_dtype=kv_dtype), max_ctas=max_ctas)
 
 
+@pytest.mark.parametrize("kv_dtype", ["bf16", "fp8"])
 @pytest.mark.parametrize("paged", [False, True])
-def test_extend_batched_ragged(paged):
-    _extend_and_check(_cfg(batch=4, S0=0, S0_range=(10, 3000), paged=paged, gamma=7, cap_slack=8, W=128, seed=31))
+def test_extend_batched_ragged(paged, kv_dtype):
+    _extend_and_check(_cfg(batch=4, S0=0, S0_range=(10, 3000), paged=paged, gamma=7, cap_slack=8, W=128, seed=31, kv_dtype=kv_dtype,
+                           key_scale=(0.5, 2.0) if kv_dtype == "fp8" else None))
 
 
-def test_extend_at_long_context():
-    _extend_and_check(wi.scaled(wi.CONFIGS[1], gamma=7, cap_slack=6, name="ext_s128k"))
+@pytest.mark.parametrize("kv_dtype", ["bf16", "fp8"])
+def test_extend_at_long_context(kv_dtype):
+    _extend_and_check(wi.scaled(wi.CONFIGS[1], gamma=7, cap_slack=6, kv_dtype=kv_dtype, name="ext_s128k_" + kv_dtype))
+
+
+@pytest.mark.parametrize("D", [128, 256])
+def test_extend_fp8_group_sizes_and_query_chunks(D):
+    """fp8 store, six new tokens (two passes: a chunk of four queries and one of two), three query heads per KV head
+    (heads beyond the group read as zero in the MMA tile), distinct scales per KV head."""
+    _extend_and_check(_cfg(S0=700, D=D, Hq=6, Hkv=2, gamma=6, cap_slack=8, W=128, seed=77, kv_dtype="fp8", key_scale=(0.5, 2.0)))
 
 
 def test_extend_needs_slack_slots():
