@@ -89,9 +89,8 @@ struct Cfg {
     static constexpr int kStealChunk = kStealChunkBytes / (2 * kTileBytes);
     static_assert(kStealChunk % kPair == 0, "a cursor step hands out whole stages");
     static constexpr int kStealMinTiles = 8 * kStealChunk;   // ranges shorter than this are streamed statically
-    // columns of d merged per pass of a flush: the two-group configurations of the streaming form trade a second pass
-    // for shared memory (stage depth); the cluster form, fed from L2, has the room
-    static constexpr int kPassCols = (kGroups == 2 && !CL) ? 64 : 128;
+    // columns of d merged per pass of a flush: the two-group configurations trade a second pass for shared memory
+    static constexpr int kPassCols = (kGroups == 2) ? 64 : 128;
     static constexpr int kScratchRow = kPassCols + 4;
     static constexpr int kMergeFloats = kGroupWarps * kMaxGroup * kScratchRow;
     static constexpr int kScratchFloats = kMergeFloats > kCombineFloats ? kMergeFloats : kCombineFloats;
