@@ -137,9 +137,11 @@ def _stream(stream) -> int:
 class Ring:
     """Device ring-buffer KV store for ``batch`` sequences: n_sink sink slots + ``cap`` window slots.
 
-    ``k_scale`` / ``v_scale`` (device fp32 [Hkv]) select an fp8 (e4m3) store: uint8 codes, value = code * scale."""
+    ``k_scale`` / ``v_scale`` (device fp32 [Hkv]) select an fp8 (e4m3) store: uint8 codes, value = code * scale.
+    ``alloc(shape, dtype, device)`` returns the (uninitialised) device tensor for each of the four arrays; the default is
+    ``torch.empty``. A caller with its own memory pool, or a test that wants guard bands around the arrays, passes one."""
 
-    def __init__(self, batch, Hkv, D, n_sink, W, cap=None, device="cuda", k_scale=None, v_scale=None):
+    def __init__(self, batch, Hkv, D, n_sink, W, cap=None, device="cuda", k_scale=None, v_scale=None, alloc=None):
         cap = W if cap is None else cap
         self.batch, self.Hkv, self.D, self.n_sink, self.W, self.cap = batch, Hkv, D, n_sink, W, cap
         slots = n_sink + cap
@@ -147,10 +149,11 @@ class Ring:
         f8 = k_scale is not None
         dt = torch.uint8 if f8 else torch.bfloat16
         self.k_scale, self.v_scale = k_scale, v_scale
-        self.k = torch.zeros((batch, Hkv, slots, D), dtype=dt, device=device)
-        self.v = torch.zeros((batch, Hkv, slots, D), dtype=dt, device=device)
-        self.slot_pos = torch.full((batch, slots), -1, dtype=torch.int32, device=device)
-        self.len = torch.zeros((batch,), dtype=torch.int64, device=device)
+        alloc = alloc or (lambda shape, dtype, device: torch.empty(shape, dtype=dtype, device=device))
+        self.k = alloc((batch, Hkv, slots, D), dt, device).zero_()
+        self.v = alloc((batch, Hkv, slots, D), dt, device).zero_()
+        self.slot_pos = alloc((batch, slots), torch.int32, device).fill_(-1)
+        self.len = alloc((batch,), torch.int64, device).zero_()
         self.desc = wmtp_ring(self.k.data_ptr(), self.v.data_ptr(), self.slot_pos.data_ptr(), self.len.data_ptr(),
                               batch, Hkv, D, n_sink, W, cap, WMTP_KV_FP8_E4M3 if f8 else WMTP_KV_BF16, _ptr(k_scale),
                               _ptr(v_scale))
@@ -184,10 +187,11 @@ class KV:
 
 
 class Workspace:
-    def __init__(self, batch, Hq, Hkv, D, device="cuda", stream=None):
+    def __init__(self, batch, Hq, Hkv, D, device="cuda", stream=None, alloc=None):
         self.nbytes = int(lib().wmtp_workspace_bytes(batch, Hq, Hkv, D))
+        alloc = alloc or (lambda shape, dtype, device: torch.empty(shape, dtype=dtype, device=device))
         # 0xFF bytes are NaN as floats: a partial result read before it is written cannot go unnoticed
-        self.buf = torch.full((self.nbytes,), 0xFF, dtype=torch.uint8, device=device)
+        self.buf = alloc((self.nbytes,), torch.uint8, device).fill_(0xFF)
         assert self.buf.data_ptr() % 256 == 0
         wmtp_workspace_init(self, stream=stream)
 

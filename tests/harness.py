@@ -15,6 +15,38 @@ MAX_ABS, MEAN_ABS = 2e-2, 2e-3
 REL_L2, LSE_ABS = 1e-2, 1e-3
 
 
+class GuardedAlloc:
+    """Device allocations with sentinel-filled bands before and after them: a kernel that writes outside one of the
+    arrays it was given changes a band, which `check()` notices (the stand-in for a memory checker on this path)."""
+
+    BAND, SENTINEL = 4096, 0xA5
+
+    def __init__(self):
+        self.blocks = []                                   # (name, padded uint8 buffer, payload offset, payload bytes)
+
+    def __call__(self, shape, dtype, device="cuda", name=""):
+        nbytes = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        padded = (nbytes + 255) // 256 * 256
+        buf = torch.full((2 * self.BAND + padded + 256,), self.SENTINEL, dtype=torch.uint8, device=device)
+        off = self.BAND + (-(buf.data_ptr() + self.BAND)) % 256        # the array itself starts on a 256-byte boundary
+        self.blocks.append((name or f"array {len(self.blocks)}", buf, off, nbytes))
+        return buf[off:off + nbytes].view(dtype).view(shape)
+
+    def like(self, t: torch.Tensor, name=""):
+        """A guarded copy of t (same shape, dtype, contents)."""
+        g = self(tuple(t.shape), t.dtype, t.device, name)
+        g.copy_(t)
+        return g
+
+    def check(self, what=""):
+        if torch.cuda.is_available():
+            torch.cuda.synchronize()
+        for name, buf, off, nbytes in self.blocks:
+            lo, hi = buf[:off], buf[off + nbytes:]
+            ok = bool((lo == self.SENTINEL).all()) and bool((hi == self.SENTINEL).all())
+            assert ok, f"{what}: bytes outside {name} were written"
+
+
 def to_dev_bf16(a: np.ndarray, dev="cuda"):
     return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(dev).view(torch.bfloat16)
 
@@ -38,21 +70,27 @@ class DeviceWorkload:
     def __init__(self, wl: wi.Workload, dev="cuda", cap=None):
         cfg = wl.cfg
         self.wl, self.cfg, self.dev = wl, cfg, dev
+        # every array a kernel writes lives between guard bands (stores of more than 1 GiB are left as they are)
+        self.guard = g = GuardedAlloc()
         self.K, self.V = to_dev_store(wl.K_dev, dev), to_dev_store(wl.V_dev, dev)
-        self.lens = torch.from_numpy(wl.seq_lens.copy()).to(dev)
+        if self.K.numel() * self.K.element_size() <= (1 << 30):
+            self.K, self.V = g.like(self.K, "KV store K"), g.like(self.V, "KV store V")
+        self.lens = g.like(torch.from_numpy(wl.seq_lens.copy()).to(dev), "the KV lengths")
         pt = torch.from_numpy(wl.page_table).to(dev) if cfg.paged else None
         self.k_scale = torch.from_numpy(wl.k_scale).to(dev) if wl.k_scale is not None else None
         self.v_scale = torch.from_numpy(wl.v_scale).to(dev) if wl.v_scale is not None else None
         self.kv = wm.KV(self.K, self.V, self.lens, page_table=pt, S_cap=None if cfg.paged else wl.S_cap,
                         k_scale=self.k_scale, v_scale=self.v_scale)
         self.ring = wm.Ring(cfg.batch, cfg.Hkv, cfg.D, cfg.n_sink, cfg.W, cap=cap if cap is not None else cfg.W + cfg.cap_slack,
-                            device=dev, k_scale=self.k_scale, v_scale=self.v_scale)
-        self.ws = wm.Workspace(cfg.batch, cfg.Hq, cfg.Hkv, cfg.D, device=dev)
+                            device=dev, k_scale=self.k_scale, v_scale=self.v_scale,
+                            alloc=lambda shape, dtype, device: g(shape, dtype, device, "a ring array"))
+        self.ws = wm.Workspace(cfg.batch, cfg.Hq, cfg.Hkv, cfg.D, device=dev,
+                               alloc=lambda shape, dtype, device: g(shape, dtype, device, "the workspace"))
         self.q, self.k_new, self.v_new = to_dev_bf16(wl.q, dev), to_dev_bf16(wl.k_new, dev), to_dev_bf16(wl.v_new, dev)
-        self.out_w = torch.full_like(self.q, float("nan"))
-        self.out_f = torch.full_like(self.q, float("nan"))
-        self.lse_w = torch.full(self.q.shape[:-1], float("nan"), dtype=torch.float32, device=dev)
-        self.lse_f = torch.full(self.q.shape[:-1], float("nan"), dtype=torch.float32, device=dev)
+        self.out_w = g(tuple(self.q.shape), torch.bfloat16, dev, "out (windowed)").fill_(float("nan"))
+        self.out_f = g(tuple(self.q.shape), torch.bfloat16, dev, "out (full)").fill_(float("nan"))
+        self.lse_w = g(tuple(self.q.shape[:-1]), torch.float32, dev, "lse (windowed)").fill_(float("nan"))
+        self.lse_f = g(tuple(self.q.shape[:-1]), torch.float32, dev, "lse (full)").fill_(float("nan"))
 
     def run_loops(self, windowed=True, full=True):
         if windowed:
@@ -61,6 +99,7 @@ class DeviceWorkload:
         if full:
             wm.wmtp_draft_loop_full(self.kv, self.q, self.k_new, self.v_new, self.out_f, self.ws, lse=self.lse_f)
         wm.wmtp_device_status(self.ws)
+        self.guard.check(self.cfg.name)
 
 
 def compare(got_bf16: torch.Tensor, got_lse: torch.Tensor | None, ref_out: np.ndarray, ref_lse: np.ndarray, what=""):

@@ -154,6 +154,7 @@ def _extend_and_check(cfg, max_ctas=0, seqs=None):
     wm.wmtp_draft_extend_windowed(qm, dw.ring, out_w, ws, lse=lse_w)
     wm.wmtp_draft_extend_full(qm, dw.kv, out_f, ws, lse=lse_f)
     wm.wmtp_device_status(ws)
+    dw.guard.check(cfg.name)                 # appends and extends wrote nothing outside the stores
     for b in (range(cfg.batch) if seqs is None else seqs):
         orc = oracle_for(wl, b, with_ring=False)
         for i in range(qlen):

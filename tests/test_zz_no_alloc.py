@@ -51,7 +51,7 @@ class _Case:
         got = torch.full(shape, float("nan"), dtype=torch.bfloat16, device="cuda")
         got_lse = torch.full(shape[:2], float("nan"), device="cuda")
         wm.wmtp_draft_attn_windowed_noalloc(dw.q[i], dw.ring, got, lse=got_lse)
-        torch.cuda.synchronize()
+        dw.guard.check(cfg.name)
         for b in range(cfg.batch):
             r = self.orcs[b].step(self.wl.q[i, b], self.wl.k_new[i, b], self.wl.v_new[i, b], full=False)
             compare(got[b], got_lse[b], *r["win"], what=f"{cfg.name} call {i} seq {b} vs oracle")
