@@ -128,6 +128,20 @@ wmtp_status wmtp_device_status(void* workspace, void* stream);
 wmtp_status wmtp_ring_reset(const wmtp_ring* ring, void* stream);
 
 /*
+ * Snapshot and restore of a ring. The paper defines no checkpoint format: this is the store of Appendix A (RING) copied
+ * as it stands -- K rows, V rows, slot_pos, len, in that order, each starting on a 256-byte boundary of the blob.
+ * wmtp_ring_state_bytes: size of the snapshot (0 for an invalid descriptor). wmtp_ring_export copies the four arrays
+ * into `blob`, wmtp_ring_import copies them back into a ring of the same geometry (batch, Hkv, D, n_sink, cap,
+ * kv_dtype are the caller's to keep; only the size is checked; the scales of an fp8 ring are not part of the state).
+ * `blob` is device memory or page-locked host memory, 16-byte aligned, blob_bytes >= wmtp_ring_state_bytes(ring);
+ * the copies are asynchronous on `stream`. A ring restored from a snapshot taken between two draft steps continues
+ * bit-identically.
+ */
+size_t      wmtp_ring_state_bytes(const wmtp_ring* ring);
+wmtp_status wmtp_ring_export(const wmtp_ring* ring, void* blob, size_t blob_bytes, void* stream);
+wmtp_status wmtp_ring_import(const wmtp_ring* ring, const void* blob, size_t blob_bytes, void* stream);
+
+/*
  * Seeds the ring from a context KV holding S = kv->len[r] tokens per sequence: copies positions
  * [0, min(S, n_sink)) and [max(n_sink, S - cap), S) into their slots, sets slot_pos and len = S.
  * The result is bit-identical to S sequential wmtp_ring_append calls (Section 6, "Prefill

@@ -54,6 +54,9 @@ _SIGNATURES = {
     "wmtp_device_status": (c_int, [c_void_p, c_void_p]),
     "wmtp_ring_reset": (c_int, [POINTER(wmtp_ring), c_void_p]),
     "wmtp_ring_init_from_kv": (c_int, [POINTER(wmtp_ring), POINTER(wmtp_kv), c_void_p]),
+    "wmtp_ring_state_bytes": (c_size_t, [POINTER(wmtp_ring)]),
+    "wmtp_ring_export": (c_int, [POINTER(wmtp_ring), c_void_p, c_size_t, c_void_p]),
+    "wmtp_ring_import": (c_int, [POINTER(wmtp_ring), c_void_p, c_size_t, c_void_p]),
     "wmtp_ring_append": (c_int, [POINTER(wmtp_ring), c_void_p, c_void_p, c_void_p]),
     "wmtp_kv_append": (c_int, [POINTER(wmtp_kv), c_void_p, c_void_p, c_void_p, c_void_p]),
     "wmtp_draft_attn_windowed": (c_int, [c_void_p, c_int, POINTER(wmtp_ring), c_float, c_void_p, c_void_p, c_void_p,
@@ -235,6 +238,19 @@ def wmtp_device_status(ws: Workspace, stream=None) -> None:
 
 def wmtp_ring_reset(ring: Ring, stream=None) -> None:
     _check(lib().wmtp_ring_reset(byref(ring.desc), _stream(stream)))
+
+
+def wmtp_ring_state_bytes(ring: Ring) -> int:
+    return int(lib().wmtp_ring_state_bytes(byref(ring.desc)))
+
+
+def wmtp_ring_export(ring: Ring, blob, stream=None) -> None:
+    """blob: uint8 tensor (device or pinned host) of at least wmtp_ring_state_bytes(ring) bytes."""
+    _check(lib().wmtp_ring_export(byref(ring.desc), _ptr(blob), blob.numel() * blob.element_size(), _stream(stream)))
+
+
+def wmtp_ring_import(ring: Ring, blob, stream=None) -> None:
+    _check(lib().wmtp_ring_import(byref(ring.desc), _ptr(blob), blob.numel() * blob.element_size(), _stream(stream)))
 
 
 def wmtp_ring_init_from_kv(ring: Ring, kv: KV, stream=None) -> None:

@@ -385,6 +385,52 @@ wmtp_status wmtp_ring_reset(const wmtp_ring* ring, void* stream) {
     return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "ring reset launch");
 }
 
+// ---- snapshot / restore of a ring: four plain copies, each part on a 256-byte boundary of the blob
+namespace {
+struct RingState { size_t kv_bytes, pos_bytes, len_bytes, off_v, off_pos, off_len, total; };
+RingState ring_state(const wmtp_ring* r) {
+    RingState s;
+    const size_t slots = (size_t)r->n_sink + (size_t)r->cap;
+    s.kv_bytes = (size_t)r->batch * r->Hkv * slots * r->D * (r->kv_dtype == WMTP_KV_FP8_E4M3 ? 1 : 2);
+    s.pos_bytes = (size_t)r->batch * slots * sizeof(int32_t);
+    s.len_bytes = (size_t)r->batch * sizeof(int64_t);
+    s.off_v = round_up(s.kv_bytes, 256);
+    s.off_pos = s.off_v + round_up(s.kv_bytes, 256);
+    s.off_len = s.off_pos + round_up(s.pos_bytes, 256);
+    s.total = s.off_len + round_up(s.len_bytes, 256);
+    return s;
+}
+wmtp_status ring_copy(const wmtp_ring* ring, void* blob, size_t blob_bytes, cudaStream_t st, bool to_blob) {
+    if (wmtp_status s = check_ring(ring)) return s;
+    if (!blob || !aligned(blob, 16)) return fail(WMTP_ERR_INVALID_ARG, "blob is NULL or not 16-byte aligned");
+    const RingState rs = ring_state(ring);
+    if (blob_bytes < rs.total) return fail(WMTP_ERR_CAPACITY, "blob of %zu bytes, the ring's state takes %zu", blob_bytes, rs.total);
+    char* b = static_cast<char*>(blob);
+    struct Part { void* ring_ptr; size_t off, bytes; };
+    const Part parts[4] = {{ring->k, 0, rs.kv_bytes}, {ring->v, rs.off_v, rs.kv_bytes}, {ring->slot_pos, rs.off_pos, rs.pos_bytes},
+                           {ring->len, rs.off_len, rs.len_bytes}};
+    for (const Part& pt : parts) {
+        const cudaError_t e = to_blob ? cudaMemcpyAsync(b + pt.off, pt.ring_ptr, pt.bytes, cudaMemcpyDefault, st)
+                                      : cudaMemcpyAsync(pt.ring_ptr, b + pt.off, pt.bytes, cudaMemcpyDefault, st);
+        if (e != cudaSuccess) return cuda_fail(e, to_blob ? "ring export copy" : "ring import copy");
+    }
+    return WMTP_OK;
+}
+}  // namespace
+
+size_t wmtp_ring_state_bytes(const wmtp_ring* ring) {
+    if (check_ring(ring) != WMTP_OK) return 0;
+    return ring_state(ring).total;
+}
+
+wmtp_status wmtp_ring_export(const wmtp_ring* ring, void* blob, size_t blob_bytes, void* stream) {
+    return ring_copy(ring, blob, blob_bytes, (cudaStream_t)stream, true);
+}
+
+wmtp_status wmtp_ring_import(const wmtp_ring* ring, const void* blob, size_t blob_bytes, void* stream) {
+    return ring_copy(ring, const_cast<void*>(blob), blob_bytes, (cudaStream_t)stream, false);
+}
+
 wmtp_status wmtp_ring_init_from_kv(const wmtp_ring* ring, const wmtp_kv* kv, void* stream) {
     if (wmtp_status s = check_ring(ring)) return s;
     if (wmtp_status s = check_kv(kv)) return s;

@@ -45,6 +45,23 @@ def test_sizes():
     assert wm.wmtp_status_string(0) == "ok" and "bounds" in wm.wmtp_status_string(7)
 
 
+def test_ring_snapshot_size_and_arguments_rejected_on_host():
+    L = wm.lib()
+    good = _ring_desc()
+    # K and V rows (2 KV heads x 12 slots x 128 x 2 bytes), slot_pos (12 x 4), len (8): each part on a 256-byte boundary
+    assert L.wmtp_ring_state_bytes(ctypes.byref(good)) == 2 * 6144 + 256 + 256
+    f8 = _ring_desc(kv_dtype=1, k_scale=4096, v_scale=4096)
+    assert L.wmtp_ring_state_bytes(ctypes.byref(f8)) == 2 * 3072 + 256 + 256
+    assert L.wmtp_ring_state_bytes(ctypes.byref(_ring_desc(W=0))) == 0
+    need = L.wmtp_ring_state_bytes(ctypes.byref(good))
+    for fn in (L.wmtp_ring_export, L.wmtp_ring_import):
+        assert fn(ctypes.byref(good), None, need, None) == 1                       # no blob
+        assert fn(ctypes.byref(good), 4104, need, None) == 1                       # misaligned blob
+        assert fn(ctypes.byref(good), 4096, need - 1, None) == 3                   # blob too small
+        assert "takes" in wm.wmtp_last_error()
+        assert fn(ctypes.byref(_ring_desc(cap=4)), 4096, need, None) == 1          # bad descriptor
+
+
 def _ring_desc(**kw):
     d = dict(k=4096, v=8192, slot_pos=4096, len=4096, batch=1, Hkv=2, D=128, n_sink=4, W=8, cap=8)
     d.update(kw)

@@ -324,3 +324,48 @@ def test_one_workspace_serves_two_batch_sizes_in_turn():
                 r = orcs[name][b].step(wl.q[i + j, b], wl.k_new[i + j, b], wl.v_new[i + j, b], full=False)
                 compare(ow[j, b], lw[j, b], *r["win"], what=f"{name} step {i + j} seq {b}")
         done[name] += steps
+
+
+# ------------------------------------------------------------------------------------------ snapshot / restore
+@pytest.mark.parametrize("kv_dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("where", ["device", "pinned host"])
+def test_ring_snapshot_restores_a_ring_that_continues_bit_identically(kv_dtype, where):
+    """Three draft steps, snapshot, two more steps; a second ring restored from the snapshot and given the same two steps
+    ends with the same bits in every array and gave the same outputs; the blob's bytes beyond the state are untouched."""
+    cfg = _cfg(S0=500, D=128, W=64, gamma=5, cap_slack=3, seed=4242, kv_dtype=kv_dtype,
+               key_scale=(0.5, 2.0) if kv_dtype == "fp8" else None)
+    wl = wi.make_workload(cfg)
+    dw = DeviceWorkload(wl)
+    wm.wmtp_ring_init_from_kv(dw.ring, dw.kv)
+    need = wm.wmtp_ring_state_bytes(dw.ring)
+    blob = torch.full((need + 512,), 0x5A, dtype=torch.uint8, device="cuda" if where == "device" else "cpu")
+    if where != "device":
+        blob = blob.pin_memory()
+    q, kn, vn = dw.q, dw.k_new, dw.v_new
+    outs = torch.full_like(q, float("nan"))
+    wm.wmtp_draft_loop_windowed(dw.ring, q[:3], kn[:3], vn[:3], outs[:3], dw.ws)
+    wm.wmtp_ring_export(dw.ring, blob)
+    wm.wmtp_draft_loop_windowed(dw.ring, q[3:], kn[3:], vn[3:], outs[3:], dw.ws)
+    torch.cuda.synchronize()
+    assert (blob[need:] == 0x5A).all()
+    twin = wm.Ring(cfg.batch, cfg.Hkv, cfg.D, cfg.n_sink, cfg.W, cap=cfg.W + cfg.cap_slack, k_scale=dw.k_scale, v_scale=dw.v_scale)
+    twin.k.fill_(3); twin.v.fill_(3)                              # stale contents the import must replace
+    wm.wmtp_ring_import(twin, blob)
+    outs2 = torch.full_like(q[3:], float("nan"))
+    wm.wmtp_draft_loop_windowed(twin, q[3:], kn[3:], vn[3:], outs2, dw.ws)
+    wm.wmtp_device_status(dw.ws)
+    dw.guard.check(cfg.name)
+    assert torch.equal(bits_t(twin.k), bits_t(dw.ring.k)) and torch.equal(bits_t(twin.v), bits_t(dw.ring.v))
+    assert torch.equal(twin.slot_pos, dw.ring.slot_pos) and torch.equal(twin.len, dw.ring.len)
+    assert torch.equal(outs2.view(torch.int16), outs[3:].view(torch.int16))
+    # and the continued ring is the oracle's ring
+    orc = oracle_for(wl, 0)
+    for i in range(cfg.gamma):
+        r = orc.step(wl.q[i, 0], wl.k_new[i, 0], wl.v_new[i, 0], full=False)
+        if i >= 3:
+            compare(outs2[i - 3, 0], None, *r["win"], what=f"restored ring step {i}")
+    check_ring_against_sim(twin, 0, orc.ring, "restored ring")
+
+
+def bits_t(t):
+    return t if t.dtype == torch.uint8 else t.view(torch.int16)
