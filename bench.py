@@ -395,6 +395,52 @@ def main():
         lens.copy_(torch.from_numpy(cur_lens).to(dev))
         wm.wmtp_ring_init_from_kv(ring, kv)
         torch.cuda.synchronize()
+    # ---- index structures of a paged store: the O(W) reduced block table of the windowed draft against the O(S) token
+    #      index a full-context draft rebuilds every step (a paged view of the same lengths when the store is contiguous)
+    index_build = None
+    try:
+        ps = 64
+        S_max = int(cur_lens.max())
+        mp = (S_max + ps - 1) // ps + 1
+        if cfg.paged:
+            kv_p = kv
+        else:
+            pt_i = torch.arange(B * mp, dtype=torch.int32, device=dev).view(B, mp)
+            dummy = torch.empty((1, cfg.Hkv, ps, cfg.D), dtype=K.dtype, device=dev)
+            kv_p = wm.KV(dummy.expand(B * mp, -1, -1, -1), dummy.expand(B * mp, -1, -1, -1), lens, page_table=pt_i, **scales)
+        width = wm.wmtp_reduced_block_table_width(cfg.n_sink, cfg.W, ps)
+        table = torch.empty((B, width), dtype=torch.int32, device=dev)
+        meta = torch.empty((B, 5), dtype=torch.int32, device=dev)
+        index = torch.empty((B, (S_max + 64 + 3) // 4 * 4), dtype=torch.int32, device=dev)
+
+        def time_calls(fn):
+            # replayed from a CUDA graph: an eager loop of such short launches measures the host's launch rate
+            gs2 = torch.cuda.Stream()
+            g2 = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(gs2):
+                fn()
+                torch.cuda.synchronize()
+                with torch.cuda.graph(g2, stream=gs2):
+                    for _ in range(reps):
+                        fn()
+            torch.cuda.synchronize()
+            g2.replay()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(3):
+                g2.replay()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) * 1e3 / (3 * reps)
+        us_table = time_calls(lambda: wm.wmtp_reduced_block_table(kv_p, cfg.n_sink, cfg.W, table, meta, ws))
+        us_index = time_calls(lambda: wm.wmtp_full_token_index(kv_p, index, ws))
+        wm.wmtp_device_status(ws)
+        index_build = {"reduced_block_table_us": us_table, "reduced_table_entries_per_sequence": width,
+                       "full_token_index_us": us_index, "full_index_entries_per_sequence": int(index.shape[1]),
+                       "note": "O(W / page) against O(S): what the windowed and the full-context draft of a paged serving stack "
+                               "rebuild before each attention call; this library's kernels need neither"}
+    except Exception as exc:
+        log(f"[bench] index-build comparison skipped: {exc}")
     # ---- draft-extend after a verify step: q_len = 4 tokens per sequence (3 accepted + the bonus token) appended to
     #      a ring with slack slots and to the KV store, then attended in one launch each
     ext = None
@@ -640,6 +686,7 @@ def main():
                          "us_per_attention_call": us_full_call,
                          "us_per_step_graph_replay": us_full_graph},
                 "draft_extend": ext,
+                "index_build": index_build,
                 "fp8_kv": f8,
             },
             "windowed_flatness": flat,

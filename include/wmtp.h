@@ -246,6 +246,17 @@ int         wmtp_reduced_block_table_width(int n_sink, int W, int page_size);
 wmtp_status wmtp_reduced_block_table(const wmtp_kv* kv, int n_sink, int W, int32_t* table, int table_stride, int32_t* meta,
                                      void* workspace, void* stream);
 
+/*
+ * The O(S) counterpart, for comparison: the pool row of every token of a paged store, which a full-context (native)
+ * draft rebuilds before every attention call (Section 3, t_ctx; Appendix B, per-kernel table: the draft's KV index
+ * build). index[r][s] = page_table[r][s / page_size] * page_size + s mod page_size for s < len[r], -1 for
+ * len[r] <= s < index_stride; `index` is device int32 [batch][index_stride]. A length beyond index_stride or a page id
+ * outside the pool is flagged WMTP_ERR_DEVICE_BOUNDS in `workspace` (may be NULL) and the entry is -1. The attention
+ * entry points of this library never need it (they walk the page table arithmetically); it exists so that the O(S)
+ * and the O(W) structure can be timed side by side.
+ */
+wmtp_status wmtp_full_token_index(const wmtp_kv* kv, int32_t* index, int64_t index_stride, void* workspace, void* stream);
+
 /* ---- after verification: rollback and draft-extend -------------------------------------------- */
 
 /*

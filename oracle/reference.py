@@ -199,6 +199,16 @@ def reduced_block_table(S: int, n_sink: int, W: int, page_row, page_size: int):
     return pages, meta
 
 
+def full_token_index(S: int, page_row, page_size: int, stride: int):
+    """The O(S) structure a full-context draft over a paged store rebuilds every step (Section 3, t_ctx; Appendix B,
+    per-kernel table: the draft's KV index build): for each token position s < S the pool row that holds it,
+    page_row[s // page_size] * page_size + s % page_size; -1 from S up to ``stride``.  One entry per token."""
+    out = [-1] * stride
+    for s in range(min(S, stride)):
+        out[s] = int(page_row[s // page_size]) * page_size + s % page_size
+    return out
+
+
 class WindowStore:
     """Explicit sink list + window list; the key set is their concatenation."""
 

@@ -79,6 +79,7 @@ _SIGNATURES = {
                                             c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "wmtp_reduced_block_table_width": (c_int, [c_int, c_int, c_int]),
     "wmtp_reduced_block_table": (c_int, [POINTER(wmtp_kv), c_int, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
+    "wmtp_full_token_index": (c_int, [POINTER(wmtp_kv), c_void_p, c_int64, c_void_p, c_void_p]),
     "wmtp_ring_rewind": (c_int, [POINTER(wmtp_ring), c_void_p, c_void_p, c_void_p]),
     "wmtp_ring_append_many": (c_int, [POINTER(wmtp_ring), c_int, c_void_p, c_void_p, c_void_p]),
     "wmtp_ring_replace_tail": (c_int, [POINTER(wmtp_ring), c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -374,6 +375,12 @@ def wmtp_attn_mass_diagnostics(out_win, lse_win, out_full, lse_full, mass=None, 
     rows = out_win.numel() // D
     _check(lib().wmtp_attn_mass_diagnostics(_ptr(out_win), _ptr(lse_win), _ptr(out_full), _ptr(lse_full), rows, D, _ptr(mass),
                                             _ptr(perturb), _ptr(tail), _stream(stream)))
+
+
+def wmtp_full_token_index(kv: KV, index, ws: Workspace | None = None, stream=None) -> None:
+    """index: device int32 [batch][stride]; entry s of a row is the pool row of token s, -1 beyond the length."""
+    _check(lib().wmtp_full_token_index(byref(kv.desc), _ptr(index), index.shape[1], ws.ptr if ws is not None else None,
+                                       _stream(stream)))
 
 
 def wmtp_reduced_block_table_width(n_sink: int, W: int, page_size: int) -> int:

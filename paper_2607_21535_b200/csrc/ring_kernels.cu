@@ -249,6 +249,52 @@ __global__ void reduced_block_table_kernel(KvParams kv, int n_sink, int W, int32
     }
 }
 
+// The structure a full-context draft over a paged store rebuilds before every attention call (Appendix B, per-kernel
+// table: the draft's KV index build, O(S) per step): the pool row of every token, index[b][s] = page * page_size +
+// s mod page_size for s < len[b], -1 beyond. Built here to be measured against the O(W) table above; the attention
+// kernels of this library walk the page table directly and need neither.
+__global__ void full_token_index_kernel(KvParams kv, int32_t* __restrict__ index, int64_t stride, int vec4, int* status) {
+    const int b = blockIdx.y, ps = kv.page_size;
+    const int64_t S = kv.len[b];
+    if (S > stride && blockIdx.x == 0 && threadIdx.x == 0 && status) atomicCAS(status, 0, kErrBounds);
+    const int32_t* pt = kv.page_table + (int64_t)b * kv.max_pages;
+    auto row_of = [&](int64_t s, int page) { return page * ps + (int32_t)(s % ps); };
+    auto page_of = [&](int64_t s) {
+        const int page = pt[s / ps];
+        if (page < 0 || page >= kv.num_pages) { if (status) atomicCAS(status, 0, kErrBounds); return -1; }
+        return page;
+    };
+    const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, dt = (int64_t)gridDim.x * blockDim.x;
+    if (vec4) {
+        // four consecutive tokens lie in one page (page_size and stride are multiples of 4): one lookup, one 16-byte store
+        int4* out = reinterpret_cast<int4*>(index + (int64_t)b * stride);
+        for (int64_t i = t0; i < stride / 4; i += dt) {
+            const int64_t s = 4 * i;
+            int4 r = make_int4(-1, -1, -1, -1);
+            if (s < S) {
+                const int page = page_of(s);
+                if (page >= 0) {
+                    const int32_t r0 = row_of(s, page);
+                    r.x = r0;
+                    if (s + 1 < S) r.y = r0 + 1;
+                    if (s + 2 < S) r.z = r0 + 2;
+                    if (s + 3 < S) r.w = r0 + 3;
+                }
+            }
+            out[i] = r;
+        }
+    } else {
+        for (int64_t s = t0; s < stride; s += dt) {
+            int32_t row = -1;
+            if (s < S) {
+                const int page = page_of(s);
+                if (page >= 0) row = row_of(s, page);
+            }
+            index[(int64_t)b * stride + s] = row;
+        }
+    }
+}
+
 // Rollback and append in one launch (the draft's state update after a verify step): drop the last n_drop[b] tokens, then
 // append n_tok new ones at the positions that follow. Slots of dropped positions that are not rewritten are marked
 // empty. Same conditions as ring_rewind_kernel; a violation leaves the sequence unchanged and is flagged.
@@ -377,6 +423,15 @@ cudaError_t launch_kv_append_many(const KvParams& kv, int n_tok, const void* k_n
 cudaError_t launch_reduced_block_table(const KvParams& kv, int n_sink, int W, int32_t* table, int stride, int32_t* meta, int* status,
                                        cudaStream_t st) {
     reduced_block_table_kernel<<<kv.B, 128, 0, st>>>(kv, n_sink, W, table, stride, meta, status);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_full_token_index(const KvParams& kv, int32_t* index, int64_t stride, int* status, cudaStream_t st) {
+    const int vec4 = kv.page_size % 4 == 0 && stride % 4 == 0 && reinterpret_cast<uintptr_t>(index) % 16 == 0;
+    const int64_t per_seq = ((vec4 ? stride / 4 : stride) + 255) / 256;
+    const unsigned gx = (unsigned)(per_seq < 1 ? 1 : (per_seq > 1024 ? 1024 : per_seq));
+    full_token_index_kernel<<<dim3(gx, kv.B), 256, 0, st>>>(kv, index, stride, vec4, status);
     count_launch(1);
     return cudaGetLastError();
 }

@@ -626,6 +626,17 @@ wmtp_status wmtp_reduced_block_table(const wmtp_kv* kv, int n_sink, int W, int32
     return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "reduced block table launch");
 }
 
+wmtp_status wmtp_full_token_index(const wmtp_kv* kv, int32_t* index, int64_t index_stride, void* workspace, void* stream) {
+    if (wmtp_status s = check_kv(kv)) return s;
+    if (!kv->page_table) return fail(WMTP_ERR_INVALID_ARG, "a token index needs a paged store");
+    if (!index || !aligned(index, 4)) return fail(WMTP_ERR_INVALID_ARG, "index is NULL or misaligned");
+    if (index_stride < 1) return fail(WMTP_ERR_INVALID_ARG, "index_stride=%lld must be positive", (long long)index_stride);
+    if ((int64_t)kv->num_pages * kv->page_size > INT32_MAX)
+        return fail(WMTP_ERR_UNSUPPORTED, "pool rows do not fit the 32-bit index");
+    cudaError_t e = launch_full_token_index(kv_params(kv), index, index_stride, static_cast<int*>(workspace), (cudaStream_t)stream);
+    return e == cudaSuccess ? WMTP_OK : cuda_fail(e, "token index launch");
+}
+
 wmtp_status wmtp_draft_loop_windowed_kv(const wmtp_kv* kv, int n_sink, int W, int gamma, const void* q, int Hq,
                                         const void* k_new, const void* v_new, float sm_scale, void* out, float* lse,
                                         void* workspace, size_t ws_bytes, void* stream) {

@@ -119,6 +119,7 @@ cudaError_t launch_ring_replace_tail(const RingParams& r, const int32_t* n_drop,
                                      int* status, cudaStream_t st);
 cudaError_t launch_reduced_block_table(const KvParams& kv, int n_sink, int W, int32_t* table, int stride, int32_t* meta, int* status,
                                        cudaStream_t st);
+cudaError_t launch_full_token_index(const KvParams& kv, int32_t* index, int64_t stride, int* status, cudaStream_t st);
 // The TMA descriptors of a store's K and V tensors. They depend on the store only (base pointers, rows, head_dim, entry
 // size), so a chain of launches on one store encodes them once.
 struct AttnMaps { CUtensorMap k, v; };

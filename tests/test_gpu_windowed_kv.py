@@ -137,3 +137,34 @@ def test_reduced_block_table_needs_a_wide_enough_table_and_a_paged_store():
     with pytest.raises(wm.WmtpError) as ei:
         wm.wmtp_reduced_block_table(dc.kv, 4, 256, torch.zeros((2, 8), dtype=torch.int32, device="cuda"), meta)
     assert ei.value.status == 1
+
+
+# ------------------------------------------------------------------------------------------ the O(S) counterpart
+def test_full_token_index_bit_exact_and_flags_a_short_table():
+    cfg = wi.DraftConfig("fti", 7, 0, 16, 2, 128, 64, 4, 1, seed=77, S0_range=(1, 9000), paged=True)
+    wl = wi.make_workload(cfg)
+    dw = DeviceWorkload(wl)
+    lens = wl.seq_lens.copy()
+    lens[0], lens[1], lens[2] = 0, 1, 64
+    dw.lens.copy_(torch.from_numpy(lens))
+    stride = int(lens.max()) + 37
+    index = dw.guard((cfg.batch, stride), torch.int32, "cuda", "the token index").fill_(-7)
+    wm.wmtp_full_token_index(dw.kv, index, dw.ws)
+    wm.wmtp_device_status(dw.ws)
+    dw.guard.check("token index")
+    got = index.cpu().numpy()
+    for b in range(cfg.batch):
+        assert got[b].tolist() == R.full_token_index(int(lens[b]), wl.page_table[b], 64, stride), b
+    # a table shorter than the longest sequence: its entries are still right, the overflow is flagged
+    short = torch.full((cfg.batch, 100), -7, dtype=torch.int32, device="cuda")
+    wm.wmtp_full_token_index(dw.kv, short, dw.ws)
+    with pytest.raises(wm.WmtpError) as ei:
+        wm.wmtp_device_status(dw.ws)
+    assert ei.value.status == 7
+    sh = short.cpu().numpy()
+    for b in range(cfg.batch):
+        assert sh[b].tolist() == R.full_token_index(int(lens[b]), wl.page_table[b], 64, 100)
+    dc = DeviceWorkload(wi.make_workload(wi.scaled(cfg, paged=False, S0=300, S0_range=None)))
+    with pytest.raises(wm.WmtpError) as ei:
+        wm.wmtp_full_token_index(dc.kv, short)
+    assert ei.value.status == 1

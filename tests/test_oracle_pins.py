@@ -499,3 +499,23 @@ def test_reduced_block_table_expands_to_the_keep_set(n_sink, W, ps):
             rows += [(pages[n_s + i], r) for r in range(lo, hi)]
         want = [(int(page_row[p // ps]), p % ps) for p in R.keep_set(S, n_sink, W)]        # brute force, token by token
         assert rows == want, (S, meta)
+
+
+@pytest.mark.parametrize("ps", [64, 16])
+def test_full_token_index_gathers_the_logical_sequence_from_the_pool(ps):
+    """The index is right when reading the pool through it gives back every sequence's keys in order: pool rows are
+    filled from the logical K by the input generator's own scatter (page by page), the index must invert it."""
+    cfg = wi.DraftConfig("idx", 3, 0, 4, 2, 128, 32, 2, 1, seed=5150 + ps, S0_range=(1, 5 * ps + 3), paged=True, page_size=ps)
+    wl = wi.make_workload(cfg, poison_unused=False)
+    pool = wl.K_dev                                              # [num_pages][Hkv][ps][D]
+    rows = np.ascontiguousarray(np.swapaxes(pool, 0, 1)).reshape(cfg.Hkv, -1, cfg.D)     # per KV head: pool row -> key
+    stride = int(wl.seq_lens.max()) + 5
+    for b in range(cfg.batch):
+        S = int(wl.seq_lens[b])
+        idx = R.full_token_index(S, wl.page_table[b], ps, stride)
+        assert len(idx) == stride and all(i == -1 for i in idx[S:]) and all(i >= 0 for i in idx[:S])
+        assert len(set(idx[:S])) == S                            # no pool row twice
+        for g in range(cfg.Hkv):
+            assert (rows[g][idx[:S]] == wl.K[b][g][:S]).all()
+    # a table shorter than the sequence keeps its first entries
+    assert R.full_token_index(10, [7, 3], 4, 6) == [28, 29, 30, 31, 12, 13]
