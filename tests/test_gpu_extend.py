@@ -369,3 +369,22 @@ def test_ring_snapshot_restores_a_ring_that_continues_bit_identically(kv_dtype, 
 
 def bits_t(t):
     return t if t.dtype == torch.uint8 else t.view(torch.int16)
+
+
+# ------------------------------------------------------------------------------------------ seeded random shapes
+@pytest.mark.parametrize("idx", range(20))
+def test_extend_random_shape(idx):
+    """Draft-extend (windowed and full-context, multi-query kernel and per-query path alike) on seeded random shapes:
+    group sizes that leave MMA columns empty, 1 to 9 sequences, 2 to 7 new tokens (one or two passes of four queries),
+    both store types and layouts, CTA caps."""
+    rs = np.random.RandomState(4100 + idx)
+    Hkv = int(rs.choice([1, 2, 4]))
+    G = int(rs.choice([1, 2, 3, 4, 7, 8]))
+    q_len = int(rs.choice([2, 3, 4, 5, 7]))
+    kv_dtype = str(rs.choice(["bf16", "fp8"]))
+    cfg = wi.DraftConfig(
+        name=f"extrand{idx}", batch=int(rs.choice([1, 1, 2, 3, 9])), S0=0, Hq=G * Hkv, Hkv=Hkv, D=int(rs.choice([128, 256])),
+        W=int(rs.choice([16, 64, 200, 1024])), n_sink=int(rs.choice([0, 1, 4, 64])), gamma=q_len, seed=4200 + idx,
+        S0_range=(1, int(rs.choice([200, 3000, 30000]))), paged=bool(rs.randint(2)), cap_slack=q_len - 1 + int(rs.choice([0, 3])),
+        kv_dtype=kv_dtype, key_scale=(0.5, 2.0) if Hkv > 1 and rs.randint(2) else None)
+    _extend_and_check(cfg, max_ctas=int(rs.choice([0, 0, 1, 5, 64])))
