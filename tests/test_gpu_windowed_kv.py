@@ -102,6 +102,17 @@ def test_window_view_rejects_bad_window():
     assert ei.value.status == 1
 
 
+@pytest.mark.parametrize("kv_dtype,D", [("fp8", 128), ("fp8", 256), ("bf16", 128)])
+@pytest.mark.parametrize("paged", [False, True])
+def test_window_view_long_enough_for_the_streaming_form(kv_dtype, D, paged):
+    """A window of 40000 tokens is served by the cooperative (streaming) form: with an fp8 head_dim-128 store its tiles
+    travel in pairs, and with three sink tiles (n_sink = 130) one pair holds the last sink tile and the first window
+    tile -- rows from two places of the store, each with its own row bounds."""
+    cfg = _cfg(S0=90001, n_sink=130, W=40000, D=D, Hq=8, Hkv=1, gamma=2, paged=paged, seed=611, kv_dtype=kv_dtype)
+    _run(cfg)
+    _run(cfg, max_ctas=5)
+
+
 # ------------------------------------------------------------------------------------------ the reduced block table itself
 @pytest.mark.parametrize("n_sink,W", [(4, 64), (0, 100), (64, 252), (70, 130), (4, 2048)])
 def test_reduced_block_table_bit_exact(n_sink, W):
