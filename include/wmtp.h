@@ -281,8 +281,10 @@ wmtp_status wmtp_full_token_index(const wmtp_kv* kv, int32_t* index, int64_t ind
  *   store. Query i of a sequence attends as a decode step would have at length len - (q_len - 1 - i): over sink + last W
  *   of that length (windowed; needs cap >= W + q_len - 1) or over all positions below it (full). out: device bf16
  *   [batch][q_len][Hq][D]; lse: device fp32 [batch][q_len][Hq] or NULL. The workspace must be sized for
- *   batch * q_len sequences: wmtp_workspace_bytes(batch * q_len, Hq, Hkv, D). One launch; K/V are read once per
- *   query from L2/HBM.
+ *   batch * q_len sequences: wmtp_workspace_bytes(batch * q_len, Hq, Hkv, D). The windowed form is one launch (the
+ *   ring is L2-resident; each query reads it). The full-context form reads every K/V tile from HBM once for up to four
+ *   queries of a sequence (one attention launch and one small merge launch; bf16 and fp8 stores); only a batch whose
+ *   per-sequence tables do not fit the kernel's shared memory is served query by query in a single launch.
  */
 wmtp_status wmtp_ring_rewind(const wmtp_ring* ring, const int32_t* n_drop, void* workspace, void* stream);
 wmtp_status wmtp_ring_append_many(const wmtp_ring* ring, int n_tok, const void* k_new, const void* v_new, void* stream);
