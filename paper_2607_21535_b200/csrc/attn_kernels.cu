@@ -66,9 +66,11 @@ constexpr int kStealChunkBytes = 262144;        // bytes of K/V handed out per c
 // contrib[kMaxContrib][4] = {seg, b, g, slot}, reg_k[kMaxContrib] (slot of the group's i-th contribution, producer -> group)
 constexpr int kGroupInts = 4 + 5 * kMaxContrib;
 
-// D: head_dim; F8: the store holds e4m3 codes (one byte per entry) instead of bf16; CL: the cluster form of the kernel.
-template <int D, bool F8, bool CL = false>
+// D: head_dim; F8: the store holds e4m3 codes (one byte per entry) instead of bf16; CL: the cluster form of the kernel;
+// ONE (cluster form only): one consumer group whatever the tile size -- for launches that leave a CTA a handful of tiles.
+template <int D, bool F8, bool CL = false, bool ONE = false>
 struct Cfg {
+    static_assert(CL || !ONE, "the one-group variant exists in the cluster form only");
     static constexpr int kElemBytes = F8 ? 1 : 2;
     static constexpr int kChunks = D * kElemBytes / 128;      // 128-byte column chunks per row
     static constexpr int kChunkBytes = kTileKeys * 128;       // one TMA box: 64 rows x 128 B
@@ -79,7 +81,7 @@ struct Cfg {
     static constexpr int kPair = (F8 && D == 128 && !CL) ? 2 : 1;
     static constexpr int kStageBytes = kPair * 2 * kTileBytes;
     // consumer groups: a tile of fewer bytes brings the same softmax work, so the smaller tiles get two groups
-    static constexpr int kGroups = (D == 256 && !F8) ? 1 : 2;
+    static constexpr int kGroups = ((D == 256 && !F8) || ONE) ? 1 : 2;
     // Stages of the shared-memory ring. What counts for the streaming rate is the bytes a CTA keeps in flight (about
     // 190 KB per SM saturate HBM at the loaded latency of ~4 us): the host takes as many stages as fit beside the
     // batch-dependent tables, up to kMaxStages, in multiples of the group count (a stage then always serves one group).
@@ -396,11 +398,11 @@ __device__ __noinline__ void patch_new_row(const void* new_rows, int64_t row_ind
 //     launch is an ordinary one (no CTA waits for another cluster), and the cluster that finishes last -- a ticket in
 //     the workspace header -- advances the lengths of a fused append. Tile processing is the same code in both forms.
 // ---------------------------------------------------------------------------------------------
-template <int D, bool F8, bool CL>
-__global__ void __launch_bounds__(Cfg<D, F8, CL>::kThreads, 1)
+template <int D, bool F8, bool ONE, bool CL>
+__global__ void __launch_bounds__(Cfg<D, F8, CL, ONE>::kThreads, 1)
 attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                const __grid_constant__ AttnParams p) {
-    using C = Cfg<D, F8, CL>;
+    using C = Cfg<D, F8, CL, ONE>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     // Shared memory: the fixed-size part first (compile-time offsets), then the stage ring (1024-byte aligned for the
@@ -1414,41 +1416,41 @@ cudaError_t launch_fused(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaSt
         cudaGetDevice(&dev);
         std::lock_guard<std::mutex> lock(mu);
         if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-            cudaError_t e = cudaFuncSetAttribute(attn_fused_tma<D, F8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+            cudaError_t e = cudaFuncSetAttribute(attn_fused_tma<D, F8, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
             if (e != cudaSuccess) return e;
             if (dev >= 0 && dev < 64) attr_set[dev] = true;
         }
     }
     void* args[] = {&mk, &mv, &p};
     // cooperative: the CTAs wait on one another in the combine, so they must all be resident
-    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(attn_fused_tma<D, F8, false>), dim3(p.num_ctas), dim3(Cfg<D, F8>::kThreads), args, smem, st);
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(attn_fused_tma<D, F8, false, false>), dim3(p.num_ctas), dim3(Cfg<D, F8>::kThreads), args, smem, st);
 }
 
 // ---- cluster form ----
 // Stages of the cluster form: as many as fit beside the groups' partial buffers (the data comes from L2: depth matters less
 // than in the streaming form).
-template <int D, bool F8>
+template <int D, bool F8, bool ONE>
 constexpr int cluster_stages() {
-    using C = Cfg<D, F8, true>;
+    using C = Cfg<D, F8, true, ONE>;
     int stages = C::kMaxStages;
     while (stages > C::kGroups &&
            1024 + C::kFixedBytes + stages * C::kStageBytes + (int)sizeof(float) * C::kGroups * (kMaxGroup * D + kMaxGroup) + 16 > 227 * 1024)
         stages -= C::kGroups;
     return stages;
 }
-template <int D, bool F8>
+template <int D, bool F8, bool ONE>
 size_t cluster_smem_bytes() {
-    using C = Cfg<D, F8, true>;
-    return 1024 + (size_t)C::kFixedBytes + (size_t)cluster_stages<D, F8>() * C::kStageBytes +
+    using C = Cfg<D, F8, true, ONE>;
+    return 1024 + (size_t)C::kFixedBytes + (size_t)cluster_stages<D, F8, ONE>() * C::kStageBytes +
            sizeof(float) * C::kGroups * (kMaxGroup * D + kMaxGroup) + 16;
 }
-static_assert(cluster_stages<256, false>() == 3 && cluster_stages<256, true>() >= 4 && cluster_stages<128, false>() >= 4 &&
-              cluster_stages<128, true>() >= 4, "cluster form: stages that fit shared memory");
+static_assert(cluster_stages<256, false, false>() == 3 && cluster_stages<256, true, false>() >= 4 && cluster_stages<128, false, false>() >= 4 &&
+              cluster_stages<128, true, false>() >= 4 && cluster_stages<128, false, true>() >= 4, "cluster form: stages that fit shared memory");
 
 // One-time set-up per device: shared-memory opt-in, non-portable cluster sizes, and how many clusters of each size the
 // device holds at once (index: log2 of the cluster size).
 struct ClusterInfo { bool ready; int sms; int active[kMaxCluster + 1]; };   // active[c]: resident clusters of c CTAs
-template <int D, bool F8>
+template <int D, bool F8, bool ONE>
 cudaError_t cluster_info(const ClusterInfo** out) {
     static std::mutex mu;
     static ClusterInfo info[64] = {};
@@ -1457,14 +1459,14 @@ cudaError_t cluster_info(const ClusterInfo** out) {
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     std::lock_guard<std::mutex> lock(mu);
     if (!info[dev].ready) {
-        auto* fn = attn_fused_tma<D, F8, true>;
+        auto* fn = attn_fused_tma<D, F8, ONE, true>;
         cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
         if (cudaDeviceGetAttribute(&info[dev].sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) info[dev].sms = 0;
         for (int cl = 1; cl <= kMaxCluster; ++cl) {
             cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(cl); cfg.blockDim = dim3(Cfg<D, F8, true>::kThreads); cfg.dynamicSmemBytes = cluster_smem_bytes<D, F8>();
+            cfg.gridDim = dim3(cl); cfg.blockDim = dim3(Cfg<D, F8, true, ONE>::kThreads); cfg.dynamicSmemBytes = cluster_smem_bytes<D, F8, ONE>();
             cudaLaunchAttribute at[1];
             at[0].id = cudaLaunchAttributeClusterDimension;
             at[0].val.clusterDim.x = (unsigned)cl; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
@@ -1479,12 +1481,18 @@ cudaError_t cluster_info(const ClusterInfo** out) {
     return cudaSuccess;
 }
 
-template <int D, bool F8>
+template <int D, bool F8, bool ONE>
 cudaError_t launch_cluster(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cudaStream_t st) {
-    using C = Cfg<D, F8, true>;
-    p.stages = cluster_stages<D, F8>();
+    using C = Cfg<D, F8, true, ONE>;
+    if constexpr (ONE) {
+        // this variant's own one-time set-up (the shared-memory and cluster-size opt-ins); its CTAs use no more shared
+        // memory than the two-group variant's, whose resident-cluster counts chose the cluster size
+        const ClusterInfo* unused = nullptr;
+        if (cudaError_t e = cluster_info<D, F8, ONE>(&unused); e != cudaSuccess) return e;
+    }
+    p.stages = cluster_stages<D, F8, ONE>();
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.num_ctas); cfg.blockDim = dim3(C::kThreads); cfg.dynamicSmemBytes = cluster_smem_bytes<D, F8>(); cfg.stream = st;
+    cfg.gridDim = dim3(p.num_ctas); cfg.blockDim = dim3(C::kThreads); cfg.dynamicSmemBytes = cluster_smem_bytes<D, F8, ONE>(); cfg.stream = st;
     cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = (unsigned)p.cluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
@@ -1492,7 +1500,7 @@ cudaError_t launch_cluster(CUtensorMap& mk, CUtensorMap& mv, AttnParams& p, cuda
     at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at; cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, attn_fused_tma<D, F8, true>, mk, mv, p);
+    return cudaLaunchKernelEx(&cfg, attn_fused_tma<D, F8, ONE, true>, mk, mv, p);
 }
 
 }  // namespace
@@ -1516,8 +1524,9 @@ cudaError_t launch_attention(const AttnParams& p_in, const AttnMaps& maps, cudaS
     CUtensorMap mk = maps.k, mv = maps.v;
     cudaError_t e;
     if (p.cluster > 0) {
-        if (p.f8) e = p.D == 128 ? launch_cluster<128, true>(mk, mv, p, st) : launch_cluster<256, true>(mk, mv, p, st);
-        else e = p.D == 128 ? launch_cluster<128, false>(mk, mv, p, st) : launch_cluster<256, false>(mk, mv, p, st);
+        if (p.f8) e = p.D == 128 ? launch_cluster<128, true, false>(mk, mv, p, st) : launch_cluster<256, true, false>(mk, mv, p, st);
+        else if (p.D == 256) e = launch_cluster<256, false, false>(mk, mv, p, st);
+        else e = p.one_group ? launch_cluster<128, false, true>(mk, mv, p, st) : launch_cluster<128, false, false>(mk, mv, p, st);
     } else {
         if (p.f8) e = p.D == 128 ? launch_fused<128, true>(mk, mv, p, st) : launch_fused<256, true>(mk, mv, p, st);
         else e = p.D == 128 ? launch_fused<128, false>(mk, mv, p, st) : launch_fused<256, false>(mk, mv, p, st);
@@ -1529,11 +1538,12 @@ cudaError_t launch_attention(const AttnParams& p_in, const AttnMaps& maps, cudaS
 // CTAs per cluster for a launch of `nseg` segments of at most `tiles` tiles each through the cluster form of the kernel,
 // or 0 when the cooperative form should serve it: the largest power of two (at most 16, at most `max_ctas` CTAs in all
 // when that is positive) whose clusters are all resident at once, as long as that leaves a CTA a handful of tiles.
-int pick_cluster(int D, int f8, int nseg, int64_t tiles, int max_ctas) {
+int pick_cluster(int D, int f8, int nseg, int64_t tiles, int max_ctas, int* one_group) {
+    *one_group = 0;
     const ClusterInfo* info = nullptr;
     cudaError_t e;
-    if (f8) e = D == 128 ? cluster_info<128, true>(&info) : cluster_info<256, true>(&info);
-    else e = D == 128 ? cluster_info<128, false>(&info) : cluster_info<256, false>(&info);
+    if (f8) e = D == 128 ? cluster_info<128, true, false>(&info) : cluster_info<256, true, false>(&info);
+    else e = D == 128 ? cluster_info<128, false, false>(&info) : cluster_info<256, false, false>(&info);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return 0; }
     // the largest cluster all of whose copies are resident at once (a second wave of clusters would double the time)
     int best = 0;
@@ -1552,6 +1562,9 @@ int pick_cluster(int D, int f8, int nseg, int64_t tiles, int max_ctas) {
     const int64_t per_coop = (tiles * nseg + coop_ctas - 1) / (coop_ctas > 0 ? coop_ctas : 1);
     const int tile_ns = f8 ? (D == 256 ? kTileNsF8D256 : kTileNsF8D128) : (D == 256 ? kTileNsD256 : kTileNsD128);
     if ((per_cta - per_coop) * tile_ns > kClusterFixedGainNs) return 0;
+    // With a handful of tiles per CTA one consumer group is the faster arrangement for the 32 KB tiles of a bf16
+    // head_dim-128 store too (one flush pass, half as many partials to merge); two groups win from about ten tiles on.
+    *one_group = !f8 && D == 128 && per_cta <= kOneGroupMaxTiles;
     return best;
 }
 

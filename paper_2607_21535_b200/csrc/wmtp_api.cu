@@ -214,7 +214,7 @@ wmtp_status attn_windowed(const void* q, int Hq, const wmtp_ring* ring, float sm
     bind_ring(p, ring, k_new, v_new);
     const int nseg = ring->batch * q_len * ring->Hkv;
     const int64_t tiles_per_seg = (p.rows_per_head + kTileKeys - 1) / kTileKeys, tiles = tiles_per_seg * nseg;
-    p.cluster = pick_cluster(p.D, p.f8, nseg, tiles_per_seg, g_max_ctas.load());
+    p.cluster = pick_cluster(p.D, p.f8, nseg, tiles_per_seg, g_max_ctas.load(), &p.one_group);
     if (p.cluster > 0) {
         p.num_ctas = nseg * p.cluster;
     } else {
@@ -254,7 +254,7 @@ wmtp_status attn_full(const void* q, int Hq, const wmtp_kv* kv, float sm_scale, 
     // extend, which re-reads rows through L2, measured slower on fewer SMs)
     const bool streaming = W == 0 && !p.f8 && q_len == 1 && kv->batch * kv->Hkv <= 8;
     const int nseg = kv->batch * q_len * kv->Hkv;
-    if (W > 0) p.cluster = pick_cluster(p.D, p.f8, nseg, tiles_per_seg, g_max_ctas.load());
+    if (W > 0) p.cluster = pick_cluster(p.D, p.f8, nseg, tiles_per_seg, g_max_ctas.load(), &p.one_group);
     if (p.cluster > 0) {
         p.num_ctas = nseg * p.cluster;
     } else {

@@ -21,6 +21,7 @@ constexpr int kMaxCluster = 16;                                  // CTAs in a th
 // measured with the ring in L2) and what the cluster form saves in fixed cost (launch overlap, no grid-wide combine).
 constexpr int kTileNsD256 = 1000, kTileNsD128 = 500, kTileNsF8D256 = 800, kTileNsF8D128 = 450;
 constexpr int kClusterFixedGainNs = 5500;
+constexpr int kOneGroupMaxTiles = 6;   // tiles per CTA up to which the one-group cluster variant is used (bf16, head_dim 128)
 constexpr int kExtendChunk = 4;     // new tokens of a sequence whose queries share one pass over its K/V (draft-extend)
 constexpr size_t kCursorBytes = 1024;                                          // int cur[kMaxCtas], padded
 constexpr size_t kWorkspaceZeroBytes = 256 + kCursorBytes + 2 * (8 + 4 + 4) * kMaxSegments;   // header + cursors + two copies of the per-segment words
@@ -92,6 +93,7 @@ struct AttnParams {
     int stages;               // stages of the kernel's shared-memory ring (set by the launcher)
     uint32_t spin_limit;      // polls a CTA spends waiting for another CTA's global word before it gives up
     int cluster;              // > 0: the cluster form of the kernel, one cluster of this many CTAs per segment (num_ctas = segments * cluster)
+    int one_group;            // cluster form, bf16 head_dim 128: the variant with one consumer group (few tiles per CTA)
 };
 
 struct RingParams {
@@ -126,7 +128,7 @@ struct AttnMaps { CUtensorMap k, v; };
 cudaError_t make_attention_maps(const AttnParams& p, AttnMaps* maps);
 // One launch: optional append of (k_new, v_new), split-KV partials, LSE combine (cooperative or cluster form: p.cluster).
 cudaError_t launch_attention(const AttnParams& p, const AttnMaps& maps, cudaStream_t st);
-int pick_cluster(int D, int f8, int nseg, int64_t tiles_per_segment, int max_ctas);
+int pick_cluster(int D, int f8, int nseg, int64_t tiles_per_segment, int max_ctas, int* one_group);
 
 // Full-context draft-extend with shared K/V tiles: p.B counts sequences, p.q_len their new tokens;
 // partial results go to p.part_lse / p.part_o, (p.num_ctas + streams) * min(q_len, kExtendChunk) rows of G (x D) floats.
