@@ -21,7 +21,7 @@ constexpr int kMaxCluster = 16;                                  // CTAs in a th
 // measured with the ring in L2) and what the cluster form saves in fixed cost (launch overlap, no grid-wide combine).
 constexpr int kTileNsD256 = 1000, kTileNsD128 = 500, kTileNsF8D256 = 800, kTileNsF8D128 = 450;
 constexpr int kClusterFixedGainNs = 5500;
-constexpr int kOneGroupMaxTiles = 6;   // tiles per CTA up to which the one-group cluster variant is used (bf16, head_dim 128)
+constexpr int kOneGroupMaxTiles = 5;   // tiles per CTA up to which the one-group cluster variant is used (bf16, head_dim 128)
 constexpr int kExtendChunk = 4;     // new tokens of a sequence whose queries share one pass over its K/V (draft-extend)
 constexpr size_t kCursorBytes = 1024;                                          // int cur[kMaxCtas], padded
 constexpr size_t kWorkspaceZeroBytes = 256 + kCursorBytes + 2 * (8 + 4 + 4) * kMaxSegments;   // header + cursors + two copies of the per-segment words
