@@ -244,6 +244,11 @@ def test_config_sweep_shape_fp8():
     _run_and_check(wi.scaled(wi.CONFIGS[4], S0=262144, W=4096, gamma=3, kv_dtype="fp8", name="sweep_fp8"))
 
 
+def test_config_sweep_shape_fp8_at_full_size():
+    """The head_dim-128 shape at the size the benchmark times it (S = 1,048,576; tiles in pairs), first and last step."""
+    _run_and_check(wi.scaled(wi.CONFIGS[4], kv_dtype="fp8", name="sweep_fp8_full_size"), steps={0, 6})
+
+
 @pytest.mark.parametrize("kv_dtype,D", [("fp8", 256), ("fp8", 128), ("bf16", 128), ("bf16", 256)])
 def test_very_large_batch_leaves_room_for_fewer_stages(kv_dtype, D):
     """1000 sequences: the batch-sized tables take shared memory from the stage ring, the kernel runs with fewer stages."""
