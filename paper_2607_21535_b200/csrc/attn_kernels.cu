@@ -92,9 +92,13 @@ struct Cfg {
     static_assert(kStealChunk % kPair == 0, "a cursor step hands out whole stages");
     static constexpr int kStealMinTiles = 8 * kStealChunk;   // ranges shorter than this are streamed statically
     // columns of d merged per pass of a flush: the two-group configurations trade a second pass for shared memory
-    static constexpr int kPassCols = (kGroups == 2) ? 64 : 128;
+    // (A cluster-form CTA with one group is done with its stages when it flushes: the warp merge then runs in stage
+    // memory, all of d in one pass.)
+    static constexpr bool kFlushInStages = CL && kGroups == 1;
+    static constexpr int kPassCols = kFlushInStages ? D : ((kGroups == 2) ? 64 : 128);
     static constexpr int kScratchRow = kPassCols + 4;
-    static constexpr int kMergeFloats = kGroupWarps * kMaxGroup * kScratchRow;
+    static constexpr int kMergeFloats = kFlushInStages ? 0 : kGroupWarps * kMaxGroup * kScratchRow;
+    static_assert(!kFlushInStages || kGroupWarps * kMaxGroup * kScratchRow * 4 <= kStageBytes, "the warp merge fits one stage");
     static constexpr int kScratchFloats = kMergeFloats > kCombineFloats ? kMergeFloats : kCombineFloats;
     // With two groups the CTA has 9 warps and a thread at most 168 registers: the query fragments (the same in all four
     // warps of a group) then live in shared memory, one copy per group, instead of D / 8 registers per thread.
@@ -793,6 +797,8 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     const int grp = threadIdx.x / kGroupThreads, tid = threadIdx.x % kGroupThreads;   // group, thread within the group
     const int warp = tid >> 5;                           // warp within the group: owns keys [16 warp, 16 warp + 16) of a tile
     float* scratch = scratch_all + grp * C::kScratchFloats;
+    // where a flush merges the four warps' accumulators: the group's scratch, or the first stage (see kFlushInStages)
+    float* fscratch = C::kFlushInStages ? reinterpret_cast<float*>(stages) : scratch;
     float* sm_m = sm_stats + grp * 3 * kGroupWarps * kMaxGroup;
     float* sm_l = sm_m + kGroupWarps * kMaxGroup;
     float* sm_le = sm_l + kGroupWarps * kMaxGroup;
@@ -910,7 +916,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 const int mb = pass * (C::kPassCols / 16) + mbl;
                 // accumulator rows g8 and g8 + 8 of block mb hold d = 16 mb + g8 and + 8 (bf16 store), or, for an fp8
                 // store whose V fragments come out of the transposed load with d pairs interleaved, d = 16 mb + 2 g8 and + 1
-                float* row0 = scratch + (warp * kMaxGroup + 2 * t4) * kScratchRow + mbl * 16 + (F8 ? 2 * g8 : g8);
+                float* row0 = fscratch + (warp * kMaxGroup + 2 * t4) * kScratchRow + mbl * 16 + (F8 ? 2 * g8 : g8);
                 float* row1 = row0 + kScratchRow;
                 constexpr int kSecond = F8 ? 1 : 8;
                 row0[0] = o[mb][0] * f[0]; row1[0] = o[mb][1] * f[1];
@@ -921,7 +927,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 const int h = idx / C::kPassCols, dd = idx % C::kPassCols;
                 float acc = 0.f;
 #pragma unroll
-                for (int w = 0; w < kGroupWarps; ++w) acc += scratch[(w * kMaxGroup + h) * kScratchRow + dd];
+                for (int w = 0; w < kGroupWarps; ++w) acc += fscratch[(w * kMaxGroup + h) * kScratchRow + dd];
                 dst_o[h * D + pass * C::kPassCols + dd] = acc;
             }
         }
