@@ -571,26 +571,17 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                                 row = ((int64_t)kv_seq(p, csg.b) * p.Hkv + csg.g) * p.rows_per_head + src * kTileKeys;
                             }
                             const uint32_t dstK = stage0 + s * C::kStageBytes, dstV = dstK + C::kTileBytes;
-                            stage_tile[s] = c_lo + base + j;       // ordered before the consumers' wait by the arrive below
-                            mbar_expect_tx(bar_fullK + 8 * s, C::kTileBytes);
+                            // One barrier for both tensors: the data comes from L2 well ahead of its use, and the consumers
+                            // know their tiles by number (group q takes c_lo + q, c_lo + q + kGroups, ... in order), so
+                            // this form has neither a second wait per tile nor tags nor end markers.
+                            mbar_expect_tx(bar_fullK + 8 * s, 2 * C::kTileBytes);
                             tma_load_3d(dstK, &mapK, (int)row, bar_fullK + 8 * s);
-                            mbar_expect_tx(bar_fullV + 8 * s, C::kTileBytes);
-                            tma_load_3d(dstV, &mapV, (int)row, bar_fullV + 8 * s);
+                            tma_load_3d(dstV, &mapV, (int)row, bar_fullK + 8 * s);
                         }
                     }
                 }
             }
-            if (lane == 0) {
-                // one end marker per consumer group
-                for (int q = 0; q < C::kGroups; ++q, ++it, ps = (ps + 1 == nst ? 0 : ps + 1), pph ^= (ps == 0)) {
-                    const uint32_t s = ps, ph = pph;
-                    const uint32_t gq = it % C::kGroups;
-                    mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, p.status);
-                    stage_tile[s] = -1;
-                    mbar_arrive(bar_fullK0 + 8 * (gq * C::kMaxStages + s));
-                    mbar_arrive(bar_fullV0 + 8 * (gq * C::kMaxStages + s));
-                }
-            }
+            (void)bar_fullV0;
             __syncwarp();
             cluster_sync_all();                  // the two barriers of the cluster's merge (the consumers' work lies between them)
             cluster_sync_all();
@@ -1166,7 +1157,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
                 pb[h][1] = movmatrix_trans(pc);
             }
         }
-        mbar_wait(bar_fullV + 8 * s, ph, abort_flag, p.status);
+        if constexpr (!CL) mbar_wait(bar_fullV + 8 * s, ph, abort_flag, p.status);      // (cluster form: K and V share a barrier)
         if (__builtin_expect(any_new, 0)) {
 #pragma unroll
             for (int h = 0; h < NH; ++h)
@@ -1245,11 +1236,18 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         if (__builtin_expect(need_enter, 0)) { enter_segment(tt); need_enter = false; }
         const uint32_t s = cs, ph = cph;             // stage of tile `it` and the parity of this group's use count of it
         if (!have_tile) {
-            const bool landed = mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
-            tt = *reinterpret_cast<volatile int64_t*>(stage_tile + s);
-            if (C::kPair == 2 && tt >= 0) { tcnt = (int)(tt & 1) + 1; tt >>= 1; }          // (first tile << 1) | (tiles - 1)
-            const bool end = tt < 0 || !landed;
-            const bool outside = sg.seg < 0 || tt < sg.seg_start || tt >= sg.seg_start + sg.tiles;
+            bool end, outside;
+            if constexpr (CL) {
+                tt = c_lo + (int)it;                                   // this CTA's tiles in order: nothing to look up
+                end = tt >= c_hi || !mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
+                outside = false;                                       // one segment per cluster
+            } else {
+                const bool landed = mbar_wait(bar_fullK + 8 * s, ph, abort_flag, p.status);
+                tt = *reinterpret_cast<volatile int64_t*>(stage_tile + s);
+                if (C::kPair == 2 && tt >= 0) { tcnt = (int)(tt & 1) + 1; tt >>= 1; }      // (first tile << 1) | (tiles - 1)
+                end = tt < 0 || !landed;
+                outside = sg.seg < 0 || tt < sg.seg_start || tt >= sg.seg_start + sg.tiles;
+            }
             if (__builtin_expect((end || outside) && sg.seg >= 0 && seg_tiles_done > 0, 0)) flush_segment();
             if (__builtin_expect(end || ncontrib == kMaxContrib, 0)) {
                 combine_outstanding();           // every segment this group contributed to (normally: once, at the end)
