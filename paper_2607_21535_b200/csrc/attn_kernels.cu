@@ -92,10 +92,10 @@ struct Cfg {
     static_assert(kStealChunk % kPair == 0, "a cursor step hands out whole stages");
     static constexpr int kStealMinTiles = 8 * kStealChunk;   // ranges shorter than this are streamed statically
     // columns of d merged per pass of a flush: the two-group configurations trade a second pass for shared memory
-    // (A cluster-form CTA with one group is done with its stages when it flushes: the warp merge then runs in stage
-    // memory, all of d in one pass.)
-    static constexpr bool kFlushInStages = CL && kGroups == 1;
-    static constexpr int kPassCols = kFlushInStages ? D : ((kGroups == 2) ? 64 : 128);
+    // (A group of a cluster-form CTA is done with its own stages when it flushes: the warp merge then runs in the group's
+    // first stage, all of d in one pass with one group, 128 columns at a time with two; 16 KB stages are too small.)
+    static constexpr bool kFlushInStages = CL && (kGroups == 1 || kStageBytes >= 32768);
+    static constexpr int kPassCols = kFlushInStages ? (kGroups == 1 ? D : 128) : ((kGroups == 2) ? 64 : 128);
     static constexpr int kScratchRow = kPassCols + 4;
     static constexpr int kMergeFloats = kFlushInStages ? 0 : kGroupWarps * kMaxGroup * kScratchRow;
     static_assert(!kFlushInStages || kGroupWarps * kMaxGroup * kScratchRow * 4 <= kStageBytes, "the warp merge fits one stage");
@@ -789,7 +789,7 @@ attn_fused_tma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
     const int warp = tid >> 5;                           // warp within the group: owns keys [16 warp, 16 warp + 16) of a tile
     float* scratch = scratch_all + grp * C::kScratchFloats;
     // where a flush merges the four warps' accumulators: the group's scratch, or the first stage (see kFlushInStages)
-    float* fscratch = C::kFlushInStages ? reinterpret_cast<float*>(stages) : scratch;
+    float* fscratch = C::kFlushInStages ? reinterpret_cast<float*>(stages + grp * C::kStageBytes) : scratch;
     float* sm_m = sm_stats + grp * 3 * kGroupWarps * kMaxGroup;
     float* sm_l = sm_m + kGroupWarps * kMaxGroup;
     float* sm_le = sm_l + kGroupWarps * kMaxGroup;
