@@ -411,3 +411,45 @@ def test_config_sweep_shape_at_full_size():
     # Hq=32, Hkv=4, D=128 at S=1,048,576 (the two-consumer-group kernel at the size the benchmark times), default CTAs;
     # first and last draft step
     _run_and_check(wi.scaled(wi.CONFIGS[4], name="sweep_full_size"), steps={0, 6})
+
+
+def test_two_host_threads_on_their_own_streams_and_workspaces():
+    """Two host threads drive their own stores, workspaces and streams at the same time (the library's per-device caches
+    are shared between them; cooperative launches of the two streams take the GPU in turn): both must match the oracle."""
+    import threading
+
+    cfgs = [wi.DraftConfig("thrA", 1, 3000, 16, 2, 256, 256, 4, 3, seed=91),
+            wi.DraftConfig("thrB", 2, 0, 8, 2, 128, 64, 4, 3, seed=92, S0_range=(500, 5000), paged=True)]
+    wls = [wi.make_workload(c) for c in cfgs]
+    dws = [DeviceWorkload(w) for w in wls]
+    streams = [torch.cuda.Stream() for _ in cfgs]
+    errors = []
+
+    def run(i):
+        try:
+            dw, st = dws[i], streams[i]
+            with torch.cuda.stream(st):
+                for _ in range(3):                                   # the same loops three times over: lengths restored in between
+                    dw.lens.copy_(torch.from_numpy(wls[i].seq_lens.copy()), non_blocking=False)
+                    wm.wmtp_ring_init_from_kv(dw.ring, dw.kv, stream=st.cuda_stream)
+                    wm.wmtp_draft_loop_windowed(dw.ring, dw.q, dw.k_new, dw.v_new, dw.out_w, dw.ws, lse=dw.lse_w, stream=st.cuda_stream)
+                    wm.wmtp_draft_loop_full(dw.kv, dw.q, dw.k_new, dw.v_new, dw.out_f, dw.ws, lse=dw.lse_f, stream=st.cuda_stream)
+                wm.wmtp_device_status(dw.ws, stream=st.cuda_stream)
+        except Exception as exc:                                     # surfaces in the main thread below
+            errors.append(exc)
+
+    threads = [threading.Thread(target=run, args=(i,)) for i in range(len(cfgs))]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    for i, (cfg, wl, dw) in enumerate(zip(cfgs, wls, dws)):
+        dw.guard.check(cfg.name)
+        for b in range(cfg.batch):
+            orc = oracle_for(wl, b)
+            for s in range(cfg.gamma):
+                r = orc.step(wl.q[s, b], wl.k_new[s, b], wl.v_new[s, b])
+                compare(dw.out_w[s, b], dw.lse_w[s, b], *r["win"], what=f"{cfg.name} seq={b} step={s} windowed")
+                compare(dw.out_f[s, b], dw.lse_f[s, b], *r["full"], what=f"{cfg.name} seq={b} step={s} full")
